@@ -1,0 +1,305 @@
+"""Algorithm 1 ("2M Ozaki-II") step by step in exact integers -- TEST INFRASTRUCTURE ONLY.
+
+Every function follows one passage of the paper, in its notation, with no blocking or fusion:
+
+  is_2m_modulus, greedy_2m_moduli   Section 2 (definition of a 2M modulus) and Section 4 (greedy coprime set in [1, 256])
+  sqrt_minus_one, inv2              Section 2: s^2 = -1 (mod m); 2^-1 = (m+1)/2
+  pre_2m, mul_2m, post_2m           Eq. (2a), (2b), (2c)
+  crt, lift                         Section 3.1 (CRT formula) and Algorithm 1 steps 5-6
+  scaling_targets, scaling_exponents, quantise, unscale   Algorithm 1 steps 2, 3, 7
+
+Readings taken where the paper is silent (they are the library's documented readings too):
+  * s is the smallest positive root (any root gives the same C);
+  * residues are kept as symmetric representatives in [-(m-1)/2, (m-1)/2];
+  * scale factors are powers of two chosen from the largest part-magnitude of each row of A /
+    column of B so that every entry of the integer product is bounded by 2^P_t <= (M-1)/2
+    (Cauchy-Schwarz), see `scaling_exponents`;
+  * quantisation truncates toward zero (keeps that bound rigorous);
+  * the CRT sum is reduced mod M and lifted to [-(M-1)/2, (M-1)/2];
+  * the lifted integer is rounded once (nearest-even) to the output precision, then scaled by 2^(e_i+f_j).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------- moduli (Sections 2, 4)
+def prime_factors(n: int):
+    out = []
+    p = 2
+    while p * p <= n:
+        while n % p == 0:
+            out.append(p)
+            n //= p
+        p += 1
+    if n > 1:
+        out.append(n)
+    return out
+
+
+def is_2m_modulus(m: int) -> bool:
+    """Section 2: m odd and a product of primes congruent to 1 mod 4 (equivalently s with s^2 = -1 exists)."""
+    return m > 1 and m % 2 == 1 and all(p % 4 == 1 for p in prime_factors(m))
+
+
+def greedy_2m_moduli(limit: int = 256):
+    """Section 4: walk down from `limit`, keep every 2M modulus coprime to all those already kept."""
+    kept = []
+    for cand in range(limit, 1, -1):
+        if is_2m_modulus(cand) and all(math.gcd(cand, q) == 1 for q in kept):
+            kept.append(cand)
+    return kept
+
+
+def sqrt_minus_one(m: int) -> int:
+    """Smallest positive s with s^2 = -1 (mod m) (Section 2)."""
+    for s in range(1, m):
+        if (s * s + 1) % m == 0:
+            return s
+    raise ValueError(f"{m} is not a 2M modulus")
+
+
+def inv2(m: int) -> int:
+    """Section 2: 2^-1 = (m+1)/2 mod m."""
+    return (m + 1) // 2
+
+
+def sym(x, m: int):
+    """Symmetric representative of x mod m (m odd): in [-(m-1)/2, (m-1)/2]."""
+    h = (m - 1) // 2
+    return (x + h) % m - h
+
+
+# ----------------------------------------------------------------------------- 2M multiplication (Eq. 2a-2c)
+def pre_2m(Xr, Xi, m: int, s: int):
+    """Eq. (2a): X+ = Xr + s Xi, X- = Xr - s Xi (mod m), symmetric representatives."""
+    return sym(Xr + s * Xi, m), sym(Xr - s * Xi, m)
+
+
+def _exact_matmul(P, Q):
+    """Exact integer matrix product of small-integer matrices (a library matmul used as one step)."""
+    P = np.asarray(P)
+    Q = np.asarray(Q)
+    k = P.shape[1]
+    pm = int(np.abs(P).max(initial=0))
+    qm = int(np.abs(Q).max(initial=0))
+    if max(k, 1) * pm * qm < 2 ** 52:              # exact in float64, BLAS does the work
+        return np.rint(P.astype(np.float64) @ Q.astype(np.float64)).astype(np.int64)
+    return P.astype(object) @ Q.astype(object)
+
+
+def mul_2m(Ap, Bp, m: int):
+    """Eq. (2b): C+- = A+- B+- (mod m)."""
+    return sym(_exact_matmul(Ap, Bp), m)
+
+
+def post_2m(Cp, Cm, m: int, s: int):
+    """Eq. (2c): C = 2^-1 (C- + C+) + i s 2^-1 (C- - C+) (mod m)."""
+    h = inv2(m)
+    return sym(h * (Cm + Cp), m), sym(s * h * (Cm - Cp), m)
+
+
+# ----------------------------------------------------------------------------- CRT (Section 3.1, Algorithm 1 steps 5-6)
+def product(moduli):
+    M = 1
+    for q in moduli:
+        M *= int(q)
+    return M
+
+
+def crt(residues, moduli):
+    """X = ( sum_l ((x_l q_l) mod m_l) (M/m_l) ) mod M with q_l = (M/m_l mod m_l)^-1 mod m_l, in [0, M)."""
+    M = product(moduli)
+    acc = 0
+    for x, ml in zip(residues, moduli):
+        ml = int(ml)
+        Wl = M // ml
+        ql = pow(Wl % ml, -1, ml)
+        x = np.asarray(x).astype(object) if isinstance(x, np.ndarray) else int(x)
+        acc = acc + ((x * ql) % ml) * Wl
+    return acc % M
+
+
+def lift(X, M: int):
+    """Algorithm 1 step 6: representative in [-M/2, M/2); M is odd so this is [-(M-1)/2, (M-1)/2]."""
+    h = (M - 1) // 2
+    return (X + h) % M - h
+
+
+# ----------------------------------------------------------------------------- scaling (Algorithm 1 steps 2, 3, 7)
+def scaling_targets(M: int, k: int, herk: bool = False):
+    """P_t = floor(log2((M-1)/2)); the row budget P_A and column budget P_B split it (equal for HERK);
+    c_k = ceil(log2(2k)/2) accounts for the 2k real terms of a row's 2-norm."""
+    Pt = ((M - 1) // 2).bit_length() - 1
+    PA, PB = -((-Pt) // 2), Pt // 2
+    if herk:
+        PA = PB = Pt // 2
+    ck = 0
+    while 4 ** ck < 2 * max(k, 1):
+        ck += 1
+    return Pt, PA, PB, ck
+
+
+def scaling_exponents(Z, axis: int, P: int, ck: int):
+    """sigma_i = 2^e_i (axis=1: per row of A) or tau_j = 2^f_j (axis=0: per column of B).
+    mu = largest |Re| or |Im| in the row/column, x = floor(log2 mu), e = x + 1 + c_k - P; zero rows get e = 0.
+    Then |z'| <= |z| 2^-e < 2^(P - c_k), so the row's 2-norm is at most sqrt(2k) 2^(P-c_k) <= 2^P."""
+    Z = np.asarray(Z)
+    mags = np.maximum(np.abs(Z.real), np.abs(Z.imag)).astype(np.float64)
+    mu = mags.max(axis=axis, initial=0.0)
+    _, ex = np.frexp(mu)                       # mu = f 2^ex with 0.5 <= f < 1, so floor(log2 mu) = ex - 1
+    e = ex.astype(np.int64) + ck - P
+    return np.where(mu > 0, e, 0).astype(np.int64)
+
+
+def _quantise_part(x, e):
+    """trunc(x 2^-e) exactly, elementwise; x float array, e broadcastable integer array.  Object array of ints."""
+    x = np.asarray(x, dtype=np.float64)
+    mant, ex = np.frexp(x)
+    Mi = np.ldexp(mant, 53).astype(np.int64)             # x = Mi 2^(ex-53), |Mi| < 2^53, exact
+    sh = ex.astype(np.int64) - 53 - e                    # x 2^-e = Mi 2^sh
+    sgn = np.sign(Mi)
+    mag = np.abs(Mi)
+    right = np.minimum(np.maximum(-sh, 0), 63)
+    out = (sgn * (mag >> right)).astype(object)          # truncation toward zero on the magnitude
+    pos = sh > 0
+    if np.any(pos):
+        flat_out = out.ravel()
+        flat_M = Mi.ravel()
+        flat_sh = np.broadcast_to(sh, x.shape).ravel()
+        for idx in np.flatnonzero(pos.ravel()):
+            flat_out[idx] = int(flat_M[idx]) << int(flat_sh[idx])
+        out = flat_out.reshape(x.shape)
+    return out
+
+
+def quantise(Z, e, axis: int):
+    """Algorithm 1 step 3 with truncation: (Zr', Zi') = trunc(parts of Z / 2^e) with e per row (axis=1) or column (axis=0)."""
+    Z = np.asarray(Z)
+    eb = e[:, None] if axis == 1 else e[None, :]
+    return _quantise_part(Z.real, eb), _quantise_part(Z.imag, eb)
+
+
+def round_int_nearest_even(X: int, bits: int):
+    """X ~ Y 2^t with |Y| <= 2^bits, round-to-nearest-even once."""
+    a = abs(X)
+    n = a.bit_length()
+    if n <= bits:
+        return X, 0
+    t = n - bits
+    q, r = divmod(a, 1 << t)
+    half = 1 << (t - 1)
+    if r > half or (r == half and (q & 1)):
+        q += 1
+    return (q if X >= 0 else -q), t
+
+
+def unscale(X, e_row, f_col, bits: int = 53):
+    """Algorithm 1 step 7: c_ij sigma_i tau_j with one rounding of the integer to `bits` significant bits."""
+    m, n = X.shape
+    out = np.zeros((m, n), dtype=np.float64)
+    for i in range(m):
+        for j in range(n):
+            y, t = round_int_nearest_even(int(X[i, j]), bits)
+            out[i, j] = math.ldexp(float(y), t + int(e_row[i]) + int(f_col[j]))
+    return out
+
+
+def _small(a):
+    """Object array of ints -> int64 when it fits (faster residues)."""
+    if a.size == 0:
+        return a.astype(np.int64)
+    mx = max(abs(int(a.max())), abs(int(a.min())))
+    return a.astype(np.int64) if mx < 2 ** 62 else a
+
+
+def _residue_planes(Zr, Zi, moduli, roots):
+    Zr, Zi = _small(Zr), _small(Zi)
+    planes = []
+    for ml, sl in zip(moduli, roots):
+        # reduce first so that s * Zi stays small in int64
+        zr = Zr % ml
+        zi = Zi % ml
+        p, q = pre_2m(zr, zi, ml, sl)
+        planes.append((np.asarray(p).astype(np.int64), np.asarray(q).astype(np.int64)))
+    return planes
+
+
+# ----------------------------------------------------------------------------- whole paths
+def gemm2m_int_staged(Ar, Ai, Br, Bi, nmod: int):
+    """Integer 2M multiplication (Section 2) + CRT over the first `nmod` moduli.  Returns a dict of stages."""
+    moduli = greedy_2m_moduli()[:nmod]
+    roots = [sqrt_minus_one(q) for q in moduli]
+    M = product(moduli)
+    Ar, Ai, Br, Bi = (np.asarray(x).astype(object) for x in (Ar, Ai, Br, Bi))
+    Apl = _residue_planes(Ar, Ai, moduli, roots)
+    Bpl = _residue_planes(Br, Bi, moduli, roots)
+    Cpm, res_r, res_i = [], [], []
+    for (Ap, Am), (Bp, Bm), ml, sl in zip(Apl, Bpl, moduli, roots):
+        Cp, Cm = mul_2m(Ap, Bp, ml), mul_2m(Am, Bm, ml)
+        Cpm.append((Cp, Cm))
+        r, i = post_2m(Cp, Cm, ml, sl)
+        res_r.append(r)
+        res_i.append(i)
+    Xr, Xi = lift(crt(res_r, moduli), M), lift(crt(res_i, moduli), M)
+    return dict(moduli=moduli, roots=roots, M=M, Apm=Apl, Bpm=Bpl, Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi)
+
+
+def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto: str = "all"):
+    """Algorithm 1 on floating-point A (m x k), B (k x n).  For herk=True pass B = A^H.
+    upto = "pre" stops after the residue planes (cheap at large sizes)."""
+    A = np.asarray(A)
+    B = np.asarray(B)
+    k = A.shape[1]
+    moduli = greedy_2m_moduli()[:nmod]                            # step 1
+    roots = [sqrt_minus_one(q) for q in moduli]
+    M = product(moduli)
+    Pt, PA, PB, ck = scaling_targets(M, k, herk)
+    eA = scaling_exponents(A, 1, PA, ck)                           # step 2
+    eB = scaling_exponents(B, 0, PB, ck)
+    Aq = quantise(A, eA, 1)                                        # step 3
+    Bq = quantise(B, eB, 0)
+    Apl = _residue_planes(Aq[0], Aq[1], moduli, roots)             # step 4: (2a)
+    Bpl = _residue_planes(Bq[0], Bq[1], moduli, roots)
+    st = dict(moduli=moduli, roots=roots, M=M, Pt=Pt, PA=PA, PB=PB, ck=ck, eA=eA, eB=eB, Aq=Aq, Bq=Bq,
+              Apm=Apl, Bpm=Bpl)
+    if upto == "pre":
+        return st
+    Cpm, res_r, res_i = [], [], []
+    for (Ap, Am), (Bp, Bm), ml, sl in zip(Apl, Bpl, moduli, roots):
+        Cp, Cm = mul_2m(Ap, Bp, ml), mul_2m(Am, Bm, ml)            # (2b)
+        Cpm.append((Cp, Cm))
+        r, i = post_2m(Cp, Cm, ml, sl)                             # (2c)
+        res_r.append(r)
+        res_i.append(i)
+    Xr, Xi = lift(crt(res_r, moduli), M), lift(crt(res_i, moduli), M)   # steps 5, 6
+    C = unscale(Xr, eA, eB, out_bits) + 1j * unscale(Xi, eA, eB, out_bits)   # step 7
+    st.update(Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi, C=C)
+    return st
+
+
+def staged_samples(st, pairs, out_bits: int = 53):
+    """Exact lifted integers and final values for sampled entries, from the quantised matrices of a
+    `zgemm2m_staged(..., upto="pre")` result: the 4M product of the quantised Gaussian integers reduced
+    mod M -- the value steps 4-6 must reproduce whatever multiplication method is used (Section 6)."""
+    M = st["M"]
+    Ar, Ai = st["Aq"]
+    Br, Bi = st["Bq"]
+    vals = np.zeros(len(pairs), dtype=np.complex128)
+    Xs = []
+    for t, (i, j) in enumerate(np.asarray(pairs).tolist()):
+        ar = [int(v) for v in Ar[i, :]]
+        ai = [int(v) for v in Ai[i, :]]
+        br = [int(v) for v in Br[:, j]]
+        bi = [int(v) for v in Bi[:, j]]
+        cr = sum(x * y for x, y in zip(ar, br)) - sum(x * y for x, y in zip(ai, bi))
+        ci = sum(x * y for x, y in zip(ar, bi)) + sum(x * y for x, y in zip(ai, br))
+        xr, xi = lift(cr, M), lift(ci, M)
+        Xs.append((xr, xi))
+        sc = int(st["eA"][i]) + int(st["eB"][j])
+        yr, tr = round_int_nearest_even(xr, out_bits)
+        yi, ti = round_int_nearest_even(xi, out_bits)
+        vals[t] = complex(math.ldexp(float(yr), tr + sc), math.ldexp(float(yi), ti + sc))
+    return Xs, vals

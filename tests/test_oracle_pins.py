@@ -1,0 +1,285 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, brute force, library routines.
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a wrong sign, a
+transposed operand, a wrong constant) fails it.  None of these needs a GPU.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import direct, staged
+from paper_2609_05419_b200 import inputs
+from conftest import read_golden
+
+
+@pytest.fixture(scope="module")
+def printed(golden_dir):
+    return read_golden(os.path.join(golden_dir, "moduli_printed.txt"))
+
+
+# ------------------------------------------------------------------ constants
+def test_moduli_match_printed_list(printed):
+    mods = staged.greedy_2m_moduli()
+    assert mods[:14] == printed["m2m_prefix"]
+    assert mods[-2:] == printed["m2m_suffix"]
+    assert len(mods) == 22
+    assert round(math.log2(staged.product(mods[:16])) - 0.5) == printed["m2m_log2_first16"][0]   # 2^117.69
+    assert round(math.log2(staged.product(mods))) == printed["m2m_log2_all"][0]                  # 2^152.08
+    for a in mods:
+        for b in mods:
+            assert a == b or math.gcd(a, b) == 1
+
+
+def test_greedy_reading_reproduces_real_modulus_set(printed):
+    # the same greedy walk without the 2M filter must give the paper's real-Ozaki-II list
+    kept = []
+    for cand in range(256, 1, -1):
+        if all(math.gcd(cand, q) == 1 for q in kept):
+            kept.append(cand)
+    assert kept[:10] == printed["mreal_prefix"]
+    n117 = printed["mreal_count_for_117"][0]
+    assert 117 <= math.log2(staged.product(kept[:n117])) < 118
+    assert round(math.log2(staged.product(kept))) == printed["mreal_log2_all"][0]
+
+
+def test_2m_modulus_criterion_by_brute_force():
+    # Section 2: s with s^2 = -1 (mod m) exists iff m is a product of primes = 1 (mod 4), m odd
+    for m in range(3, 258, 2):
+        exists = any((s * s + 1) % m == 0 for s in range(m))
+        assert exists == staged.is_2m_modulus(m), m
+
+
+def test_roots_two_derivations():
+    for m in staged.greedy_2m_moduli():
+        s = staged.sqrt_minus_one(m)
+        assert (s * s) % m == m - 1
+        assert (2 * staged.inv2(m)) % m == 1
+        # Section 2.1: m = u^2 + v^2 with gcd(u, v) = 1 and s = -u v^-1 (mod m), up to sign / choice of root
+        found = False
+        for u in range(1, 16):
+            v2 = m - u * u
+            v = math.isqrt(v2) if v2 > 0 else 0
+            if v > 0 and v * v == v2 and math.gcd(u, v) == 1:
+                cand = (-u * pow(v, -1, m)) % m
+                assert (cand * cand) % m == m - 1
+                found = found or cand in (s, m - s)
+        assert found, m
+    assert staged.sqrt_minus_one(241) == 64 and (-15 * pow(4, -1, 241)) % 241 == 241 - 64
+
+
+def test_2m_identity_brute_force():
+    # (2c) applied to (2b) of (2a) equals the complex product mod m, for every small Gaussian integer pair
+    rng = range(-3, 4)
+    for m in staged.greedy_2m_moduli():
+        s = staged.sqrt_minus_one(m)
+        for ar in rng:
+            for ai in rng:
+                ap, am = staged.pre_2m(ar, ai, m, s)
+                for br in rng:
+                    for bi in rng:
+                        bp, bm = staged.pre_2m(br, bi, m, s)
+                        cp, cm = staged.sym(ap * bp, m), staged.sym(am * bm, m)
+                        # (2b): C+- = (ArBr - AiBi) +- s (ArBi + AiBr)
+                        assert (cp - ((ar * br - ai * bi) + s * (ar * bi + ai * br))) % m == 0
+                        assert (cm - ((ar * br - ai * bi) - s * (ar * bi + ai * br))) % m == 0
+                        cr, ci = staged.post_2m(cp, cm, m, s)
+                        assert (cr - (ar * br - ai * bi)) % m == 0
+                        assert (ci - (ar * bi + ai * br)) % m == 0
+                        assert abs(cr) <= (m - 1) // 2 and abs(ci) <= (m - 1) // 2
+
+
+def test_2m_hand_example():
+    # m = 241, s = 64, a = 3 + 2i, b = 1 - 4i, ab = 11 - 10i, worked through (2a)-(2c) by hand
+    m, s = 241, 64
+    ap, am = staged.pre_2m(3, 2, m, s)
+    bp, bm = staged.pre_2m(1, -4, m, s)
+    assert (ap % m, am % m, bp % m, bm % m) == (131, 116, 227, 16)
+    cp, cm = (ap * bp) % m, (am * bm) % m
+    assert (cp, cm) == (94, 169)
+    assert staged.inv2(m) == 121
+    assert staged.post_2m(cp, cm, m, s) == (11, -10)
+
+
+def test_crt_roundtrip_known_integers():
+    rng = np.random.default_rng(5)
+    for nmod in (1, 2, 3, 8, 16, 22):
+        mods = staged.greedy_2m_moduli()[:nmod]
+        M = staged.product(mods)
+        h = (M - 1) // 2
+        for x in [0, 1, -1, h, -h, h - 1] + [int(rng.integers(-2 ** 62, 2 ** 62)) % M - h for _ in range(20)]:
+            res = [staged.sym(x, q) for q in mods]
+            assert staged.lift(staged.crt(res, mods), M) == staged.lift(x, M)
+        # one step beyond the range wraps around, as the definition says
+        assert staged.lift(staged.crt([staged.sym(h + 1, q) for q in mods], mods), M) == -h
+
+
+# ------------------------------------------------------------------ O-int
+@pytest.mark.parametrize("shape", [(1, 1, 1), (2, 3, 1), (3, 2, 5), (7, 5, 3), (4, 4, 9)])
+def test_int128_product_vs_python_ints(shape):
+    m, n, k = shape
+    rng = np.random.default_rng(11 + m * n * k)
+    big = 2 ** 55
+    Ar, Ai = rng.integers(-big, big, size=(m, k)), rng.integers(-big, big, size=(m, k))
+    Br, Bi = rng.integers(-big, big, size=(k, n)), rng.integers(-big, big, size=(k, n))
+    cr, ci = direct.gauss4m_exact(Ar, Ai, Br, Bi)
+    pr, pi = direct.gauss4m_python(Ar, Ai, Br, Bi)
+    assert (cr == pr).all() and (ci == pi).all()
+
+
+def test_int128_product_vs_numpy_complex_matmul():
+    # int8-range data: numpy's complex matmul is exact here (all values far below 2^53)
+    Ar, Ai, Br, Bi = inputs.gaussian_int_inputs(33, 17, 70, seed=3)
+    cr, ci = direct.gauss4m_exact(Ar, Ai, Br, Bi)
+    Z = (Ar.astype(np.float64) + 1j * Ai) @ (Br.astype(np.float64) + 1j * Bi)
+    assert (cr.astype(np.float64) == Z.real).all() and (ci.astype(np.float64) == Z.imag).all()
+    # asymmetric shapes catch a transposed operand; the scalar case pins the sign convention i^2 = -1
+    cr1, ci1 = direct.gauss4m_exact([[3]], [[2]], [[1]], [[-4]])
+    assert (int(cr1[0, 0]), int(ci1[0, 0])) == (11, -10)
+
+
+def test_symmetric_residue_definition():
+    M = 241 * 233
+    h = (M - 1) // 2
+    for x in range(-3 * M, 3 * M, 997):
+        r = direct.symmetric_residue(x, M)
+        assert -h <= r <= h and (r - x) % M == 0
+
+
+# ------------------------------------------------------------------ O-fp
+def test_dd_product_vs_exact_rationals():
+    A, B = inputs.complex_inputs(3, 4, 6, seed=2, dist="phi", phi=2.0)
+    C, D = direct.zgemm4m_dd(A, B)
+    for i in range(3):
+        for j in range(4):
+            er = sum(Fraction(A[i, p].real) * Fraction(B[p, j].real) - Fraction(A[i, p].imag) * Fraction(B[p, j].imag) for p in range(6))
+            ei = sum(Fraction(A[i, p].real) * Fraction(B[p, j].imag) + Fraction(A[i, p].imag) * Fraction(B[p, j].real) for p in range(6))
+            d = sum(abs(A[i, p]) * abs(B[p, j]) for p in range(6))
+            # correctly rounded up to the last bit of the larger product (double-double carries 100+ bits)
+            assert abs(Fraction(C[i, j].real) - er) <= Fraction(d) * Fraction(1, 2 ** 52)
+            assert abs(Fraction(C[i, j].imag) - ei) <= Fraction(d) * Fraction(1, 2 ** 52)
+            assert abs(D[i, j] - d) <= 1e-15 * d
+
+
+def test_dd_product_recovers_cancellation():
+    # ar*br - ai*bi with massive cancellation: plain double loses everything, double-double must not
+    a = np.array([[(1 + 2.0 ** -30) + 1j * (1 - 2.0 ** -30)]], order="F")
+    b = np.array([[(1 + 2.0 ** -30) + 1j * (1 + 2.0 ** -30)]], order="F")
+    C, _ = direct.zgemm4m_dd(a, b)
+    exact_r = Fraction(a[0, 0].real) * Fraction(b[0, 0].real) - Fraction(a[0, 0].imag) * Fraction(b[0, 0].imag)
+    assert Fraction(C[0, 0].real) == exact_r        # exactly representable: 2^-29 + 2^-59 ... fits a double
+
+
+def test_dd_product_equals_integer_product_on_integer_data():
+    Ar, Ai, Br, Bi = inputs.gaussian_int_inputs(20, 31, 45, seed=8)
+    A = np.asfortranarray(Ar.astype(np.float64) + 1j * Ai)
+    B = np.asfortranarray(Br.astype(np.float64) + 1j * Bi)
+    C, D = direct.zgemm4m_dd(A, B)
+    cr, ci = direct.gauss4m_exact(Ar, Ai, Br, Bi)
+    assert (C.real == cr.astype(np.float64)).all() and (C.imag == ci.astype(np.float64)).all()
+    assert np.allclose(D, np.abs(A) @ np.abs(B), rtol=1e-13)
+
+
+def test_dd_product_vs_library_matmul_and_samples():
+    A, B = inputs.complex_inputs(40, 23, 64, seed=4)
+    C, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(A @ B, C, D) < 64 * 2.3e-16
+    pairs = inputs.sample_indices(40, 23, 50, seed=1, tile=16)
+    Cs, Ds = direct.zgemm4m_dd_samples(A, B, pairs)
+    assert (Cs == C[pairs[:, 0], pairs[:, 1]]).all() and (Ds == D[pairs[:, 0], pairs[:, 1]]).all()
+
+
+# ------------------------------------------------------------------ staged Algorithm 1
+@pytest.mark.parametrize("nmod", [1, 2, 3, 8])
+def test_staged_integer_path_equals_4m_definition(nmod):
+    # Section 6: the multiplication method (2M vs 4M) cannot change the integer result
+    Ar, Ai, Br, Bi = inputs.gaussian_int_inputs(24, 19, 37, seed=nmod)
+    st = staged.gemm2m_int_staged(Ar, Ai, Br, Bi, nmod)
+    er, ei = direct.gauss4m_mod(Ar, Ai, Br, Bi, st["M"])
+    assert (st["Xr"].astype(np.int64) == er).all() and (st["Xi"].astype(np.int64) == ei).all()
+    if nmod == 3:        # |c| <= 2*37*16^2 < M/2: no wrap, equals the exact product
+        cr, ci = direct.gauss4m_exact(Ar, Ai, Br, Bi)
+        assert (st["Xr"] == cr).all() and (st["Xi"] == ci).all()
+    if nmod == 1:        # M = 241 wraps for sure
+        cr, _ = direct.gauss4m_exact(Ar, Ai, Br, Bi)
+        assert (st["Xr"] != cr).any()
+
+
+def test_scaling_rule_and_truncation_invariants():
+    A, B = inputs.complex_inputs(17, 13, 300, seed=6, dist="phi", phi=2.0)
+    A[3, :] = 0                                   # zero row: exponent 0, quantises to zero
+    for nmod in (3, 7, 16, 22):
+        st = staged.zgemm2m_staged(A, B, nmod, upto="pre")
+        assert st["eA"][3] == 0
+        for (qr, qi), e, Z, axis, P in ((st["Aq"], st["eA"], A, 1, st["PA"]), (st["Bq"], st["eB"], B, 0, st["PB"])):
+            eb = e[:, None] if axis == 1 else e[None, :]
+            for q, part in ((qr, Z.real), (qi, Z.imag)):
+                for idx in np.ndindex(q.shape):
+                    exact = Fraction(float(part[idx])) / Fraction(2) ** int(np.broadcast_to(eb, q.shape)[idx])
+                    assert abs(q[idx]) <= abs(exact) < abs(q[idx]) + 1        # truncation toward zero
+                    assert (q[idx] >= 0) == (exact >= 0) or q[idx] == 0
+            # the row/column 2-norm bound that makes |X| <= 2^Pt
+            sq = (qr.astype(object) ** 2 + qi.astype(object) ** 2).sum(axis=axis)
+            assert all(int(v) <= 4 ** P for v in sq)
+        assert st["PA"] + st["PB"] == st["Pt"] and 2 ** st["Pt"] <= (st["M"] - 1) // 2 < 2 ** (st["Pt"] + 1)
+
+
+@pytest.mark.parametrize("nmod", [14, 16, 22])
+def test_staged_float_path_meets_error_bound_and_equals_4m_on_quantised(nmod):
+    A, B = inputs.complex_inputs(12, 9, 100, seed=9, dist="phi", phi=0.5)
+    st = staged.zgemm2m_staged(A, B, nmod)
+    assert all(abs(int(v)) <= 2 ** st["Pt"] for v in st["Xr"].ravel())
+    assert all(abs(int(v)) <= 2 ** st["Pt"] for v in st["Xi"].ravel())
+    # the 2M route reproduces the plain integer product of the quantised matrices (no wrap by the bound)
+    pairs = np.array([(i, j) for i in range(12) for j in range(9)])
+    Xs, vals = staged.staged_samples(st, pairs)
+    assert all(int(st["Xr"][i, j]) == xr and int(st["Xi"][i, j]) == xi for (i, j), (xr, xi) in zip(pairs.tolist(), Xs))
+    assert (vals == st["C"][pairs[:, 0], pairs[:, 1]]).all()
+    Cref, D = direct.zgemm4m_dd(A, B)
+    err = direct.componentwise_error(st["C"], Cref, D)
+    assert err <= (1e-13 if nmod == 14 else 1e-14)
+
+
+def test_staged_error_falls_with_modulus_count():
+    # Section 3.1: error ~ O(M^-1/2): each extra modulus (~2^7.5) buys about 2^3.7 until the rounding floor
+    A, B = inputs.complex_inputs(10, 8, 64, seed=12)
+    Cref, D = direct.zgemm4m_dd(A, B)
+    errs = [direct.componentwise_error(staged.zgemm2m_staged(A, B, n)["C"], Cref, D) for n in (6, 8, 10, 12)]
+    assert all(a > 20 * b for a, b in zip(errs, errs[1:])), errs
+    M6, M12 = (staged.product(staged.greedy_2m_moduli()[:n]) for n in (6, 12))
+    ratio = math.log2(errs[0] / errs[-1]) / math.log2(M12 / M6)
+    assert 0.4 < ratio < 0.6, ratio
+
+
+def test_staged_complex64_rounding():
+    A, B = inputs.complex_inputs(9, 7, 50, seed=13, dtype=np.complex64)
+    st = staged.zgemm2m_staged(A, B, 7, out_bits=24)
+    C32 = st["C"].astype(np.complex64)
+    assert (C32.astype(np.complex128) == st["C"]).all()          # already on the float32 grid
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(C32, Cref, D) <= 2e-6
+
+
+def test_round_int_nearest_even_vs_python_float():
+    rng = np.random.default_rng(3)
+    xs = [int(rng.integers(-2 ** 62, 2 ** 62)) * int(rng.integers(1, 2 ** 60)) + int(rng.integers(-5, 5)) for _ in range(300)]
+    xs += [2 ** 53 + 1, 2 ** 53 + 2, 2 ** 53 + 3, -(2 ** 54 + 2), 3 * 2 ** 52 + 0, (2 ** 53 - 1) * 2 ** 40 + 2 ** 39]
+    for x in xs:
+        y, t = staged.round_int_nearest_even(x, 53)
+        assert math.ldexp(float(y), t) == float(x)               # Python's int -> float is round-half-even
+
+
+def test_herk_symmetry_and_equivalence():
+    A = inputs.herk_input(11, 40, seed=14)
+    B = np.asfortranarray(A.conj().T)
+    st = staged.zgemm2m_staged(A, B, 16, herk=True)
+    assert st["Pt"] % 2 == 0
+    for (Ap, Am), (Bp, Bm), (Cp, Cm) in zip(st["Apm"], st["Bpm"], st["Cpm"]):
+        assert (Bp == Am.T).all() and (Bm == Ap.T).all()         # residues of A^H are the swapped planes, transposed
+        assert (Cm == Cp.T).all()                                # Section 5: C- = C+^T
+    assert (st["Xr"] == st["Xr"].T).all() and (st["Xi"] == -st["Xi"].T).all()
+    assert all(int(v) == 0 for v in np.diag(st["Xi"]))
+    st2 = staged.zgemm2m_staged(A, B, 16, herk=False)            # Pt even: same scaling, identical integers
+    assert (st2["Xr"] == st["Xr"]).all() and (st2["Xi"] == st["Xi"]).all()
