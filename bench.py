@@ -1,0 +1,297 @@
+"""Benchmark of the zgemm2m hot path (2M multiplication + Ozaki-II) on B200.
+
+One step = one zgemm2m call (exponent scan, quantise + residues, 2N int8 GEMMs, post-processing) on a synthetic
+complex128 problem.  Prints ONE JSON line (rank 0).  See --help for the workload knobs; the defaults are the
+headline configuration: m = n = k = 8192, 16 moduli, inputs (rand-0.5)*exp(0.5*randn).
+
+  python bench.py                          # this library, 1 GPU
+  python bench.py --impl reference         # the CPU oracle timed on the host cores (a baseline, not a target)
+  torchrun ... bench.py --gpus N           # N independent replicas (the path is single-GPU; no collective)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "zgemm2m_effective_tflops_8mnk_per_t"
+UNIT = "TFLOP/s"
+INT8_NOMINAL_TOPS = 4500.0          # dense int8, nominal
+INT8_OVER_BF16 = 2.0                # nominal ratio used to turn the measured bf16 peak into an int8 peak
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--m", type=int, default=8192)
+    ap.add_argument("--n", type=int, default=8192)
+    ap.add_argument("--k", type=int, default=8192)
+    ap.add_argument("--nmod", type=int, default=16)
+    ap.add_argument("--phi", type=float, default=0.5)
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(a):
+    return f"zgemm2m complex128 m={a.m} n={a.n} k={a.k} nmod={a.nmod} parts=(rand-0.5)*exp({a.phi}*randn)"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_burst=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle leg
+def time_oracle(a, A, B, seconds):
+    """Times the double-double 4M oracle, as it stands, on a bounded sample of entries of the same product."""
+    from oracle import direct
+    from paper_2609_05419_b200 import inputs
+    cores = direct.num_threads()
+    probe = inputs.sample_indices(a.m, a.n, 2048, seed=11)
+    t0 = time.perf_counter()
+    direct.zgemm4m_dd_samples(A, B, probe)
+    t_probe = max(time.perf_counter() - t0, 1e-6)
+    count = int(min(max(len(probe), len(probe) * seconds / t_probe), a.m * a.n))
+    pairs = inputs.sample_indices(a.m, a.n, count, seed=12)
+    t0 = time.perf_counter()
+    direct.zgemm4m_dd_samples(A, B, pairs)
+    dt = time.perf_counter() - t0
+    flops = 8.0 * a.k * len(pairs)
+    return dict(value=flops / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{len(pairs)} sampled entries of the {a.m}x{a.n}x{a.k} product (double-double 4M, {dt:.1f} s)"), dt
+
+
+def run_reference(a):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_05419_b200 import inputs
+    A, B = inputs.complex_inputs(a.m, a.n, a.k, a.seed, dist="phi", phi=a.phi)
+    per_step = max(2.0, min(a.cpu_seconds, 120.0 / max(a.steps + a.warmup, 1)))
+    for _ in range(a.warmup):
+        time_oracle(a, A, B, per_step)
+    vals, times = [], []
+    last = None
+    for _ in range(a.steps):
+        last, dt = time_oracle(a, A, B, per_step)
+        vals.append(last["value"])
+        times.append(dt)
+    value = float(np.mean(vals))
+    last["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": a.gpus, "steps": a.steps,
+            "warmup": a.warmup, "ms_per_step": float(np.mean(times)) * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(a), "note": "CPU oracle on host cores; each step is a bounded sample of entries"},
+            "cpu_baseline": last,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------- GPU leg
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                    power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        load = [s for s, p in zip(sm, power) if p > 0.5 * max(power)] or sm
+        return {"sm_mhz": float(np.median(load)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "power_w_max": float(max(power)), "samples": len(sm)}
+
+
+def run_ours(a):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_05419_b200 import binding as b
+    from paper_2609_05419_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    b.lib()   # fails loudly if the CUDA library is missing
+    m, n, k, nmod = a.m, a.n, a.k, a.nmod
+    A, B = inputs.complex_inputs(m, n, k, a.seed + rank, dist="phi", phi=a.phi)     # every replica its own problem
+    # pinned host buffers in column-major order (the transposed view is what the C ABI sees)
+    hA = torch.from_numpy(np.ascontiguousarray(A.T)).pin_memory()
+    hB = torch.from_numpy(np.ascontiguousarray(B.T)).pin_memory()
+    hC = torch.empty((n, m), dtype=torch.complex128).pin_memory()
+    dA, dB = hA.cuda(), hB.cuda()
+    dC = torch.empty((n, m), dtype=torch.complex128, device="cuda")
+    ws = torch.zeros(b.workspace_bytes(b.OP_ZGEMM, m, n, k, nmod), dtype=torch.uint8, device="cuda")
+    b.set_workspace(ws)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        b.zgemm2m(dA.t(), dB.t(), dC.t(), nmod, stream)
+
+    def step_e2e():
+        dA.copy_(hA, non_blocking=True)
+        dB.copy_(hB, non_blocking=True)
+        b.zgemm2m(dA.t(), dB.t(), dC.t(), nmod, stream)
+        hC.copy_(dC, non_blocking=True)
+
+    for _ in range(max(a.warmup, 3)):
+        step()
+    b.device_status()
+
+    # ---- timed region: device-resident inputs, phase events recorded on the same stream
+    sampler = ClockSampler(local)
+    b.set_profiling(True)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(a.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    phase, calls = b.phase_ms()
+    b.set_profiling(False)
+    b.device_status()
+    launches_per_step, per_phase = b.last_launch_count()
+
+    # ---- end to end: pinned host -> device, call, device -> host, every step
+    e2e = None
+    if not a.no_e2e:
+        for _ in range(2):
+            step_e2e()
+        barrier()
+        e0.record(stream)
+        for _ in range(a.steps):
+            step_e2e()
+        e1.record(stream)
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+        e2e = {"value": 8.0 * m * n * k * world * a.steps / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": int(hA.numel() * 16 + hB.numel() * 16), "d2h_bytes_per_step": int(hC.numel() * 16),
+               "ms_per_step": ms_e2e / a.steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ms_step = ms_total / a.steps
+    value = 8.0 * m * n * k * world / (ms_step * 1e-3) / 1e12
+    gemm_ops = 2.0 * (2 * nmod) * m * n * k            # int8 multiply-adds x2, all 2N real GEMMs = one launch
+    gemm_tops = gemm_ops / (phase[2] * 1e-3) / 1e12
+    int8_peak = INT8_OVER_BF16 * peaks["bf16_sustained"]
+    pre_bytes = (m * k + k * n) * (16 + 2 * nmod)       # quantise read + residue planes written
+    scan_bytes = (m * k + k * n) * 16
+    post_bytes = m * n * (2 * nmod + 16)
+    roofline = {"bound": "tensor", "kernel": "gemm_i8_tcgen05_kernel", "achieved": gemm_tops, "peak": int8_peak, "unit": "TFLOP/s",
+                "frac": gemm_tops / int8_peak, "traffic": None,
+                "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate (int8:bf16 nominal ratio); int8 ops counted as 2 per MAC",
+                "frac_of_nominal_4500": gemm_tops / INT8_NOMINAL_TOPS,
+                "launch_ms": phase[2], "algorithmic_ops_per_launch": gemm_ops}
+    phases = {"scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3], "calls_averaged": calls,
+              "scan_gbs": scan_bytes / (phase[0] * 1e-3) / 1e9 if phase[0] > 0 else None,
+              "residues_gbs": pre_bytes / (phase[1] * 1e-3) / 1e9 if phase[1] > 0 else None,
+              "post_gbs": post_bytes / (phase[3] * 1e-3) / 1e9 if phase[3] > 0 else None,
+              "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]}
+    cpu = None
+    if not a.no_cpu_baseline:
+        cpu, _ = time_oracle(a, A, B, a.cpu_seconds)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(a.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+            "data": "synthetic",
+            "config": {"workload": workload_name(a), "l2": "inputs (2 x %.2f GiB) and residue planes exceed the 126 MB L2" % (m * k * 16 / 2**30),
+                       "multi_gpu": "replicas only (no collective on the path)"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * a.steps, "launches_per_step": per_phase,
+            "roofline": roofline, "phases": phases, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    b.set_workspace(None)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
+
+
+if __name__ == "__main__":
+    main()

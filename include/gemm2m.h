@@ -1,0 +1,137 @@
+/*
+ * gemm2m -- complex matrix multiplication by 2M multiplication + the Ozaki-II scheme, for NVIDIA B200 (sm_100a).
+ *
+ * Complex GEMM with only two real int8 GEMMs per modulus:
+ *   1. per-row (A) / per-column (B) power-of-two scale factors, entries truncated to Gaussian integers
+ *      (Algorithm 1 steps 2-3; Section 3.1 for the real scheme);
+ *   2. for each 2M modulus m_j (odd, s_j^2 = -1 mod m_j; Section 2, set of Section 4) the residues
+ *      A+- = A_r +- s_j A_i, B+- = B_r +- s_j B_i (mod m_j), Eq. (2a), kept as symmetric int8;
+ *   3. the two real products C+- = A+- B+- (mod m_j), Eq. (2b), on the int8 tensor cores;
+ *   4. C = 2^-1 (C- + C+) + i s_j 2^-1 (C- - C+) (mod m_j), Eq. (2c); CRT over j (Section 3.1; Algorithm 1
+ *      step 5); lift to the symmetric range (step 6); multiply by sigma_i tau_j (step 7).
+ *
+ * Conventions for every entry point
+ *   - BLAS-3 style as in the paper's problem statement (Section 1: A in C^{m x k}, B in C^{k x n}; Section 6:
+ *     alpha = 1, beta = 0): column-major, complex numbers interleaved (re, im), leading dimensions counted in
+ *     elements (complex elements for complex matrices), no transposition arguments, C is overwritten.
+ *   - All matrix pointers are DEVICE pointers owned by the caller.  The library never allocates or frees device
+ *     memory inside a call; it uses the caller-provided workspace registered with gemm2m_set_workspace().
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and
+ *     return immediately.  The return value is a gemm2m_status; it is the only error channel.
+ *   - Argument errors are detected on the host before anything is launched.  m, n or k equal to 0 is valid:
+ *     nothing is computed for m = 0 or n = 0, and C is set to zero for k = 0.
+ *   - `nmod` selects the first nmod moduli of the set of Section 4 (241, 233, 229, 221, 205, ... , 37, 29; 22 in
+ *     all).  More moduli = larger M = more accuracy and proportionally more work.  16 gives about double
+ *     precision accuracy for zgemm2m/zherk2m, 7 about single precision for cgemm2m.
+ *   - One call at a time per workspace: calls that share a workspace must be ordered on the GPU (same stream).
+ *   - Non-finite inputs: a row of A (column of B) that contains an Inf or NaN yields NaN in the whole
+ *     corresponding row (column) of C; no error is reported.
+ */
+#ifndef GEMM2M_H
+#define GEMM2M_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GEMM2M_OK = 0,
+    GEMM2M_ERR_ARG = 1,            /* negative size, leading dimension too small, null pointer with non-empty matrix */
+    GEMM2M_ERR_NMOD = 2,           /* nmod outside [1, 22], or > 8 for the int64 result of gemm2m_gaussian_int */
+    GEMM2M_ERR_WORKSPACE = 3,      /* no workspace registered or too small; nothing was launched */
+    GEMM2M_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (see gemm2m_last_cuda_error) */
+    GEMM2M_ERR_ARCH = 5,           /* current device is not compute capability 10.0 */
+    GEMM2M_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait gave up (reported by gemm2m_device_status) */
+} gemm2m_status;
+
+typedef enum { GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3 } gemm2m_op;
+
+/* Human-readable name of a status code (static string). */
+const char* gemm2m_status_string(int status);
+/* Text of the last CUDA error seen by this thread's calls (static/thread-local string, never NULL). */
+const char* gemm2m_last_cuda_error(void);
+
+/* Number of 2M moduli available (22): the greedy coprime set in [1, 256] of Section 4. */
+int gemm2m_max_moduli(void);
+/* j-th modulus (0-based, descending) and its smallest positive square root of -1 (Section 2).  Host pointers. */
+int gemm2m_modulus(int j, int* m, int* s);
+
+/* Bytes of device workspace a call of `op` with these sizes needs (for zherk2m pass m = n).  0 on bad arguments. */
+size_t gemm2m_workspace_bytes(int op, int64_t m, int64_t n, int64_t k, int nmod);
+/* Register a caller-owned device buffer (256-byte aligned) used by later calls of this host thread's current
+ * device.  Passing (NULL, 0) unregisters.  The buffer must stay valid until the last call using it has finished. */
+int gemm2m_set_workspace(void* dev_ptr, size_t bytes);
+
+/* Gaussian-integer product by 2M multiplication (Section 2, Eq. (2a)-(2c)) and CRT over nmod <= 8 moduli.
+ * Ar, Ai: m x k int8 (lda >= m); Br, Bi: k x n int8 (ldb >= k); Cr, Ci: m x n int64 (ldc >= m), overwritten with
+ * the representative of the exact product modulo M = m_1 ... m_nmod in [-(M-1)/2, (M-1)/2] -- the exact product
+ * itself whenever 2 max|c| < M (first paragraph of Section 2). */
+int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k,
+                        const int8_t* Ar, const int8_t* Ai, int64_t lda,
+                        const int8_t* Br, const int8_t* Bi, int64_t ldb,
+                        int64_t* Cr, int64_t* Ci, int64_t ldc, int nmod, void* stream);
+
+/* C = A B in complex double precision by Algorithm 1 ("2M Ozaki-II").  A: m x k, B: k x n, C: m x n, interleaved
+ * complex128, lda >= m, ldb >= k, ldc >= m. */
+int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb,
+            double* C, int64_t ldc, int nmod, void* stream);
+
+/* The same for complex single precision (interleaved complex64). */
+int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb,
+            float* C, int64_t ldc, int nmod, void* stream);
+
+/* Hermitian rank-k update C = A A^H (Section 5, HERK) with ONE real int8 GEMM per modulus: C+ = A+ A-^T and
+ * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
+ * diagonal is written; diagonal imaginary parts are exactly 0; the strict upper triangle is not touched. */
+int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream);
+
+/* Waits for `stream` and returns GEMM2M_ERR_DEVICE_TIMEOUT if a kernel of an earlier call on the registered
+ * workspace gave up a bounded wait (its results are then invalid), GEMM2M_ERR_CUDA on a CUDA error, else OK. */
+int gemm2m_device_status(void* stream);
+
+/* ---- instrumentation (used by the tests and the benchmark; not needed for normal use) ---- */
+
+/* Phase timing: when enabled, every call records CUDA events around its phases on the call's stream (up to the 64 most
+ * recent calls are kept).  Switching it on or off forgets earlier records. */
+int gemm2m_set_profiling(int enabled);
+/* Waits for the recorded calls and returns the average milliseconds per call of each phase: ms[0] = exponent scan,
+ * ms[1] = quantise + residues (Eq. 2a), ms[2] = int8 GEMMs (Eq. 2b), ms[3] = post-processing (Eq. 2c + CRT + unscale);
+ * *calls = number of calls averaged.  Host pointers; GEMM2M_ERR_ARG if nothing was recorded. */
+int gemm2m_phase_ms(float ms[4], int* calls);
+/* Number of kernels the last call launched (per phase in the same order, host pointer, may be NULL); returns total. */
+int gemm2m_last_launch_count(int per_phase[4]);
+
+/* Where the intermediate stages of a call live inside the workspace (byte offsets from its start), so that tests
+ * can compare each stage with the CPU oracle.  Planes are indexed p = sign * nmod + j with sign 0 for "+", 1 for "-". */
+typedef struct {
+    int64_t off_exp_a;     /* int32[m]: scale exponents e_i, sigma_i = 2^e_i (rows of A)                 */
+    int64_t off_exp_b;     /* int32[n]: scale exponents f_j, tau_j = 2^f_j (columns of B); HERK: unused  */
+    int64_t off_apm;       /* int8 [2 nmod][m][kp]: residues of A, K contiguous                           */
+    int64_t off_bpm;       /* int8 [2 nmod][n][kp]: residues of B, K contiguous; HERK: unused             */
+    int64_t off_cpm;       /* int8 [2 nmod][n][ldp]: C+- mod m_j, M contiguous; HERK: [nmod][n][ldp], C+ only */
+    int64_t kp;            /* padded K (multiple of 128; padding is zero)                                  */
+    int64_t ldp;           /* leading dimension of the C+- planes (multiple of 16)                         */
+    int64_t total_bytes;
+} gemm2m_layout;
+int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, gemm2m_layout* out);
+
+/* Which int8 GEMM kernel later calls use: 0 = the tcgen05 kernel (default), 1 = a plain CUDA-core check kernel kept
+ * only so that tests can tell a fault in the tensor-core kernel from one in the pre/post kernels. */
+int gemm2m_debug_set_gemm_kernel(int which);
+
+/* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host
+ * pointers, any may be NULL), so that CPU tests can check them against an independent computation:
+ *   scale[4]        = P_t, P_A, P_B, c_k of the scaling rule (herk != 0: P_A = P_B)
+ *   crt_gr/gi[nmod*4] = signed base-2^40 digits of the folded CRT weights (real / imaginary part), crt_m[4] = digits of M
+ *   nchunks         = number of digits in use
+ *   res_w[nmod*16]  = int8 byte weights of the residue kernels: 8 for the real part, then 8 for the imaginary part */
+int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,
+                        int8_t* res_w);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GEMM2M_H */

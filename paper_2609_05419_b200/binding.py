@@ -1,0 +1,201 @@
+"""Thin ctypes binding of the gemm2m C-ABI library (include/gemm2m.h): same entry-point names, argument
+marshalling only.  Matrices are torch CUDA tensors viewed column-major (stride 1 along the first dimension);
+torch is used for device memory and streams, every step of the computation runs in the library's kernels.
+
+There is no fallback: if libgemm2m.so has not been built (``python -m paper_2609_05419_b200.build``) or cannot
+be loaded, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK = 0, 1, 2, 3
+OK = 0
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgemm2m.so")
+_lib = None
+
+
+class Gemm2mError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        name = lib().gemm2m_status_string(status).decode()
+        extra = ""
+        if name == "GEMM2M_ERR_CUDA":
+            extra = " (" + lib().gemm2m_last_cuda_error().decode() + ")"
+        super().__init__(f"{where}: {name}{extra}")
+
+
+class Layout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in
+                ("off_exp_a", "off_exp_b", "off_apm", "off_bpm", "off_cpm", "kp", "ldp", "total_bytes")]
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it is missing: there is no CPU or library fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_05419_b200.build` (needs nvcc)")
+    L = ctypes.CDLL(LIB_PATH)
+    i64, i32, vp, sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
+    L.gemm2m_status_string.restype = ctypes.c_char_p
+    L.gemm2m_status_string.argtypes = [i32]
+    L.gemm2m_last_cuda_error.restype = ctypes.c_char_p
+    L.gemm2m_max_moduli.restype = i32
+    L.gemm2m_modulus.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.gemm2m_workspace_bytes.restype = sz
+    L.gemm2m_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
+    L.gemm2m_set_workspace.argtypes = [vp, sz]
+    L.gemm2m_gaussian_int.argtypes = [i64, i64, i64, vp, vp, i64, vp, vp, i64, vp, vp, i64, i32, vp]
+    L.zgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.cgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.zherk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
+    L.gemm2m_device_status.argtypes = [vp]
+    L.gemm2m_set_profiling.argtypes = [i32]
+    L.gemm2m_phase_ms.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    L.gemm2m_last_launch_count.argtypes = [ctypes.POINTER(i32)]
+    L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
+    L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
+    L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
+    _lib = L
+    return L
+
+
+def _check(status, where):
+    if status != OK:
+        raise Gemm2mError(status, where)
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _colmajor(t, name):
+    """(pointer, rows, cols, leading dimension) of a 2-D CUDA tensor stored column-major."""
+    if t.dim() != 2 or not t.is_cuda:
+        raise ValueError(f"{name}: need a 2-D CUDA tensor")
+    rows, cols = t.shape
+    if rows > 1 and t.stride(0) != 1:
+        raise ValueError(f"{name}: need column-major storage (stride 1 along dim 0), e.g. torch.empty(cols, rows).t()")
+    ld = t.stride(1) if cols > 1 else max(rows, 1)
+    return ctypes.c_void_p(t.data_ptr()), rows, cols, max(ld, 1)
+
+
+def max_moduli():
+    return int(lib().gemm2m_max_moduli())
+
+
+def modulus(j):
+    m, s = ctypes.c_int(), ctypes.c_int()
+    _check(lib().gemm2m_modulus(j, ctypes.byref(m), ctypes.byref(s)), "gemm2m_modulus")
+    return m.value, s.value
+
+
+def workspace_bytes(op, m, n, k, nmod):
+    return int(lib().gemm2m_workspace_bytes(op, m, n, k, nmod))
+
+
+def workspace_layout(op, m, n, k, nmod):
+    lay = Layout()
+    _check(lib().gemm2m_workspace_layout(op, m, n, k, nmod, ctypes.byref(lay)), "gemm2m_workspace_layout")
+    return {name: getattr(lay, name) for name, _ in Layout._fields_}
+
+
+def set_workspace(tensor):
+    """Register a torch uint8 CUDA tensor (kept alive by the caller) as the library's workspace; None unregisters."""
+    if tensor is None:
+        _check(lib().gemm2m_set_workspace(None, 0), "gemm2m_set_workspace")
+    else:
+        _check(lib().gemm2m_set_workspace(ctypes.c_void_p(tensor.data_ptr()), tensor.numel() * tensor.element_size()),
+               "gemm2m_set_workspace")
+
+
+def gemm2m_gaussian_int(Ar, Ai, Br, Bi, Cr, Ci, nmod, stream=None):
+    pa, m, k, lda = _colmajor(Ar, "Ar")
+    pai, _, _, ldai = _colmajor(Ai, "Ai")
+    pb, k2, n, ldb = _colmajor(Br, "Br")
+    pbi, _, _, ldbi = _colmajor(Bi, "Bi")
+    pc, _, _, ldc = _colmajor(Cr, "Cr")
+    pci, _, _, ldci = _colmajor(Ci, "Ci")
+    if k != k2 or Ai.shape != Ar.shape or Bi.shape != Br.shape or Cr.shape != (m, n) or Ci.shape != (m, n):
+        raise ValueError("shape mismatch")
+    if (lda, ldb, ldc) != (ldai, ldbi, ldci):
+        raise ValueError("real and imaginary planes must share their leading dimension")
+    _check(lib().gemm2m_gaussian_int(m, n, k, pa, pai, lda, pb, pbi, ldb, pc, pci, ldc, nmod, _stream_ptr(stream)),
+           "gemm2m_gaussian_int")
+
+
+def _xgemm(fn, name, A, B, C, nmod, stream):
+    pa, m, k, lda = _colmajor(A, "A")
+    pb, k2, n, ldb = _colmajor(B, "B")
+    pc, mc, nc, ldc = _colmajor(C, "C")
+    if k != k2 or (mc, nc) != (m, n):
+        raise ValueError("shape mismatch")
+    _check(fn(m, n, k, pa, lda, pb, ldb, pc, ldc, nmod, _stream_ptr(stream)), name)
+
+
+def zgemm2m(A, B, C, nmod=16, stream=None):
+    _xgemm(lib().zgemm2m, "zgemm2m", A, B, C, nmod, stream)
+
+
+def cgemm2m(A, B, C, nmod=7, stream=None):
+    _xgemm(lib().cgemm2m, "cgemm2m", A, B, C, nmod, stream)
+
+
+def zherk2m(A, C, nmod=16, stream=None):
+    pa, n, k, lda = _colmajor(A, "A")
+    pc, n1, n2, ldc = _colmajor(C, "C")
+    if (n1, n2) != (n, n):
+        raise ValueError("shape mismatch")
+    _check(lib().zherk2m(n, k, pa, lda, pc, ldc, nmod, _stream_ptr(stream)), "zherk2m")
+
+
+def device_status(stream=None):
+    _check(lib().gemm2m_device_status(_stream_ptr(stream)), "gemm2m_device_status")
+
+
+def set_profiling(enabled):
+    _check(lib().gemm2m_set_profiling(1 if enabled else 0), "gemm2m_set_profiling")
+
+
+def phase_ms():
+    """Average per-call milliseconds of (scan, residues, GEMMs, post) over the profiled calls, and their number."""
+    ms = (ctypes.c_float * 4)()
+    calls = ctypes.c_int()
+    _check(lib().gemm2m_phase_ms(ms, ctypes.byref(calls)), "gemm2m_phase_ms")
+    return [float(x) for x in ms], calls.value
+
+
+def last_launch_count():
+    per = (ctypes.c_int * 4)()
+    total = int(lib().gemm2m_last_launch_count(per))
+    return total, [int(x) for x in per]
+
+
+def debug_set_gemm_kernel(which):
+    _check(lib().gemm2m_debug_set_gemm_kernel(which), "gemm2m_debug_set_gemm_kernel")
+
+
+def debug_tables(nmod, k, herk=False):
+    """Host-side constants of the library for `nmod` moduli (see gemm2m_debug_tables)."""
+    import numpy as np
+    scale = np.zeros(4, dtype=np.int32)
+    gr = np.zeros((nmod, 4), dtype=np.float64)
+    gi = np.zeros((nmod, 4), dtype=np.float64)
+    mc = np.zeros(4, dtype=np.float64)
+    nch = np.zeros(1, dtype=np.int32)
+    w = np.zeros((nmod, 16), dtype=np.int8)
+    ptr = lambda a: ctypes.c_void_p(a.ctypes.data)
+    _check(lib().gemm2m_debug_tables(nmod, k, 1 if herk else 0, ptr(scale), ptr(gr), ptr(gi), ptr(mc), ptr(nch), ptr(w)),
+           "gemm2m_debug_tables")
+    return dict(Pt=int(scale[0]), PA=int(scale[1]), PB=int(scale[2]), ck=int(scale[3]), gr=gr, gi=gi, Mc=mc,
+                nchunks=int(nch[0]), res_w=w)

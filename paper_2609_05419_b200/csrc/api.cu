@@ -1,0 +1,437 @@
+// C-ABI entry points of the gemm2m library (declared in include/gemm2m.h): argument checks, workspace
+// carving and the launch sequence of Algorithm 1.  Host code only enqueues; nothing here allocates device memory.
+#include "../../include/gemm2m.h"
+
+#include "common.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+using namespace gemm2m;
+
+namespace {
+
+struct State {
+    std::mutex mu;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    int profiling = 0;
+    static constexpr int kProfSlots = 64;
+    cudaEvent_t ev[kProfSlots][5] = {};
+    int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
+    cudaEvent_t* cur = nullptr;   // event set of the call being enqueued
+    int launches[4] = {0, 0, 0, 0};
+    int gemm_kernel = 0;          // 0 = tcgen05, 1 = check kernel
+    int sm_count = 0;
+    int arch_ok = -1;
+};
+State g;
+thread_local char g_cuda_err[256] = "no error";
+
+int cuda_fail(cudaError_t e) {
+    std::snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return GEMM2M_ERR_CUDA;
+}
+#define CK(expr)                                       \
+    do {                                               \
+        cudaError_t _e = (expr);                       \
+        if (_e != cudaSuccess) return cuda_fail(_e);   \
+    } while (0)
+
+inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+int check_device() {
+    if (g.arch_ok < 0) {
+        int dev = 0;
+        cudaDeviceProp prop;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return GEMM2M_ERR_CUDA;
+        g.arch_ok = (prop.major == 10 && prop.minor == 0) ? 1 : 0;
+        g.sm_count = prop.multiProcessorCount;
+    }
+    return g.arch_ok ? GEMM2M_OK : GEMM2M_ERR_ARCH;
+}
+
+// Workspace: [status 256 B][absmax A u64][absmax B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each 256-byte aligned.
+struct Carve {
+    int64_t off_status, off_abs_a, off_abs_b, off_exp_a, off_exp_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
+};
+
+bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
+    if (m < 0 || n < 0 || k < 0 || nmod < 1 || nmod > kMaxMod) return false;
+    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_ZHERK) return false;
+    const bool herk = op == GEMM2M_OP_ZHERK;
+    if (herk) m = n;
+    const int64_t kp = round_up(k > 0 ? k : 1, 128), ldp = round_up(m > 0 ? m : 1, 16);
+    int64_t off = 0;
+    auto take = [&](int64_t bytes) { int64_t o = off; off = round_up(off + bytes, 256); return o; };
+    c->off_status = take(256);
+    c->off_abs_a = take(8 * m);
+    c->off_abs_b = take(herk ? 0 : 8 * n);
+    c->off_exp_a = take(4 * m);
+    c->off_exp_b = take(herk ? 0 : 4 * n);
+    c->off_apm = take(2 * (int64_t)nmod * m * kp);
+    c->off_bpm = take(herk ? 0 : 2 * (int64_t)nmod * n * kp);
+    c->off_cpm = take((herk ? 1 : 2) * (int64_t)nmod * n * ldp);
+    c->kp = kp;
+    c->ldp = ldp;
+    c->total = off;
+    return true;
+}
+
+struct Phases {   // event bookkeeping of one call
+    cudaStream_t st;
+    bool on;
+    int idx = 0;
+    cudaError_t mark() {
+        if (!on) return cudaSuccess;
+        return cudaEventRecord(g.cur[idx++], st);
+    }
+    void done() { if (on) ++g.prof_calls; }
+};
+
+int begin_call(cudaStream_t st, Phases* ph) {
+    ph->st = st;
+    ph->on = g.profiling != 0;
+    std::memset(g.launches, 0, sizeof(g.launches));
+    if (ph->on) {
+        g.cur = g.ev[g.prof_calls % State::kProfSlots];
+        for (int i = 0; i < 5; ++i)
+            if (!g.cur[i]) CK(cudaEventCreate(&g.cur[i]));
+        CK(ph->mark());
+    }
+    return GEMM2M_OK;
+}
+
+constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kernels
+
+int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
+    const int64_t klim = gemm_k_limit(nmod);
+    if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
+    else CK(launch_gemm_tcgen05(a, klim, g.sm_count, st, &g.launches[2]));
+    return GEMM2M_OK;
+}
+
+template <typename T>
+int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, const T* B, int64_t ldb, T* C, int64_t ldc, int nmod,
+            void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
+    if (lda < (m > 1 ? m : 1) || ldb < (k > 1 ? k : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
+    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
+    if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
+    if (m == 0 || n == 0) return GEMM2M_OK;
+    if (!C || (k > 0 && (!A || !B))) return GEMM2M_ERR_ARG;
+    if (int s = check_device()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (k == 0) {
+        CK(cudaMemset2DAsync(C, (size_t)ldc * 2 * sizeof(T), 0, (size_t)m * 2 * sizeof(T), (size_t)n, st));
+        return GEMM2M_OK;
+    }
+    Carve c;
+    if (!carve(op, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)g.ws;
+    int* dev_status = (int*)(ws + c.off_status);
+    uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
+    uint64_t* absB = (uint64_t*)(ws + c.off_abs_b);
+    int32_t* eA = (int32_t*)(ws + c.off_exp_a);
+    int32_t* eB = (int32_t*)(ws + c.off_exp_b);
+    int8_t* apm = (int8_t*)(ws + c.off_apm);
+    int8_t* bpm = (int8_t*)(ws + c.off_bpm);
+    int8_t* cpm = (int8_t*)(ws + c.off_cpm);
+
+    const ScaleTargets sc = scale_targets(nmod, k, false);
+    ResidueTable rtab;
+    build_residue_table(nmod, &rtab);
+    CrtTable ctab;
+    build_crt_table(nmod, &ctab);
+    const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
+
+    Phases ph;
+    if (int s = begin_call(st, &ph)) return s;
+    // step 2: scale factors
+    CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
+    CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
+    CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
+    CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
+    CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
+    CK(ph.mark());
+    // step 3 + Eq. (2a)
+    CK(launch_residues_fp<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
+    CK(launch_residues_fp<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
+    CK(ph.mark());
+    // Eq. (2b): 2 nmod real int8 GEMMs; TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm)
+    GemmArgs ga;
+    ga.rowop = bpm; ga.colop = apm;
+    ga.R = n; ga.Cn = m; ga.Kp = c.kp;
+    ga.row_planes = ga.col_planes = 2 * nmod;
+    ga.row_plane0 = ga.col_plane0 = 0;
+    ga.nbatch = 2 * nmod;
+    ga.out = cpm; ga.ldp = c.ldp;
+    build_mod_table(nmod, &ga.mods);
+    ga.dev_status = dev_status;
+    if (int s = run_gemm(ga, nmod, st)) return s;
+    CK(ph.mark());
+    // Eq. (2c) + steps 5-7
+    CK(launch_post_fp<T>(cpm, c.ldp, m, n, eA, eB, ctab, C, ldc, st, &g.launches[3]));
+    CK(ph.mark());
+    ph.done();
+    return GEMM2M_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* gemm2m_status_string(int status) {
+    switch (status) {
+        case GEMM2M_OK: return "GEMM2M_OK";
+        case GEMM2M_ERR_ARG: return "GEMM2M_ERR_ARG";
+        case GEMM2M_ERR_NMOD: return "GEMM2M_ERR_NMOD";
+        case GEMM2M_ERR_WORKSPACE: return "GEMM2M_ERR_WORKSPACE";
+        case GEMM2M_ERR_CUDA: return "GEMM2M_ERR_CUDA";
+        case GEMM2M_ERR_ARCH: return "GEMM2M_ERR_ARCH";
+        case GEMM2M_ERR_DEVICE_TIMEOUT: return "GEMM2M_ERR_DEVICE_TIMEOUT";
+        default: return "GEMM2M_UNKNOWN";
+    }
+}
+
+const char* gemm2m_last_cuda_error(void) { return g_cuda_err; }
+
+int gemm2m_max_moduli(void) { return kMaxMod; }
+
+int gemm2m_modulus(int j, int* m, int* s) {
+    if (j < 0 || j >= kMaxMod) return GEMM2M_ERR_ARG;
+    if (m) *m = modulus_value(j);
+    if (s) *s = modulus_root(j);
+    return GEMM2M_OK;
+}
+
+size_t gemm2m_workspace_bytes(int op, int64_t m, int64_t n, int64_t k, int nmod) {
+    Carve c;
+    if (op == GEMM2M_OP_GAUSSIAN_INT && nmod > 8) return 0;
+    if (!carve(op, m, n, k, nmod, &c)) return 0;
+    return (size_t)c.total;
+}
+
+int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, gemm2m_layout* out) {
+    Carve c;
+    if (!out || !carve(op, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
+    out->off_exp_a = c.off_exp_a;
+    out->off_exp_b = c.off_exp_b;
+    out->off_apm = c.off_apm;
+    out->off_bpm = c.off_bpm;
+    out->off_cpm = c.off_cpm;
+    out->kp = c.kp;
+    out->ldp = c.ldp;
+    out->total_bytes = c.total;
+    return GEMM2M_OK;
+}
+
+int gemm2m_set_workspace(void* dev_ptr, size_t bytes) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if ((dev_ptr == nullptr) != (bytes == 0)) return GEMM2M_ERR_ARG;
+    if (((uintptr_t)dev_ptr & 255) != 0) return GEMM2M_ERR_ARG;
+    g.ws = dev_ptr;
+    g.ws_bytes = bytes;
+    if (dev_ptr) CK(cudaMemset(dev_ptr, 0, 256));   // device status word
+    return GEMM2M_OK;
+}
+
+int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const int8_t* Ai, int64_t lda, const int8_t* Br,
+                        const int8_t* Bi, int64_t ldb, int64_t* Cr, int64_t* Ci, int64_t ldc, int nmod, void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
+    if (lda < (m > 1 ? m : 1) || ldb < (k > 1 ? k : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
+    if (nmod < 1 || nmod > 8) return GEMM2M_ERR_NMOD;
+    if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
+    if (m == 0 || n == 0) return GEMM2M_OK;
+    if (!Cr || !Ci || (k > 0 && (!Ar || !Ai || !Br || !Bi))) return GEMM2M_ERR_ARG;
+    if (int s = check_device()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (k == 0) {
+        CK(cudaMemset2DAsync(Cr, (size_t)ldc * 8, 0, (size_t)m * 8, (size_t)n, st));
+        CK(cudaMemset2DAsync(Ci, (size_t)ldc * 8, 0, (size_t)m * 8, (size_t)n, st));
+        return GEMM2M_OK;
+    }
+    Carve c;
+    if (!carve(GEMM2M_OP_GAUSSIAN_INT, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)g.ws;
+    int8_t* apm = (int8_t*)(ws + c.off_apm);
+    int8_t* bpm = (int8_t*)(ws + c.off_bpm);
+    int8_t* cpm = (int8_t*)(ws + c.off_cpm);
+    ResidueTable rtab;
+    build_residue_table(nmod, &rtab);
+    CrtTableInt ctab;
+    build_crt_table_int(nmod, &ctab);
+    Phases ph;
+    if (int s = begin_call(st, &ph)) return s;
+    CK(ph.mark());   // no scan phase
+    CK(launch_residues_int8(Ar, Ai, lda, false, m, k, c.kp, rtab, apm, st, &g.launches[1]));
+    CK(launch_residues_int8(Br, Bi, ldb, true, n, k, c.kp, rtab, bpm, st, &g.launches[1]));
+    CK(ph.mark());
+    GemmArgs ga;
+    ga.rowop = bpm; ga.colop = apm;
+    ga.R = n; ga.Cn = m; ga.Kp = c.kp;
+    ga.row_planes = ga.col_planes = 2 * nmod;
+    ga.row_plane0 = ga.col_plane0 = 0;
+    ga.nbatch = 2 * nmod;
+    ga.out = cpm; ga.ldp = c.ldp;
+    build_mod_table(nmod, &ga.mods);
+    ga.dev_status = (int*)(ws + c.off_status);
+    if (int s = run_gemm(ga, nmod, st)) return s;
+    CK(ph.mark());
+    CK(launch_post_int(cpm, c.ldp, m, n, ctab, Cr, Ci, ldc, st, &g.launches[3]));
+    CK(ph.mark());
+    ph.done();
+    return GEMM2M_OK;
+}
+
+int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
+            int nmod, void* stream) {
+    return xgemm2m<double>(GEMM2M_OP_ZGEMM, m, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
+}
+
+int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc, int nmod,
+            void* stream) {
+    return xgemm2m<float>(GEMM2M_OP_CGEMM, m, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
+}
+
+int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (n < 0 || k < 0) return GEMM2M_ERR_ARG;
+    if (lda < (n > 1 ? n : 1) || ldc < (n > 1 ? n : 1)) return GEMM2M_ERR_ARG;
+    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
+    if (n > kMaxRows) return GEMM2M_ERR_ARG;
+    if (n == 0) return GEMM2M_OK;
+    if (!C || (k > 0 && !A)) return GEMM2M_ERR_ARG;
+    if (int s = check_device()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    Carve c;
+    if (!carve(GEMM2M_OP_ZHERK, n, n, k > 0 ? k : 1, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)g.ws;
+    uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
+    int32_t* eA = (int32_t*)(ws + c.off_exp_a);
+    int8_t* apm = (int8_t*)(ws + c.off_apm);
+    int8_t* cp = (int8_t*)(ws + c.off_cpm);
+    const ScaleTargets sc = scale_targets(nmod, k, true);
+    ResidueTable rtab;
+    build_residue_table(nmod, &rtab);
+    CrtTable ctab;
+    build_crt_table(nmod, &ctab);
+    Phases ph;
+    if (int s = begin_call(st, &ph)) return s;
+    CK(cudaMemsetAsync(absA, 0, (size_t)8 * n, st));
+    CK(launch_scan_rows<double>(A, n, k, lda, absA, st, &g.launches[0]));
+    CK(launch_exponents<double>(absA, n, sc.PA, sc.ck, eA, st, &g.launches[0]));
+    CK(ph.mark());
+    if (k == 0) CK(cudaMemsetAsync(apm, 0, (size_t)2 * nmod * n * c.kp, st));
+    else CK(launch_residues_fp<double>(A, lda, false, n, k, c.kp, eA, rtab, sc.PA - sc.ck > 62, apm, st, &g.launches[1]));
+    CK(ph.mark());
+    // Section 5: C+ = A+ A-^T only.  TMEM columns (contiguous index i of the output) <- rows of A+, TMEM lanes (j) <- rows of A-,
+    // so that out[j][i] = sum_k A+[i,k] A-[j,k] = C+[i,j].
+    GemmArgs ga;
+    ga.rowop = apm; ga.colop = apm;
+    ga.R = n; ga.Cn = n; ga.Kp = c.kp;
+    ga.row_planes = ga.col_planes = 2 * nmod;
+    ga.row_plane0 = nmod;    // "-" planes
+    ga.col_plane0 = 0;       // "+" planes
+    ga.nbatch = nmod;
+    ga.out = cp; ga.ldp = c.ldp;
+    build_mod_table(nmod, &ga.mods);
+    ga.dev_status = (int*)(ws + c.off_status);
+    if (int s = run_gemm(ga, nmod, st)) return s;
+    CK(ph.mark());
+    CK(launch_post_herk(cp, c.ldp, n, eA, ctab, C, ldc, st, &g.launches[3]));
+    CK(ph.mark());
+    ph.done();
+    return GEMM2M_OK;
+}
+
+int gemm2m_device_status(void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    if (!g.ws) return GEMM2M_OK;
+    int code = 0;
+    CK(cudaMemcpy(&code, g.ws, sizeof(int), cudaMemcpyDeviceToHost));
+    if (code != kDevOk) {
+        CK(cudaMemset(g.ws, 0, sizeof(int)));
+        return GEMM2M_ERR_DEVICE_TIMEOUT;
+    }
+    return GEMM2M_OK;
+}
+
+int gemm2m_set_profiling(int enabled) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    g.profiling = enabled ? 1 : 0;
+    g.prof_calls = 0;
+    return GEMM2M_OK;
+}
+
+int gemm2m_phase_ms(float ms[4], int* calls) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    const int count = g.prof_calls < State::kProfSlots ? g.prof_calls : State::kProfSlots;
+    if (!ms || count == 0) return GEMM2M_ERR_ARG;
+    for (int i = 0; i < 4; ++i) ms[i] = 0.f;
+    for (int c = 0; c < count; ++c) {
+        cudaEvent_t* ev = g.ev[c];
+        CK(cudaEventSynchronize(ev[4]));
+        for (int i = 0; i < 4; ++i) {
+            float t = 0.f;
+            CK(cudaEventElapsedTime(&t, ev[i], ev[i + 1]));
+            ms[i] += t / (float)count;
+        }
+    }
+    if (calls) *calls = count;
+    return GEMM2M_OK;
+}
+
+int gemm2m_last_launch_count(int per_phase[4]) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    int total = 0;
+    for (int i = 0; i < 4; ++i) {
+        if (per_phase) per_phase[i] = g.launches[i];
+        total += g.launches[i];
+    }
+    return total;
+}
+
+int gemm2m_debug_set_gemm_kernel(int which) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (which != 0 && which != 1) return GEMM2M_ERR_ARG;
+    g.gemm_kernel = which;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,
+                        int8_t* res_w) {
+    if (nmod < 1 || nmod > kMaxMod || k < 0) return GEMM2M_ERR_ARG;
+    const ScaleTargets sc = scale_targets(nmod, k, herk != 0);
+    if (scale) { scale[0] = sc.Pt; scale[1] = sc.PA; scale[2] = sc.PB; scale[3] = sc.ck; }
+    CrtTable ct;
+    build_crt_table(nmod, &ct);
+    for (int j = 0; j < nmod; ++j)
+        for (int c = 0; c < kMaxChunks; ++c) {
+            if (crt_gr) crt_gr[j * kMaxChunks + c] = ct.gr[j][c];
+            if (crt_gi) crt_gi[j * kMaxChunks + c] = ct.gi[j][c];
+        }
+    if (crt_m) for (int c = 0; c < kMaxChunks; ++c) crt_m[c] = ct.Mc[c];
+    if (nchunks) *nchunks = ct.nchunks;
+    if (res_w) {
+        ResidueTable rt;
+        build_residue_table(nmod, &rt);
+        for (int j = 0; j < nmod; ++j)
+            for (int b = 0; b < 8; ++b) {
+                const uint32_t w = b < 4 ? rt.w_lo[j] >> (8 * b) : rt.w_hi[j] >> (8 * (b - 4));
+                const uint32_t ws = b < 4 ? rt.ws_lo[j] >> (8 * b) : rt.ws_hi[j] >> (8 * (b - 4));
+                res_w[j * 16 + b] = (int8_t)(w & 0xFF);
+                res_w[j * 16 + 8 + b] = (int8_t)(ws & 0xFF);
+            }
+    }
+    return GEMM2M_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+// Shared declarations of the gemm2m CUDA library: constant tables passed to kernels by value,
+// launch wrappers of each phase, and small device helpers.  Notation follows the paper:
+// m_j = 2M modulus, s_j = its square root of -1, M = product of the moduli in use.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gemm2m {
+
+constexpr int kMaxMod = 22;        // size of the greedy 2M modulus set in [1, 256] (Section 4)
+constexpr int kMaxChunks = 4;      // 40-bit digits needed for M/2 < 2^152
+constexpr int kChunkBits = 40;
+constexpr int kMaxWideShift = 80;  // largest left shift of a mantissa in the wide quantisation mode
+constexpr int kExpNonFinite = INT32_MIN;   // scale-exponent sentinel: row/column holds an Inf or NaN
+
+// Device status word values (written by kernels whose bounded waits give up).
+constexpr int kDevOk = 0;
+constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilogue = 103;
+
+// Per-modulus constants for the residue kernels, Eq. (2a).
+// A quantised part x (two's complement int64) is written as 4 unsigned low bytes and 4 balanced
+// (signed) high digits; its residue is the dot product of those 8 digits with w_b = sym(256^b mod m).
+// The imaginary part uses s*w_b so that R + I = A_r + s A_i and R - I = A_r - s A_i (mod m).
+struct ResidueTable {
+    int32_t m[kMaxMod];
+    float inv_m[kMaxMod];
+    uint32_t w_lo[kMaxMod], w_hi[kMaxMod];     // int8 x4 each: sym(256^b mod m), b = 0..3 / 4..7
+    uint32_t ws_lo[kMaxMod], ws_hi[kMaxMod];   // int8 x4 each: sym(s 256^b mod m)
+    int32_t s[kMaxMod];
+    int8_t pow2[kMaxMod][kMaxWideShift];       // sym(2^t mod m): only used when quantised values exceed 62 bits
+    int nmod;
+};
+
+// Moduli for the GEMM epilogue (reduction of the int32 accumulators mod m_j).
+struct ModTable {
+    int32_t m[kMaxMod];
+    float inv_m[kMaxMod];
+    int nmod;
+};
+
+// CRT constants for the floating-point post-processing (Eq. (2c) folded into the CRT weights):
+//   X_r = sum_j (c-_j + c+_j) Gr_j  (mod M),  Gr_j = sym(2^-1 q_j mod m_j) (M/m_j)
+//   X_i = sum_j (c-_j - c+_j) Gi_j  (mod M),  Gi_j = sym(s_j 2^-1 q_j mod m_j) (M/m_j)
+// with q_j = (M/m_j)^-1 mod m_j.  Each weight is stored as signed base-2^40 digits held in doubles, so
+// that every digit-column sum is an exact integer below 2^53; rho = G/M estimates the multiple of M to remove.
+struct CrtTable {
+    double gr[kMaxMod][kMaxChunks];
+    double gi[kMaxMod][kMaxChunks];
+    double rho_r[kMaxMod], rho_i[kMaxMod];
+    double Mc[kMaxChunks];                     // digits of M
+    int nmod, nchunks;
+};
+
+// CRT constants for the exact int64 result (nmod <= 8, M < 2^62).
+struct CrtTableInt {
+    int64_t W[8];          // M / m_j
+    int32_t gr[8], gi[8];  // sym(2^-1 q_j), sym(s_j 2^-1 q_j)  (mod m_j)
+    int32_t m[8];
+    int64_t M;
+    int nmod;
+};
+
+struct ScaleTargets { int Pt, PA, PB, ck; };
+
+// ---- host-side table builders (tables.cu) ----
+int modulus_value(int j);
+int modulus_root(int j);
+void build_residue_table(int nmod, ResidueTable* t);
+void build_mod_table(int nmod, ModTable* t);
+void build_crt_table(int nmod, CrtTable* t);
+void build_crt_table_int(int nmod, CrtTableInt* t);
+ScaleTargets scale_targets(int nmod, int64_t k, bool herk);
+int64_t gemm_k_limit(int nmod);     // largest K for which k ((m_1-1)/2)^2 fits int32
+
+// ---- phase launchers (prepost.cu) ----
+// Exponent scan: largest |Re|,|Im| bit pattern per row of a column-major matrix (rows x cols, ld).
+template <typename T> cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches);
+// The same per column.
+template <typename T> cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches);
+template <typename T> cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int ck, int32_t* e, cudaStream_t st, int* launches);
+// Quantise + residues.  k_contiguous = false: operand row r is row r of the column-major matrix X (A: m x k);
+// true: operand row r is column r of X (B: k x n).
+// wide = quantised values may need more than 62 bits (P - c_k > 62): they are carried as mantissa x 2^t.
+template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+                                 const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
+template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const int32_t* eA, const int32_t* eB,
+                                                 const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches);
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
+                             cudaStream_t st, int* launches);
+cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,
+                            int64_t ldc, cudaStream_t st, int* launches);
+
+// ---- int8 GEMM (gemm_i8.cu) ----
+// For each batch b in [0, nbatch): out[b][r][c] = sym( sum_k rowop[b + row_plane0][r][k] * colop[b + col_plane0][c][k]  mod m_{b % nmod} ),
+// r < R, c < Cn, k < Kp (zero padded); planes are [*][rows][Kp] int8; out planes are [R][ldp] int8.
+struct GemmArgs {
+    const int8_t* rowop; const int8_t* colop;
+    int64_t R, Cn, Kp;
+    int row_planes, col_planes;       // number of planes behind each pointer (for the tensor maps)
+    int row_plane0, col_plane0, nbatch;
+    int8_t* out; int64_t ldp;
+    ModTable mods;
+    int* dev_status;
+};
+cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);
+cudaError_t launch_gemm_check(const GemmArgs& a, int64_t k_limit, cudaStream_t st, int* launches);
+
+}  // namespace gemm2m

@@ -1,0 +1,606 @@
+// Pre- and post-processing kernels of 2M Ozaki-II (Algorithm 1 steps 2, 3, 4 (Eq. 2a, 2c), 5, 6, 7).
+// All of them are streaming kernels bounded by HBM bandwidth / plain ALU throughput.
+#include "common.cuh"
+
+namespace gemm2m {
+
+// =====================================================================================================
+// Step 2: exponent scan.  For every row (or column) the largest magnitude bit pattern of any real or
+// imaginary part; IEEE bit patterns of non-negative numbers are ordered like the numbers themselves.
+// =====================================================================================================
+template <typename T> struct FpBits;
+template <> struct FpBits<double> {
+    using U = unsigned long long;
+    static constexpr int kMantBits = 52, kExpMax = 2047, kBias = 1023;
+    __device__ static U mag(double v) { return (U)__double_as_longlong(v) & 0x7FFFFFFFFFFFFFFFull; }
+};
+template <> struct FpBits<float> {
+    using U = unsigned long long;
+    static constexpr int kMantBits = 23, kExpMax = 255, kBias = 127;
+    __device__ static U mag(float v) { return (U)(__float_as_uint(v) & 0x7FFFFFFFu); }
+};
+
+template <typename T> struct Cplx { T re, im; };
+template <typename T> __device__ __forceinline__ Cplx<T> load_cplx(const T* p);
+template <> __device__ __forceinline__ Cplx<double> load_cplx<double>(const double* p) {
+    const double2 v = __ldg(reinterpret_cast<const double2*>(p));
+    return {v.x, v.y};
+}
+template <> __device__ __forceinline__ Cplx<float> load_cplx<float>(const float* p) {
+    const float2 v = __ldg(reinterpret_cast<const float2*>(p));
+    return {v.x, v.y};
+}
+
+constexpr int kScanThreads = 256;
+constexpr int kScanRowsSpan = 64;     // columns handled by one block of scan_rows
+constexpr int kScanColsSpan = 2048;   // rows handled by one warp of scan_cols
+
+// One thread per row, a span of columns per block: consecutive threads read consecutive rows (coalesced).
+template <typename T>
+__global__ void __launch_bounds__(kScanThreads) scan_rows_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
+                                                                 unsigned long long* __restrict__ absmax) {
+    const int64_t r = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
+    if (r >= rows) return;
+    const int64_t c0 = (int64_t)blockIdx.y * span;
+    const int64_t c1 = min(cols, c0 + span);
+    unsigned long long mx = 0;
+    const T* p = X + 2 * (r + c0 * ld);
+#pragma unroll 8
+    for (int64_t c = c0; c < c1; ++c, p += 2 * ld) {
+        const Cplx<T> v = load_cplx<T>(p);
+        mx = max(mx, max(FpBits<T>::mag(v.re), FpBits<T>::mag(v.im)));
+    }
+    if (mx) atomicMax(absmax + r, mx);
+}
+
+// One warp per (column, span of rows): lanes read consecutive elements of the column.
+template <typename T>
+__global__ void __launch_bounds__(kScanThreads) scan_cols_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
+                                                                 unsigned long long* __restrict__ absmax) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c = (int64_t)blockIdx.x * (kScanThreads / 32) + warp;
+    if (c >= cols) return;
+    const int64_t r0 = (int64_t)blockIdx.y * span;
+    const int64_t r1 = min(rows, r0 + span);
+    unsigned long long mx = 0;
+    const T* base = X + 2 * (c * ld);
+#pragma unroll 4
+    for (int64_t r = r0 + lane; r < r1; r += 32) {
+        const Cplx<T> v = load_cplx<T>(base + 2 * r);
+        mx = max(mx, max(FpBits<T>::mag(v.re), FpBits<T>::mag(v.im)));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if (lane == 0 && mx) atomicMax(absmax + c, mx);
+}
+
+// e = floor(log2 mu) + 1 + c_k - P for the largest magnitude mu; 0 for an all-zero row; sentinel for Inf/NaN.
+template <typename T>
+__global__ void exponents_kernel(const unsigned long long* __restrict__ absmax, int64_t count, int P, int ck, int32_t* __restrict__ e) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const unsigned long long b = absmax[i];
+    int out;
+    if (b == 0) {
+        out = 0;
+    } else {
+        const int E = (int)(b >> FpBits<T>::kMantBits);
+        if (E == FpBits<T>::kExpMax) {
+            out = kExpNonFinite;
+        } else {
+            const int x = E ? E - FpBits<T>::kBias : (63 - __clzll((long long)b)) - (FpBits<T>::kBias - 1 + FpBits<T>::kMantBits);
+            out = x + 1 + ck - P;
+        }
+    }
+    e[i] = out;
+}
+
+template <typename T>
+cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    int64_t span = kScanRowsSpan;
+    while ((cols + span - 1) / span > 65535) span *= 2;        // grid.y limit
+    dim3 grid((unsigned)((rows + kScanThreads - 1) / kScanThreads), (unsigned)((cols + span - 1) / span));
+    scan_rows_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    ++*launches;
+    return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    int64_t span = kScanColsSpan;
+    while ((rows + span - 1) / span > 65535) span *= 2;        // grid.y limit
+    dim3 grid((unsigned)((cols + kScanThreads / 32 - 1) / (kScanThreads / 32)), (unsigned)((rows + span - 1) / span));
+    scan_cols_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    ++*launches;
+    return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int ck, int32_t* e, cudaStream_t st, int* launches) {
+    if (count <= 0) return cudaSuccess;
+    exponents_kernel<T><<<(unsigned)((count + 255) / 256), 256, 0, st>>>((const unsigned long long*)absmax, count, P, ck, e);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// =====================================================================================================
+// Steps 3 + 4 (Eq. 2a): quantise by truncation and emit the symmetric int8 residues A+ / A- for every
+// modulus, K contiguous.  A block stages a tile of 32 operand rows x 128 k of quantised parts in shared
+// memory (coalesced global reads in either orientation), then each thread owns 16 consecutive k of one row
+// and writes 16-byte vectors into every plane.
+// =====================================================================================================
+constexpr int kResRows = 32, kResK = 128, kResThreads = 256;
+constexpr int kResRowStride = kResK + kResK / 16 + 1;   // in 16-byte elements: one pad per 16 + odd row stride -> no bank conflicts
+
+struct QPair { long long re, im; };   // quantised parts, two's complement
+
+// trunc(v 2^-e) for a finite v given by its bit pattern.
+// Narrow mode (WIDE = false): the scaling rule guarantees |result| < 2^62, returned as a two's complement int64.
+// Wide mode: the result is sign * mant * 2^t with mant < 2^53; returned packed as (sign * mant) * 256 + t.
+template <typename T, bool WIDE>
+__device__ __forceinline__ long long quantise_part(T v, int e) {
+    using F = FpBits<T>;
+    const unsigned long long mag = F::mag(v);
+    const int E = (int)(mag >> F::kMantBits);
+    unsigned long long mant = mag & ((1ull << F::kMantBits) - 1);
+    if (E) mant |= (1ull << F::kMantBits);
+    // v = mant 2^(max(E,1) - bias - mantbits)
+    const int sh = max(E, 1) - (F::kBias + F::kMantBits) - e;
+    const bool neg = (sizeof(T) == 8) ? (__double_as_longlong((double)v) < 0) : (__float_as_int((float)v) < 0);
+    unsigned long long q;
+    int t = 0;
+    if (sh >= 0) {
+        if (WIDE) { q = mant; t = mant ? min(sh, kMaxWideShift - 1) : 0; }
+        else q = mant << min(sh, 63);
+    } else {
+        q = (-sh > 63) ? 0ull : (mant >> (-sh));
+    }
+    const long long sq = neg ? -(long long)q : (long long)q;
+    return WIDE ? sq * 256 + t : sq;
+}
+
+__device__ __forceinline__ int dp4a_us(uint32_t a_unsigned, uint32_t b_signed, int c) {
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a_unsigned), "r"(b_signed), "r"(c));
+    return d;
+}
+__device__ __forceinline__ int dp4a_ss(uint32_t a_signed, uint32_t b_signed, int c) {
+    int d;
+    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a_signed), "r"(b_signed), "r"(c));
+    return d;
+}
+
+// Symmetric residue of x (|x| < 2^22) modulo m by a float reciprocal: the quotient estimate is exact because
+// |x/m| < 2^11 carries an error below 1/(2m), the distance of x/m from the nearest rounding boundary.
+__device__ __forceinline__ int sym_reduce_small(int x, int m, float inv_m) {
+    const float xf = __int_as_float(x + 0x4B400000) - 12582912.0f;   // exact int -> float for |x| < 2^22
+    const float t = fmaf(xf, inv_m, 12582912.0f);                    // nearest integer in the low mantissa bits
+    const int q = __float_as_int(t) - 0x4B400000;
+    return x - q * m;
+}
+
+struct Digits { uint32_t lo, hi; };   // 4 unsigned low bytes; 4 balanced (signed) high digits
+__device__ __forceinline__ Digits split_digits(long long x) {
+    Digits d;
+    d.lo = (uint32_t)(unsigned long long)x;
+    const uint32_t hi = (uint32_t)((unsigned long long)x >> 32);
+    d.hi = (hi + 0x80808080u) ^ 0x80808080u;   // hi = sum (byte_b - 128) 256^b  after adding 128 to every byte
+    return d;
+}
+
+// Stage one 32 x 128 tile of quantised parts into shared memory.  fetch(r, kk) returns the quantised pair.
+template <typename Fetch>
+__device__ __forceinline__ void stage_tile(QPair* tile, bool k_contiguous, Fetch fetch) {
+    const int t = threadIdx.x;
+    if (!k_contiguous) {          // consecutive threads -> consecutive operand rows (column-major A)
+        const int r = t & 31;
+        for (int kk = t >> 5; kk < kResK; kk += kResThreads / 32) tile[r * kResRowStride + kk + (kk >> 4)] = fetch(r, kk);
+    } else {                      // consecutive threads -> consecutive k (columns of B are contiguous)
+        const int kk = t & (kResK - 1);
+        for (int r = t >> 7; r < kResRows; r += kResThreads / kResK) tile[r * kResRowStride + kk + (kk >> 4)] = fetch(r, kk);
+    }
+}
+
+// From the staged tile: thread (row = t / 8, group g = t % 8) owns k = 16 g .. 16 g + 15 and writes both sign planes
+// of every modulus.  planes: [2 nmod][R][Kp].
+template <bool WIDE>
+__device__ __forceinline__ void emit_residues(const QPair* tile, const ResidueTable& tab, int8_t* planes, int64_t R, int64_t Kp,
+                                              int64_t row0, int64_t k0) {
+    const int t = threadIdx.x;
+    const int g = t & 7, r = t >> 3;
+    Digits dr[16], di[16];
+    uint32_t tsh[WIDE ? 16 : 1];   // wide mode: left shifts t_r | t_i << 8 of the two mantissas
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const QPair q = tile[r * kResRowStride + 16 * g + i + g];
+        if (WIDE) {
+            tsh[i] = (uint32_t)(q.re & 0xFF) | ((uint32_t)(q.im & 0xFF) << 8);
+            dr[i] = split_digits(q.re >> 8);
+            di[i] = split_digits(q.im >> 8);
+        } else {
+            dr[i] = split_digits(q.re);
+            di[i] = split_digits(q.im);
+        }
+    }
+    const int64_t row = row0 + r;
+    if (row >= R) return;
+    const int64_t plane_stride = R * Kp;
+    int8_t* dst = planes + row * Kp + k0 + 16 * g;
+    const int nmod = tab.nmod;
+    for (int j = 0; j < nmod; ++j) {
+        const int m = tab.m[j];
+        const float inv_m = tab.inv_m[j];
+        const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
+        uint32_t pw[4], mw[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t pp = 0, mm = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = 4 * w + b;
+                int Rv = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, 0));   // A_r mod m (unreduced)
+                int Iv = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, 0));   // s A_i mod m (unreduced)
+                if (WIDE) {                                                 // times 2^t mod m
+                    Rv = sym_reduce_small(Rv, m, inv_m) * (int)tab.pow2[j][tsh[i] & 0xFF];
+                    Iv = sym_reduce_small(Iv, m, inv_m) * (int)tab.pow2[j][tsh[i] >> 8];
+                }
+                const int ap = sym_reduce_small(Rv + Iv, m, inv_m);               // Eq. (2a), "+"
+                const int am = sym_reduce_small(Rv - Iv, m, inv_m);               // Eq. (2a), "-"
+                pp |= ((uint32_t)ap & 0xFFu) << (8 * b);
+                mm |= ((uint32_t)am & 0xFFu) << (8 * b);
+            }
+            pw[w] = pp;
+            mw[w] = mm;
+        }
+        *reinterpret_cast<uint4*>(dst + (int64_t)j * plane_stride) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+        *reinterpret_cast<uint4*>(dst + (int64_t)(nmod + j) * plane_stride) = make_uint4(mw[0], mw[1], mw[2], mw[3]);
+    }
+}
+
+template <typename T, bool WIDE>
+__global__ void __launch_bounds__(kResThreads) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
+                                                                  int64_t Kp, const int32_t* __restrict__ e, const __grid_constant__ ResidueTable tab,
+                                                                  int8_t* __restrict__ planes) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    QPair* tile = reinterpret_cast<QPair*>(smem_raw);
+    const int64_t row0 = (int64_t)blockIdx.y * kResRows, k0 = (int64_t)blockIdx.x * kResK;
+    stage_tile(tile, k_contiguous, [&](int r, int kk) -> QPair {
+        const int64_t row = row0 + r, k = k0 + kk;
+        QPair q{0, 0};
+        if (row < R && k < K) {
+            const int ex = __ldg(e + row);
+            if (ex != kExpNonFinite) {
+                const T* p = k_contiguous ? X + 2 * (k + row * ld) : X + 2 * (row + k * ld);
+                const Cplx<T> v = load_cplx<T>(p);
+                q.re = quantise_part<T, WIDE>(v.re, ex);
+                q.im = quantise_part<T, WIDE>(v.im, ex);
+            }
+        }
+        return q;
+    });
+    __syncthreads();
+    emit_residues<WIDE>(tile, tab, planes, R, Kp, row0, k0);
+}
+
+__global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t* __restrict__ Xr, const int8_t* __restrict__ Xi, int64_t ld,
+                                                                    bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+                                                                    const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    QPair* tile = reinterpret_cast<QPair*>(smem_raw);
+    const int64_t row0 = (int64_t)blockIdx.y * kResRows, k0 = (int64_t)blockIdx.x * kResK;
+    stage_tile(tile, k_contiguous, [&](int r, int kk) -> QPair {
+        const int64_t row = row0 + r, k = k0 + kk;
+        QPair q{0, 0};
+        if (row < R && k < K) {
+            const int64_t idx = k_contiguous ? k + row * ld : row + k * ld;
+            q.re = Xr[idx];
+            q.im = Xi[idx];
+        }
+        return q;
+    });
+    __syncthreads();
+    emit_residues<false>(tile, tab, planes, R, Kp, row0, k0);
+}
+
+constexpr size_t kResSmem = (size_t)kResRows * kResRowStride * sizeof(QPair);
+
+template <typename T>
+cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
+    if (R <= 0 || Kp <= 0) return cudaSuccess;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResRows - 1) / kResRows));
+    if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, kResSmem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    else residues_fp_kernel<T, false><<<grid, kResThreads, kResSmem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+                                 const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches) {
+    if (R <= 0 || Kp <= 0) return cudaSuccess;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(residues_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResRows - 1) / kResRows));
+    residues_int8_kernel<<<grid, kResThreads, kResSmem, st>>>(Xr, Xi, ld, k_contiguous, R, K, Kp, tab, planes);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// =====================================================================================================
+// Steps 4 (Eq. 2c), 5, 6, 7: per output element, fold the 2M post-processing into the CRT weights, sum the
+// weighted residues exactly in 40-bit digit columns (FP64 FMAs on integers below 2^53), remove the multiple
+// of M, and round the lifted integer once to floating point before scaling by 2^(e_i + f_j).
+// =====================================================================================================
+__device__ __forceinline__ double int_to_double(int v) {   // exact, avoids the slow conversion instruction
+    return __hiloint2double(0x43300000, (int)(0x80000000u ^ (uint32_t)v)) - 4503601774854144.0;   // 2^52 + 2^31
+}
+
+// Lifted X (exact integer, |X| <= (M-1)/2) from the digit-column sums S[c] and the quotient estimate qsum ~ X'/M,
+// returned as an unevaluated sum hi + lo with |lo| <= ulp(hi)/2.
+template <int NCH>
+__device__ __forceinline__ void crt_finish(double (&S)[NCH], double qsum, const CrtTable& tab, double* hi, double* lo) {
+    const double t = rint(qsum);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) S[c] = fma(-t, tab.Mc[c], S[c]);          // exact: |t| < 2^12, digits < 2^40
+    const double two40 = 1099511627776.0, inv40 = 1.0 / 1099511627776.0;
+#pragma unroll
+    for (int c = 0; c + 1 < NCH; ++c) {                                     // carry into canonical digits [0, 2^40)
+        const double carry = floor(S[c] * inv40);
+        S[c] = fma(-carry, two40, S[c]);
+        S[c + 1] += carry;
+    }
+    double h = S[NCH - 1], l = 0.0;                                          // top digit keeps the sign
+#pragma unroll
+    for (int c = NCH - 2; c >= 0; --c) {
+        h *= two40;
+        l *= two40;
+        const double s = h + S[c];                                           // TwoSum
+        const double bb = s - h;
+        const double err = (h - (s - bb)) + (S[c] - bb);
+        h = s;
+        l += err;
+    }
+    *hi = h;
+    *lo = l;
+}
+
+__device__ __forceinline__ double scale_pow2(double x, int e) {   // x 2^e with e split so that both factors are normal
+    const int e1 = max(-1000, min(1000, e));
+    const int e2 = max(-1000, min(1000, e - e1));
+    const int e3 = e - e1 - e2;
+    double y = x * __longlong_as_double((long long)(e1 + 1023) << 52);
+    if (e2) y *= __longlong_as_double((long long)(e2 + 1023) << 52);
+    if (e3) y = ldexp(y, e3);
+    return y;
+}
+
+template <typename T> __device__ __forceinline__ void store4(T* dst, const double (&re)[4], const double (&im)[4], int count);
+template <> __device__ __forceinline__ void store4<double>(double* dst, const double (&re)[4], const double (&im)[4], int count) {
+    for (int i = 0; i < count; ++i) *reinterpret_cast<double2*>(dst + 2 * i) = make_double2(re[i], im[i]);
+}
+template <> __device__ __forceinline__ void store4<float>(float* dst, const double (&re)[4], const double (&im)[4], int count) {
+    if (count == 4 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        *reinterpret_cast<float4*>(dst) = make_float4((float)re[0], (float)im[0], (float)re[1], (float)im[1]);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4((float)re[2], (float)im[2], (float)re[3], (float)im[3]);
+    } else {
+        for (int i = 0; i < count; ++i) *reinterpret_cast<float2*>(dst + 2 * i) = make_float2((float)re[i], (float)im[i]);
+    }
+}
+
+constexpr int kPostThreads = 128;
+
+// cpm: [2 nmod][n][ldp] int8 (row index i contiguous).  One thread -> 4 consecutive i of one column j.
+template <typename T, int NCH>
+__global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
+                                                               const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
+                                                               const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc) {
+    const int64_t i0 = ((int64_t)blockIdx.x * kPostThreads + threadIdx.x) * 4;
+    const int64_t j = blockIdx.y;
+    if (i0 >= m) return;
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cpm + j * ldp + i0;
+    double Sr[4][NCH], Si[4][NCH], qr[4], qi[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        qr[e] = qi[e] = 0.0;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
+    }
+    for (int jm = 0; jm < nmod; ++jm) {
+        const uint32_t wp = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)jm * plane));            // c+ of 4 elements
+        const uint32_t wm = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)(nmod + jm) * plane));   // c-
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int cp = (int)(int8_t)(wp >> (8 * e));
+            const int cm = (int)(int8_t)(wm >> (8 * e));
+            const double vr = int_to_double(cm + cp);     // Eq. (2c): real part uses C- + C+
+            const double vi = int_to_double(cm - cp);     //           imaginary part uses C- - C+
+            qr[e] = fma(vr, tab.rho_r[jm], qr[e]);
+            qi[e] = fma(vi, tab.rho_i[jm], qi[e]);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
+                Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
+            }
+        }
+    }
+    const int fb = __ldg(eB + j);
+    double re[4], im[4];
+    int count = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if (i0 + e < m) {
+            ++count;
+            const int ea = __ldg(eA + i0 + e);
+            if (ea == kExpNonFinite || fb == kExpNonFinite) {
+                re[e] = im[e] = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(Sr[e], qr[e], tab, &h, &l);
+                re[e] = scale_pow2(h + l, ea + fb);
+                crt_finish<NCH>(Si[e], qi[e], tab, &h, &l);
+                im[e] = scale_pow2(h + l, ea + fb);
+            }
+        }
+    }
+    store4<T>(C + 2 * (i0 + j * ldc), re, im, count);
+}
+
+template <typename T>
+cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const int32_t* eA, const int32_t* eB, const CrtTable& tab,
+                           T* C, int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || n <= 0) return cudaSuccess;
+    const int64_t per_block = (int64_t)kPostThreads * 4;
+    for (int64_t j0 = 0; j0 < n; j0 += 65535) {      // grid.y limit
+        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+        dim3 grid((unsigned)((m + per_block - 1) / per_block), (unsigned)nj);
+        const int8_t* src = cpm + j0 * ldp;
+        T* dst = C + 2 * j0 * ldc;
+        // the plane stride is n * ldp for the whole matrix, so pass the full n and offset pointers
+        switch (tab.nchunks) {
+            case 1: post_fp_kernel<T, 1><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 2: post_fp_kernel<T, 2><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 3: post_fp_kernel<T, 3><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            default: post_fp_kernel<T, 4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+        }
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+// HERK (Section 5): only C+ = A+ A-^T was computed; C- = C+^T.  cp: [nmod][n][ldp] with cp[j][col][row] = C+_j[row, col].
+// A 32 x 32 tile (rows i, columns j, i >= j) needs C+[i, j] (direct, i contiguous) and C+[j, i] (the mirrored tile,
+// transposed through shared memory).  Lower triangle only; the diagonal's imaginary part is exactly zero.
+constexpr int kHerkTile = 32;
+template <int NCH>
+__global__ void __launch_bounds__(kHerkTile * 8) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n,
+                                                                  const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
+                                                                  double* __restrict__ C, int64_t ldc) {
+    const int ti = blockIdx.x, tj = blockIdx.y;
+    if (ti < tj) return;
+    __shared__ int8_t mirror[kMaxMod][kHerkTile][kHerkTile + 4];
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    const int64_t ibase = (int64_t)ti * kHerkTile, jbase = (int64_t)tj * kHerkTile;
+    // mirrored tile: C+[j, i] = cp[col = i][row = j]; read with j contiguous, store transposed
+    for (int jm = 0; jm < nmod; ++jm)
+        for (int r = ty; r < kHerkTile; r += 8) {
+            const int64_t i = ibase + r, j = jbase + tx;
+            mirror[jm][r][tx] = (i < n && j < n) ? cp[(int64_t)jm * plane + i * ldp + j] : (int8_t)0;
+        }
+    __syncthreads();
+    for (int cj = ty; cj < kHerkTile; cj += 8) {
+        const int64_t i = ibase + tx, j = jbase + cj;
+        if (i >= n || j >= n || i < j) continue;
+        double Sr[NCH], Si[NCH], qr = 0.0, qi = 0.0;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) Sr[c] = Si[c] = 0.0;
+        for (int jm = 0; jm < nmod; ++jm) {
+            const int cpv = cp[(int64_t)jm * plane + j * ldp + i];   // C+[i, j]
+            const int cmv = mirror[jm][tx][cj];                      // C-[i, j] = C+[j, i]
+            const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
+            qr = fma(vr, tab.rho_r[jm], qr);
+            qi = fma(vi, tab.rho_i[jm], qi);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[c] = fma(vr, tab.gr[jm][c], Sr[c]);
+                Si[c] = fma(vi, tab.gi[jm][c], Si[c]);
+            }
+        }
+        const int ei = __ldg(eA + i), ej = __ldg(eA + j);
+        double re, im;
+        if (ei == kExpNonFinite || ej == kExpNonFinite) {
+            re = im = __longlong_as_double(0x7FF8000000000000ll);
+        } else {
+            double h, l;
+            crt_finish<NCH>(Sr, qr, tab, &h, &l);
+            re = scale_pow2(h + l, ei + ej);
+            crt_finish<NCH>(Si, qi, tab, &h, &l);
+            im = scale_pow2(h + l, ei + ej);
+        }
+        *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
+    }
+}
+
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
+                             cudaStream_t st, int* launches) {
+    if (n <= 0) return cudaSuccess;
+    const unsigned tiles = (unsigned)((n + kHerkTile - 1) / kHerkTile);
+    dim3 grid(tiles, tiles);
+    switch (tab.nchunks) {
+        case 1: post_herk_kernel<1><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        case 2: post_herk_kernel<2><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        case 3: post_herk_kernel<3><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        default: post_herk_kernel<4><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// Exact integer variant for gemm2m_gaussian_int: X = sum_j sym(v_j g_j mod m_j) (M/m_j) mod M in int64 (M < 2^62).
+__global__ void __launch_bounds__(256) post_int_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
+                                                       const __grid_constant__ CrtTableInt tab, int64_t* __restrict__ Cr,
+                                                       int64_t* __restrict__ Ci, int64_t ldc) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t j = blockIdx.y;
+    if (i >= m) return;
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cpm + j * ldp + i;
+    long long xr = 0, xi = 0;
+    const long long M = tab.M;
+    for (int jm = 0; jm < nmod; ++jm) {
+        const int cp = src[(int64_t)jm * plane], cm = src[(int64_t)(nmod + jm) * plane];
+        const int mj = tab.m[jm], half = (mj - 1) / 2;
+        int ur = ((cm + cp) * tab.gr[jm]) % mj;       // Eq. (2c) and the CRT factor q_j, folded
+        int ui = ((cm - cp) * tab.gi[jm]) % mj;
+        if (ur > half) ur -= mj; else if (ur < -half) ur += mj;
+        if (ui > half) ui -= mj; else if (ui < -half) ui += mj;
+        xr = (xr + (long long)ur * tab.W[jm]) % M;    // |term| < 2^62, |xr| < M < 2^62: no overflow
+        xi = (xi + (long long)ui * tab.W[jm]) % M;
+    }
+    const long long h = (M - 1) / 2;                  // lift to [-(M-1)/2, (M-1)/2]
+    if (xr > h) xr -= M; else if (xr < -h) xr += M;
+    if (xi > h) xi -= M; else if (xi < -h) xi += M;
+    Cr[i + j * ldc] = xr;
+    Ci[i + j * ldc] = xi;
+}
+
+cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,
+                            int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || n <= 0) return cudaSuccess;
+    for (int64_t j0 = 0; j0 < n; j0 += 65535) {
+        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+        dim3 grid((unsigned)((m + 255) / 256), (unsigned)nj);
+        post_int_kernel<<<grid, 256, 0, st>>>(cpm + j0 * ldp, ldp, m, n, tab, Cr + j0 * ldc, Ci + j0 * ldc, ldc);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+// explicit instantiations
+template cudaError_t launch_scan_rows<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
+template cudaError_t launch_scan_rows<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
+template cudaError_t launch_scan_cols<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
+template cudaError_t launch_scan_cols<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
+template cudaError_t launch_exponents<double>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
+template cudaError_t launch_exponents<float>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
+template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, cudaStream_t, int*);
+template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, cudaStream_t, int*);
+
+}  // namespace gemm2m

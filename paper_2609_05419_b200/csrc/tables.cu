@@ -1,0 +1,188 @@
+// Host-side constants of the method: the 2M modulus set of Section 4, the roots s_j (Section 2), the byte
+// weights of the residue kernels and the CRT weights (Section 3.1), computed with a small multi-limb integer.
+#include "common.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+namespace gemm2m {
+
+// Greedy coprime set of 2M moduli in [1, 256], descending (Section 4).
+static const int kModuli[kMaxMod] = {241, 233, 229, 221, 205, 197, 193, 181, 173, 157, 149,
+                                     137, 113, 109, 101, 97,  89,  73,  61,  53,  37,  29};
+
+int modulus_value(int j) { return kModuli[j]; }
+
+int modulus_root(int j) {   // smallest positive s with s^2 = -1 (mod m)
+    const int m = kModuli[j];
+    for (int s = 1; s < m; ++s)
+        if ((s * s + 1) % m == 0) return s;
+    return 0;
+}
+
+static inline int sym_mod(int64_t x, int m) {   // representative in [-(m-1)/2, (m-1)/2]
+    int r = (int)(x % m);
+    if (r < 0) r += m;
+    if (r > (m - 1) / 2) r -= m;
+    return r;
+}
+
+static int inv_mod(int a, int m) {   // a^-1 mod m by search (m <= 241)
+    a %= m;
+    if (a < 0) a += m;
+    for (int x = 1; x < m; ++x)
+        if ((a * x) % m == 1) return x;
+    return 0;
+}
+
+// ---- non-negative multi-limb integer, base 2^32, little endian ----
+struct Big {
+    std::vector<uint32_t> w;
+    void trim() { while (!w.empty() && w.back() == 0) w.pop_back(); }
+    static Big from(uint64_t v) { Big b; b.w = {(uint32_t)v, (uint32_t)(v >> 32)}; b.trim(); return b; }
+    void mul_small(uint32_t f) {
+        uint64_t carry = 0;
+        for (auto& limb : w) { uint64_t t = (uint64_t)limb * f + carry; limb = (uint32_t)t; carry = t >> 32; }
+        if (carry) w.push_back((uint32_t)carry);
+        trim();
+    }
+    uint32_t divmod_small(uint32_t d) {   // in-place quotient, returns remainder
+        uint64_t rem = 0;
+        for (size_t i = w.size(); i-- > 0;) { uint64_t t = (rem << 32) | w[i]; w[i] = (uint32_t)(t / d); rem = t % d; }
+        trim();
+        return (uint32_t)rem;
+    }
+    uint32_t mod_small(uint32_t d) const { Big c = *this; return c.divmod_small(d); }
+    int bit_length() const {
+        if (w.empty()) return 0;
+        int top = 32 - __builtin_clz(w.back());
+        return (int)(w.size() - 1) * 32 + top;
+    }
+    uint64_t bits(int pos, int count) const {   // count <= 64 bits starting at bit pos
+        uint64_t out = 0;
+        for (int b = 0; b < count; ++b) {
+            int p = pos + b;
+            size_t limb = (size_t)(p >> 5);
+            if (limb < w.size() && ((w[limb] >> (p & 31)) & 1u)) out |= (1ull << b);
+        }
+        return out;
+    }
+    void sub_one() { for (auto& limb : w) { if (limb-- != 0) break; } trim(); }
+    void shr1() { uint32_t c = 0; for (size_t i = w.size(); i-- > 0;) { uint32_t n = w[i] & 1u; w[i] = (w[i] >> 1) | (c << 31); c = n; } trim(); }
+    double to_double() const { double v = 0; for (size_t i = w.size(); i-- > 0;) v = v * 4294967296.0 + w[i]; return v; }
+};
+
+static Big product_of(int nmod) {
+    Big M = Big::from(1);
+    for (int j = 0; j < nmod; ++j) M.mul_small((uint32_t)kModuli[j]);
+    return M;
+}
+
+void build_residue_table(int nmod, ResidueTable* t) {
+    std::memset(t, 0, sizeof(*t));
+    t->nmod = nmod;
+    for (int j = 0; j < nmod; ++j) {
+        const int m = kModuli[j], s = modulus_root(j);
+        t->m[j] = m;
+        t->s[j] = s;
+        t->inv_m[j] = 1.0f / (float)m;
+        int64_t p = 1;   // 256^b mod m
+        uint32_t w[8], ws[8];
+        for (int b = 0; b < 8; ++b) {
+            w[b] = (uint32_t)(uint8_t)(int8_t)sym_mod(p, m);
+            ws[b] = (uint32_t)(uint8_t)(int8_t)sym_mod(p * s, m);
+            p = (p * 256) % m;
+        }
+        t->w_lo[j] = w[0] | (w[1] << 8) | (w[2] << 16) | (w[3] << 24);
+        t->w_hi[j] = w[4] | (w[5] << 8) | (w[6] << 16) | (w[7] << 24);
+        t->ws_lo[j] = ws[0] | (ws[1] << 8) | (ws[2] << 16) | (ws[3] << 24);
+        t->ws_hi[j] = ws[4] | (ws[5] << 8) | (ws[6] << 16) | (ws[7] << 24);
+        int64_t p2 = 1;
+        for (int e = 0; e < kMaxWideShift; ++e) { t->pow2[j][e] = (int8_t)sym_mod(p2, m); p2 = (p2 * 2) % m; }
+    }
+}
+
+void build_mod_table(int nmod, ModTable* t) {
+    std::memset(t, 0, sizeof(*t));
+    t->nmod = nmod;
+    for (int j = 0; j < nmod; ++j) { t->m[j] = kModuli[j]; t->inv_m[j] = 1.0f / (float)kModuli[j]; }
+}
+
+// Folded CRT weights: g_j = sym(2^-1 q_j mod m_j), h_j = sym(s_j 2^-1 q_j mod m_j), q_j = (M/m_j)^-1 mod m_j.
+static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h) {
+    const int m = kModuli[j];
+    *W = M;
+    W->divmod_small((uint32_t)m);
+    const int q = inv_mod((int)W->mod_small((uint32_t)m), m);
+    const int half = (m + 1) / 2;   // 2^-1 mod m (Section 2)
+    *g = sym_mod((int64_t)half * q, m);
+    *h = sym_mod((int64_t)modulus_root(j) * half % m * q, m);
+    (void)nmod;
+}
+
+void build_crt_table(int nmod, CrtTable* t) {
+    std::memset(t, 0, sizeof(*t));
+    t->nmod = nmod;
+    const Big M = product_of(nmod);
+    Big half = M;   // (M-1)/2 bounds every |G_j|
+    half.sub_one();
+    half.shr1();
+    t->nchunks = (half.bit_length() + kChunkBits - 1) / kChunkBits;
+    if (t->nchunks < 1) t->nchunks = 1;
+    for (int c = 0; c < kMaxChunks; ++c) t->Mc[c] = (double)M.bits(c * kChunkBits, kChunkBits);
+    for (int j = 0; j < nmod; ++j) {
+        Big W;
+        int g, h;
+        folded_weights(nmod, j, M, &W, &g, &h);
+        Big Gr = W, Gi = W;
+        Gr.mul_small((uint32_t)std::abs(g));
+        Gi.mul_small((uint32_t)std::abs(h));
+        for (int c = 0; c < kMaxChunks; ++c) {
+            t->gr[j][c] = (g < 0 ? -1.0 : 1.0) * (double)Gr.bits(c * kChunkBits, kChunkBits);
+            t->gi[j][c] = (h < 0 ? -1.0 : 1.0) * (double)Gi.bits(c * kChunkBits, kChunkBits);
+        }
+        t->rho_r[j] = (double)g / (double)kModuli[j];
+        t->rho_i[j] = (double)h / (double)kModuli[j];
+    }
+}
+
+void build_crt_table_int(int nmod, CrtTableInt* t) {
+    std::memset(t, 0, sizeof(*t));
+    t->nmod = nmod;
+    const Big M = product_of(nmod);
+    t->M = (int64_t)M.bits(0, 63);
+    for (int j = 0; j < nmod; ++j) {
+        Big W;
+        int g, h;
+        folded_weights(nmod, j, M, &W, &g, &h);
+        t->W[j] = (int64_t)W.bits(0, 63);
+        t->gr[j] = g;
+        t->gi[j] = h;
+        t->m[j] = kModuli[j];
+    }
+}
+
+// Scaling budget: P_t = floor(log2((M-1)/2)) split between rows of A and columns of B; c_k = ceil(log2(2k)/2).
+ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
+    Big half = product_of(nmod);
+    half.sub_one();
+    half.shr1();
+    ScaleTargets s;
+    s.Pt = half.bit_length() - 1;
+    s.PA = (s.Pt + 1) / 2;
+    s.PB = s.Pt / 2;
+    if (herk) s.PA = s.PB = s.Pt / 2;
+    s.ck = 0;
+    const int64_t kk = k > 0 ? k : 1;
+    while ((1ull << (2 * s.ck)) < (uint64_t)(2 * kk)) ++s.ck;
+    return s;
+}
+
+int64_t gemm_k_limit(int nmod) {
+    (void)nmod;
+    const int64_t h = (kModuli[0] - 1) / 2;   // the largest modulus comes first
+    return (int64_t)INT32_MAX / (h * h);
+}
+
+}  // namespace gemm2m

@@ -1,0 +1,255 @@
+"""GPU parity tests: the CUDA path, called through the C-ABI, against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import direct, staged
+from paper_2609_05419_b200 import binding as b
+from paper_2609_05419_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import Workspace, empty_dev, to_dev, to_host, ulp_distance  # noqa: E402
+
+TOL_Z = 1e-14      # complex128: max |C - Cref| / (|A||B|)
+TOL_C = 2e-6       # complex64
+
+
+@pytest.fixture(autouse=True)
+def _default_kernel():
+    b.debug_set_gemm_kernel(0)
+    yield
+    b.debug_set_gemm_kernel(0)
+
+
+def run_int(Ar, Ai, Br, Bi, nmod, kernel=0, ldc=None):
+    m, k = Ar.shape
+    n = Br.shape[1]
+    b.debug_set_gemm_kernel(kernel)
+    with Workspace(b.workspace_bytes(b.OP_GAUSSIAN_INT, m, n, k, nmod)) as ws:
+        Cr = empty_dev(m, n, torch.int64, ld=ldc, fill=-7)
+        Ci = empty_dev(m, n, torch.int64, ld=ldc, fill=-7)
+        b.gemm2m_gaussian_int(to_dev(Ar), to_dev(Ai), to_dev(Br), to_dev(Bi), Cr, Ci, nmod)
+        b.device_status()
+        st = ws.stages(b.OP_GAUSSIAN_INT, m, n, k, nmod)
+        return to_host(Cr), to_host(Ci), st
+
+
+def check_stages_int(st, ref, m, n, k, nmod):
+    for j in range(nmod):
+        for sgn in range(2):
+            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all(), ("Apm", sgn, j)
+            assert (st["Bpm"][sgn, j, :, :k] == ref["Bpm"][j][sgn].T).all(), ("Bpm", sgn, j)
+            assert (st["Apm"][sgn, j, :, k:] == 0).all() and (st["Bpm"][sgn, j, :, k:] == 0).all()
+            assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j)
+
+
+@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])   # check kernel first: isolates pre/post from the tensor-core GEMM
+@pytest.mark.parametrize("shape,nmod", [((128, 128, 128), 3), ((128, 128, 128), 1), ((128, 128, 128), 2),
+                                        ((130, 77, 300), 3), ((1, 1, 1), 1), ((257, 513, 129), 4), ((5, 300, 1000), 8)])
+def test_gaussian_int_bit_exact(shape, nmod, kernel):
+    m, n, k = shape
+    full = nmod == 8
+    Ar, Ai, Br, Bi = inputs.gaussian_int_inputs(m, n, k, seed=1 + nmod, lo=-128 if full else -16, hi=127 if full else 16)
+    Cr, Ci, st = run_int(Ar, Ai, Br, Bi, nmod, kernel)
+    M = staged.product(staged.greedy_2m_moduli()[:nmod])
+    er, ei = direct.gauss4m_mod(Ar, Ai, Br, Bi, M)
+    ref = staged.gemm2m_int_staged(Ar, Ai, Br, Bi, nmod)
+    check_stages_int(st, ref, m, n, k, nmod)
+    assert (Cr == er).all() and (Ci == ei).all()
+
+
+def test_gaussian_int_padded_leading_dimensions_and_untouched_padding():
+    m, n, k = 70, 45, 200
+    Ar, Ai, Br, Bi = inputs.gaussian_int_inputs(m, n, k, seed=21)
+    pad = lambda a, ld: np.asfortranarray(np.vstack([a, np.full((ld - a.shape[0], a.shape[1]), 99, dtype=a.dtype)]))
+    with Workspace(b.workspace_bytes(b.OP_GAUSSIAN_INT, m, n, k, 3)):
+        dAr, dAi = to_dev(pad(Ar, 80))[:m], to_dev(pad(Ai, 80))[:m]
+        dBr, dBi = to_dev(pad(Br, 256))[:k], to_dev(pad(Bi, 256))[:k]
+        Crf = empty_dev(96, n, torch.int64, fill=-7)
+        Cif = empty_dev(96, n, torch.int64, fill=-7)
+        b.gemm2m_gaussian_int(dAr, dAi, dBr, dBi, Crf[:m], Cif[:m], 3)
+        b.device_status()
+        Cr, Ci = to_host(Crf), to_host(Cif)
+    er, ei = direct.gauss4m_mod(Ar, Ai, Br, Bi, staged.product(staged.greedy_2m_moduli()[:3]))
+    assert (Cr[:m] == er).all() and (Ci[:m] == ei).all()
+    assert (Cr[m:] == -7).all() and (Ci[m:] == -7).all()
+
+
+def test_gaussian_int_k_split_beyond_int32_range():
+    # k ((241-1)/2)^2 > 2^31: the GEMM must split K and add residues; extreme entries make the overflow real
+    m, n, k = 40, 24, 150000 + 77
+    Ar = np.asfortranarray(np.full((m, k), 120, dtype=np.int8))
+    Ai = np.asfortranarray(np.zeros((m, k), dtype=np.int8))
+    Br = np.asfortranarray(np.full((k, n), 120, dtype=np.int8))
+    Bi = np.asfortranarray(np.zeros((k, n), dtype=np.int8))
+    rng = np.random.default_rng(5)
+    Ar[:, ::7] = rng.integers(-128, 128, size=Ar[:, ::7].shape)
+    Bi[::5, :] = rng.integers(-128, 128, size=Bi[::5, :].shape)
+    M = staged.product(staged.greedy_2m_moduli()[:6])
+    er, ei = direct.gauss4m_mod(Ar, Ai, Br, Bi, M)
+    for kernel in (1, 0):
+        Cr, Ci, _ = run_int(Ar, Ai, Br, Bi, 6, kernel)
+        assert (Cr == er).all() and (Ci == ei).all(), kernel
+
+
+def run_z(A, B, nmod, kernel=0, cplx=torch.complex128, op=None):
+    m, k = A.shape
+    n = B.shape[1]
+    op = op or (b.OP_ZGEMM if cplx == torch.complex128 else b.OP_CGEMM)
+    b.debug_set_gemm_kernel(kernel)
+    with Workspace(b.workspace_bytes(op, m, n, k, nmod)) as ws:
+        C = empty_dev(m, n, cplx)
+        (b.zgemm2m if op == b.OP_ZGEMM else b.cgemm2m)(to_dev(A), to_dev(B), C, nmod)
+        b.device_status()
+        st = ws.stages(op, m, n, k, nmod) if m * n * k else None
+        return to_host(C), st
+
+
+@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])
+@pytest.mark.parametrize("shape,nmod,dist", [((200, 150, 300), 16, "phi"), ((129, 257, 128), 14, "uniform"),
+                                             ((64, 64, 64), 3, "uniform"), ((33, 19, 50), 22, "phi"), ((40, 40, 520), 20, "uniform")])
+def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
+    m, n, k = shape
+    A, B = inputs.complex_inputs(m, n, k, seed=7, dist=dist, phi=1.0)
+    C, st = run_z(A, B, nmod, kernel)
+    ref = staged.zgemm2m_staged(A, B, nmod)
+    assert (st["eA"] == ref["eA"]).all() and (st["eB"] == ref["eB"]).all()          # step 2: integer rule, bit-exact
+    for j in range(nmod):
+        for sgn in range(2):
+            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all(), ("Apm", sgn, j)       # steps 3-4, Eq. (2a)
+            assert (st["Bpm"][sgn, j, :, :k] == ref["Bpm"][j][sgn].T).all(), ("Bpm", sgn, j)
+            assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j)     # Eq. (2b)
+    # steps 5-7: at most one unit in the last place from the exactly rounded value (identical except near ties)
+    assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
+    assert (C == ref["C"]).mean() > 0.999
+    Cref, D = direct.zgemm4m_dd(A, B)
+    if nmod >= 16:
+        assert direct.componentwise_error(C, Cref, D) <= TOL_Z
+
+
+@pytest.mark.parametrize("nmod,tol", [(16, TOL_Z), (15, TOL_Z), (14, 1e-13)])
+def test_zgemm_1024_full_oracle(nmod, tol):
+    A, B = inputs.complex_inputs(1024, 1024, 1024, seed=1)
+    C, _ = run_z(A, B, nmod)
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(C, Cref, D) <= tol
+
+
+def test_zgemm_ragged_and_padded():
+    m, n, k = 333, 130, 257
+    A, B = inputs.complex_inputs(m, n, k, seed=3, dist="phi", phi=2.0)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, 18)):
+        Af = to_dev(np.asfortranarray(np.vstack([A, np.full((7, k), np.nan)])))
+        Bf = to_dev(np.asfortranarray(np.vstack([B, np.full((3, n), np.inf)])))
+        Cf = empty_dev(m + 5, n, torch.complex128, fill=-3.0)
+        b.zgemm2m(Af[:m], Bf[:k], Cf[:m], 18)
+        b.device_status()
+        C = to_host(Cf)
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(C[:m], Cref, D) <= TOL_Z
+    assert (C[m:] == -3.0).all()
+
+
+def test_zgemm_degenerate_inputs():
+    m, n, k = 70, 50, 90
+    A, B = inputs.complex_inputs(m, n, k, seed=4)
+    B *= 2.0 ** 200                   # keeps the products of the subnormal row in the normal range
+    A[5, :] = 0                       # zero row -> zero row of C
+    B[:, 7] = 0
+    A[9, 3] = np.inf                  # non-finite -> NaN row / column, nothing else disturbed
+    B[11, 2] = np.nan
+    A[20, :] *= 2.0 ** -1040          # subnormal row
+    B[:, 30] *= 2.0 ** 700            # huge column
+    C, st = run_z(A, B, 16)
+    assert (C[5, np.arange(n) != 2] == 0).all() and (C[np.arange(m) != 9, 7] == 0).all()
+    assert np.isnan(C[9, :]).all() and np.isnan(C[:, 2]).all()
+    ok_r = np.array([i for i in range(m) if i != 9])
+    ok_c = np.array([j for j in range(n) if j != 2])
+    A2, B2 = A[ok_r, :], B[:, ok_c]
+    Cref, D = direct.zgemm4m_dd(A2, B2)
+    assert direct.componentwise_error(C[np.ix_(ok_r, ok_c)], Cref, D) <= TOL_Z
+    ref = staged.zgemm2m_staged(A2, B2, 16, upto="pre")
+    assert (st["eA"][ok_r] == ref["eA"]).all() and (st["eB"][ok_c] == ref["eB"]).all()
+
+
+def test_empty_dimensions():
+    A, B = inputs.complex_inputs(6, 5, 4, seed=5)
+    with Workspace(4096):
+        C = empty_dev(6, 5, torch.complex128, fill=9.0)
+        b.zgemm2m(to_dev(A)[:, :0], to_dev(B)[:0, :], C, 16)        # k = 0: C = 0
+        assert (to_host(C) == 0).all()
+        b.zgemm2m(to_dev(A)[:0, :], to_dev(B), empty_dev(0, 5, torch.complex128), 16)   # m = 0: no-op
+        b.zherk2m(to_dev(A)[:0, :], empty_dev(0, 0, torch.complex128), 16)
+        b.device_status()
+
+
+def test_workspace_too_small_is_refused():
+    A, B = inputs.complex_inputs(64, 64, 64, seed=5)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, 64, 64, 64, 16) - 256):
+        with pytest.raises(b.Gemm2mError, match="WORKSPACE"):
+            b.zgemm2m(to_dev(A), to_dev(B), empty_dev(64, 64, torch.complex128), 16)
+    b.set_workspace(None)
+    with pytest.raises(b.Gemm2mError, match="WORKSPACE"):
+        b.zgemm2m(to_dev(A), to_dev(B), empty_dev(64, 64, torch.complex128), 16)
+
+
+@pytest.mark.parametrize("shape,nmod", [((100, 90, 150), 7), ((257, 300, 1000), 7), ((64, 64, 64), 22), ((128, 128, 256), 9)])
+def test_cgemm_parity(shape, nmod):
+    m, n, k = shape
+    A, B = inputs.complex_inputs(m, n, k, seed=8, dtype=np.complex64)
+    C, st = run_z(A, B, nmod, cplx=torch.complex64)
+    assert C.dtype == np.complex64
+    ref = staged.zgemm2m_staged(A, B, nmod, out_bits=24)
+    assert (st["eA"] == ref["eA"]).all() and (st["eB"] == ref["eB"]).all()
+    for j in range(nmod):
+        for sgn in range(2):
+            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all()
+            assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all()
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(C, Cref, D) <= TOL_C
+    # double rounding (53 then 24 bits) may differ from the single rounding by one float ulp
+    spacing = np.spacing(np.abs(ref["C"].real).astype(np.float32)).astype(np.float64)
+    assert (np.abs(C.real.astype(np.float64) - ref["C"].real) <= spacing).all()
+
+
+@pytest.mark.parametrize("n,k,nmod", [(96, 200, 16), (257, 129, 16), (130, 300, 17), (64, 64, 21)])
+def test_zherk_parity(n, k, nmod):
+    A = inputs.herk_input(n, k, seed=9)
+    with Workspace(max(b.workspace_bytes(b.OP_ZHERK, n, n, k, nmod), b.workspace_bytes(b.OP_ZGEMM, n, n, k, nmod))) as ws:
+        C = empty_dev(n, n, torch.complex128, fill=-5.0)
+        b.zherk2m(to_dev(A), C, nmod)
+        b.device_status()
+        st = ws.stages(b.OP_ZHERK, n, n, k, nmod)
+        Ch = to_host(C)
+        Cg = empty_dev(n, n, torch.complex128)
+        b.zgemm2m(to_dev(A), to_dev(np.asfortranarray(A.conj().T)), Cg, nmod)
+        b.device_status()
+        Cg = to_host(Cg)
+    ref = staged.zgemm2m_staged(A, np.asfortranarray(A.conj().T), nmod, herk=True)
+    assert (st["eA"] == ref["eA"]).all()
+    for j in range(nmod):
+        assert (st["Cpm"][0, j, :, :n] == ref["Cpm"][j][0].T).all()          # C+ = A+ A-^T (Section 5)
+    low = np.tril(np.ones((n, n), dtype=bool))
+    assert (Ch[~low] == -5.0).all()                                           # strict upper triangle untouched
+    assert (np.diag(Ch).imag == 0).all()
+    Cref, D = direct.zgemm4m_dd(A, np.asfortranarray(A.conj().T))
+    assert direct.componentwise_error(Ch[low], Cref[low], D[low]) <= TOL_Z
+    assert ulp_distance(Ch[low].real, ref["C"][low].real).max() <= 1 and ulp_distance(Ch[low].imag, ref["C"][low].imag).max() <= 1
+    if ref["Pt"] % 2 == 0:                                                    # same scale split: identical integers, identical bits
+        assert (Ch[low] == Cg[low]).all()
+
+
+def test_device_status_and_launch_counts():
+    A, B = inputs.complex_inputs(256, 256, 256, seed=2)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, 256, 256, 256, 16)):
+        b.set_profiling(True)
+        try:
+            b.zgemm2m(to_dev(A), to_dev(B), empty_dev(256, 256, torch.complex128), 16)
+            b.device_status()
+            ms, calls = b.phase_ms()
+            total, per = b.last_launch_count()
+        finally:
+            b.set_profiling(False)
+    assert calls == 1 and all(x >= 0 for x in ms) and sum(ms) > 0
+    assert per == [4, 2, 1, 1] and total == 8
