@@ -124,7 +124,11 @@ class ClockSampler:
             os.close(fd)
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.out, stderr=subprocess.DEVNULL)
+            t0 = time.time()                     # wait for the first sample so that the timed region is covered
+            while time.time() - t0 < 5.0 and os.path.getsize(self.path) == 0:
+                self.out.flush()
+                time.sleep(0.02)
         except Exception:
             self.proc = None
 
