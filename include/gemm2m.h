@@ -88,6 +88,25 @@ int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const 
  * diagonal is written; diagonal imaginary parts are exactly 0; the strict upper triangle is not touched. */
 int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream);
 
+/* (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
+ * Scale exponents without any allocation.  Some programs that would like to use this library are not allowed to
+ * allocate device memory at the point of the call: a plug-in running inside a host application that handed the whole
+ * GPU to its own memory pool at start-up, a service with a fixed memory budget that forbids cudaMalloc after
+ * initialisation, or code on a latency-critical path where an allocation's implicit synchronisation is unacceptable.
+ * They cannot provide the workspace the other entry points need.  This call computes, for the rows of A (m x k
+ * complex128, column-major, lda >= m, device pointer), exactly the scale exponents e_i (sigma_i = 2^e_i, Algorithm 1
+ * step 2) that zgemm2m(m, *, k, ..., nmod) uses, and writes them to e (int32[m], device pointer), using a scratch array
+ * that is built into the library instead of a workspace.  It calls no cudaMalloc/cudaFree and no allocating library.
+ *   - At most GEMM2M_STATIC_MAX_ROWS rows; more returns GEMM2M_ERR_WORKSPACE and launches nothing.
+ *   - The built-in scratch (8 bytes per row of the maximum, 512 KB) is held by every GPU that loads the library until the
+ *     process exits, is shared by all calls and keeps the last call's contents; the call clears what it uses.  Two calls
+ *     that overlap on the same GPU (different streams) race on it: order them.
+ *   - The first call on each device looks up the scratch's device address (with that device current).  Make that first
+ *     call before starting any stream capture.
+ *   - gemm2m_last_cuda_error is not updated by this entry point. */
+#define GEMM2M_STATIC_MAX_ROWS 65536
+int gemm2m_zscale_exponents_static(int64_t m, int64_t k, const double* A, int64_t lda, int nmod, int32_t* e, void* stream);
+
 /* Waits for `stream` and returns GEMM2M_ERR_DEVICE_TIMEOUT if a kernel of an earlier call on the registered
  * workspace gave up a bounded wait (its results are then invalid), GEMM2M_ERR_CUDA on a CUDA error, else OK. */
 int gemm2m_device_status(void* stream);

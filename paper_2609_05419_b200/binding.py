@@ -55,6 +55,7 @@ def lib():
     L.cgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.zherk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
     L.gemm2m_device_status.argtypes = [vp]
+    L.gemm2m_zscale_exponents_static.argtypes = [i64, i64, vp, i64, i32, vp, vp]
     L.gemm2m_set_profiling.argtypes = [i32]
     L.gemm2m_phase_ms.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     L.gemm2m_last_launch_count.argtypes = [ctypes.POINTER(i32)]
@@ -157,6 +158,22 @@ def zherk2m(A, C, nmod=16, stream=None):
     if (n1, n2) != (n, n):
         raise ValueError("shape mismatch")
     _check(lib().zherk2m(n, k, pa, lda, pc, ldc, nmod, _stream_ptr(stream)), "zherk2m")
+
+
+STATIC_MAX_ROWS = 65536
+
+
+def zscale_exponents_static(A, e, nmod=16, stream=None):
+    """Scale exponents of the rows of A (the ones zgemm2m uses for `nmod` moduli) into the int32 CUDA tensor `e`, for
+    callers that may not allocate device memory: the library's built-in scratch replaces the workspace.  At most
+    STATIC_MAX_ROWS rows; calls on one GPU must not overlap."""
+    pa, m, k, lda = _colmajor(A, "A")
+    if m > STATIC_MAX_ROWS:
+        raise ValueError(f"zscale_exponents_static: {m} rows exceed the built-in scratch ({STATIC_MAX_ROWS} rows)")
+    if e.numel() != m or not e.is_cuda or e.element_size() != 4 or not e.is_contiguous():
+        raise ValueError("e: need a contiguous int32 CUDA tensor with one entry per row of A")
+    _check(lib().gemm2m_zscale_exponents_static(m, k, pa, lda, nmod, ctypes.c_void_p(e.data_ptr()), _stream_ptr(stream)),
+           "gemm2m_zscale_exponents_static")
 
 
 def device_status(stream=None):
