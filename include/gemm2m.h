@@ -137,8 +137,9 @@ typedef struct {
 } gemm2m_layout;
 int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, gemm2m_layout* out);
 
-/* Which int8 GEMM kernel later calls use: 0 = the tcgen05 kernel (default), 1 = a plain CUDA-core check kernel kept
- * only so that tests can tell a fault in the tensor-core kernel from one in the pre/post kernels. */
+/* Which int8 GEMM kernel later calls use: 0 = the tcgen05 kernel on CTA pairs (default), 1 = a plain CUDA-core check
+ * kernel kept only so that tests can tell a fault in a tensor-core kernel from one in the pre/post kernels, 2 = the
+ * tcgen05 kernel with one CTA per tile. */
 int gemm2m_debug_set_gemm_kernel(int which);
 
 /* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host

@@ -22,7 +22,7 @@ struct State {
     int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
     cudaEvent_t* cur = nullptr;   // event set of the call being enqueued
     int launches[4] = {0, 0, 0, 0};
-    int gemm_kernel = 0;          // 0 = tcgen05, 1 = check kernel
+    int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
     int sm_count = 0;
     int arch_ok = -1;
 };
@@ -108,7 +108,8 @@ constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kern
 int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
     const int64_t klim = gemm_k_limit(nmod);
     if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
-    else CK(launch_gemm_tcgen05(a, klim, g.sm_count, st, &g.launches[2]));
+    else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(a, klim, g.sm_count, st, &g.launches[2]));
+    else CK(launch_gemm_tcgen05_pair(a, klim, g.sm_count, st, &g.launches[2]));
     return GEMM2M_OK;
 }
 
@@ -401,7 +402,7 @@ int gemm2m_last_launch_count(int per_phase[4]) {
 
 int gemm2m_debug_set_gemm_kernel(int which) {
     std::lock_guard<std::mutex> lock(g.mu);
-    if (which != 0 && which != 1) return GEMM2M_ERR_ARG;
+    if (which < 0 || which > 2) return GEMM2M_ERR_ARG;
     g.gemm_kernel = which;
     return GEMM2M_OK;
 }

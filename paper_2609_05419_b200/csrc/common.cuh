@@ -42,12 +42,13 @@ struct ModTable {
 //   X_r = sum_j (c-_j + c+_j) Gr_j  (mod M),  Gr_j = sym(2^-1 q_j mod m_j) (M/m_j)
 //   X_i = sum_j (c-_j - c+_j) Gi_j  (mod M),  Gi_j = sym(s_j 2^-1 q_j mod m_j) (M/m_j)
 // with q_j = (M/m_j)^-1 mod m_j.  Each weight is stored as signed base-2^40 digits held in doubles, so
-// that every digit-column sum is an exact integer below 2^53; rho = G/M estimates the multiple of M to remove.
+// that every digit-column sum is an exact integer below 2^53.  The multiple of M to remove is estimated from the
+// two leading digit-column sums: t = rint(S_top q_hi + S_(top-1) q_lo), q_hi = 2^(40 top)/M, q_lo = q_hi 2^-40.
 struct CrtTable {
     double gr[kMaxMod][kMaxChunks];
     double gi[kMaxMod][kMaxChunks];
-    double rho_r[kMaxMod], rho_i[kMaxMod];
     double Mc[kMaxChunks];                     // digits of M
+    double q_hi, q_lo;
     int nmod, nchunks;
 };
 
@@ -104,7 +105,8 @@ struct GemmArgs {
     ModTable mods;
     int* dev_status;
 };
-cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);
+cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);        // one CTA per tile
+cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);   // CTA pairs (default)
 cudaError_t launch_gemm_check(const GemmArgs& a, int64_t k_limit, cudaStream_t st, int* launches);
 
 }  // namespace gemm2m

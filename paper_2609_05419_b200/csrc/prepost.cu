@@ -125,13 +125,10 @@ cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int c
 
 // =====================================================================================================
 // Steps 3 + 4 (Eq. 2a): quantise by truncation and emit the symmetric int8 residues A+ / A- for every
-// modulus, K contiguous.  A block stages a tile of 32 operand rows x 128 k of quantised parts in shared
-// memory (coalesced global reads in either orientation), then each thread owns 16 consecutive k of one row
-// and writes 16-byte vectors into every plane.
+// modulus, K contiguous.  Tiles of operand rows x 128 k are staged in shared memory (coalesced global
+// reads in either orientation), then each thread owns a run of consecutive k of one row and writes
+// vectors into every plane.
 // =====================================================================================================
-constexpr int kResRows = 32, kResK = 128, kResThreads = 256;
-constexpr int kResRowStride = kResK + kResK / 16 + 1;   // in 16-byte elements: one pad per 16 + odd row stride -> no bank conflicts
-
 struct QPair { long long re, im; };   // quantised parts, two's complement
 
 // trunc(v 2^-e) for a finite v given by its bit pattern.
@@ -179,6 +176,19 @@ __device__ __forceinline__ int sym_reduce_small(int x, int m, float inv_m) {
     return x - q * m;
 }
 
+// The same for the pair (Rv + Iv, Rv - Iv); the two symmetric residues come back in the low bytes of bp / bm (two's
+// complement).  y = 1.5 2^23 + x holds x exactly in its mantissa; after q = rint(x/m), fma(-q, m, y) = 1.5 2^23 + (x - q m)
+// is exact and its low mantissa byte is the residue.  Plain FP32 adds and FMAs: they issue to both FMA pipes, whereas the
+// packed two-lane forms and integer multiply-adds only use one of them, which the dp4a's already keep busy.
+__device__ __forceinline__ void sym_reduce_pm(int Rv, int Iv, float neg_m, float inv_m, uint32_t* bp, uint32_t* bm) {
+    const float magic = 12582912.0f;
+    const float yp = __int_as_float(Rv + Iv + 0x4B400000), ym = __int_as_float(Rv - Iv + 0x4B400000);
+    const float qp = fmaf(yp - magic, inv_m, magic) - magic;
+    const float qm = fmaf(ym - magic, inv_m, magic) - magic;
+    *bp = __float_as_uint(fmaf(qp, neg_m, yp));
+    *bm = __float_as_uint(fmaf(qm, neg_m, ym));
+}
+
 struct Digits { uint32_t lo, hi; };   // 4 unsigned low bytes; 4 balanced (signed) high digits
 __device__ __forceinline__ Digits split_digits(long long x) {
     Digits d;
@@ -188,53 +198,22 @@ __device__ __forceinline__ Digits split_digits(long long x) {
     return d;
 }
 
-// Stage one 32 x 128 tile of quantised parts into shared memory.  fetch(r, kk) returns the quantised pair.
-template <typename Fetch>
-__device__ __forceinline__ void stage_tile(QPair* tile, bool k_contiguous, Fetch fetch) {
-    const int t = threadIdx.x;
-    if (!k_contiguous) {          // consecutive threads -> consecutive operand rows (column-major A)
-        const int r = t & 31;
-        for (int kk = t >> 5; kk < kResK; kk += kResThreads / 32) tile[r * kResRowStride + kk + (kk >> 4)] = fetch(r, kk);
-    } else {                      // consecutive threads -> consecutive k (columns of B are contiguous)
-        const int kk = t & (kResK - 1);
-        for (int r = t >> 7; r < kResRows; r += kResThreads / kResK) tile[r * kResRowStride + kk + (kk >> 4)] = fetch(r, kk);
-    }
-}
-
-// From the staged tile: thread (row = t / 8, group g = t % 8) owns k = 16 g .. 16 g + 15 and writes both sign planes
-// of every modulus.  planes: [2 nmod][R][Kp].
-template <bool WIDE>
-__device__ __forceinline__ void emit_residues(const QPair* tile, const ResidueTable& tab, int8_t* planes, int64_t R, int64_t Kp,
-                                              int64_t row0, int64_t k0) {
-    const int t = threadIdx.x;
-    const int g = t & 7, r = t >> 3;
-    Digits dr[16], di[16];
-    uint32_t tsh[WIDE ? 16 : 1];   // wide mode: left shifts t_r | t_i << 8 of the two mantissas
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const QPair q = tile[r * kResRowStride + 16 * g + i + g];
-        if (WIDE) {
-            tsh[i] = (uint32_t)(q.re & 0xFF) | ((uint32_t)(q.im & 0xFF) << 8);
-            dr[i] = split_digits(q.re >> 8);
-            di[i] = split_digits(q.im >> 8);
-        } else {
-            dr[i] = split_digits(q.re);
-            di[i] = split_digits(q.im);
-        }
-    }
-    const int64_t row = row0 + r;
-    if (row >= R) return;
-    const int64_t plane_stride = R * Kp;
-    int8_t* dst = planes + row * Kp + k0 + 16 * g;
+// Residues of NE consecutive elements of one operand row for every modulus, written as NE-byte vectors into both sign
+// planes.  dst points at plane 0, this row, first k of the run; tsh (wide mode) holds the mantissa shifts t_r | t_i << 8.
+template <int NE, bool WIDE>
+__device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tsh, const ResidueTable& tab,
+                                         int8_t* dst, int64_t plane_stride) {
+    static_assert(NE == 8 || NE == 16, "runs of 8 or 16 elements");
     const int nmod = tab.nmod;
+#pragma unroll 1
     for (int j = 0; j < nmod; ++j) {
         const int m = tab.m[j];
-        const float inv_m = tab.inv_m[j];
+        const float inv_m = tab.inv_m[j], neg_m = -(float)m;
         const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
-        uint32_t pw[4], mw[4];
+        uint32_t pw[NE / 4], mw[NE / 4];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            uint32_t pp = 0, mm = 0;
+        for (int w = 0; w < NE / 4; ++w) {
+            uint32_t bp[4], bm[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const int i = 4 * w + b;
@@ -244,51 +223,169 @@ __device__ __forceinline__ void emit_residues(const QPair* tile, const ResidueTa
                     Rv = sym_reduce_small(Rv, m, inv_m) * (int)tab.pow2[j][tsh[i] & 0xFF];
                     Iv = sym_reduce_small(Iv, m, inv_m) * (int)tab.pow2[j][tsh[i] >> 8];
                 }
-                const int ap = sym_reduce_small(Rv + Iv, m, inv_m);               // Eq. (2a), "+"
-                const int am = sym_reduce_small(Rv - Iv, m, inv_m);               // Eq. (2a), "-"
-                pp |= ((uint32_t)ap & 0xFFu) << (8 * b);
-                mm |= ((uint32_t)am & 0xFFu) << (8 * b);
+                sym_reduce_pm(Rv, Iv, neg_m, inv_m, &bp[b], &bm[b]);        // Eq. (2a): "+" and "-"
             }
-            pw[w] = pp;
-            mw[w] = mm;
+            pw[w] = __byte_perm(__byte_perm(bp[0], bp[1], 0x0040), __byte_perm(bp[2], bp[3], 0x0040), 0x5410);
+            mw[w] = __byte_perm(__byte_perm(bm[0], bm[1], 0x0040), __byte_perm(bm[2], bm[3], 0x0040), 0x5410);
         }
-        *reinterpret_cast<uint4*>(dst + (int64_t)j * plane_stride) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-        *reinterpret_cast<uint4*>(dst + (int64_t)(nmod + j) * plane_stride) = make_uint4(mw[0], mw[1], mw[2], mw[3]);
+        int8_t* dp = dst + (int64_t)j * plane_stride;
+        int8_t* dm = dst + (int64_t)(nmod + j) * plane_stride;
+        if (NE == 16) {
+            *reinterpret_cast<uint4*>(dp) = make_uint4(pw[0], pw[1], pw[2 % (NE / 4)], pw[3 % (NE / 4)]);
+            *reinterpret_cast<uint4*>(dm) = make_uint4(mw[0], mw[1], mw[2 % (NE / 4)], mw[3 % (NE / 4)]);
+        } else {
+            *reinterpret_cast<uint2*>(dp) = make_uint2(pw[0], pw[1]);
+            *reinterpret_cast<uint2*>(dm) = make_uint2(mw[0], mw[1]);
+        }
     }
 }
 
+// ---- floating-point inputs: persistent blocks, raw elements copied asynchronously into a two-stage ring -------------
+constexpr int kResRows = 16, kResK = 128, kResThreads = 256, kResRun = 8;
+constexpr int kResRowStride = kResK + kResK / kResRun + 1;   // in elements: one pad per run of 8 + odd row stride -> no bank conflicts
+constexpr int kResStages = 2;
+
+template <typename T> struct RawCplx;
+template <> struct RawCplx<double> { using type = double2; };
+template <> struct RawCplx<float> { using type = float2; };
+
+template <int BYTES>
+__device__ __forceinline__ void cp_async_zfill(void* smem_dst, const void* gmem_src, bool valid) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const int src_bytes = valid ? BYTES : 0;   // 0 source bytes: the destination is filled with zeros
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"(d), "l"(gmem_src), "n"(BYTES), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <typename T, bool WIDE>
-__global__ void __launch_bounds__(kResThreads) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
-                                                                  int64_t Kp, const int32_t* __restrict__ e, const __grid_constant__ ResidueTable tab,
-                                                                  int8_t* __restrict__ planes) {
+__global__ void __launch_bounds__(kResThreads, 3) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
+                                                                     int64_t Kp, const int32_t* __restrict__ e,
+                                                                     const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
+    using Raw = typename RawCplx<T>::type;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    QPair* tile = reinterpret_cast<QPair*>(smem_raw);
-    const int64_t row0 = (int64_t)blockIdx.y * kResRows, k0 = (int64_t)blockIdx.x * kResK;
-    stage_tile(tile, k_contiguous, [&](int r, int kk) -> QPair {
-        const int64_t row = row0 + r, k = k0 + kk;
-        QPair q{0, 0};
-        if (row < R && k < K) {
-            const int ex = __ldg(e + row);
-            if (ex != kExpNonFinite) {
-                const T* p = k_contiguous ? X + 2 * (k + row * ld) : X + 2 * (row + k * ld);
-                const Cplx<T> v = load_cplx<T>(p);
-                q.re = quantise_part<T, WIDE>(v.re, ex);
-                q.im = quantise_part<T, WIDE>(v.im, ex);
+    Raw* ring = reinterpret_cast<Raw*>(smem_raw);
+    constexpr int kStageElems = kResRows * kResRowStride;
+    const int t = threadIdx.x;
+    const int64_t ktiles = Kp / kResK;
+    const int64_t total = ((R + kResRows - 1) / kResRows) * ktiles;
+    const int64_t plane_stride = R * Kp;
+
+    auto issue = [&](int64_t tile, int stage) {
+        const int64_t row0 = (tile / ktiles) * kResRows, k0 = (tile % ktiles) * kResK;
+        Raw* dst = ring + stage * kStageElems;
+        if (!k_contiguous) {          // consecutive threads -> consecutive operand rows (rows of a column-major matrix)
+            const int r = t & (kResRows - 1);
+            const int64_t row = row0 + r;
+#pragma unroll
+            for (int kk = t / kResRows; kk < kResK; kk += kResThreads / kResRows) {
+                const int64_t k = k0 + kk;
+                const bool ok = row < R && k < K;
+                cp_async_zfill<sizeof(Raw)>(dst + r * kResRowStride + kk + (kk >> 3), ok ? X + 2 * (row + k * ld) : X, ok);
+            }
+        } else {                      // consecutive threads -> consecutive k (columns of the matrix are contiguous)
+            const int kk = t & (kResK - 1);
+            const int64_t k = k0 + kk;
+#pragma unroll
+            for (int r = t / kResK; r < kResRows; r += kResThreads / kResK) {
+                const int64_t row = row0 + r;
+                const bool ok = row < R && k < K;
+                cp_async_zfill<sizeof(Raw)>(dst + r * kResRowStride + kk + (kk >> 3), ok ? X + 2 * (k + row * ld) : X, ok);
             }
         }
-        return q;
-    });
-    __syncthreads();
-    emit_residues<WIDE>(tile, tab, planes, R, Kp, row0, k0);
+        cp_async_commit();
+    };
+
+    int64_t tile = blockIdx.x;
+    if (tile >= total) return;
+    issue(tile, 0);
+    for (int it = 0; tile < total; tile += gridDim.x, ++it) {
+        const int64_t next = tile + gridDim.x;
+        if (next < total) { issue(next, (it + 1) & 1); cp_async_wait_group<1>(); }
+        else cp_async_wait_group<0>();
+        __syncthreads();
+        const Raw* src = ring + (it & 1) * kStageElems;
+        const int64_t row0 = (tile / ktiles) * kResRows, k0 = (tile % ktiles) * kResK;
+        const int g = t & (kResK / kResRun - 1), r = t / (kResK / kResRun);
+        const int64_t row = row0 + r;
+        if (row < R) {
+            const int ex = __ldg(e + row);
+            // Narrow mode, ordinary exponents: x 2^-e is an exact FP64 product (or underflows towards zero, where the
+            // truncation is zero anyway) and its truncation to int64 is one conversion; |x 2^-e| < 2^62 by the scaling rule.
+            const bool fast = !WIDE && ex > -1000 && ex < 1000;
+            const double scale = __longlong_as_double((long long)(1023 - (fast ? ex : 0)) << 52);
+            Digits dr[kResRun], di[kResRun];
+            uint32_t tsh[WIDE ? kResRun : 1];
+#pragma unroll
+            for (int i = 0; i < kResRun; ++i) {
+                const Raw v = src[r * kResRowStride + kResRun * g + g + i];
+                long long qr = 0, qi = 0;
+                if (fast) {
+                    qr = __double2ll_rz((double)v.x * scale);
+                    qi = __double2ll_rz((double)v.y * scale);
+                } else if (ex != kExpNonFinite) {
+                    qr = quantise_part<T, WIDE>(v.x, ex);
+                    qi = quantise_part<T, WIDE>(v.y, ex);
+                }
+                if (WIDE) {
+                    tsh[i] = (uint32_t)(qr & 0xFF) | ((uint32_t)(qi & 0xFF) << 8);
+                    qr >>= 8;
+                    qi >>= 8;
+                }
+                dr[i] = split_digits(qr);
+                di[i] = split_digits(qi);
+            }
+            emit_run<kResRun, WIDE>(dr, di, tsh, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
+        }
+        __syncthreads();   // everyone is done with this stage before it is refilled
+    }
 }
+
+constexpr size_t kResSmemBytes(size_t elem) { return (size_t)kResStages * kResRows * kResRowStride * elem; }
+
+static int cached_sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
+    return sms;
+}
+
+template <typename T>
+cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
+    if (R <= 0 || Kp <= 0) return cudaSuccess;
+    constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
+    }
+    const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
+    const int64_t resident = (int64_t)cached_sm_count() * 3;
+    const unsigned grid = (unsigned)(total < resident ? total : resident);
+    if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    else residues_fp_kernel<T, false><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// ---- int8 Gaussian-integer inputs (no scaling): one 32 x 128 tile per block, loaded synchronously ---------------------
+constexpr int kResIRows = 32, kResIRun = 16;
+constexpr int kResIRowStride = kResK + kResK / kResIRun + 1;
 
 __global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t* __restrict__ Xr, const int8_t* __restrict__ Xi, int64_t ld,
                                                                     bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                                                     const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     QPair* tile = reinterpret_cast<QPair*>(smem_raw);
-    const int64_t row0 = (int64_t)blockIdx.y * kResRows, k0 = (int64_t)blockIdx.x * kResK;
-    stage_tile(tile, k_contiguous, [&](int r, int kk) -> QPair {
+    const int64_t row0 = (int64_t)blockIdx.y * kResIRows, k0 = (int64_t)blockIdx.x * kResK;
+    const int t = threadIdx.x;
+    auto fetch = [&](int r, int kk) -> QPair {
         const int64_t row = row0 + r, k = k0 + kk;
         QPair q{0, 0};
         if (row < R && k < K) {
@@ -297,42 +394,40 @@ __global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t
             q.im = Xi[idx];
         }
         return q;
-    });
-    __syncthreads();
-    emit_residues<false>(tile, tab, planes, R, Kp, row0, k0);
-}
-
-constexpr size_t kResSmem = (size_t)kResRows * kResRowStride * sizeof(QPair);
-
-template <typename T>
-cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
-    if (R <= 0 || Kp <= 0) return cudaSuccess;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
-        if (err != cudaSuccess) return err;
-        attr_set = true;
+    };
+    if (!k_contiguous) {
+        const int r = t & 31;
+        for (int kk = t >> 5; kk < kResK; kk += kResThreads / 32) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
+    } else {
+        const int kk = t & (kResK - 1);
+        for (int r = t >> 7; r < kResIRows; r += kResThreads / kResK) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
     }
-    dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResRows - 1) / kResRows));
-    if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, kResSmem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
-    else residues_fp_kernel<T, false><<<grid, kResThreads, kResSmem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
-    ++*launches;
-    return cudaGetLastError();
+    __syncthreads();
+    const int g = t & 7, r = t >> 3;
+    Digits dr[kResIRun], di[kResIRun];
+#pragma unroll
+    for (int i = 0; i < kResIRun; ++i) {
+        const QPair q = tile[r * kResIRowStride + kResIRun * g + i + g];
+        dr[i] = split_digits(q.re);
+        di[i] = split_digits(q.im);
+    }
+    const int64_t row = row0 + r;
+    if (row >= R) return;
+    emit_run<kResIRun, false>(dr, di, nullptr, tab, planes + row * Kp + k0 + kResIRun * g, R * Kp);
 }
 
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
+    constexpr size_t smem = (size_t)kResIRows * kResIRowStride * sizeof(QPair);
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(residues_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResSmem);
+        cudaError_t err = cudaFuncSetAttribute(residues_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         attr_set = true;
     }
-    dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResRows - 1) / kResRows));
-    residues_int8_kernel<<<grid, kResThreads, kResSmem, st>>>(Xr, Xi, ld, k_contiguous, R, K, Kp, tab, planes);
+    dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResIRows - 1) / kResIRows));
+    residues_int8_kernel<<<grid, kResThreads, smem, st>>>(Xr, Xi, ld, k_contiguous, R, K, Kp, tab, planes);
     ++*launches;
     return cudaGetLastError();
 }
@@ -346,11 +441,12 @@ __device__ __forceinline__ double int_to_double(int v) {   // exact, avoids the 
     return __hiloint2double(0x43300000, (int)(0x80000000u ^ (uint32_t)v)) - 4503601774854144.0;   // 2^52 + 2^31
 }
 
-// Lifted X (exact integer, |X| <= (M-1)/2) from the digit-column sums S[c] and the quotient estimate qsum ~ X'/M,
-// returned as an unevaluated sum hi + lo with |lo| <= ulp(hi)/2.
+// Lifted X (exact integer, |X| <= (M-1)/2) from the digit-column sums S[c], returned as an unevaluated sum hi + lo with
+// |lo| <= ulp(hi)/2.  The weighted sum X' = sum_c S[c] 2^(40c) is X + t M with |t| < 2^12; |X/M| stays below 0.494 by the
+// scaling rule, so rounding X'/M (from the two leading sums; the rest is below 2^-60 M) gives t exactly.
 template <int NCH>
-__device__ __forceinline__ void crt_finish(double (&S)[NCH], double qsum, const CrtTable& tab, double* hi, double* lo) {
-    const double t = rint(qsum);
+__device__ __forceinline__ void crt_finish(double (&S)[NCH], const CrtTable& tab, double* hi, double* lo) {
+    const double t = rint(NCH > 1 ? fma(S[NCH - 1], tab.q_hi, S[NCH > 1 ? NCH - 2 : 0] * tab.q_lo) : S[0] * tab.q_hi);
 #pragma unroll
     for (int c = 0; c < NCH; ++c) S[c] = fma(-t, tab.Mc[c], S[c]);          // exact: |t| < 2^12, digits < 2^40
     const double two40 = 1099511627776.0, inv40 = 1.0 / 1099511627776.0;
@@ -399,36 +495,51 @@ template <> __device__ __forceinline__ void store4<float>(float* dst, const doub
 }
 
 constexpr int kPostThreads = 128;
+constexpr int kPostSpan = kPostThreads * 4;   // consecutive row indices i handled by one block
 
-// cpm: [2 nmod][n][ldp] int8 (row index i contiguous).  One thread -> 4 consecutive i of one column j.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// cpm: [2 nmod][n][ldp] int8 (row index i contiguous).  A block handles 512 consecutive i of one column j: it first pulls
+// the 2 nmod x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
+// thread combines 4 consecutive i.
 template <typename T, int NCH>
 __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
                                                                const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
                                                                const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc) {
-    const int64_t i0 = ((int64_t)blockIdx.x * kPostThreads + threadIdx.x) * 4;
+    __shared__ __align__(16) uint32_t stage[2 * kMaxMod][kPostThreads];
+    const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
     const int64_t j = blockIdx.y;
-    if (i0 >= m) return;
     const int nmod = tab.nmod;
     const int64_t plane = n * ldp;
-    const int8_t* src = cpm + j * ldp + i0;
-    double Sr[4][NCH], Si[4][NCH], qr[4], qi[4];
+    const int8_t* src = cpm + j * ldp + ib;
+    const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);   // ldp is a multiple of 16
+    for (int idx = threadIdx.x; idx < 2 * nmod * (kPostSpan / 16); idx += kPostThreads) {
+        const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
+        if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    const int64_t i0 = ib + 4 * threadIdx.x;
+    if (i0 >= m) return;
+    double Sr[4][NCH], Si[4][NCH];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        qr[e] = qi[e] = 0.0;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
     }
+#pragma unroll 2
     for (int jm = 0; jm < nmod; ++jm) {
-        const uint32_t wp = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)jm * plane));            // c+ of 4 elements
-        const uint32_t wm = __ldg(reinterpret_cast<const uint32_t*>(src + (int64_t)(nmod + jm) * plane));   // c-
+        const uint32_t wp = stage[jm][threadIdx.x];            // c+ of 4 elements
+        const uint32_t wm = stage[nmod + jm][threadIdx.x];     // c-
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int cp = (int)(int8_t)(wp >> (8 * e));
             const int cm = (int)(int8_t)(wm >> (8 * e));
             const double vr = int_to_double(cm + cp);     // Eq. (2c): real part uses C- + C+
             const double vi = int_to_double(cm - cp);     //           imaginary part uses C- - C+
-            qr[e] = fma(vr, tab.rho_r[jm], qr[e]);
-            qi[e] = fma(vi, tab.rho_i[jm], qi[e]);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
@@ -448,9 +559,9 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
                 re[e] = im[e] = __longlong_as_double(0x7FF8000000000000ll);
             } else {
                 double h, l;
-                crt_finish<NCH>(Sr[e], qr[e], tab, &h, &l);
+                crt_finish<NCH>(Sr[e], tab, &h, &l);
                 re[e] = scale_pow2(h + l, ea + fb);
-                crt_finish<NCH>(Si[e], qi[e], tab, &h, &l);
+                crt_finish<NCH>(Si[e], tab, &h, &l);
                 im[e] = scale_pow2(h + l, ea + fb);
             }
         }
@@ -462,7 +573,7 @@ template <typename T>
 cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const int32_t* eA, const int32_t* eB, const CrtTable& tab,
                            T* C, int64_t ldc, cudaStream_t st, int* launches) {
     if (m <= 0 || n <= 0) return cudaSuccess;
-    const int64_t per_block = (int64_t)kPostThreads * 4;
+    const int64_t per_block = kPostSpan;
     for (int64_t j0 = 0; j0 < n; j0 += 65535) {      // grid.y limit
         const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
         dim3 grid((unsigned)((m + per_block - 1) / per_block), (unsigned)nj);
@@ -505,15 +616,13 @@ __global__ void __launch_bounds__(kHerkTile * 8) post_herk_kernel(const int8_t* 
     for (int cj = ty; cj < kHerkTile; cj += 8) {
         const int64_t i = ibase + tx, j = jbase + cj;
         if (i >= n || j >= n || i < j) continue;
-        double Sr[NCH], Si[NCH], qr = 0.0, qi = 0.0;
+        double Sr[NCH], Si[NCH];
 #pragma unroll
         for (int c = 0; c < NCH; ++c) Sr[c] = Si[c] = 0.0;
         for (int jm = 0; jm < nmod; ++jm) {
             const int cpv = cp[(int64_t)jm * plane + j * ldp + i];   // C+[i, j]
             const int cmv = mirror[jm][tx][cj];                      // C-[i, j] = C+[j, i]
             const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
-            qr = fma(vr, tab.rho_r[jm], qr);
-            qi = fma(vi, tab.rho_i[jm], qi);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 Sr[c] = fma(vr, tab.gr[jm][c], Sr[c]);
@@ -526,9 +635,9 @@ __global__ void __launch_bounds__(kHerkTile * 8) post_herk_kernel(const int8_t* 
             re = im = __longlong_as_double(0x7FF8000000000000ll);
         } else {
             double h, l;
-            crt_finish<NCH>(Sr, qr, tab, &h, &l);
+            crt_finish<NCH>(Sr, tab, &h, &l);
             re = scale_pow2(h + l, ei + ej);
-            crt_finish<NCH>(Si, qi, tab, &h, &l);
+            crt_finish<NCH>(Si, tab, &h, &l);
             im = scale_pow2(h + l, ei + ej);
         }
         *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);

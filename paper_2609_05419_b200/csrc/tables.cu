@@ -142,9 +142,9 @@ void build_crt_table(int nmod, CrtTable* t) {
             t->gr[j][c] = (g < 0 ? -1.0 : 1.0) * (double)Gr.bits(c * kChunkBits, kChunkBits);
             t->gi[j][c] = (h < 0 ? -1.0 : 1.0) * (double)Gi.bits(c * kChunkBits, kChunkBits);
         }
-        t->rho_r[j] = (double)g / (double)kModuli[j];
-        t->rho_i[j] = (double)h / (double)kModuli[j];
     }
+    t->q_hi = std::ldexp(1.0, kChunkBits * (t->nchunks - 1)) / M.to_double();
+    t->q_lo = t->nchunks > 1 ? std::ldexp(t->q_hi, -kChunkBits) : 0.0;
 }
 
 void build_crt_table_int(int nmod, CrtTableInt* t) {

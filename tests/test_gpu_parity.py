@@ -44,7 +44,7 @@ def check_stages_int(st, ref, m, n, k, nmod):
             assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j)
 
 
-@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])   # check kernel first: isolates pre/post from the tensor-core GEMM
+@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])   # check kernel first: isolates pre/post from the tensor-core GEMM
 @pytest.mark.parametrize("shape,nmod", [((128, 128, 128), 3), ((128, 128, 128), 1), ((128, 128, 128), 2),
                                         ((130, 77, 300), 3), ((1, 1, 1), 1), ((257, 513, 129), 4), ((5, 300, 1000), 8)])
 def test_gaussian_int_bit_exact(shape, nmod, kernel):
@@ -88,7 +88,7 @@ def test_gaussian_int_k_split_beyond_int32_range():
     Bi[::5, :] = rng.integers(-128, 128, size=Bi[::5, :].shape)
     M = staged.product(staged.greedy_2m_moduli()[:6])
     er, ei = direct.gauss4m_mod(Ar, Ai, Br, Bi, M)
-    for kernel in (1, 0):
+    for kernel in (1, 2, 0):
         Cr, Ci, _ = run_int(Ar, Ai, Br, Bi, 6, kernel)
         assert (Cr == er).all() and (Ci == ei).all(), kernel
 
@@ -106,7 +106,7 @@ def run_z(A, B, nmod, kernel=0, cplx=torch.complex128, op=None):
         return to_host(C), st
 
 
-@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])
+@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])
 @pytest.mark.parametrize("shape,nmod,dist", [((200, 150, 300), 16, "phi"), ((129, 257, 128), 14, "uniform"),
                                              ((64, 64, 64), 3, "uniform"), ((33, 19, 50), 22, "phi"), ((40, 40, 520), 20, "uniform")])
 def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
