@@ -28,6 +28,25 @@ METRIC = "zgemm2m_effective_tflops_8mnk_per_t"
 UNIT = "TFLOP/s"
 INT8_NOMINAL_TOPS = 4500.0          # dense int8, nominal
 INT8_OVER_BF16 = 2.0                # nominal ratio used to turn the measured bf16 peak into an int8 peak
+# DRAM bytes (read + write) of the GEMM launch per byte of int8 planes it touches, from the ncu capture of the 4096^3,
+# 16-modulus case (profiles/gemm_i8_tcgen05_pair_4096_nmod16.md): (1.156 + 0.519) GB over 3 x 536.9 MB of planes.
+GEMM_DRAM_BYTES_PER_PLANE_BYTE = (1.155904e9 + 0.519411968e9) / (3 * 32 * 4096 * 4096)
+
+
+def job_value(flops_per_rank_step, world, ms_per_step):
+    """Whole-job throughput in TFLOP/s: every rank processed its own problem in the (max over ranks) step time."""
+    return flops_per_rank_step * world / (ms_per_step * 1e-3) / 1e12
+
+
+def max_over_ranks(x, world, device):
+    """Max of a per-rank scalar over all ranks (any torch.distributed backend); identity for one rank."""
+    if world == 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 def parse():
@@ -182,13 +201,6 @@ def run_ours(a):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     b.lib()   # fails loudly if the CUDA library is missing
     m, n, k, nmod = a.m, a.n, a.k, a.nmod
     A, B = inputs.complex_inputs(m, n, k, a.seed + rank, dist="phi", phi=a.phi)     # every replica its own problem
@@ -227,27 +239,54 @@ def run_ours(a):
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
     phase, calls = b.phase_ms()
     b.set_profiling(False)
     b.device_status()
     launches_per_step, per_phase = b.last_launch_count()
 
-    # ---- end to end: pinned host -> device, call, device -> host, every step
+    # ---- end to end: every step copies its inputs from pinned host memory, calls the library and reads C back.
+    # Steps are pipelined the way a user streaming problems through the GPU would: uploads, compute and downloads run
+    # on three streams with two sets of device buffers, so PCIe transfers of neighbouring steps overlap the kernels.
     e2e = None
     if not a.no_e2e:
-        for _ in range(2):
-            step_e2e()
+        s_h2d, s_d2h = torch.cuda.Stream(), torch.cuda.Stream()
+        bufs = [(dA, dB, dC), (torch.empty_like(dA), torch.empty_like(dB), torch.empty_like(dC))]
+        up = [torch.cuda.Event() for _ in range(2)]
+        done = [torch.cuda.Event() for _ in range(2)]
+        freed = [torch.cuda.Event() for _ in range(2)]
+
+        def run_e2e(nsteps):
+            for i in range(nsteps):
+                A_, B_, C_ = bufs[i & 1]
+                with torch.cuda.stream(s_h2d):
+                    if i >= 2:
+                        s_h2d.wait_event(done[i & 1])         # compute of step i-2 no longer reads these inputs
+                    A_.copy_(hA, non_blocking=True)
+                    B_.copy_(hB, non_blocking=True)
+                    up[i & 1].record(s_h2d)
+                stream.wait_event(up[i & 1])
+                if i >= 2:
+                    stream.wait_event(freed[i & 1])           # download of step i-2 has left this C buffer
+                b.zgemm2m(A_.t(), B_.t(), C_.t(), nmod, stream)
+                done[i & 1].record(stream)
+                with torch.cuda.stream(s_d2h):
+                    s_d2h.wait_event(done[i & 1])
+                    hC.copy_(C_, non_blocking=True)
+                    freed[i & 1].record(s_d2h)
+            stream.wait_stream(s_d2h)
+            stream.wait_stream(s_h2d)
+
+        run_e2e(2)
         barrier()
         e0.record(stream)
-        for _ in range(a.steps):
-            step_e2e()
+        run_e2e(a.steps)
         e1.record(stream)
         barrier()
-        ms_e2e = max_over_ranks(e0.elapsed_time(e1))
-        e2e = {"value": 8.0 * m * n * k * world * a.steps / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+        e2e = {"value": job_value(8.0 * m * n * k, world, ms_e2e / a.steps), "unit": UNIT,
                "h2d_bytes_per_step": int(hA.numel() * 16 + hB.numel() * 16), "d2h_bytes_per_step": int(hC.numel() * 16),
-               "ms_per_step": ms_e2e / a.steps}
+               "ms_per_step": ms_e2e / a.steps, "pipeline": "3 streams, 2 device buffer sets; pinned host buffers"}
 
     if rank != 0:
         if world > 1:
@@ -256,15 +295,18 @@ def run_ours(a):
 
     peaks = measured_peaks()
     ms_step = ms_total / a.steps
-    value = 8.0 * m * n * k * world / (ms_step * 1e-3) / 1e12
+    value = job_value(8.0 * m * n * k, world, ms_step)
     gemm_ops = 2.0 * (2 * nmod) * m * n * k            # int8 multiply-adds x2, all 2N real GEMMs = one launch
     gemm_tops = gemm_ops / (phase[2] * 1e-3) / 1e12
     int8_peak = INT8_OVER_BF16 * peaks["bf16_sustained"]
+    c_kp, c_ldp = (k + 127) // 128 * 128, (m + 15) // 16 * 16
     pre_bytes = (m * k + k * n) * (16 + 2 * nmod)       # quantise read + residue planes written
     scan_bytes = (m * k + k * n) * 16
     post_bytes = m * n * (2 * nmod + 16)
-    roofline = {"bound": "tensor", "kernel": "gemm_i8_tcgen05_kernel", "achieved": gemm_tops, "peak": int8_peak, "unit": "TFLOP/s",
-                "frac": gemm_tops / int8_peak, "traffic": None,
+    roofline = {"bound": "tensor", "kernel": "gemm_i8_tcgen05_pair_kernel", "achieved": gemm_tops, "peak": int8_peak, "unit": "TFLOP/s",
+                "frac": gemm_tops / int8_peak,
+                "traffic": GEMM_DRAM_BYTES_PER_PLANE_BYTE * 2 * nmod * (m * c_kp + n * c_kp + n * c_ldp),
+                "traffic_source": "ncu dram__bytes_read+write of the 4096^3 launch, scaled by plane bytes",
                 "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate (int8:bf16 nominal ratio); int8 ops counted as 2 per MAC",
                 "frac_of_nominal_4500": gemm_tops / INT8_NOMINAL_TOPS,
                 "launch_ms": phase[2], "algorithmic_ops_per_launch": gemm_ops}

@@ -20,7 +20,10 @@ constexpr int BM = 128;        // rows of the row operand per CTA (TMEM lanes); 
 constexpr int BN = 256;        // rows of the column operand per pair (TMEM columns); each CTA loads 128 of them
 constexpr int BK = kGemmBK;
 constexpr int UMMA_K = 32;
-constexpr int STAGES = 6;
+#ifndef GEMM2M_PAIR_STAGES
+#define GEMM2M_PAIR_STAGES 6
+#endif
+constexpr int STAGES = GEMM2M_PAIR_STAGES;
 constexpr int ROW_TILE_BYTES = BM * BK;          // 16 KB
 constexpr int COL_HALF_BYTES = (BN / 2) * BK;    // 16 KB
 constexpr int STAGE_BYTES = ROW_TILE_BYTES + COL_HALF_BYTES;
