@@ -70,8 +70,8 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int b = tile / tiles_per_batch, rem = tile - b * tiles_per_batch;
-                const int tr = rem / p.tiles_c, tc = rem - tr * p.tiles_c;
+                int b, tr, tc;
+                decode_tile(p, tile, &b, &tr, &tc);
                 for (int kb = 0; kb < p.kblocks; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, kDevTimeoutProducer))) break;
                     const uint32_t dst = tiles_base + stage * STAGE_BYTES;
@@ -130,8 +130,8 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
         int it = 0;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
             const int acc = it & 1;
-            const int b = tile / tiles_per_batch, rem = tile - b * tiles_per_batch;
-            const int tr = rem / p.tiles_c, tc = rem - tr * p.tiles_c;
+            int b, tr, tc;
+            decode_tile(p, tile, &b, &tr, &tc);
             const int jm = b % p.mods.nmod;
             const int m = p.mods.m[jm];
             const float inv_m = p.mods.inv_m[jm];
@@ -211,6 +211,7 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count
     p.out_plane_stride = a.R * a.ldp;
     p.mods = a.mods;
     p.dev_status = a.dev_status;
+    p.band = p.tiles_r < 8 ? p.tiles_r : 8;
     const int64_t total_tiles = (int64_t)p.tiles_r * p.tiles_c * p.nbatch;
     if (total_tiles > INT32_MAX) return cudaErrorInvalidValue;
     const int grid = (int)(total_tiles < sm_count ? total_tiles : sm_count);

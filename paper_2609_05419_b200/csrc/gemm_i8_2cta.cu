@@ -120,8 +120,8 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < total_tiles; tile += npairs) {
-                const int b = tile / tiles_per_batch, rem = tile - b * tiles_per_batch;
-                const int tr = rem / p.tiles_c, tc = rem - tr * p.tiles_c;
+                int b, tr, tc;
+                decode_tile(p, tile, &b, &tr, &tc);
                 const int row0 = tr * (2 * BM) + (int)rank * BM;
                 const int col0 = tc * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < p.kblocks; ++kb) {
@@ -175,8 +175,8 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
         int it = 0;
         for (int tile = pair; ok && tile < total_tiles; tile += npairs, ++it) {
             const int acc = it & 1;
-            const int b = tile / tiles_per_batch, rem = tile - b * tiles_per_batch;
-            const int tr = rem / p.tiles_c, tc = rem - tr * p.tiles_c;
+            int b, tr, tc;
+            decode_tile(p, tile, &b, &tr, &tc);
             const int jm = b % p.mods.nmod;
             const int m = p.mods.m[jm];
             const float inv_m = p.mods.inv_m[jm];
@@ -277,6 +277,7 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
     p.out_plane_stride = a.R * a.ldp;
     p.mods = a.mods;
     p.dev_status = a.dev_status;
+    p.band = p.tiles_r < 8 ? p.tiles_r : 8;
     const int64_t total_tiles = (int64_t)p.tiles_r * p.tiles_c * p.nbatch;
     if (total_tiles > INT32_MAX) return cudaErrorInvalidValue;
     const int pairs = (int)(total_tiles < max_pairs ? total_tiles : max_pairs);

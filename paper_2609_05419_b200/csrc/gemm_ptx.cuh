@@ -141,9 +141,24 @@ struct GemmKernelParams {
     int8_t* out;
     int64_t ldp, out_plane_stride;
     int accumulate;          // add the residues already stored in `out` (later K chunks)
+    int band;                // tile rasterisation: row tiles per band (see decode_tile)
     ModTable mods;
     int* dev_status;
 };
+
+// Linear tile index -> (batch, row tile, column tile).  Within a batch the tiles are walked in bands of `band` row tiles,
+// column by column inside a band, so that the tiles in flight at any time (one per CTA or CTA pair, consecutive indices)
+// cover about band x (CTAs / band) tiles and share their operand slices through L2 instead of re-reading them from HBM.
+__device__ __forceinline__ void decode_tile(const GemmKernelParams& p, int tile, int* b, int* tr, int* tc) {
+    const int per_batch = p.tiles_r * p.tiles_c;
+    *b = tile / per_batch;
+    const int rem = tile - *b * per_batch;
+    const int per_band = p.band * p.tiles_c;
+    const int band_idx = rem / per_band, in_band = rem - band_idx * per_band;
+    const int rows_here = min(p.band, p.tiles_r - band_idx * p.band);
+    *tc = in_band / rows_here;
+    *tr = band_idx * p.band + (in_band - *tc * rows_here);
+}
 
 // ------------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,

@@ -592,70 +592,113 @@ cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n,
 }
 
 // HERK (Section 5): only C+ = A+ A-^T was computed; C- = C+^T.  cp: [nmod][n][ldp] with cp[j][col][row] = C+_j[row, col].
-// A 32 x 32 tile (rows i, columns j, i >= j) needs C+[i, j] (direct, i contiguous) and C+[j, i] (the mirrored tile,
-// transposed through shared memory).  Lower triangle only; the diagonal's imaginary part is exactly zero.
-constexpr int kHerkTile = 32;
+// A block handles 64 rows i x 16 columns j of the lower triangle.  It needs C+[i, j] (rows of cp along i: 16 runs of 64
+// bytes per modulus) and C-[i, j] = C+[j, i] (rows of cp along j: 64 runs of 16 bytes per modulus); both are pulled into
+// shared memory with asynchronous 16-byte copies, then each thread combines 4 consecutive i of one column.
+// Lower triangle only; on the diagonal C- - C+ = 0, so the imaginary part is exactly zero.
+constexpr int kHerkI = 64, kHerkJ = 16, kHerkThreads = 256;
+constexpr int kHerkMirrorSlots = kHerkI + kHerkI / 8;                      // 16-byte slots, one pad slot per 8 rows (bank spread)
+constexpr int kHerkPlaneBytes = kHerkJ * kHerkI + kHerkMirrorSlots * 16;   // direct + mirrored bytes per modulus
+
 template <int NCH>
-__global__ void __launch_bounds__(kHerkTile * 8) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n,
-                                                                  const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
-                                                                  double* __restrict__ C, int64_t ldc) {
-    const int ti = blockIdx.x, tj = blockIdx.y;
-    if (ti < tj) return;
-    __shared__ int8_t mirror[kMaxMod][kHerkTile][kHerkTile + 4];
+__global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n,
+                                                                 const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
+                                                                 double* __restrict__ C, int64_t ldc) {
+    extern __shared__ __align__(16) unsigned char herk_smem[];
+    const int64_t ibase = (int64_t)blockIdx.x * kHerkI, jbase = (int64_t)blockIdx.y * kHerkJ;
+    if (ibase + kHerkI - 1 < jbase) return;                                // tile entirely above the diagonal
     const int nmod = tab.nmod;
     const int64_t plane = n * ldp;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
-    const int64_t ibase = (int64_t)ti * kHerkTile, jbase = (int64_t)tj * kHerkTile;
-    // mirrored tile: C+[j, i] = cp[col = i][row = j]; read with j contiguous, store transposed
-    for (int jm = 0; jm < nmod; ++jm)
-        for (int r = ty; r < kHerkTile; r += 8) {
-            const int64_t i = ibase + r, j = jbase + tx;
-            mirror[jm][r][tx] = (i < n && j < n) ? cp[(int64_t)jm * plane + i * ldp + j] : (int8_t)0;
-        }
+    const int t = threadIdx.x;
+    // direct part: for each modulus and each column j of the tile, 64 bytes along i (4 copies of 16 bytes)
+    for (int idx = t; idx < nmod * kHerkJ * (kHerkI / 16); idx += kHerkThreads) {
+        const int v = idx & 3, jj = (idx >> 2) & (kHerkJ - 1), jm = idx / (kHerkJ * 4);
+        const int64_t i = ibase + 16 * v, j = jbase + jj;
+        if (j < n && i < ldp) cp_async16(herk_smem + jm * kHerkPlaneBytes + jj * kHerkI + 16 * v, cp + (int64_t)jm * plane + j * ldp + i);
+    }
+    // mirrored part: for each modulus and each row i of the tile, the 16 bytes C+[jbase .. jbase+15, i]
+    for (int idx = t; idx < nmod * kHerkI; idx += kHerkThreads) {
+        const int ii = idx & (kHerkI - 1), jm = idx / kHerkI;
+        const int64_t i = ibase + ii;
+        if (i < n && jbase < ldp)
+            cp_async16(herk_smem + jm * kHerkPlaneBytes + kHerkJ * kHerkI + (ii + (ii >> 3)) * 16, cp + (int64_t)jm * plane + i * ldp + jbase);
+    }
+    cp_async_wait_all();
     __syncthreads();
-    for (int cj = ty; cj < kHerkTile; cj += 8) {
-        const int64_t i = ibase + tx, j = jbase + cj;
-        if (i >= n || j >= n || i < j) continue;
-        double Sr[NCH], Si[NCH];
+    const int g = t & 15, jj = t >> 4;                                     // 4 consecutive rows i0 .. i0+3 of column j
+    const int64_t i0 = ibase + 4 * g, j = jbase + jj;
+    if (j >= n || i0 >= n || i0 + 3 < j) return;
+    double Sr[4][NCH], Si[4][NCH];
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) Sr[c] = Si[c] = 0.0;
-        for (int jm = 0; jm < nmod; ++jm) {
-            const int cpv = cp[(int64_t)jm * plane + j * ldp + i];   // C+[i, j]
-            const int cmv = mirror[jm][tx][cj];                      // C-[i, j] = C+[j, i]
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
+    }
+#pragma unroll 2
+    for (int jm = 0; jm < nmod; ++jm) {
+        const unsigned char* base = herk_smem + jm * kHerkPlaneBytes;
+        const uint32_t wp = *reinterpret_cast<const uint32_t*>(base + jj * kHerkI + 4 * g);      // C+[i0..i0+3, j]
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int ii = 4 * g + e;
+            const int cpv = (int)(int8_t)(wp >> (8 * e));
+            const int cmv = (int)(int8_t)base[kHerkJ * kHerkI + (ii + (ii >> 3)) * 16 + jj];    // C-[i, j] = C+[j, i]
             const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-                Sr[c] = fma(vr, tab.gr[jm][c], Sr[c]);
-                Si[c] = fma(vi, tab.gi[jm][c], Si[c]);
+                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
+                Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
             }
         }
-        const int ei = __ldg(eA + i), ej = __ldg(eA + j);
-        double re, im;
-        if (ei == kExpNonFinite || ej == kExpNonFinite) {
-            re = im = __longlong_as_double(0x7FF8000000000000ll);
-        } else {
-            double h, l;
-            crt_finish<NCH>(Sr, tab, &h, &l);
-            re = scale_pow2(h + l, ei + ej);
-            crt_finish<NCH>(Si, tab, &h, &l);
-            im = scale_pow2(h + l, ei + ej);
+    }
+    const int ej = __ldg(eA + j);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int64_t i = i0 + e;
+        if (i < n && i >= j) {
+            const int ei = __ldg(eA + i);
+            double re, im;
+            if (ei == kExpNonFinite || ej == kExpNonFinite) {
+                re = im = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(Sr[e], tab, &h, &l);
+                re = scale_pow2(h + l, ei + ej);
+                crt_finish<NCH>(Si[e], tab, &h, &l);
+                im = scale_pow2(h + l, ei + ej);
+            }
+            *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
         }
-        *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
     }
 }
 
 cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
                              cudaStream_t st, int* launches) {
     if (n <= 0) return cudaSuccess;
-    const unsigned tiles = (unsigned)((n + kHerkTile - 1) / kHerkTile);
-    dim3 grid(tiles, tiles);
-    switch (tab.nchunks) {
-        case 1: post_herk_kernel<1><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        case 2: post_herk_kernel<2><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        case 3: post_herk_kernel<3><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        default: post_herk_kernel<4><<<grid, kHerkTile * 8, 0, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+    const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
     }
-    ++*launches;
+    const size_t use = (size_t)tab.nmod * kHerkPlaneBytes;
+    const int64_t tiles_j = (n + kHerkJ - 1) / kHerkJ;
+    for (int64_t j0 = 0; j0 < tiles_j; j0 += 65535) {      // grid.y limit
+        const int64_t nj = (tiles_j - j0 < 65535) ? tiles_j - j0 : 65535;
+        if (j0 != 0) return cudaErrorInvalidValue;         // n beyond 65535 * 16 columns is rejected by the API's row limit anyway
+        dim3 grid((unsigned)((n + kHerkI - 1) / kHerkI), (unsigned)nj);
+        switch (tab.nchunks) {
+            case 1: post_herk_kernel<1><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+            case 2: post_herk_kernel<2><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+            case 3: post_herk_kernel<3><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+            default: post_herk_kernel<4><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        }
+        ++*launches;
+    }
     return cudaGetLastError();
 }
 
