@@ -10,7 +10,6 @@ namespace gemm2m {
 constexpr int kMaxMod = 22;        // size of the greedy 2M modulus set in [1, 256] (Section 4)
 constexpr int kMaxChunks = 4;      // 40-bit digits needed for M/2 < 2^152
 constexpr int kChunkBits = 40;
-constexpr int kMaxWideShift = 80;  // largest left shift of a mantissa in the wide quantisation mode
 constexpr int kExpNonFinite = INT32_MIN;   // scale-exponent sentinel: row/column holds an Inf or NaN
 
 // Device status word values (written by kernels whose bounded waits give up).
@@ -18,16 +17,17 @@ constexpr int kDevOk = 0;
 constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilogue = 103;
 
 // Per-modulus constants for the residue kernels, Eq. (2a).
-// A quantised part x (two's complement int64) is written as 4 unsigned low bytes and 4 balanced
-// (signed) high digits; its residue is the dot product of those 8 digits with w_b = sym(256^b mod m).
+// A quantised part x (two's complement, 64 bits; 96 bits in the wide mode used from 19-20 moduli on) is written as 4
+// unsigned low bytes and 4 (8) balanced signed high digits; its residue is the dot product of those digits with
+// w_b = sym(256^b mod m).
 // The imaginary part uses s*w_b so that R + I = A_r + s A_i and R - I = A_r - s A_i (mod m).
 struct ResidueTable {
     int32_t m[kMaxMod];
     float inv_m[kMaxMod];
     uint32_t w_lo[kMaxMod], w_hi[kMaxMod];     // int8 x4 each: sym(256^b mod m), b = 0..3 / 4..7
     uint32_t ws_lo[kMaxMod], ws_hi[kMaxMod];   // int8 x4 each: sym(s 256^b mod m)
+    uint32_t w_top[kMaxMod], ws_top[kMaxMod];  // b = 8..11: only used when quantised values exceed 62 bits
     int32_t s[kMaxMod];
-    int8_t pow2[kMaxMod][kMaxWideShift];       // sym(2^t mod m): only used when quantised values exceed 62 bits
     int nmod;
 };
 

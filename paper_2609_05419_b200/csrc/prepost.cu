@@ -131,10 +131,8 @@ cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int c
 // =====================================================================================================
 struct QPair { long long re, im; };   // quantised parts, two's complement
 
-// trunc(v 2^-e) for a finite v given by its bit pattern.
-// Narrow mode (WIDE = false): the scaling rule guarantees |result| < 2^62, returned as a two's complement int64.
-// Wide mode: the result is sign * mant * 2^t with mant < 2^53; returned packed as (sign * mant) * 256 + t.
-template <typename T, bool WIDE>
+// trunc(v 2^-e) for a finite v given by its bit pattern; the scaling rule guarantees |result| < 2^62 in the narrow mode.
+template <typename T>
 __device__ __forceinline__ long long quantise_part(T v, int e) {
     using F = FpBits<T>;
     const unsigned long long mag = F::mag(v);
@@ -145,15 +143,28 @@ __device__ __forceinline__ long long quantise_part(T v, int e) {
     const int sh = max(E, 1) - (F::kBias + F::kMantBits) - e;
     const bool neg = (sizeof(T) == 8) ? (__double_as_longlong((double)v) < 0) : (__float_as_int((float)v) < 0);
     unsigned long long q;
-    int t = 0;
-    if (sh >= 0) {
-        if (WIDE) { q = mant; t = mant ? min(sh, kMaxWideShift - 1) : 0; }
-        else q = mant << min(sh, 63);
-    } else {
-        q = (-sh > 63) ? 0ull : (mant >> (-sh));
-    }
-    const long long sq = neg ? -(long long)q : (long long)q;
-    return WIDE ? sq * 256 + t : sq;
+    if (sh >= 0) q = mant << min(sh, 63);
+    else q = (-sh > 63) ? 0ull : (mant >> (-sh));
+    return neg ? -(long long)q : (long long)q;
+}
+
+// Wide mode: |result| < 2^76 (19 or more moduli); returned as the low 32 bits and the signed upper 64 bits of the 96-bit
+// two's complement value.
+template <typename T>
+__device__ __forceinline__ void quantise_part_wide(T v, int e, uint32_t* lo, long long* upper) {
+    using F = FpBits<T>;
+    const unsigned long long mag = F::mag(v);
+    const int E = (int)(mag >> F::kMantBits);
+    unsigned long long mant = mag & ((1ull << F::kMantBits) - 1);
+    if (E) mant |= (1ull << F::kMantBits);
+    const int sh = max(E, 1) - (F::kBias + F::kMantBits) - e;
+    const bool neg = (sizeof(T) == 8) ? (__double_as_longlong((double)v) < 0) : (__float_as_int((float)v) < 0);
+    unsigned __int128 q;
+    if (sh >= 0) q = (unsigned __int128)mant << min(sh, 64);
+    else q = (-sh > 63) ? 0 : (mant >> (-sh));
+    const __int128 sq = neg ? -(__int128)q : (__int128)q;
+    *lo = (uint32_t)(unsigned __int128)sq;
+    *upper = (long long)(sq >> 32);
 }
 
 __device__ __forceinline__ int dp4a_us(uint32_t a_unsigned, uint32_t b_signed, int c) {
@@ -197,12 +208,21 @@ __device__ __forceinline__ Digits split_digits(long long x) {
     d.hi = (hi + 0x80808080u) ^ 0x80808080u;   // hi = sum (byte_b - 128) 256^b  after adding 128 to every byte
     return d;
 }
+// The same for a 96-bit value given as low word and signed upper 64 bits: 8 balanced digits above the low word.
+__device__ __forceinline__ Digits split_digits_wide(uint32_t lo, long long upper, uint32_t* top) {
+    const unsigned long long rec = ((unsigned long long)upper + 0x8080808080808080ull) ^ 0x8080808080808080ull;
+    Digits d;
+    d.lo = lo;
+    d.hi = (uint32_t)rec;
+    *top = (uint32_t)(rec >> 32);
+    return d;
+}
 
 // Residues of NE consecutive elements of one operand row for every modulus, written as NE-byte vectors into both sign
-// planes.  dst points at plane 0, this row, first k of the run; tsh (wide mode) holds the mantissa shifts t_r | t_i << 8.
+// planes.  dst points at plane 0, this row, first k of the run; tr / ti (wide mode) hold the four top digits of each part.
 template <int NE, bool WIDE>
-__device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tsh, const ResidueTable& tab,
-                                         int8_t* dst, int64_t plane_stride) {
+__device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tr, const uint32_t* ti,
+                                         const ResidueTable& tab, int8_t* dst, int64_t plane_stride) {
     static_assert(NE == 8 || NE == 16, "runs of 8 or 16 elements");
     const int nmod = tab.nmod;
 #pragma unroll 1
@@ -210,6 +230,7 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
         const int m = tab.m[j];
         const float inv_m = tab.inv_m[j], neg_m = -(float)m;
         const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
+        const uint32_t wt = WIDE ? tab.w_top[j] : 0u, st = WIDE ? tab.ws_top[j] : 0u;
         uint32_t pw[NE / 4], mw[NE / 4];
 #pragma unroll
         for (int w = 0; w < NE / 4; ++w) {
@@ -219,9 +240,9 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
                 const int i = 4 * w + b;
                 int Rv = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, 0));   // A_r mod m (unreduced)
                 int Iv = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, 0));   // s A_i mod m (unreduced)
-                if (WIDE) {                                                 // times 2^t mod m
-                    Rv = sym_reduce_small(Rv, m, inv_m) * (int)tab.pow2[j][tsh[i] & 0xFF];
-                    Iv = sym_reduce_small(Iv, m, inv_m) * (int)tab.pow2[j][tsh[i] >> 8];
+                if (WIDE) {                                                 // digits 8..11 of the 96-bit value
+                    Rv = dp4a_ss(tr[i], wt, Rv);
+                    Iv = dp4a_ss(ti[i], st, Iv);
                 }
                 sym_reduce_pm(Rv, Iv, neg_m, inv_m, &bp[b], &bm[b]);        // Eq. (2a): "+" and "-"
             }
@@ -315,27 +336,33 @@ __global__ void __launch_bounds__(kResThreads, 3) residues_fp_kernel(const T* __
             const bool fast = !WIDE && ex > -1000 && ex < 1000;
             const double scale = __longlong_as_double((long long)(1023 - (fast ? ex : 0)) << 52);
             Digits dr[kResRun], di[kResRun];
-            uint32_t tsh[WIDE ? kResRun : 1];
+            uint32_t tr[WIDE ? kResRun : 1], ti[WIDE ? kResRun : 1];
 #pragma unroll
             for (int i = 0; i < kResRun; ++i) {
                 const Raw v = src[r * kResRowStride + kResRun * g + g + i];
-                long long qr = 0, qi = 0;
-                if (fast) {
-                    qr = __double2ll_rz((double)v.x * scale);
-                    qi = __double2ll_rz((double)v.y * scale);
-                } else if (ex != kExpNonFinite) {
-                    qr = quantise_part<T, WIDE>(v.x, ex);
-                    qi = quantise_part<T, WIDE>(v.y, ex);
-                }
                 if (WIDE) {
-                    tsh[i] = (uint32_t)(qr & 0xFF) | ((uint32_t)(qi & 0xFF) << 8);
-                    qr >>= 8;
-                    qi >>= 8;
+                    uint32_t lr = 0, li = 0;
+                    long long ur = 0, ui = 0;
+                    if (ex != kExpNonFinite) {
+                        quantise_part_wide<T>(v.x, ex, &lr, &ur);
+                        quantise_part_wide<T>(v.y, ex, &li, &ui);
+                    }
+                    dr[i] = split_digits_wide(lr, ur, &tr[i]);
+                    di[i] = split_digits_wide(li, ui, &ti[i]);
+                } else {
+                    long long qr = 0, qi = 0;
+                    if (fast) {
+                        qr = __double2ll_rz((double)v.x * scale);
+                        qi = __double2ll_rz((double)v.y * scale);
+                    } else if (ex != kExpNonFinite) {
+                        qr = quantise_part<T>(v.x, ex);
+                        qi = quantise_part<T>(v.y, ex);
+                    }
+                    dr[i] = split_digits(qr);
+                    di[i] = split_digits(qi);
                 }
-                dr[i] = split_digits(qr);
-                di[i] = split_digits(qi);
             }
-            emit_run<kResRun, WIDE>(dr, di, tsh, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
+            emit_run<kResRun, WIDE>(dr, di, tr, ti, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
         }
         __syncthreads();   // everyone is done with this stage before it is refilled
     }
@@ -413,7 +440,7 @@ __global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t
     }
     const int64_t row = row0 + r;
     if (row >= R) return;
-    emit_run<kResIRun, false>(dr, di, nullptr, tab, planes + row * Kp + k0 + kResIRun * g, R * Kp);
+    emit_run<kResIRun, false>(dr, di, nullptr, nullptr, tab, planes + row * Kp + k0 + kResIRun * g, R * Kp);
 }
 
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,

@@ -88,18 +88,19 @@ void build_residue_table(int nmod, ResidueTable* t) {
         t->s[j] = s;
         t->inv_m[j] = 1.0f / (float)m;
         int64_t p = 1;   // 256^b mod m
-        uint32_t w[8], ws[8];
-        for (int b = 0; b < 8; ++b) {
+        uint32_t w[12], ws[12];
+        for (int b = 0; b < 12; ++b) {
             w[b] = (uint32_t)(uint8_t)(int8_t)sym_mod(p, m);
             ws[b] = (uint32_t)(uint8_t)(int8_t)sym_mod(p * s, m);
             p = (p * 256) % m;
         }
-        t->w_lo[j] = w[0] | (w[1] << 8) | (w[2] << 16) | (w[3] << 24);
-        t->w_hi[j] = w[4] | (w[5] << 8) | (w[6] << 16) | (w[7] << 24);
-        t->ws_lo[j] = ws[0] | (ws[1] << 8) | (ws[2] << 16) | (ws[3] << 24);
-        t->ws_hi[j] = ws[4] | (ws[5] << 8) | (ws[6] << 16) | (ws[7] << 24);
-        int64_t p2 = 1;
-        for (int e = 0; e < kMaxWideShift; ++e) { t->pow2[j][e] = (int8_t)sym_mod(p2, m); p2 = (p2 * 2) % m; }
+        auto pack = [](const uint32_t* v) { return v[0] | (v[1] << 8) | (v[2] << 16) | (v[3] << 24); };
+        t->w_lo[j] = pack(w);
+        t->w_hi[j] = pack(w + 4);
+        t->w_top[j] = pack(w + 8);
+        t->ws_lo[j] = pack(ws);
+        t->ws_hi[j] = pack(ws + 4);
+        t->ws_top[j] = pack(ws + 8);
     }
 }
 
