@@ -244,6 +244,15 @@ def run_ours(a):
     b.set_profiling(False)
     b.device_status()
     launches_per_step, per_phase = b.last_launch_count()
+    # the same phases strictly one after the other (no panel overlap): what the per-phase bandwidth figures are taken from
+    b.debug_set_panels(1)
+    b.set_profiling(True)
+    for _ in range(3):
+        step()
+    serial, _ = b.phase_ms()
+    b.set_profiling(False)
+    b.debug_set_panels(4)
+    b.device_status()
 
     # ---- end to end: every step copies its inputs from pinned host memory, calls the library and reads C back.
     # Steps are pipelined the way a user streaming problems through the GPU would: uploads, compute and downloads run
@@ -296,8 +305,9 @@ def run_ours(a):
     peaks = measured_peaks()
     ms_step = ms_total / a.steps
     value = job_value(8.0 * m * n * k, world, ms_step)
-    gemm_ops = 2.0 * (2 * nmod) * m * n * k            # int8 multiply-adds x2, all 2N real GEMMs = one launch
-    gemm_tops = gemm_ops / (phase[2] * 1e-3) / 1e12
+    gemm_launches = max(per_phase[2], 1)               # one launch per column panel, each all 2N real GEMMs of its panel
+    gemm_ops = 2.0 * (2 * nmod) * m * n * k / gemm_launches   # int8 multiply-adds x2
+    gemm_tops = gemm_ops * gemm_launches / (phase[2] * 1e-3) / 1e12
     int8_peak = INT8_OVER_BF16 * peaks["bf16_sustained"]
     c_kp, c_ldp = (k + 127) // 128 * 128, (m + 15) // 16 * 16
     pre_bytes = (m * k + k * n) * (16 + 2 * nmod)       # quantise read + residue planes written
@@ -305,16 +315,19 @@ def run_ours(a):
     post_bytes = m * n * (2 * nmod + 16)
     roofline = {"bound": "tensor", "kernel": "gemm_i8_tcgen05_pair_kernel", "achieved": gemm_tops, "peak": int8_peak, "unit": "TFLOP/s",
                 "frac": gemm_tops / int8_peak,
-                "traffic": GEMM_DRAM_BYTES_PER_PLANE_BYTE * 2 * nmod * (m * c_kp + n * c_kp + n * c_ldp),
+                "traffic": GEMM_DRAM_BYTES_PER_PLANE_BYTE * 2 * nmod * (m * c_kp + n * c_kp + n * c_ldp) / gemm_launches,
                 "traffic_source": "ncu dram__bytes_read+write of the 4096^3 launch, scaled by plane bytes",
                 "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate (int8:bf16 nominal ratio); int8 ops counted as 2 per MAC",
                 "frac_of_nominal_4500": gemm_tops / INT8_NOMINAL_TOPS,
-                "launch_ms": phase[2], "algorithmic_ops_per_launch": gemm_ops}
-    phases = {"scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3], "calls_averaged": calls,
-              "scan_gbs": scan_bytes / (phase[0] * 1e-3) / 1e9 if phase[0] > 0 else None,
-              "residues_gbs": pre_bytes / (phase[1] * 1e-3) / 1e9 if phase[1] > 0 else None,
-              "post_gbs": post_bytes / (phase[3] * 1e-3) / 1e9 if phase[3] > 0 else None,
-              "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]}
+                "launch_ms": phase[2] / gemm_launches, "launches_per_step": gemm_launches, "algorithmic_ops_per_launch": gemm_ops}
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else None
+    phases = {"note": "sums of kernel durations per phase in the timed region; post-processing of a column panel runs beside the "
+                      "next panel's GEMMs, so the phases add up to more than ms_per_step",
+              "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3], "calls_averaged": calls}
+    phases_serial = {"note": "3 extra calls with the panel overlap switched off (phases strictly sequential)",
+                     "scan_ms": serial[0], "residues_ms": serial[1], "gemm_ms": serial[2], "post_ms": serial[3],
+                     "scan_gbs": gbs(scan_bytes, serial[0]), "residues_gbs": gbs(pre_bytes, serial[1]), "post_gbs": gbs(post_bytes, serial[3]),
+                     "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]}
     cpu = None
     if not a.no_cpu_baseline:
         cpu, _ = time_oracle(a, A, B, a.cpu_seconds)
@@ -324,7 +337,7 @@ def run_ours(a):
             "config": {"workload": workload_name(a), "l2": "inputs (2 x %.2f GiB) and residue planes exceed the 126 MB L2" % (m * k * 16 / 2**30),
                        "multi_gpu": "replicas only (no collective on the path)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * a.steps, "launches_per_step": per_phase,
-            "roofline": roofline, "phases": phases, "cpu_baseline": cpu}
+            "roofline": roofline, "phases": phases, "phases_serial": phases_serial, "cpu_baseline": cpu}
     print(json.dumps(line))
     b.set_workspace(None)
     if world > 1:

@@ -17,7 +17,9 @@
  *   - All matrix pointers are DEVICE pointers owned by the caller.  The library never allocates or frees device
  *     memory inside a call; it uses the caller-provided workspace registered with gemm2m_set_workspace().
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and
- *     return immediately.  The return value is a gemm2m_status; it is the only error channel.
+ *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  zgemm2m and cgemm2m
+ *     additionally use one library-owned stream, forked from and joined back into `stream` with events: work enqueued
+ *     on `stream` after the call still sees the finished result.
  *   - Argument errors are detected on the host before anything is launched.  m, n or k equal to 0 is valid:
  *     nothing is computed for m = 0 or n = 0, and C is set to zero for k = 0.
  *   - `nmod` selects the first nmod moduli of the set of Section 4 (241, 233, 229, 221, 205, ... , 37, 29; 22 in
@@ -118,7 +120,9 @@ int gemm2m_device_status(void* stream);
 int gemm2m_set_profiling(int enabled);
 /* Waits for the recorded calls and returns the average milliseconds per call of each phase: ms[0] = exponent scan,
  * ms[1] = quantise + residues (Eq. 2a), ms[2] = int8 GEMMs (Eq. 2b), ms[3] = post-processing (Eq. 2c + CRT + unscale);
- * *calls = number of calls averaged.  Host pointers; GEMM2M_ERR_ARG if nothing was recorded. */
+ * *calls = number of calls averaged.  Each figure is the sum of the durations of the phase's kernels on the stream they run
+ * on; zgemm2m/cgemm2m post-process one column panel on an internal stream while the next panel's GEMMs run, so the four
+ * figures can add up to more than the duration of the call.  Host pointers; GEMM2M_ERR_ARG if nothing was recorded. */
 int gemm2m_phase_ms(float ms[4], int* calls);
 /* Number of kernels the last call launched (per phase in the same order, host pointer, may be NULL); returns total. */
 int gemm2m_last_launch_count(int per_phase[4]);
@@ -141,6 +145,9 @@ int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, g
  * kernel kept only so that tests can tell a fault in a tensor-core kernel from one in the pre/post kernels, 2 = the
  * tcgen05 kernel with one CTA per tile. */
 int gemm2m_debug_set_gemm_kernel(int which);
+/* Largest number of column panels zgemm2m/cgemm2m cut C into (default 4).  With 1 the phases run strictly one after the
+ * other on the caller's stream, which is what per-phase bandwidth figures should be measured with. */
+int gemm2m_debug_set_panels(int max_panels);
 
 /* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host
  * pointers, any may be NULL), so that CPU tests can check them against an independent computation:

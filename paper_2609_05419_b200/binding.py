@@ -61,6 +61,7 @@ def lib():
     L.gemm2m_last_launch_count.argtypes = [ctypes.POINTER(i32)]
     L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
+    L.gemm2m_debug_set_panels.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
     _lib = L
     return L
@@ -200,6 +201,10 @@ def last_launch_count():
 
 def debug_set_gemm_kernel(which):
     _check(lib().gemm2m_debug_set_gemm_kernel(which), "gemm2m_debug_set_gemm_kernel")
+
+
+def debug_set_panels(max_panels):
+    _check(lib().gemm2m_debug_set_panels(max_panels), "gemm2m_debug_set_panels")
 
 
 def debug_tables(nmod, k, herk=False):

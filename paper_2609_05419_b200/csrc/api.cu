@@ -17,10 +17,16 @@ struct State {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     int profiling = 0;
-    static constexpr int kProfSlots = 64;
-    cudaEvent_t ev[kProfSlots][5] = {};
+    static constexpr int kProfSlots = 64, kMaxIntervals = 24, kMaxPanels = 8;
+    struct Interval { cudaEvent_t a = nullptr, b = nullptr; int phase = 0; };
+    struct Slot { Interval iv[kMaxIntervals]; int n = 0; };
+    Slot slots[kProfSlots];       // timed intervals (phase, start, end) of the profiled calls
     int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
-    cudaEvent_t* cur = nullptr;   // event set of the call being enqueued
+    Slot* cur = nullptr;          // slot of the call being enqueued
+    cudaStream_t side = nullptr;  // library-owned stream on which the post-processing of a column panel overlaps the next panel's GEMMs
+    cudaEvent_t panel_done[kMaxPanels] = {};
+    cudaEvent_t side_done = nullptr;
+    int max_panels = 4;           // column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
     int sm_count = 0;
@@ -79,27 +85,39 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     return true;
 }
 
-struct Phases {   // event bookkeeping of one call
-    cudaStream_t st;
-    bool on;
-    int idx = 0;
-    cudaError_t mark() {
-        if (!on) return cudaSuccess;
-        return cudaEventRecord(g.cur[idx++], st);
+struct Phases {   // event bookkeeping of one call: every phase is a set of intervals, each on the stream its kernels run on
+    bool on = false;
+    cudaError_t begin(int phase, cudaStream_t st) {
+        if (!on || g.cur->n >= State::kMaxIntervals) return cudaSuccess;
+        State::Interval& iv = g.cur->iv[g.cur->n];
+        iv.phase = phase;
+        if (!iv.a) { cudaError_t e = cudaEventCreate(&iv.a); if (e != cudaSuccess) return e; }
+        if (!iv.b) { cudaError_t e = cudaEventCreate(&iv.b); if (e != cudaSuccess) return e; }
+        return cudaEventRecord(iv.a, st);
+    }
+    cudaError_t end(cudaStream_t st) {
+        if (!on || g.cur->n >= State::kMaxIntervals) return cudaSuccess;
+        return cudaEventRecord(g.cur->iv[g.cur->n++].b, st);
     }
     void done() { if (on) ++g.prof_calls; }
 };
 
-int begin_call(cudaStream_t st, Phases* ph) {
-    ph->st = st;
+int begin_call(Phases* ph) {
     ph->on = g.profiling != 0;
     std::memset(g.launches, 0, sizeof(g.launches));
     if (ph->on) {
-        g.cur = g.ev[g.prof_calls % State::kProfSlots];
-        for (int i = 0; i < 5; ++i)
-            if (!g.cur[i]) CK(cudaEventCreate(&g.cur[i]));
-        CK(ph->mark());
+        g.cur = &g.slots[g.prof_calls % State::kProfSlots];
+        g.cur->n = 0;
     }
+    return GEMM2M_OK;
+}
+
+// Side stream and ordering events, created on first use (no device memory involved).
+int ensure_side_stream() {
+    if (!g.side) CK(cudaStreamCreateWithFlags(&g.side, cudaStreamNonBlocking));
+    for (auto& e : g.panel_done)
+        if (!e) CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    if (!g.side_done) CK(cudaEventCreateWithFlags(&g.side_done, cudaEventDisableTiming));
     return GEMM2M_OK;
 }
 
@@ -150,19 +168,24 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
 
     Phases ph;
-    if (int s = begin_call(st, &ph)) return s;
+    if (int s = begin_call(&ph)) return s;
     // step 2: scale factors
+    CK(ph.begin(0, st));
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
     CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
     CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
     CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
     CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
-    CK(ph.mark());
+    CK(ph.end(st));
     // step 3 + Eq. (2a)
+    CK(ph.begin(1, st));
     CK(launch_residues_fp<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
     CK(launch_residues_fp<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
-    CK(ph.mark());
-    // Eq. (2b): 2 nmod real int8 GEMMs; TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm)
+    CK(ph.end(st));
+    // Eq. (2b): 2 nmod real int8 GEMMs; TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
+    // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
+    // panel p run on the library's side stream, on the SM resources the GEMM kernel leaves free.  (Forming the residues of
+    // later panels of B beside the GEMMs as well was measured and brought nothing: the GEMMs slow down by what is hidden.)
     GemmArgs ga;
     ga.rowop = bpm; ga.colop = apm;
     ga.R = n; ga.Cn = m; ga.Kp = c.kp;
@@ -172,11 +195,32 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     ga.out = cpm; ga.ldp = c.ldp;
     build_mod_table(nmod, &ga.mods);
     ga.dev_status = dev_status;
-    if (int s = run_gemm(ga, nmod, st)) return s;
-    CK(ph.mark());
-    // Eq. (2c) + steps 5-7
-    CK(launch_post_fp<T>(cpm, c.ldp, m, n, eA, eB, ctab, C, ldc, st, &g.launches[3]));
-    CK(ph.mark());
+    int panels = (int)(n / 1024);
+    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
+    const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
+    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
+    for (int pnl = 0; pnl < panels; ++pnl) {
+        const int64_t j0 = pnl * panel_cols, j1 = (j0 + panel_cols < n) ? j0 + panel_cols : n;
+        if (j0 >= j1) break;
+        ga.row_begin = j0;
+        ga.row_end = j1;
+        CK(ph.begin(2, st));
+        if (int s = run_gemm(ga, nmod, st)) return s;
+        CK(ph.end(st));
+        const bool last = j1 >= n;
+        cudaStream_t ps = last ? st : g.side;
+        if (!last) {
+            CK(cudaEventRecord(g.panel_done[pnl], st));
+            CK(cudaStreamWaitEvent(g.side, g.panel_done[pnl], 0));
+        }
+        CK(ph.begin(3, ps));
+        CK(launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]));
+        CK(ph.end(ps));
+    }
+    if (panels > 1) {   // join: the call is complete on the caller's stream only when the side stream has finished
+        CK(cudaEventRecord(g.side_done, g.side));
+        CK(cudaStreamWaitEvent(st, g.side_done, 0));
+    }
     ph.done();
     return GEMM2M_OK;
 }
@@ -268,11 +312,11 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     CrtTableInt ctab;
     build_crt_table_int(nmod, &ctab);
     Phases ph;
-    if (int s = begin_call(st, &ph)) return s;
-    CK(ph.mark());   // no scan phase
+    if (int s = begin_call(&ph)) return s;
+    CK(ph.begin(1, st));
     CK(launch_residues_int8(Ar, Ai, lda, false, m, k, c.kp, rtab, apm, st, &g.launches[1]));
     CK(launch_residues_int8(Br, Bi, ldb, true, n, k, c.kp, rtab, bpm, st, &g.launches[1]));
-    CK(ph.mark());
+    CK(ph.end(st));
     GemmArgs ga;
     ga.rowop = bpm; ga.colop = apm;
     ga.R = n; ga.Cn = m; ga.Kp = c.kp;
@@ -282,10 +326,13 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     ga.out = cpm; ga.ldp = c.ldp;
     build_mod_table(nmod, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
+    ga.row_begin = 0; ga.row_end = n;
+    CK(ph.begin(2, st));
     if (int s = run_gemm(ga, nmod, st)) return s;
-    CK(ph.mark());
+    CK(ph.end(st));
+    CK(ph.begin(3, st));
     CK(launch_post_int(cpm, c.ldp, m, n, ctab, Cr, Ci, ldc, st, &g.launches[3]));
-    CK(ph.mark());
+    CK(ph.end(st));
     ph.done();
     return GEMM2M_OK;
 }
@@ -324,14 +371,16 @@ int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64
     CrtTable ctab;
     build_crt_table(nmod, &ctab);
     Phases ph;
-    if (int s = begin_call(st, &ph)) return s;
+    if (int s = begin_call(&ph)) return s;
+    CK(ph.begin(0, st));
     CK(cudaMemsetAsync(absA, 0, (size_t)8 * n, st));
     CK(launch_scan_rows<double>(A, n, k, lda, absA, st, &g.launches[0]));
     CK(launch_exponents<double>(absA, n, sc.PA, sc.ck, eA, st, &g.launches[0]));
-    CK(ph.mark());
+    CK(ph.end(st));
+    CK(ph.begin(1, st));
     if (k == 0) CK(cudaMemsetAsync(apm, 0, (size_t)2 * nmod * n * c.kp, st));
     else CK(launch_residues_fp<double>(A, lda, false, n, k, c.kp, eA, rtab, sc.PA - sc.ck > 62, apm, st, &g.launches[1]));
-    CK(ph.mark());
+    CK(ph.end(st));
     // Section 5: C+ = A+ A-^T only.  TMEM columns (contiguous index i of the output) <- rows of A+, TMEM lanes (j) <- rows of A-,
     // so that out[j][i] = sum_k A+[i,k] A-[j,k] = C+[i,j].
     GemmArgs ga;
@@ -344,10 +393,13 @@ int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64
     ga.out = cp; ga.ldp = c.ldp;
     build_mod_table(nmod, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
+    ga.row_begin = 0; ga.row_end = n;
+    CK(ph.begin(2, st));
     if (int s = run_gemm(ga, nmod, st)) return s;
-    CK(ph.mark());
+    CK(ph.end(st));
+    CK(ph.begin(3, st));
     CK(launch_post_herk(cp, c.ldp, n, eA, ctab, C, ldc, st, &g.launches[3]));
-    CK(ph.mark());
+    CK(ph.end(st));
     ph.done();
     return GEMM2M_OK;
 }
@@ -378,12 +430,12 @@ int gemm2m_phase_ms(float ms[4], int* calls) {
     if (!ms || count == 0) return GEMM2M_ERR_ARG;
     for (int i = 0; i < 4; ++i) ms[i] = 0.f;
     for (int c = 0; c < count; ++c) {
-        cudaEvent_t* ev = g.ev[c];
-        CK(cudaEventSynchronize(ev[4]));
-        for (int i = 0; i < 4; ++i) {
+        const State::Slot& slot = g.slots[c];
+        for (int i = 0; i < slot.n; ++i) {
             float t = 0.f;
-            CK(cudaEventElapsedTime(&t, ev[i], ev[i + 1]));
-            ms[i] += t / (float)count;
+            CK(cudaEventSynchronize(slot.iv[i].b));
+            CK(cudaEventElapsedTime(&t, slot.iv[i].a, slot.iv[i].b));
+            ms[slot.iv[i].phase] += t / (float)count;
         }
     }
     if (calls) *calls = count;
@@ -398,6 +450,13 @@ int gemm2m_last_launch_count(int per_phase[4]) {
         total += g.launches[i];
     }
     return total;
+}
+
+int gemm2m_debug_set_panels(int max_panels) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (max_panels < 1 || max_panels > State::kMaxPanels) return GEMM2M_ERR_ARG;
+    g.max_panels = max_panels;
+    return GEMM2M_OK;
 }
 
 int gemm2m_debug_set_gemm_kernel(int which) {

@@ -86,7 +86,8 @@ template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, boo
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
-template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const int32_t* eA, const int32_t* eB,
+// Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).
+template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
                                                  const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches);
 cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
                              cudaStream_t st, int* launches);
@@ -99,6 +100,7 @@ cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n
 struct GemmArgs {
     const int8_t* rowop; const int8_t* colop;
     int64_t R, Cn, Kp;
+    int64_t row_begin, row_end;       // rows of the row operand handled by this launch (multiples of 256, or R)
     int row_planes, col_planes;       // number of planes behind each pointer (for the tensor maps)
     int row_plane0, col_plane0, nbatch;
     int8_t* out; int64_t ldp;

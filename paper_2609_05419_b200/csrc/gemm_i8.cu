@@ -188,7 +188,7 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
 
 cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches) {
     using namespace cfg;
-    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0) return cudaSuccess;
+    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0 || a.row_end <= a.row_begin) return cudaSuccess;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(gemm_i8_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
@@ -201,7 +201,8 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count
     GemmKernelParams p;
     p.R = a.R;
     p.Cn = a.Cn;
-    p.tiles_r = (int)((a.R + BM - 1) / BM);
+    p.tr0 = (int)(a.row_begin / BM);
+    p.tiles_r = (int)((a.row_end - a.row_begin + BM - 1) / BM);
     p.tiles_c = (int)((a.Cn + BN - 1) / BN);
     p.nbatch = a.nbatch;
     p.row_plane0 = a.row_plane0;
@@ -231,11 +232,12 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count
 // Plain CUDA-core version of the same contract (one thread per output entry, dp4a over K).  Only for tests.
 __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __restrict__ rowop, const int8_t* __restrict__ colop, int64_t R,
                                                             int64_t Cn, int64_t Kp, int64_t k_chunk, int row_plane0, int col_plane0,
-                                                            int8_t* __restrict__ out, int64_t ldp, const __grid_constant__ ModTable mods) {
+                                                            int8_t* __restrict__ out, int64_t ldp, const __grid_constant__ ModTable mods,
+                                                            int64_t row_begin, int64_t row_end) {
     const int64_t c = (int64_t)blockIdx.x * 16 + (threadIdx.x & 15);
-    const int64_t r = (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
+    const int64_t r = row_begin + (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
     const int b = blockIdx.z;
-    if (r >= R || c >= Cn) return;
+    if (r >= R || r >= row_end || c >= Cn) return;
     const int jm = b % mods.nmod;
     const int m = mods.m[jm];
     const int* pr = reinterpret_cast<const int*>(rowop + ((int64_t)(row_plane0 + b) * R + r) * Kp);
@@ -253,11 +255,12 @@ __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __rest
 }
 
 cudaError_t launch_gemm_check(const GemmArgs& a, int64_t k_limit, cudaStream_t st, int* launches) {
-    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0) return cudaSuccess;
+    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0 || a.row_end <= a.row_begin) return cudaSuccess;
     int64_t chunk = (k_limit / cfg::BK) * cfg::BK;
     if (chunk <= 0) chunk = cfg::BK;
-    dim3 grid((unsigned)((a.Cn + 15) / 16), (unsigned)((a.R + 15) / 16), (unsigned)a.nbatch);
-    gemm_i8_check_kernel<<<grid, 256, 0, st>>>(a.rowop, a.colop, a.R, a.Cn, a.Kp, chunk, a.row_plane0, a.col_plane0, a.out, a.ldp, a.mods);
+    dim3 grid((unsigned)((a.Cn + 15) / 16), (unsigned)((a.row_end - a.row_begin + 15) / 16), (unsigned)a.nbatch);
+    gemm_i8_check_kernel<<<grid, 256, 0, st>>>(a.rowop, a.colop, a.R, a.Cn, a.Kp, chunk, a.row_plane0, a.col_plane0, a.out, a.ldp, a.mods,
+                                               a.row_begin, a.row_end);
     ++*launches;
     return cudaGetLastError();
 }

@@ -237,7 +237,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
 
 cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches) {
     using namespace cfg2;
-    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0) return cudaSuccess;
+    if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0 || a.row_end <= a.row_begin) return cudaSuccess;
     static bool attr_set = false;
     static int max_pairs = 0;
     if (!attr_set) {
@@ -267,7 +267,8 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
     GemmKernelParams p;
     p.R = a.R;
     p.Cn = a.Cn;
-    p.tiles_r = (int)((a.R + 2 * BM - 1) / (2 * BM));
+    p.tr0 = (int)(a.row_begin / (2 * BM));
+    p.tiles_r = (int)((a.row_end - a.row_begin + 2 * BM - 1) / (2 * BM));
     p.tiles_c = (int)((a.Cn + BN - 1) / BN);
     p.nbatch = a.nbatch;
     p.row_plane0 = a.row_plane0;

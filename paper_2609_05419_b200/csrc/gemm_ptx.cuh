@@ -142,6 +142,7 @@ struct GemmKernelParams {
     int64_t ldp, out_plane_stride;
     int accumulate;          // add the residues already stored in `out` (later K chunks)
     int band;                // tile rasterisation: row tiles per band (see decode_tile)
+    int tr0;                 // first row tile of this launch (tiles_r counts the row tiles of the launch)
     ModTable mods;
     int* dev_status;
 };
@@ -157,7 +158,7 @@ __device__ __forceinline__ void decode_tile(const GemmKernelParams& p, int tile,
     const int band_idx = rem / per_band, in_band = rem - band_idx * per_band;
     const int rows_here = min(p.band, p.tiles_r - band_idx * p.band);
     *tc = in_band / rows_here;
-    *tr = band_idx * p.band + (in_band - *tc * rows_here);
+    *tr = p.tr0 + band_idx * p.band + (in_band - *tc * rows_here);
 }
 
 // ------------------------------------------------------------------------------------------------ host side

@@ -262,7 +262,12 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
 }
 
 // ---- floating-point inputs: persistent blocks, raw elements copied asynchronously into a two-stage ring -------------
-constexpr int kResRows = 16, kResK = 128, kResThreads = 256, kResRun = 8;
+#ifndef GEMM2M_RES_ROWS
+#define GEMM2M_RES_ROWS 8
+#endif
+constexpr int kResRows = GEMM2M_RES_ROWS, kResK = 128, kResRun = 8, kResThreads = kResRows * kResK / kResRun;
+constexpr int kResBlocksPerSm = 768 / kResThreads;
+constexpr int kResIThreads = 256;
 constexpr int kResRowStride = kResK + kResK / kResRun + 1;   // in elements: one pad per run of 8 + odd row stride -> no bank conflicts
 constexpr int kResStages = 2;
 
@@ -280,7 +285,7 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <typename T, bool WIDE>
-__global__ void __launch_bounds__(kResThreads, 3) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
+__global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
                                                                      int64_t Kp, const int32_t* __restrict__ e,
                                                                      const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
     using Raw = typename RawCplx<T>::type;
@@ -393,7 +398,7 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_
         attr_set = true;
     }
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
-    const int64_t resident = (int64_t)cached_sm_count() * 3;
+    const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
     if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
     else residues_fp_kernel<T, false><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
@@ -405,7 +410,7 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_
 constexpr int kResIRows = 32, kResIRun = 16;
 constexpr int kResIRowStride = kResK + kResK / kResIRun + 1;
 
-__global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t* __restrict__ Xr, const int8_t* __restrict__ Xi, int64_t ld,
+__global__ void __launch_bounds__(kResIThreads) residues_int8_kernel(const int8_t* __restrict__ Xr, const int8_t* __restrict__ Xi, int64_t ld,
                                                                     bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                                                     const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -424,10 +429,10 @@ __global__ void __launch_bounds__(kResThreads) residues_int8_kernel(const int8_t
     };
     if (!k_contiguous) {
         const int r = t & 31;
-        for (int kk = t >> 5; kk < kResK; kk += kResThreads / 32) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
+        for (int kk = t >> 5; kk < kResK; kk += kResIThreads / 32) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
     } else {
         const int kk = t & (kResK - 1);
-        for (int r = t >> 7; r < kResIRows; r += kResThreads / kResK) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
+        for (int r = t >> 7; r < kResIRows; r += kResIThreads / kResK) tile[r * kResIRowStride + kk + (kk >> 4)] = fetch(r, kk);
     }
     __syncthreads();
     const int g = t & 7, r = t >> 3;
@@ -454,7 +459,7 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
         attr_set = true;
     }
     dim3 grid((unsigned)(Kp / kResK), (unsigned)((R + kResIRows - 1) / kResIRows));
-    residues_int8_kernel<<<grid, kResThreads, smem, st>>>(Xr, Xi, ld, k_contiguous, R, K, Kp, tab, planes);
+    residues_int8_kernel<<<grid, kResIThreads, smem, st>>>(Xr, Xi, ld, k_contiguous, R, K, Kp, tab, planes);
     ++*launches;
     return cudaGetLastError();
 }
@@ -597,12 +602,12 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
 }
 
 template <typename T>
-cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const int32_t* eA, const int32_t* eB, const CrtTable& tab,
-                           T* C, int64_t ldc, cudaStream_t st, int* launches) {
-    if (m <= 0 || n <= 0) return cudaSuccess;
+cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                           const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
     const int64_t per_block = kPostSpan;
-    for (int64_t j0 = 0; j0 < n; j0 += 65535) {      // grid.y limit
-        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+    for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {      // grid.y limit
+        const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
         dim3 grid((unsigned)((m + per_block - 1) / per_block), (unsigned)nj);
         const int8_t* src = cpm + j0 * ldp;
         T* dst = C + 2 * j0 * ldc;
@@ -779,7 +784,7 @@ template cudaError_t launch_exponents<double>(const uint64_t*, int64_t, int, int
 template cudaError_t launch_exponents<float>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
 template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
 template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
-template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, cudaStream_t, int*);
-template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, cudaStream_t, int*);
+template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, cudaStream_t, int*);
+template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, cudaStream_t, int*);
 
 }  // namespace gemm2m
