@@ -28,9 +28,9 @@ METRIC = "zgemm2m_effective_tflops_8mnk_per_t"
 UNIT = "TFLOP/s"
 INT8_NOMINAL_TOPS = 4500.0          # dense int8, nominal
 INT8_OVER_BF16 = 2.0                # nominal ratio used to turn the measured bf16 peak into an int8 peak
-# DRAM bytes (read + write) of the GEMM launch per byte of int8 planes it touches, from the ncu capture of the 4096^3,
-# 16-modulus case (profiles/gemm_i8_tcgen05_pair_4096_nmod16.md): (1.156 + 0.519) GB over 3 x 536.9 MB of planes.
-GEMM_DRAM_BYTES_PER_PLANE_BYTE = (1.155904e9 + 0.519411968e9) / (3 * 32 * 4096 * 4096)
+# DRAM bytes (read + write) of a GEMM launch per byte of the int8 planes it touches, from the ncu capture of one panel launch of
+# the 4096^3, 16-modulus case (profiles/gemm_i8_tcgen05_pair_4096_nmod16.md): (673.9 + 123.9) MB over 805.3 MB of planes.
+GEMM_DRAM_BYTES_PER_PLANE_BYTE = (673.872384e6 + 123.916288e6) / (32 * 4096 * (4096 + 1024 + 1024))
 
 
 def job_value(flops_per_rank_step, world, ms_per_step):
@@ -315,8 +315,8 @@ def run_ours(a):
     post_bytes = m * n * (2 * nmod + 16)
     roofline = {"bound": "tensor", "kernel": "gemm_i8_tcgen05_pair_kernel", "achieved": gemm_tops, "peak": int8_peak, "unit": "TFLOP/s",
                 "frac": gemm_tops / int8_peak,
-                "traffic": GEMM_DRAM_BYTES_PER_PLANE_BYTE * 2 * nmod * (m * c_kp + n * c_kp + n * c_ldp) / gemm_launches,
-                "traffic_source": "ncu dram__bytes_read+write of the 4096^3 launch, scaled by plane bytes",
+                "traffic": GEMM_DRAM_BYTES_PER_PLANE_BYTE * 2 * nmod * (m * c_kp + (n * c_kp + n * c_ldp) / gemm_launches),
+                "traffic_source": "ncu dram__bytes_read+write of one panel launch at 4096^3, scaled by the plane bytes a launch touches",
                 "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS rate (int8:bf16 nominal ratio); int8 ops counted as 2 per MAC",
                 "frac_of_nominal_4500": gemm_tops / INT8_NOMINAL_TOPS,
                 "launch_ms": phase[2] / gemm_launches, "launches_per_step": gemm_launches, "algorithmic_ops_per_launch": gemm_ops}
