@@ -253,3 +253,46 @@ def test_device_status_and_launch_counts():
             b.set_profiling(False)
     assert calls == 1 and all(x >= 0 for x in ms) and sum(ms) > 0
     assert per == [4, 2, 1, 1] and total == 8
+
+
+def test_panel_pipeline_is_bitwise_identical_and_joins_the_callers_stream():
+    # zgemm2m cuts C into column panels and post-processes them on an internal stream; the result must not depend on the
+    # number of panels, and work queued on the caller's stream right after the call must see all of C.
+    m, n, k = 300, 2304, 256                      # 2304 columns -> 2 panels of 1280 / 1024
+    A, B = inputs.complex_inputs(m, n, k, seed=17, dist="phi", phi=1.0)
+    dA, dB = to_dev(A), to_dev(B)
+    outs = []
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, 16)):
+        side = torch.cuda.Stream()
+        for panels in (1, 4, 2, 4):
+            b.debug_set_panels(panels)
+            C = empty_dev(m, n, torch.complex128, fill=7.0)
+            snap = torch.empty_like(C)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                b.zgemm2m(dA, dB, C, 16, side)
+                snap.copy_(C)                     # same stream, no synchronisation in between
+            side.synchronize()
+            b.device_status(side)
+            outs.append((to_host(C), to_host(snap)))
+        b.debug_set_panels(4)
+    ref = staged.zgemm2m_staged(A, B, 16)["C"]
+    for C, snap in outs:
+        assert (C == outs[0][0]).all() and (snap == C).all()
+    assert ulp_distance(outs[0][0].real, ref.real).max() <= 1 and ulp_distance(outs[0][0].imag, ref.imag).max() <= 1
+
+
+def test_back_to_back_calls_of_different_sizes_share_a_workspace():
+    shapes = [(512, 2048, 128), (100, 130, 200), (256, 4096, 64), (64, 1100, 300)]
+    need = max(b.workspace_bytes(b.OP_ZGEMM, m, n, k, 16) for m, n, k in shapes)
+    data = [inputs.complex_inputs(m, n, k, seed=20 + i) for i, (m, n, k) in enumerate(shapes)]
+    with Workspace(need):
+        dev = [(to_dev(A), to_dev(B), empty_dev(A.shape[0], B.shape[1], torch.complex128)) for A, B in data]
+        for _ in range(2):
+            for dA, dB, dC in dev:                # no synchronisation between the calls
+                b.zgemm2m(dA, dB, dC, 16)
+        b.device_status()
+        got = [to_host(dC) for _, _, dC in dev]
+    for (A, B), C in zip(data, got):
+        Cref, D = direct.zgemm4m_dd(A, B)
+        assert direct.componentwise_error(C, Cref, D) <= TOL_Z
