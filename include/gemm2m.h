@@ -49,7 +49,10 @@ typedef enum {
     GEMM2M_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait gave up (reported by gemm2m_device_status) */
 } gemm2m_status;
 
-typedef enum { GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3 } gemm2m_op;
+typedef enum {
+    GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3,
+    GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6
+} gemm2m_op;
 
 /* Human-readable name of a status code (static string). */
 const char* gemm2m_status_string(int status);
@@ -61,7 +64,7 @@ int gemm2m_max_moduli(void);
 /* j-th modulus (0-based, descending) and its smallest positive square root of -1 (Section 2).  Host pointers. */
 int gemm2m_modulus(int j, int* m, int* s);
 
-/* Bytes of device workspace a call of `op` with these sizes needs (for zherk2m pass m = n).  0 on bad arguments. */
+/* Bytes of device workspace a call of `op` with these sizes needs (for the rank-k family pass m = n).  0 on bad arguments. */
 size_t gemm2m_workspace_bytes(int op, int64_t m, int64_t n, int64_t k, int nmod);
 /* Register a caller-owned device buffer (256-byte aligned) used by later calls of this host thread's current
  * device.  Passing (NULL, 0) unregisters.  The buffer must stay valid until the last call using it has finished. */
@@ -89,6 +92,23 @@ int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const 
  * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
  * diagonal is written; diagonal imaginary parts are exactly 0; the strict upper triangle is not touched. */
 int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream);
+
+/* Hermitian rank-2k update C = A B^H + B A^H (Section 5, HER2K) with TWO real int8 GEMMs per modulus instead of four:
+ * with one scale vector for A and B (sigma = tau) the sum moves into the residue domain,
+ * C+ = A+ B-^T + B+ A-^T (mod m_j) and C- = C+^T.  A, B: n x k complex128 (lda, ldb >= n).  Lower triangle of C as for
+ * zherk2m. */
+int zher2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc, int nmod,
+             void* stream);
+
+/* Real symmetric rank-k update C = A A^T (Section 5, SYRK) as the real part of the HERK of Z = A1 + i A2, where A1, A2 are
+ * the two halves of the k dimension (a zero column is appended when k is odd): one real int8 GEMM of half the inner
+ * dimension per modulus.  A: n x k real doubles (lda >= n); C: n x n real doubles (ldc >= n), lower triangle written. */
+int dsyrk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream);
+
+/* Real symmetric rank-2k update C = A B^T + B A^T (Section 5, SYR2K) as the real part of the HER2K of Z_A = A1 + i A2 and
+ * Z_B = B1 + i B2.  A, B: n x k real doubles; C as for dsyrk2m. */
+int dsyr2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc, int nmod,
+             void* stream);
 
 /* (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
  * Scale exponents without any allocation.  Some programs that would like to use this library are not allowed to

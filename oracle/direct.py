@@ -6,6 +6,8 @@
   symmetric_residue  representative of x mod M in [-(M-1)/2, (M-1)/2] (Section 2, first paragraph;
                      Algorithm 1 step 6).
   zgemm4m_dd         4M complex product with double-double accumulation plus D = |A||B|.
+  zherk_dd, zher2k_dd, dsyrk_dd, dsyr2k_dd   the rank-k definitions of Section 5 (C = A A^H, A B^H + B A^H, A A^T,
+                     A B^T + B A^T), each entry one double-double accumulation.
   componentwise_error  max_ij |C - Cref| / D_ij, the acceptance metric.
 """
 from __future__ import annotations
@@ -128,6 +130,46 @@ def zgemm4m_dd_samples(A, B, pairs):
         lib().oracle_zgemm4m_dd_samples(_i64(k), _p(A), _i64(max(m, 1)), _p(B), _i64(max(k, 1)), _i64(S),
                                         _p(rows), _p(cols), _p(C), _p(D))
     return C, D
+
+
+def zgemm4m_dd2(A1, B1, A2, B2):
+    """C = A1 B1 + A2 B2 accumulated in double-double over both products, and D = |A1||B1| + |A2||B2|."""
+    A1, B1, A2, B2 = _as_z(A1), _as_z(B1), _as_z(A2), _as_z(B2)
+    m, k = A1.shape
+    n = B1.shape[1]
+    assert A2.shape == (m, k) and B1.shape == (k, n) and B2.shape == (k, n)
+    C = np.zeros((m, n), dtype=np.complex128, order="F")
+    D = np.zeros((m, n), dtype=np.float64, order="F")
+    if m and n:
+        lib().oracle_zgemm4m_dd2(_i64(m), _i64(n), _i64(k), _p(A1), _i64(max(m, 1)), _p(B1), _i64(max(k, 1)),
+                                 _p(A2), _i64(max(m, 1)), _p(B2), _i64(max(k, 1)), _p(C), _i64(max(m, 1)), _p(D), _i64(max(m, 1)))
+    return C, D
+
+
+def zherk_dd(A):
+    """Section 5, HERK: C = A A^H."""
+    A = _as_z(A)
+    return zgemm4m_dd(A, A.conj().T)
+
+
+def zher2k_dd(A, B):
+    """Section 5, HER2K: C = A B^H + B A^H."""
+    A, B = _as_z(A), _as_z(B)
+    return zgemm4m_dd2(A, B.conj().T, B, A.conj().T)
+
+
+def dsyrk_dd(A):
+    """Section 5, SYRK: C = A A^T for real A (returned real)."""
+    A = np.asarray(A, dtype=np.float64)
+    C, D = zgemm4m_dd(A.astype(np.complex128), A.T.astype(np.complex128))
+    return np.asfortranarray(C.real), D
+
+
+def dsyr2k_dd(A, B):
+    """Section 5, SYR2K: C = A B^T + B A^T for real A, B (returned real)."""
+    A, B = np.asarray(A, dtype=np.float64), np.asarray(B, dtype=np.float64)
+    C, D = zgemm4m_dd2(A.astype(np.complex128), B.T.astype(np.complex128), B.astype(np.complex128), A.T.astype(np.complex128))
+    return np.asfortranarray(C.real), D
 
 
 def componentwise_error(C, Cref, D):

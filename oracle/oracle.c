@@ -11,6 +11,8 @@
  *                         real dot products accumulated in double-double (about 106 bits),
  *                         rounded once to double; also D = |A||B| with complex moduli.
  *   oracle_zgemm4m_dd_samples : the same for a list of (i, j) entries only.
+ *   oracle_zgemm4m_dd2  : C = A1 B1 + A2 B2 (the two-product sums of the rank-2k updates of Section 5), one double-double
+ *                         accumulation over both products, rounded once.
  *
  * All matrices are column-major; complex matrices are interleaved (re, im) doubles with the
  * leading dimension counted in complex elements.
@@ -158,5 +160,38 @@ void oracle_zgemm4m_dd_samples(int64_t k, const double* A, int64_t lda, const do
             D[s] = d;
         }
         free(arow);
+    }
+}
+
+/* C = A1 B1 + A2 B2 with A1, A2: m x k and B1, B2: k x n (all interleaved complex, column-major); D = |A1||B1| + |A2||B2|. */
+void oracle_zgemm4m_dd2(int64_t m, int64_t n, int64_t k,
+                        const double* A1, int64_t lda1, const double* B1, int64_t ldb1,
+                        const double* A2, int64_t lda2, const double* B2, int64_t ldb2,
+                        double* C, int64_t ldc, double* D, int64_t ldd) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < m; ++i) {
+        for (int64_t j = 0; j < n; ++j) {
+            dd rr = {0, 0}, ii = {0, 0}, ri = {0, 0}, ir = {0, 0};
+            double d = 0.0;
+            for (int pass = 0; pass < 2; ++pass) {
+                const double* A = pass ? A2 : A1;
+                const double* B = pass ? B2 : B1;
+                const int64_t lda = pass ? lda2 : lda1, ldb = pass ? ldb2 : ldb1;
+                for (int64_t p = 0; p < k; ++p) {
+                    double ar = A[2 * (i + p * lda)], ai = A[2 * (i + p * lda) + 1];
+                    double br = B[2 * (p + j * ldb)], bi = B[2 * (p + j * ldb) + 1];
+                    rr = dd_mac(rr, ar, br);
+                    ii = dd_mac(ii, ai, bi);
+                    ri = dd_mac(ri, ar, bi);
+                    ir = dd_mac(ir, ai, br);
+                    d += hypot(ar, ai) * hypot(br, bi);
+                }
+            }
+            dd r = dd_add(rr, dd_neg(ii));
+            dd im = dd_add(ri, ir);
+            C[2 * (i + j * ldc)] = r.hi + r.lo;
+            C[2 * (i + j * ldc) + 1] = im.hi + im.lo;
+            D[i + j * ldd] = d;
+        }
     }
 }

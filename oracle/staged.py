@@ -280,6 +280,46 @@ def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto
     return st
 
 
+def syrk_complexify(X):
+    """Section 5, SYRK paragraph: split real X (n x k) evenly in the k dimension, X = [X1 | X2] (a zero column is appended
+    when k is odd), and form Z = X1 + i X2; then X X^T = Re(Z Z^H)."""
+    X = np.asarray(X, dtype=np.float64)
+    n, k = X.shape
+    k2 = (k + 1) // 2
+    Z = np.zeros((n, k2), dtype=np.complex128, order="F")
+    Z.real = X[:, :k2]
+    Z.imag[:, : k - k2] = X[:, k2:]
+    return Z
+
+
+def zher2k2m_staged(A, B, nmod: int, out_bits: int = 53):
+    """Section 5, HER2K with 2M Ozaki-II: one scale vector for A and B (sigma = tau), then per modulus
+    C+ = A+ B-^T + B+ A-^T and C- = A- B+^T + B- A+^T (mod m), Eq. (2c), CRT, lift, unscale."""
+    A = np.asarray(A)
+    B = np.asarray(B)
+    n, k = A.shape
+    moduli = greedy_2m_moduli()[:nmod]
+    roots = [sqrt_minus_one(q) for q in moduli]
+    M = product(moduli)
+    Pt, P, _, ck = scaling_targets(M, 2 * k, herk=True)     # an entry is an inner product of rows of 2k complex numbers
+    eA = scaling_exponents(np.concatenate([A, B], axis=1), 1, P, ck)
+    Aq, Bq = quantise(A, eA, 1), quantise(B, eA, 1)
+    Apl = _residue_planes(Aq[0], Aq[1], moduli, roots)
+    Bpl = _residue_planes(Bq[0], Bq[1], moduli, roots)
+    Cpm, res_r, res_i = [], [], []
+    for (Ap, Am), (Bp, Bm), ml, sl in zip(Apl, Bpl, moduli, roots):
+        Cp = sym(_exact_matmul(Ap, Bm.T) + _exact_matmul(Bp, Am.T), ml)
+        Cm = sym(_exact_matmul(Am, Bp.T) + _exact_matmul(Bm, Ap.T), ml)
+        Cpm.append((Cp, Cm))
+        r, i = post_2m(Cp, Cm, ml, sl)
+        res_r.append(r)
+        res_i.append(i)
+    Xr, Xi = lift(crt(res_r, moduli), M), lift(crt(res_i, moduli), M)
+    C = unscale(Xr, eA, eA, out_bits) + 1j * unscale(Xi, eA, eA, out_bits)
+    return dict(moduli=moduli, roots=roots, M=M, Pt=Pt, P=P, ck=ck, eA=eA, Aq=Aq, Bq=Bq, Apm=Apl, Bpm=Bpl, Cpm=Cpm,
+                Xr=Xr, Xi=Xi, C=C)
+
+
 def staged_samples(st, pairs, out_bits: int = 53):
     """Exact lifted integers and final values for sampled entries, from the quantised matrices of a
     `zgemm2m_staged(..., upto="pre")` result: the 4M product of the quantised Gaussian integers reduced

@@ -10,7 +10,7 @@ from __future__ import annotations
 import ctypes
 import os
 
-OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK = 0, 1, 2, 3
+OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K = 0, 1, 2, 3, 4, 5, 6
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -54,6 +54,9 @@ def lib():
     L.zgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.cgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.zherk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
+    L.dsyrk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
+    L.zher2k2m.argtypes = [i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.dsyr2k2m.argtypes = [i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.gemm2m_device_status.argtypes = [vp]
     L.gemm2m_zscale_exponents_static.argtypes = [i64, i64, vp, i64, i32, vp, vp]
     L.gemm2m_set_profiling.argtypes = [i32]
@@ -175,6 +178,32 @@ def zscale_exponents_static(A, e, nmod=16, stream=None):
         raise ValueError("e: need a contiguous int32 CUDA tensor with one entry per row of A")
     _check(lib().gemm2m_zscale_exponents_static(m, k, pa, lda, nmod, ctypes.c_void_p(e.data_ptr()), _stream_ptr(stream)),
            "gemm2m_zscale_exponents_static")
+
+
+def _rank(fn, name, A, B, C, nmod, stream):
+    pa, n, k, lda = _colmajor(A, "A")
+    pc, n1, n2, ldc = _colmajor(C, "C")
+    if (n1, n2) != (n, n):
+        raise ValueError("shape mismatch")
+    if B is None:
+        _check(fn(n, k, pa, lda, pc, ldc, nmod, _stream_ptr(stream)), name)
+    else:
+        pb, nb, kb, ldb = _colmajor(B, "B")
+        if (nb, kb) != (n, k):
+            raise ValueError("shape mismatch")
+        _check(fn(n, k, pa, lda, pb, ldb, pc, ldc, nmod, _stream_ptr(stream)), name)
+
+
+def zher2k2m(A, B, C, nmod=16, stream=None):
+    _rank(lib().zher2k2m, "zher2k2m", A, B, C, nmod, stream)
+
+
+def dsyrk2m(A, C, nmod=16, stream=None):
+    _rank(lib().dsyrk2m, "dsyrk2m", A, None, C, nmod, stream)
+
+
+def dsyr2k2m(A, B, C, nmod=16, stream=None):
+    _rank(lib().dsyr2k2m, "dsyr2k2m", A, B, C, nmod, stream)
 
 
 def device_status(stream=None):

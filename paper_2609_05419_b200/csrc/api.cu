@@ -60,14 +60,17 @@ int check_device() {
 
 // Workspace: [status 256 B][absmax A u64][absmax B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each 256-byte aligned.
 struct Carve {
-    int64_t off_status, off_abs_a, off_abs_b, off_exp_a, off_exp_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
+    int64_t off_status, off_abs_a, off_abs_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
 };
 
 bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     if (m < 0 || n < 0 || k < 0 || nmod < 1 || nmod > kMaxMod) return false;
-    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_ZHERK) return false;
-    const bool herk = op == GEMM2M_OP_ZHERK;
+    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_DSYR2K) return false;
+    const bool herk = op >= GEMM2M_OP_ZHERK;                                   // the rank-k family: one scale vector, C+ only
+    const bool two = op == GEMM2M_OP_ZHER2K || op == GEMM2M_OP_DSYR2K;         // rank-2k: two operands
+    const bool real_in = op == GEMM2M_OP_DSYRK || op == GEMM2M_OP_DSYR2K;      // real input, packed as Z = X1 + i X2
     if (herk) m = n;
+    if (real_in) k = (k + 1) / 2;
     const int64_t kp = round_up(k > 0 ? k : 1, 128), ldp = round_up(m > 0 ? m : 1, 16);
     int64_t off = 0;
     auto take = [&](int64_t bytes) { int64_t o = off; off = round_up(off + bytes, 256); return o; };
@@ -76,8 +79,10 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_abs_b = take(herk ? 0 : 8 * n);
     c->off_exp_a = take(4 * m);
     c->off_exp_b = take(herk ? 0 : 4 * n);
+    c->off_pack_a = take(real_in ? 16 * n * k : 0);
+    c->off_pack_b = take(real_in && two ? 16 * n * k : 0);
     c->off_apm = take(2 * (int64_t)nmod * m * kp);
-    c->off_bpm = take(herk ? 0 : 2 * (int64_t)nmod * n * kp);
+    c->off_bpm = take((herk && !two) ? 0 : 2 * (int64_t)nmod * n * kp);
     c->off_cpm = take((herk ? 1 : 2) * (int64_t)nmod * n * ldp);
     c->kp = kp;
     c->ldp = ldp;
@@ -192,7 +197,7 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     ga.row_planes = ga.col_planes = 2 * nmod;
     ga.row_plane0 = ga.col_plane0 = 0;
     ga.nbatch = 2 * nmod;
-    ga.out = cpm; ga.ldp = c.ldp;
+    ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
     build_mod_table(nmod, &ga.mods);
     ga.dev_status = dev_status;
     int panels = (int)(n / 1024);
@@ -323,7 +328,7 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     ga.row_planes = ga.col_planes = 2 * nmod;
     ga.row_plane0 = ga.col_plane0 = 0;
     ga.nbatch = 2 * nmod;
-    ga.out = cpm; ga.ldp = c.ldp;
+    ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
     build_mod_table(nmod, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
     ga.row_begin = 0; ga.row_end = n;
@@ -347,25 +352,35 @@ int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const 
     return xgemm2m<float>(GEMM2M_OP_CGEMM, m, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
 }
 
-int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {
+// The rank-k family of Section 5: HERK (B == nullptr) and HER2K on complex inputs; SYRK / SYR2K on real inputs through
+// Z = X1 + i X2 (the halves of the k dimension), whose HERK / HER2K has the wanted matrix as its real part.
+static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
+                       int nmod, void* stream) {
     std::lock_guard<std::mutex> lock(g.mu);
+    const bool two = op == GEMM2M_OP_ZHER2K || op == GEMM2M_OP_DSYR2K;
+    const bool real_in = op == GEMM2M_OP_DSYRK || op == GEMM2M_OP_DSYR2K;
     if (n < 0 || k < 0) return GEMM2M_ERR_ARG;
-    if (lda < (n > 1 ? n : 1) || ldc < (n > 1 ? n : 1)) return GEMM2M_ERR_ARG;
+    if (lda < (n > 1 ? n : 1) || ldc < (n > 1 ? n : 1) || (two && ldb < (n > 1 ? n : 1))) return GEMM2M_ERR_ARG;
     if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
     if (n > kMaxRows) return GEMM2M_ERR_ARG;
     if (n == 0) return GEMM2M_OK;
-    if (!C || (k > 0 && !A)) return GEMM2M_ERR_ARG;
+    if (!C || (k > 0 && (!A || (two && !B)))) return GEMM2M_ERR_ARG;
     if (int s = check_device()) return s;
     cudaStream_t st = (cudaStream_t)stream;
     Carve c;
-    if (!carve(GEMM2M_OP_ZHERK, n, n, k > 0 ? k : 1, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!carve(op, n, n, k > 0 ? k : 1, nmod, &c)) return GEMM2M_ERR_ARG;
     if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
     char* ws = (char*)g.ws;
     uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
     int32_t* eA = (int32_t*)(ws + c.off_exp_a);
     int8_t* apm = (int8_t*)(ws + c.off_apm);
+    int8_t* bpm = (int8_t*)(ws + c.off_bpm);
     int8_t* cp = (int8_t*)(ws + c.off_cpm);
-    const ScaleTargets sc = scale_targets(nmod, k, true);
+    const int64_t kc = real_in ? (k + 1) / 2 : k;                   // inner dimension of the complex problem
+    // One scale vector for both operands (sigma = tau).  A rank-2k entry is the inner product of two rows of 2 kc complex
+    // numbers, so its rows count 2 kc terms in the 2-norm bound.
+    const ScaleTargets sc = scale_targets(nmod, two ? 2 * kc : kc, true);
+    const bool wide = sc.PA - sc.ck > 62;
     ResidueTable rtab;
     build_residue_table(nmod, &rtab);
     CrtTable ctab;
@@ -373,18 +388,37 @@ int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64
     Phases ph;
     if (int s = begin_call(&ph)) return s;
     CK(ph.begin(0, st));
+    const double* ZA = A;
+    const double* ZB = B;
+    int64_t ldza = lda, ldzb = ldb;
+    if (real_in && k > 0) {
+        CK(launch_pack_real_pair(A, lda, n, k, (double*)(ws + c.off_pack_a), st, &g.launches[0]));
+        ZA = (const double*)(ws + c.off_pack_a);
+        ldza = n;
+        if (two) {
+            CK(launch_pack_real_pair(B, ldb, n, k, (double*)(ws + c.off_pack_b), st, &g.launches[0]));
+            ZB = (const double*)(ws + c.off_pack_b);
+            ldzb = n;
+        }
+    }
     CK(cudaMemsetAsync(absA, 0, (size_t)8 * n, st));
-    CK(launch_scan_rows<double>(A, n, k, lda, absA, st, &g.launches[0]));
+    CK(launch_scan_rows<double>(ZA, n, k > 0 ? kc : 0, ldza, absA, st, &g.launches[0]));
+    if (two) CK(launch_scan_rows<double>(ZB, n, k > 0 ? kc : 0, ldzb, absA, st, &g.launches[0]));
     CK(launch_exponents<double>(absA, n, sc.PA, sc.ck, eA, st, &g.launches[0]));
     CK(ph.end(st));
     CK(ph.begin(1, st));
-    if (k == 0) CK(cudaMemsetAsync(apm, 0, (size_t)2 * nmod * n * c.kp, st));
-    else CK(launch_residues_fp<double>(A, lda, false, n, k, c.kp, eA, rtab, sc.PA - sc.ck > 62, apm, st, &g.launches[1]));
+    if (k == 0) {
+        CK(cudaMemsetAsync(apm, 0, (size_t)2 * nmod * n * c.kp, st));
+        if (two) CK(cudaMemsetAsync(bpm, 0, (size_t)2 * nmod * n * c.kp, st));
+    } else {
+        CK(launch_residues_fp<double>(ZA, ldza, false, n, kc, c.kp, eA, rtab, wide, apm, st, &g.launches[1]));
+        if (two) CK(launch_residues_fp<double>(ZB, ldzb, false, n, kc, c.kp, eA, rtab, wide, bpm, st, &g.launches[1]));
+    }
     CK(ph.end(st));
-    // Section 5: C+ = A+ A-^T only.  TMEM columns (contiguous index i of the output) <- rows of A+, TMEM lanes (j) <- rows of A-,
-    // so that out[j][i] = sum_k A+[i,k] A-[j,k] = C+[i,j].
+    // Section 5.  HERK: C+ = A+ A-^T.  HER2K: C+ = A+ B-^T + B+ A-^T (second product accumulated mod m_j).  C- = C+^T in both.
+    // TMEM columns (contiguous index i of the output) <- rows of the "+" planes, TMEM lanes (j) <- rows of the "-" planes,
+    // so that out[j][i] = sum_k X+[i,k] Y-[j,k].
     GemmArgs ga;
-    ga.rowop = apm; ga.colop = apm;
     ga.R = n; ga.Cn = n; ga.Kp = c.kp;
     ga.row_planes = ga.col_planes = 2 * nmod;
     ga.row_plane0 = nmod;    // "-" planes
@@ -395,13 +429,36 @@ int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64
     ga.dev_status = (int*)(ws + c.off_status);
     ga.row_begin = 0; ga.row_end = n;
     CK(ph.begin(2, st));
+    ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
     if (int s = run_gemm(ga, nmod, st)) return s;
+    if (two) {
+        ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
+        if (int s = run_gemm(ga, nmod, st)) return s;
+    }
     CK(ph.end(st));
     CK(ph.begin(3, st));
-    CK(launch_post_herk(cp, c.ldp, n, eA, ctab, C, ldc, st, &g.launches[3]));
+    CK(launch_post_herk(cp, c.ldp, n, eA, ctab, C, ldc, real_in, st, &g.launches[3]));
     CK(ph.end(st));
     ph.done();
     return GEMM2M_OK;
+}
+
+int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {
+    return rank_update(GEMM2M_OP_ZHERK, n, k, A, lda, nullptr, 0, C, ldc, nmod, stream);
+}
+
+int zher2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc, int nmod,
+             void* stream) {
+    return rank_update(GEMM2M_OP_ZHER2K, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
+}
+
+int dsyrk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {
+    return rank_update(GEMM2M_OP_DSYRK, n, k, A, lda, nullptr, 0, C, ldc, nmod, stream);
+}
+
+int dsyr2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc, int nmod,
+             void* stream) {
+    return rank_update(GEMM2M_OP_DSYR2K, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
 }
 
 int gemm2m_device_status(void* stream) {

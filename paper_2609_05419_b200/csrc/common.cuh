@@ -89,8 +89,11 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).
 template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
                                                  const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches);
+// real_out: C is a real matrix (SYRK / SYR2K through Z = A1 + i A2): only the real part is formed and stored.
 cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
-                             cudaStream_t st, int* launches);
+                             bool real_out, cudaStream_t st, int* launches);
+// Z[i, p] = X[i, p] + i X[i, p + k2] for p < k2 = ceil(k / 2) (zero beyond column k): the complex matrix whose HERK is the SYRK of X.
+cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_t k, double* Z, cudaStream_t st, int* launches);
 cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,
                             int64_t ldc, cudaStream_t st, int* launches);
 
@@ -104,6 +107,7 @@ struct GemmArgs {
     int row_planes, col_planes;       // number of planes behind each pointer (for the tensor maps)
     int row_plane0, col_plane0, nbatch;
     int8_t* out; int64_t ldp;
+    int accumulate;                   // add to the residues already stored in `out` (second product of a rank-2k update)
     ModTable mods;
     int* dev_status;
 };

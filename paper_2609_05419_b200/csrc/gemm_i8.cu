@@ -221,7 +221,7 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count
     for (int kb0 = 0; kb0 < kblocks_total; kb0 += chunk) {
         p.kblock0 = kb0;
         p.kblocks = (kblocks_total - kb0 < chunk) ? kblocks_total - kb0 : chunk;
-        p.accumulate = kb0 > 0;
+        p.accumulate = (kb0 > 0 || a.accumulate) ? 1 : 0;
         gemm_i8_tcgen05_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(map_row, map_col, p);
         ++*launches;
     }
@@ -233,7 +233,7 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count
 __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __restrict__ rowop, const int8_t* __restrict__ colop, int64_t R,
                                                             int64_t Cn, int64_t Kp, int64_t k_chunk, int row_plane0, int col_plane0,
                                                             int8_t* __restrict__ out, int64_t ldp, const __grid_constant__ ModTable mods,
-                                                            int64_t row_begin, int64_t row_end) {
+                                                            int64_t row_begin, int64_t row_end, int accumulate) {
     const int64_t c = (int64_t)blockIdx.x * 16 + (threadIdx.x & 15);
     const int64_t r = row_begin + (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
     const int b = blockIdx.z;
@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __rest
     const int m = mods.m[jm];
     const int* pr = reinterpret_cast<const int*>(rowop + ((int64_t)(row_plane0 + b) * R + r) * Kp);
     const int* pc = reinterpret_cast<const int*>(colop + ((int64_t)(col_plane0 + b) * Cn + c) * Kp);
-    int res = 0;
+    int res = accumulate ? (int)out[(int64_t)b * R * ldp + r * ldp + c] : 0;
     for (int64_t k0 = 0; k0 < Kp; k0 += k_chunk) {
         const int64_t k1 = (k0 + k_chunk < Kp) ? k0 + k_chunk : Kp;
         int acc = 0;
@@ -260,7 +260,7 @@ cudaError_t launch_gemm_check(const GemmArgs& a, int64_t k_limit, cudaStream_t s
     if (chunk <= 0) chunk = cfg::BK;
     dim3 grid((unsigned)((a.Cn + 15) / 16), (unsigned)((a.row_end - a.row_begin + 15) / 16), (unsigned)a.nbatch);
     gemm_i8_check_kernel<<<grid, 256, 0, st>>>(a.rowop, a.colop, a.R, a.Cn, a.Kp, chunk, a.row_plane0, a.col_plane0, a.out, a.ldp, a.mods,
-                                               a.row_begin, a.row_end);
+                                               a.row_begin, a.row_end, a.accumulate);
     ++*launches;
     return cudaGetLastError();
 }

@@ -287,7 +287,7 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
     for (int kb0 = 0; kb0 < kblocks_total; kb0 += chunk) {
         p.kblock0 = kb0;
         p.kblocks = (kblocks_total - kb0 < chunk) ? kblocks_total - kb0 : chunk;
-        p.accumulate = kb0 > 0;
+        p.accumulate = (kb0 > 0 || a.accumulate) ? 1 : 0;
         gemm_i8_tcgen05_pair_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(map_row, map_col, p);   // cluster size is a kernel attribute
         ++*launches;
     }

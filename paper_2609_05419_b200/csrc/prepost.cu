@@ -632,7 +632,7 @@ constexpr int kHerkI = 64, kHerkJ = 16, kHerkThreads = 256;
 constexpr int kHerkMirrorSlots = kHerkI + kHerkI / 8;                      // 16-byte slots, one pad slot per 8 rows (bank spread)
 constexpr int kHerkPlaneBytes = kHerkJ * kHerkI + kHerkMirrorSlots * 16;   // direct + mirrored bytes per modulus
 
-template <int NCH>
+template <int NCH, bool REAL_OUT>
 __global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n,
                                                                  const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
                                                                  double* __restrict__ C, int64_t ldc) {
@@ -679,7 +679,7 @@ __global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* _
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
-                Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
+                if (!REAL_OUT) Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
             }
         }
     }
@@ -689,49 +689,78 @@ __global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* _
         const int64_t i = i0 + e;
         if (i < n && i >= j) {
             const int ei = __ldg(eA + i);
-            double re, im;
+            double re, im = 0.0;
             if (ei == kExpNonFinite || ej == kExpNonFinite) {
                 re = im = __longlong_as_double(0x7FF8000000000000ll);
             } else {
                 double h, l;
                 crt_finish<NCH>(Sr[e], tab, &h, &l);
                 re = scale_pow2(h + l, ei + ej);
-                crt_finish<NCH>(Si[e], tab, &h, &l);
-                im = scale_pow2(h + l, ei + ej);
+                if (!REAL_OUT) {
+                    crt_finish<NCH>(Si[e], tab, &h, &l);
+                    im = scale_pow2(h + l, ei + ej);
+                }
             }
-            *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
+            if (REAL_OUT) C[i + j * ldc] = re;
+            else *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
         }
     }
 }
 
-cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
-                             cudaStream_t st, int* launches) {
-    if (n <= 0) return cudaSuccess;
+__global__ void __launch_bounds__(256) pack_real_pair_kernel(const double* __restrict__ X, int64_t ld, int64_t n, int64_t k, int64_t k2,
+                                                             double* __restrict__ Z) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t p = blockIdx.y;
+    if (i >= n) return;
+    const double re = __ldg(X + i + p * ld);
+    const double im = (p + k2 < k) ? __ldg(X + i + (p + k2) * ld) : 0.0;
+    *reinterpret_cast<double2*>(Z + 2 * (i + p * n)) = make_double2(re, im);
+}
+
+cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_t k, double* Z, cudaStream_t st, int* launches) {
+    const int64_t k2 = (k + 1) / 2;
+    if (n <= 0 || k2 <= 0) return cudaSuccess;
+    for (int64_t p0 = 0; p0 < k2; p0 += 65535) {      // grid.y limit
+        const int64_t np = (k2 - p0 < 65535) ? k2 - p0 : 65535;
+        dim3 grid((unsigned)((n + 255) / 256), (unsigned)np);
+        pack_real_pair_kernel<<<grid, 256, 0, st>>>(X + p0 * ld, ld, n, k - p0, k2, Z + 2 * p0 * n);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+template <bool REAL_OUT>
+static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
+                                      cudaStream_t st, int* launches) {
     const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<3, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<4, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         attr_set = true;
     }
     const size_t use = (size_t)tab.nmod * kHerkPlaneBytes;
     const int64_t tiles_j = (n + kHerkJ - 1) / kHerkJ;
-    for (int64_t j0 = 0; j0 < tiles_j; j0 += 65535) {      // grid.y limit
-        const int64_t nj = (tiles_j - j0 < 65535) ? tiles_j - j0 : 65535;
-        if (j0 != 0) return cudaErrorInvalidValue;         // n beyond 65535 * 16 columns is rejected by the API's row limit anyway
-        dim3 grid((unsigned)((n + kHerkI - 1) / kHerkI), (unsigned)nj);
-        switch (tab.nchunks) {
-            case 1: post_herk_kernel<1><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-            case 2: post_herk_kernel<2><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-            case 3: post_herk_kernel<3><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-            default: post_herk_kernel<4><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        }
-        ++*launches;
+    if (tiles_j > 65535) return cudaErrorInvalidValue;     // n beyond 65535 * 16 columns: far beyond any workspace
+    dim3 grid((unsigned)((n + kHerkI - 1) / kHerkI), (unsigned)tiles_j);
+    switch (tab.nchunks) {
+        case 1: post_herk_kernel<1, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        case 2: post_herk_kernel<2, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        case 3: post_herk_kernel<3, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        default: post_herk_kernel<4, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
     }
+    ++*launches;
     return cudaGetLastError();
+}
+
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
+                             bool real_out, cudaStream_t st, int* launches) {
+    if (n <= 0) return cudaSuccess;
+    return real_out ? launch_post_herk_t<true>(cp, ldp, n, eA, tab, C, ldc, st, launches)
+                    : launch_post_herk_t<false>(cp, ldp, n, eA, tab, C, ldc, st, launches);
 }
 
 // Exact integer variant for gemm2m_gaussian_int: X = sum_j sym(v_j g_j mod m_j) (M/m_j) mod M in int64 (M < 2^62).

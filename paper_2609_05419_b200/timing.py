@@ -4,7 +4,10 @@
   python -m paper_2609_05419_b200.timing --op cgemm --m 16384 --n 16384 --k 4096 --nmod 7
   python -m paper_2609_05419_b200.timing --op zherk --n 8192 --k 8192 --nmod 16
 
-Prints one JSON line: effective TFLOP/s (8mnk/t for GEMM, 4n^2k/t for HERK), milliseconds per call and per phase.
+  python -m paper_2609_05419_b200.timing --op dsyrk --n 8192 --k 8192 --nmod 16      (also zher2k, dsyr2k)
+
+Prints one JSON line: effective TFLOP/s (BLAS flop counts: 8mnk for GEMM, 4n^2k HERK, 8n^2k HER2K, n^2k SYRK, 2n^2k SYR2K,
+divided by the time), milliseconds per call and per phase.
 """
 from __future__ import annotations
 
@@ -20,7 +23,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk"])
+    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=8192)
@@ -31,14 +34,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--seed", type=int, default=1)
     a = ap.parse_args()
-    m, n, k, nmod = (a.n if a.op == "zherk" else a.m), a.n, a.k, a.nmod
+    rank = a.op in ("zherk", "zher2k", "dsyrk", "dsyr2k")
+    m, n, k, nmod = (a.n if rank else a.m), a.n, a.k, a.nmod
     dtype = np.complex64 if a.op == "cgemm" else np.complex128
     tdtype = torch.complex64 if a.op == "cgemm" else torch.complex128
     dev = lambda x: torch.from_numpy(np.ascontiguousarray(x.T)).cuda().t()
-    if a.op == "zherk":
-        A = dev(inputs.herk_input(n, k, a.seed, a.dist, a.phi))
-        B = None
-        opcode, flops = b.OP_ZHERK, 4.0 * n * n * k
+    if rank:
+        real = a.op in ("dsyrk", "dsyr2k")
+        two = a.op in ("zher2k", "dsyr2k")
+        gen = lambda seed: inputs.herk_input(n, k, seed, a.dist, a.phi)
+        A = dev(np.asfortranarray(gen(a.seed).real.copy()) if real else gen(a.seed))
+        B = (dev(np.asfortranarray(gen(a.seed + 1).real.copy()) if real else gen(a.seed + 1))) if two else None
+        opcode = {"zherk": b.OP_ZHERK, "zher2k": b.OP_ZHER2K, "dsyrk": b.OP_DSYRK, "dsyr2k": b.OP_DSYR2K}[a.op]
+        flops = {"zherk": 4.0, "zher2k": 8.0, "dsyrk": 1.0, "dsyr2k": 2.0}[a.op] * n * n * k     # BLAS flop counts
+        tdtype = torch.float64 if real else torch.complex128
     else:
         Ah, Bh = inputs.complex_inputs(m, n, k, a.seed, a.dist, a.phi, dtype=dtype)
         A, B = dev(Ah), dev(Bh)
@@ -51,6 +60,12 @@ def main():
     def call():
         if a.op == "zherk":
             b.zherk2m(A, C, nmod, stream)
+        elif a.op == "zher2k":
+            b.zher2k2m(A, B, C, nmod, stream)
+        elif a.op == "dsyrk":
+            b.dsyrk2m(A, C, nmod, stream)
+        elif a.op == "dsyr2k":
+            b.dsyr2k2m(A, B, C, nmod, stream)
         elif a.op == "cgemm":
             b.cgemm2m(A, B, C, nmod, stream)
         else:
@@ -71,10 +86,11 @@ def main():
     b.set_profiling(False)
     b.device_status()
     total, per = b.last_launch_count()
-    gemms = nmod if a.op == "zherk" else 2 * nmod
+    gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod}.get(a.op, 2 * nmod)
+    kin = (k + 1) // 2 if a.op in ("dsyrk", "dsyr2k") else k
     print(json.dumps({"op": a.op, "m": m, "n": n, "k": k, "nmod": nmod, "ms_per_call": ms, "effective_tflops": flops / ms / 1e9,
                       "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3],
-                      "gemm_int8_tops": 2.0 * gemms * m * n * k / phase[2] / 1e9 if phase[2] > 0 else None,
+                      "gemm_int8_tops": 2.0 * gemms * m * n * kin / phase[2] / 1e9 if phase[2] > 0 else None,
                       "launches_per_call": per}))
     b.set_workspace(None)
 

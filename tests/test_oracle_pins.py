@@ -283,3 +283,64 @@ def test_herk_symmetry_and_equivalence():
     assert all(int(v) == 0 for v in np.diag(st["Xi"]))
     st2 = staged.zgemm2m_staged(A, B, 16, herk=False)            # Pt even: same scaling, identical integers
     assert (st2["Xr"] == st["Xr"]).all() and (st2["Xi"] == st["Xi"]).all()
+
+
+# ------------------------------------------------------------------ rank-k family (Section 5)
+def test_two_product_dd_sum_vs_exact_rationals():
+    rng = np.random.default_rng(21)
+    mk = lambda r, c: np.asfortranarray(rng.standard_normal((r, c)) * np.exp(2 * rng.standard_normal((r, c))) +
+                                        1j * rng.standard_normal((r, c)))
+    A1, A2, B1, B2 = mk(3, 5), mk(3, 5), mk(5, 2), mk(5, 2)
+    C, D = direct.zgemm4m_dd2(A1, B1, A2, B2)
+    for i in range(3):
+        for j in range(2):
+            er = ei = Fraction(0)
+            d = 0.0
+            for A, B in ((A1, B1), (A2, B2)):
+                for p in range(5):
+                    ar, ai, br, bi = (Fraction(float(v)) for v in (A[i, p].real, A[i, p].imag, B[p, j].real, B[p, j].imag))
+                    er += ar * br - ai * bi
+                    ei += ar * bi + ai * br
+                    d += abs(A[i, p]) * abs(B[p, j])
+            assert abs(Fraction(C[i, j].real) - er) <= Fraction(d) * Fraction(1, 2 ** 52)
+            assert abs(Fraction(C[i, j].imag) - ei) <= Fraction(d) * Fraction(1, 2 ** 52)
+            assert abs(D[i, j] - d) <= 1e-15 * d
+    # a transposed or swapped operand in the rank-2k wrappers would break Hermitian symmetry
+    A, B = mk(6, 4), mk(6, 4)
+    C2, D2 = direct.zher2k_dd(A, B)
+    assert (np.abs(C2 - C2.conj().T) <= D2 * 2.0 ** -50).all()      # Hermitian up to the final rounding
+    assert (np.abs(C2 - (A @ B.conj().T + B @ A.conj().T)) <= D2 * 1e-14).all()
+
+
+@pytest.mark.parametrize("k", [6, 7, 1])
+def test_syrk_is_real_part_of_herk_of_half_k(k):
+    # Section 5: with Z = A1 + i A2, Z Z^H = A A^T + i (A2 A1^T - A1 A2^T); exact on integer data
+    rng = np.random.default_rng(k)
+    A = rng.integers(-9, 10, size=(5, k)).astype(np.float64)
+    Bm = rng.integers(-9, 10, size=(5, k)).astype(np.float64)
+    Z, ZB = staged.syrk_complexify(A), staged.syrk_complexify(Bm)
+    assert Z.shape == (5, (k + 1) // 2)
+    assert ((Z @ Z.conj().T).real == A @ A.T).all()
+    assert ((Z @ ZB.conj().T + ZB @ Z.conj().T).real == A @ Bm.T + Bm @ A.T).all()          # SYR2K -> HER2K
+    C, D = direct.dsyrk_dd(A)
+    assert (C == A @ A.T).all()
+    C2, _ = direct.dsyr2k_dd(A, Bm)
+    assert (C2 == A @ Bm.T + Bm @ A.T).all()
+
+
+def test_her2k_staged_symmetry_exactness_and_error():
+    A = inputs.herk_input(9, 30, seed=15, dist="phi", phi=1.0)
+    B = inputs.herk_input(9, 30, seed=16, dist="phi", phi=1.0)
+    st = staged.zher2k2m_staged(A, B, 16)
+    for Cp, Cm in st["Cpm"]:
+        assert (Cm == Cp.T).all()                                    # Section 5: C- = C+^T
+    assert (st["Xr"] == st["Xr"].T).all() and (st["Xi"] == -st["Xi"].T).all()
+    assert all(abs(int(v)) <= 2 ** st["Pt"] for v in st["Xr"].ravel()) and all(abs(int(v)) <= 2 ** st["Pt"] for v in st["Xi"].ravel())
+    # the 2M route reproduces the plain integer rank-2k update of the quantised matrices
+    Ar, Ai = (q.astype(object) for q in st["Aq"])
+    Br, Bi = (q.astype(object) for q in st["Bq"])
+    Xr = Ar @ Br.T + Ai @ Bi.T + Br @ Ar.T + Bi @ Ai.T
+    Xi = Ai @ Br.T - Ar @ Bi.T + Bi @ Ar.T - Br @ Ai.T
+    assert (st["Xr"] == Xr).all() and (st["Xi"] == Xi).all()
+    Cref, D = direct.zher2k_dd(A, B)
+    assert direct.componentwise_error(st["C"], Cref, D) <= 1e-14
