@@ -153,20 +153,8 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
                         const int64_t col = col0 + c * 32 + g * 16;
                         if (col < p.ldp) {
                             uint4* dst = reinterpret_cast<uint4*>(orow + c * 32 + g * 16);
-                            uint32_t old[4] = {0, 0, 0, 0};
-                            if (p.accumulate) { const uint4 o = *dst; old[0] = o.x; old[1] = o.y; old[2] = o.z; old[3] = o.w; }
-                            uint32_t w[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                uint32_t packed = 0;
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    int x = (int)v[g * 16 + q * 4 + e] + (int)(int8_t)(old[q] >> (8 * e));
-                                    packed |= ((uint32_t)sym_reduce_acc(x, m, inv_m) & 0xFFu) << (8 * e);
-                                }
-                                w[q] = packed;
-                            }
-                            *dst = make_uint4(w[0], w[1], w[2], w[3]);
+                            if (p.accumulate) reduce_store16<true>(v + g * 16, dst, m, inv_m);
+                            else reduce_store16<false>(v + g * 16, dst, m, inv_m);
                         }
                     }
                 }

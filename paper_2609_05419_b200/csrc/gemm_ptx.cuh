@@ -127,9 +127,30 @@ __device__ __forceinline__ int sym_reduce_acc(int x, int m, float inv_m) {
     const int q = __float2int_rn(__int2float_rn(x) * inv_m);
     int r = x - q * m;
     const int h = (m - 1) >> 1;
-    r += (r < -h) ? m : 0;
-    r -= (r > h) ? m : 0;
+    if (r > h) r -= m;
+    if (r < -h) r += m;
     return r;
+}
+
+// 16 consecutive accumulators of one TMEM lane -> 16 symmetric residues packed into one 16-byte vector.
+// ACC: add the residues already stored at `dst` first (later K chunks, second product of a rank-2k update).
+template <bool ACC>
+__device__ __forceinline__ void reduce_store16(const uint32_t* v, uint4* dst, int m, float inv_m) {
+    uint32_t old[4] = {0, 0, 0, 0};
+    if (ACC) { const uint4 o = *dst; old[0] = o.x; old[1] = o.y; old[2] = o.z; old[3] = o.w; }
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t b[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            int x = (int)v[q * 4 + e];
+            if (ACC) x += (int)(int8_t)(old[q] >> (8 * e));
+            b[e] = (uint32_t)sym_reduce_acc(x, m, inv_m);
+        }
+        w[q] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+    }
+    *dst = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 struct GemmKernelParams {
