@@ -178,6 +178,14 @@ int gemm2m_debug_set_panels(int max_panels);
 int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,
                         int8_t* res_w);
 
+/* Constants of the residue kernels' reduction modulo m_j (tests only; host pointers, nmod entries each, any may be NULL):
+ *   y0_bits  = bit pattern of the float Y0 at which the real part's byte-weight sum starts
+ *   cq       = the FMA addend 1.5 2^23 - Y0/m_j
+ *   inv_m    = the float reciprocal in use
+ *   xmax     = bound on the magnitude of the reduced sums
+ *   margin   = (1/(2 m_j)) / ((Y0 + xmax) |inv_m - 1/m_j|): the quotient estimate is exact while this exceeds 1 */
+int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin);
+
 #ifdef __cplusplus
 }
 #endif

@@ -66,6 +66,7 @@ def lib():
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
     L.gemm2m_debug_set_panels.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
+    L.gemm2m_debug_residue_reduction.argtypes = [i32, vp, vp, vp, vp, vp]
     _lib = L
     return L
 
@@ -250,3 +251,17 @@ def debug_tables(nmod, k, herk=False):
            "gemm2m_debug_tables")
     return dict(Pt=int(scale[0]), PA=int(scale[1]), PB=int(scale[2]), ck=int(scale[3]), gr=gr, gi=gi, Mc=mc,
                 nchunks=int(nch[0]), res_w=w)
+
+
+def debug_residue_reduction(nmod):
+    """Constants of the residue kernels' reduction modulo m_j (see gemm2m_debug_residue_reduction)."""
+    import numpy as np
+    y0 = np.zeros(nmod, dtype=np.int32)
+    cq = np.zeros(nmod, dtype=np.float32)
+    inv = np.zeros(nmod, dtype=np.float32)
+    xmax = np.zeros(nmod, dtype=np.int32)
+    margin = np.zeros(nmod, dtype=np.float64)
+    ptr = lambda a: ctypes.c_void_p(a.ctypes.data)
+    _check(lib().gemm2m_debug_residue_reduction(nmod, ptr(y0), ptr(cq), ptr(inv), ptr(xmax), ptr(margin)),
+           "gemm2m_debug_residue_reduction")
+    return dict(y0_bits=y0, cq=cq, inv_m=inv, xmax=xmax, margin=margin)

@@ -523,6 +523,20 @@ int gemm2m_debug_set_gemm_kernel(int which) {
     return GEMM2M_OK;
 }
 
+int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin) {
+    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_ARG;
+    ResidueTable rt;
+    build_residue_table(nmod, &rt);
+    for (int j = 0; j < nmod; ++j) {
+        if (y0_bits) y0_bits[j] = rt.magic[j];
+        if (cq) cq[j] = rt.cq[j];
+        if (inv_m) inv_m[j] = rt.inv_m[j];
+        if (xmax) xmax[j] = rt.xmax[j];
+        if (margin) margin[j] = residue_reduction_margin(rt, j);
+    }
+    return GEMM2M_OK;
+}
+
 int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,
                         int8_t* res_w) {
     if (nmod < 1 || nmod > kMaxMod || k < 0) return GEMM2M_ERR_ARG;

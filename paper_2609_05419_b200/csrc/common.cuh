@@ -24,10 +24,13 @@ constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilog
 struct ResidueTable {
     int32_t m[kMaxMod];
     float inv_m[kMaxMod];
+    int32_t magic[kMaxMod];                    // bit pattern of the float 2^23 + u m, u m a multiple of 256: start of the real dp4a chain
+    float cq[kMaxMod];                         // 1.5 2^23 - u: fma(y, inv_m, cq) = 1.5 2^23 + rint(x / m) for y = 2^23 + u m + x
     uint32_t w_lo[kMaxMod], w_hi[kMaxMod];     // int8 x4 each: sym(256^b mod m), b = 0..3 / 4..7
     uint32_t ws_lo[kMaxMod], ws_hi[kMaxMod];   // int8 x4 each: sym(s 256^b mod m)
     uint32_t w_top[kMaxMod], ws_top[kMaxMod];  // b = 8..11: only used when quantised values exceed 62 bits
     int32_t s[kMaxMod];
+    int32_t xmax[kMaxMod];                     // bound on |real dp4a sum| + |imaginary dp4a sum| (host side only)
     int nmod;
 };
 
@@ -67,6 +70,7 @@ struct ScaleTargets { int Pt, PA, PB, ck; };
 int modulus_value(int j);
 int modulus_root(int j);
 void build_residue_table(int nmod, ResidueTable* t);
+double residue_reduction_margin(const ResidueTable& t, int j);
 void build_mod_table(int nmod, ModTable* t);
 void build_crt_table(int nmod, CrtTable* t);
 void build_crt_table_int(int nmod, CrtTableInt* t);

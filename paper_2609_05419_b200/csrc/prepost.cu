@@ -178,27 +178,19 @@ __device__ __forceinline__ int dp4a_ss(uint32_t a_signed, uint32_t b_signed, int
     return d;
 }
 
-// Symmetric residue of x (|x| < 2^22) modulo m by a float reciprocal: the quotient estimate is exact because
-// |x/m| < 2^11 carries an error below 1/(2m), the distance of x/m from the nearest rounding boundary.
-__device__ __forceinline__ int sym_reduce_small(int x, int m, float inv_m) {
-    const float xf = __int_as_float(x + 0x4B400000) - 12582912.0f;   // exact int -> float for |x| < 2^22
-    const float t = fmaf(xf, inv_m, 12582912.0f);                    // nearest integer in the low mantissa bits
-    const int q = __float_as_int(t) - 0x4B400000;
-    return x - q * m;
-}
-
-// The same for the pair (Rv + Iv, Rv - Iv); the two symmetric residues come back in the low bytes of bp / bm (two's
-// complement).  y = 1.5 2^23 + x holds x exactly in its mantissa; after q = rint(x/m), fma(-q, m, y) = 1.5 2^23 + (x - q m)
-// is exact and its low mantissa byte is the residue.  Plain FP32 adds and FMAs: they issue to both FMA pipes, whereas the
-// packed two-lane forms and integer multiply-adds only use one of them, which the dp4a's already keep busy.
-// Rm = Rv + 0x4B400000: the caller starts the real part's dp4a chain at the bit pattern of 1.5 2^23, which saves two adds.
-__device__ __forceinline__ void sym_reduce_pm(int Rm, int Iv, float neg_m, float inv_m, uint32_t* bp, uint32_t* bm) {
-    const float magic = 12582912.0f;
-    const float yp = __int_as_float(Rm + Iv), ym = __int_as_float(Rm - Iv);
-    const float qp = fmaf(yp - magic, inv_m, magic) - magic;
-    const float qm = fmaf(ym - magic, inv_m, magic) - magic;
-    *bp = __float_as_uint(fmaf(qp, neg_m, yp));
-    *bm = __float_as_uint(fmaf(qm, neg_m, ym));
+// Symmetric residues of the pair (x+, x-) = (Rv + Iv, Rv - Iv), returned in the low bytes of bp / bm (two's complement).
+// The caller starts the real part's dp4a chain at the bit pattern of the float Y0 = 2^23 + (a multiple of 256 m), so
+// Ry = bits(Y0) + Rv and the integer Ry +- Iv is the bit pattern of the float y = Y0 + x.  One FMA with the constant
+// cq = 1.5 2^23 - Y0/m gives t = 1.5 2^23 + rint(x/m) exactly (the table builder proves the error of inv_m stays below
+// the distance of x/m from a rounding boundary), and bits(y) - bits(t) m has the low byte of x - rint(x/m) m because the
+// bit patterns of Y0 and of 1.5 2^23 are multiples of 256.  Per residue: one integer add, one FP32 FMA, one integer
+// multiply-add.
+__device__ __forceinline__ void sym_reduce_pm(int Ry, int Iv, int neg_m, float inv_m, float cq, uint32_t* bp, uint32_t* bm) {
+    const int yp = Ry + Iv, ym = Ry - Iv;
+    const int tp = __float_as_int(fmaf(__int_as_float(yp), inv_m, cq));
+    const int tm = __float_as_int(fmaf(__int_as_float(ym), inv_m, cq));
+    *bp = (uint32_t)(tp * neg_m + yp);
+    *bm = (uint32_t)(tm * neg_m + ym);
 }
 
 struct Digits { uint32_t lo, hi; };   // 4 unsigned low bytes; 4 balanced (signed) high digits
@@ -228,8 +220,8 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
     const int nmod = tab.nmod;
 #pragma unroll 1
     for (int j = 0; j < nmod; ++j) {
-        const int m = tab.m[j];
-        const float inv_m = tab.inv_m[j], neg_m = -(float)m;
+        const int neg_m = -tab.m[j], y0 = tab.magic[j];
+        const float inv_m = tab.inv_m[j], cq = tab.cq[j];
         const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
         const uint32_t wt = WIDE ? tab.w_top[j] : 0u, st = WIDE ? tab.ws_top[j] : 0u;
         uint32_t pw[NE / 4], mw[NE / 4];
@@ -239,13 +231,13 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const int i = 4 * w + b;
-                int Rv = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, 0x4B400000));   // A_r mod m (unreduced) + bits of 1.5 2^23
+                int Rv = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
                 int Iv = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, 0));   // s A_i mod m (unreduced)
                 if (WIDE) {                                                 // digits 8..11 of the 96-bit value
                     Rv = dp4a_ss(tr[i], wt, Rv);
                     Iv = dp4a_ss(ti[i], st, Iv);
                 }
-                sym_reduce_pm(Rv, Iv, neg_m, inv_m, &bp[b], &bm[b]);        // Eq. (2a): "+" and "-"
+                sym_reduce_pm(Rv, Iv, neg_m, inv_m, cq, &bp[b], &bm[b]);        // Eq. (2a): "+" and "-"
             }
             pw[w] = __byte_perm(__byte_perm(bp[0], bp[1], 0x0040), __byte_perm(bp[2], bp[3], 0x0040), 0x5410);
             mw[w] = __byte_perm(__byte_perm(bm[0], bm[1], 0x0040), __byte_perm(bm[2], bm[3], 0x0040), 0x5410);

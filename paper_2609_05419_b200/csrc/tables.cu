@@ -3,6 +3,7 @@
 #include "common.cuh"
 
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -94,6 +95,23 @@ void build_residue_table(int nmod, ResidueTable* t) {
             ws[b] = (uint32_t)(uint8_t)(int8_t)sym_mod(p * s, m);
             p = (p * 256) % m;
         }
+        // Reduction constants.  x = (dp4a sum of the real part) +- (dp4a sum of the imaginary part) is bounded by xmax below
+        // (digits: four unsigned bytes, then up to eight balanced ones).  The real chain starts at the bit pattern of
+        // Y0 = the first multiple of 256 m that is >= 2^23 + xmax, so the integer sum is the float y = Y0 + x exactly
+        // (2^23 <= y < 2^24, one unit per ulp).  With cq = 1.5 2^23 - Y0/m (an integer), the exact value of
+        // fma(y, inv_m, cq) is 1.5 2^23 + x/m + y d, d = inv_m - 1/m, which rounds to 1.5 2^23 + rint(x/m) because
+        // |y d| < 1/(2m), the least distance of x/m from a rounding boundary (residue_reduction_margin checks it).
+        // Y0 is a multiple of 256 and so is the bit pattern of 1.5 2^23: the low byte of y - (1.5 2^23 + q) m is that of x - q m.
+        int64_t xmax = 0;
+        for (int b = 0; b < 12; ++b) {
+            const int64_t digit = b < 4 ? 255 : 128;
+            xmax += digit * (std::abs((int)(int8_t)w[b]) + std::abs((int)(int8_t)ws[b]));
+        }
+        const int64_t step = 256LL * m;
+        const int64_t y0 = (((1LL << 23) + xmax + step - 1) / step) * step;
+        t->magic[j] = (int32_t)(0x4B000000LL + (y0 - (1LL << 23)));
+        t->cq[j] = (float)(12582912LL - y0 / m);
+        t->xmax[j] = (int32_t)xmax;
         auto pack = [](const uint32_t* v) { return v[0] | (v[1] << 8) | (v[2] << 16) | (v[3] << 24); };
         t->w_lo[j] = pack(w);
         t->w_hi[j] = pack(w + 4);
@@ -102,6 +120,19 @@ void build_residue_table(int nmod, ResidueTable* t) {
         t->ws_hi[j] = pack(ws + 4);
         t->ws_top[j] = pack(ws + 8);
     }
+}
+
+// 2^e / (2 (Y0 + xmax) |n m - 2^e|) for inv_m = n 2^-e: the factor by which the error term of the residue kernels'
+// quotient estimate stays below the distance 1/(2m) of x/m from the nearest rounding boundary (must exceed 1).
+double residue_reduction_margin(const ResidueTable& t, int j) {
+    int ex = 0;
+    const float mant = std::frexp(t.inv_m[j], &ex);          // inv_m = mant 2^ex, 0.5 <= mant < 1
+    const int64_t n = (int64_t)std::ldexp((double)mant, 24); // exact: 24-bit significand
+    const int e = 24 - ex;
+    const int64_t y0 = (int64_t)(t.magic[j] - 0x4B000000) + (1LL << 23);
+    const int64_t dev = std::llabs(n * t.m[j] - (1LL << e));
+    if (dev == 0) return 1e30;
+    return (double)(1LL << e) / (2.0 * (double)(y0 + t.xmax[j]) * (double)dev);
 }
 
 void build_mod_table(int nmod, ModTable* t) {

@@ -56,6 +56,40 @@ def test_crt_and_scaling_constants_match_oracle(nmod):
             assert int(t["res_w"][j, 8 + bb]) == staged.sym(s * 256 ** bb, m)
 
 
+def test_residue_reduction_constants_are_exact_for_every_reachable_sum():
+    """The residue kernels reduce x (a sum of byte-weight products) modulo m with one FP32 FMA and one integer
+    multiply-add.  Emulate that FMA in exact integer arithmetic (float operands are dyadic rationals; round to nearest
+    even at unit spacing) for EVERY integer x the kernels can reach and require the symmetric residue in the low byte."""
+    r = b.debug_residue_reduction(22)
+    mods = staged.greedy_2m_moduli()
+    for j, m in enumerate(mods):
+        y0_bits, xmax = int(r["y0_bits"][j]), int(r["xmax"][j])
+        y0 = (y0_bits - 0x4B000000) + 2 ** 23                 # value of the float with that bit pattern (exponent 2^23)
+        assert y0 % (256 * m) == 0 and y0 - xmax >= 2 ** 23 and y0 + xmax < 2 ** 24
+        s = staged.sqrt_minus_one(m)
+        w = [abs(staged.sym(256 ** bb, m)) + abs(staged.sym(s * 256 ** bb, m)) for bb in range(12)]
+        assert xmax == 255 * sum(w[:4]) + 128 * sum(w[4:])    # four unsigned bytes, eight balanced digits, both parts
+        assert float(r["margin"][j]) > 1.0
+        mant, ex = np.frexp(np.float64(r["inv_m"][j]))
+        n, e = int(mant * 2 ** 24), 24 - int(ex)               # inv_m = n 2^-e exactly
+        assert n * 2.0 ** -e == float(r["inv_m"][j])
+        cq = int(r["cq"][j])
+        assert cq == float(r["cq"][j]) and cq == 3 * 2 ** 22 - y0 // m
+        x = np.arange(-xmax, xmax + 1, dtype=np.int64)
+        num = (y0 + x) * n + (cq << e)                          # exact value of the FMA, times 2^e
+        fl = num >> e
+        rem = num - (fl << e)
+        half = 1 << (e - 1)
+        t = fl + ((rem > half) | ((rem == half) & (fl & 1 == 1)))   # round to nearest even; 2^23 <= t < 2^24: spacing 1
+        assert t.min() >= 2 ** 23 and t.max() < 2 ** 24
+        t_bits = 0x4B000000 + (t - 2 ** 23)
+        y_bits = y0_bits + x
+        low = (y_bits - t_bits * m) & 0xFF
+        res = np.where(low >= 128, low - 256, low)
+        want = ((x + (m - 1) // 2) % m) - (m - 1) // 2
+        assert np.array_equal(res, want), m
+
+
 def test_folded_crt_weights_reproduce_eq_2c_and_crt():
     # sum_j (c- + c+) Gr_j  and  sum_j (c- - c+) Gi_j  (mod M) must equal CRT of Eq. (2c), for random residues
     rng = np.random.default_rng(0)
