@@ -178,15 +178,13 @@ __device__ __forceinline__ int dp4a_ss(uint32_t a_signed, uint32_t b_signed, int
     return d;
 }
 
-// Symmetric residues of the pair (x+, x-) = (Rv + Iv, Rv - Iv), returned in the low bytes of bp / bm (two's complement).
-// The caller starts the real part's dp4a chain at the bit pattern of the float Y0 = 2^23 + (a multiple of 256 m), so
-// Ry = bits(Y0) + Rv and the integer Ry +- Iv is the bit pattern of the float y = Y0 + x.  One FMA with the constant
-// cq = 1.5 2^23 - Y0/m gives t = 1.5 2^23 + rint(x/m) exactly (the table builder proves the error of inv_m stays below
-// the distance of x/m from a rounding boundary), and bits(y) - bits(t) m has the low byte of x - rint(x/m) m because the
-// bit patterns of Y0 and of 1.5 2^23 are multiples of 256.  Per residue: one integer add, one FP32 FMA, one integer
-// multiply-add.
-__device__ __forceinline__ void sym_reduce_pm(int Ry, int Iv, int neg_m, float inv_m, float cq, uint32_t* bp, uint32_t* bm) {
-    const int yp = Ry + Iv, ym = Ry - Iv;
+// Symmetric residues of the pair of sums x+ = Rv + Iv and x- = Rv - Iv, returned in the low bytes of bp / bm (two's
+// complement).  The caller starts the dp4a chain at the bit pattern of the float Y0 = a multiple of 256 m in [2^23, 2^24),
+// so the integers yp = bits(Y0) + x+ and ym = bits(Y0) + x- are the bit patterns of the floats Y0 + x.  One FMA with the
+// constant cq = 1.5 2^23 - Y0/m gives t = 1.5 2^23 + rint(x/m) exactly (the table builder proves that the error of inv_m
+// stays below the distance of x/m from a rounding boundary), and bits(y) - bits(t) m has the low byte of x - rint(x/m) m
+// because the bit patterns of Y0 and of 1.5 2^23 are multiples of 256.  Per residue: one FP32 FMA, one integer multiply-add.
+__device__ __forceinline__ void sym_reduce_pm(int yp, int ym, int neg_m, float inv_m, float cq, uint32_t* bp, uint32_t* bm) {
     const int tp = __float_as_int(fmaf(__int_as_float(yp), inv_m, cq));
     const int tm = __float_as_int(fmaf(__int_as_float(ym), inv_m, cq));
     *bp = (uint32_t)(tp * neg_m + yp);
@@ -231,13 +229,14 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const int i = 4 * w + b;
-                int Rv = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
-                int Iv = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, 0));   // s A_i mod m (unreduced)
-                if (WIDE) {                                                 // digits 8..11 of the 96-bit value
-                    Rv = dp4a_ss(tr[i], wt, Rv);
-                    Iv = dp4a_ss(ti[i], st, Iv);
-                }
-                sym_reduce_pm(Rv, Iv, neg_m, inv_m, cq, &bp[b], &bm[b]);        // Eq. (2a): "+" and "-"
+                int Ry = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
+                if (WIDE) Ry = dp4a_ss(tr[i], wt, Ry);                      // digits 8..11 of the 96-bit value
+                // The imaginary part's weights continue the same chain: no separate addition for the "+" sum of Eq. (2a),
+                // and the "-" sum is 2 Ry - yp, a three-input integer add that does not compete with the dp4a's for their pipe.
+                int yp = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, Ry));
+                if (WIDE) yp = dp4a_ss(ti[i], st, yp);
+                const int ym = (int)(2u * (uint32_t)Ry - (uint32_t)yp);     // the doubled bit pattern wraps, the difference does not
+                sym_reduce_pm(yp, ym, neg_m, inv_m, cq, &bp[b], &bm[b]);
             }
             pw[w] = __byte_perm(__byte_perm(bp[0], bp[1], 0x0040), __byte_perm(bp[2], bp[3], 0x0040), 0x5410);
             mw[w] = __byte_perm(__byte_perm(bm[0], bm[1], 0x0040), __byte_perm(bm[2], bm[3], 0x0040), 0x5410);
@@ -259,7 +258,7 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
 #define GEMM2M_RES_ROWS 8
 #endif
 constexpr int kResRows = GEMM2M_RES_ROWS, kResK = 128, kResRun = 8, kResThreads = kResRows * kResK / kResRun;
-constexpr int kResBlocksPerSm = 768 / kResThreads;
+constexpr int kResBlocksPerSm = 640 / kResThreads;   // 5 blocks of 128: up to 96 registers per thread measured faster than 6 blocks at 80
 constexpr int kResIThreads = 256;
 constexpr int kResRowStride = kResK + kResK / kResRun + 1;   // in elements: one pad per run of 8 + odd row stride -> no bank conflicts
 constexpr int kResStages = 2;
