@@ -5,12 +5,15 @@ Every function follows one passage of the paper, in its notation, with no blocki
   is_2m_modulus, greedy_2m_moduli   Section 2 (definition of a 2M modulus) and Section 4 (greedy coprime set in [1, 256])
   sqrt_minus_one, inv2              Section 2: s^2 = -1 (mod m); 2^-1 = (m+1)/2
   pre_2m, mul_2m, post_2m           Eq. (2a), (2b), (2c)
+  hybrid_moduli, pre_3m, mul_3m, post_3m   Section 3 (hybrid 2M/3M remark) and Section 4 (non-2M moduli once the 2M set is
+                                    exhausted); Eq. (1) applied after the reduction modulo m
   crt, lift                         Section 3.1 (CRT formula) and Algorithm 1 steps 5-6
   scaling_targets, scaling_exponents, quantise, unscale   Algorithm 1 steps 2, 3, 7
 
 Readings taken where the paper is silent (they are the library's documented readings too):
   * s is the smallest positive root (any root gives the same C);
-  * residues are kept as symmetric representatives in [-(m-1)/2, (m-1)/2];
+  * residues are kept as symmetric representatives in [-(m-1)/2, (m-1)/2] (even m, hybrid only: [-m/2, m/2 - 1]);
+  * hybrid: all 22 2M moduli first, then the greedy walk down from 256 over the remaining coprime (non-2M) moduli;
   * scale factors are powers of two chosen from the largest part-magnitude of each row of A /
     column of B so that every entry of the integer product is bounded by 2^P_t <= (M-1)/2
     (Cauchy-Schwarz), see `scaling_exponents`;
@@ -67,9 +70,23 @@ def inv2(m: int) -> int:
 
 
 def sym(x, m: int):
-    """Symmetric representative of x mod m (m odd): in [-(m-1)/2, (m-1)/2]."""
-    h = (m - 1) // 2
+    """Symmetric representative of x mod m: in [-(m-1)/2, (m-1)/2] for odd m, in [-m/2, m/2 - 1] for even m."""
+    h = m // 2
     return (x + h) % m - h
+
+
+def hybrid_moduli(n: int, limit: int = 256):
+    """Sections 3 and 4: the 2M moduli first; when they are exhausted, further moduli come from the same greedy walk
+    down from `limit` over the numbers coprime to everything kept (none of them is a 2M modulus, or the first walk
+    would have kept it).  Returns the first n moduli."""
+    kept = greedy_2m_moduli(limit)
+    if n > len(kept):
+        for cand in range(limit, 1, -1):
+            if len(kept) >= n:
+                break
+            if all(math.gcd(cand, q) == 1 for q in kept):
+                kept.append(cand)
+    return kept[:n]
 
 
 # ----------------------------------------------------------------------------- 2M multiplication (Eq. 2a-2c)
@@ -101,6 +118,23 @@ def post_2m(Cp, Cm, m: int, s: int):
     return sym(h * (Cm + Cp), m), sym(s * h * (Cm - Cp), m)
 
 
+# ----------------------------------------------------------------------------- 3M multiplication modulo m (Eq. 1, Section 3)
+def pre_3m(Xr, Xi, m: int):
+    """Residues of Xr, Xi and Xr + Xi (the sum is formed after the reduction, Section 3)."""
+    r, i = sym(Xr, m), sym(Xi, m)
+    return r, i, sym(r + i, m)
+
+
+def mul_3m(A3, B3, m: int):
+    """The three real products of Eq. (1) modulo m: Ar Br, Ai Bi, (Ar + Ai)(Br + Bi)."""
+    return tuple(sym(_exact_matmul(a, b), m) for a, b in zip(A3, B3))
+
+
+def post_3m(P1, P2, P3, m: int):
+    """Eq. (1): C = (P1 - P2) + i (P3 - P1 - P2) (mod m)."""
+    return sym(P1 - P2, m), sym(P3 - P1 - P2, m)
+
+
 # ----------------------------------------------------------------------------- CRT (Section 3.1, Algorithm 1 steps 5-6)
 def product(moduli):
     M = 1
@@ -123,8 +157,8 @@ def crt(residues, moduli):
 
 
 def lift(X, M: int):
-    """Algorithm 1 step 6: representative in [-M/2, M/2); M is odd so this is [-(M-1)/2, (M-1)/2]."""
-    h = (M - 1) // 2
+    """Algorithm 1 step 6: representative in [-M/2, M/2); for odd M this is [-(M-1)/2, (M-1)/2]."""
+    h = M // 2
     return (X + h) % M - h
 
 
@@ -216,33 +250,50 @@ def _small(a):
 
 
 def _residue_planes(Zr, Zi, moduli, roots):
+    """Per modulus: (X+, X-) for a 2M modulus (root given), (Xr, Xi, Xr + Xi) for a 3M modulus (root None)."""
     Zr, Zi = _small(Zr), _small(Zi)
     planes = []
     for ml, sl in zip(moduli, roots):
         # reduce first so that s * Zi stays small in int64
         zr = Zr % ml
         zi = Zi % ml
-        p, q = pre_2m(zr, zi, ml, sl)
-        planes.append((np.asarray(p).astype(np.int64), np.asarray(q).astype(np.int64)))
+        pl = pre_2m(zr, zi, ml, sl) if sl is not None else pre_3m(zr, zi, ml)
+        planes.append(tuple(np.asarray(p).astype(np.int64) for p in pl))
     return planes
+
+
+def roots_of(moduli):
+    """s_l for the 2M moduli, None for the others (they take 3M multiplication)."""
+    return [sqrt_minus_one(q) if is_2m_modulus(q) else None for q in moduli]
+
+
+def _multiply_and_post(Apl, Bpl, moduli, roots):
+    Cpm, res_r, res_i = [], [], []
+    for Ap, Bp, ml, sl in zip(Apl, Bpl, moduli, roots):
+        if sl is not None:
+            Cp, Cm = mul_2m(Ap[0], Bp[0], ml), mul_2m(Ap[1], Bp[1], ml)   # (2b)
+            Cpm.append((Cp, Cm))
+            r, i = post_2m(Cp, Cm, ml, sl)                                 # (2c)
+        else:
+            P = mul_3m(Ap, Bp, ml)                                         # Eq. (1) modulo m
+            Cpm.append(P)
+            r, i = post_3m(P[0], P[1], P[2], ml)
+        res_r.append(r)
+        res_i.append(i)
+    return Cpm, res_r, res_i
 
 
 # ----------------------------------------------------------------------------- whole paths
 def gemm2m_int_staged(Ar, Ai, Br, Bi, nmod: int):
-    """Integer 2M multiplication (Section 2) + CRT over the first `nmod` moduli.  Returns a dict of stages."""
-    moduli = greedy_2m_moduli()[:nmod]
-    roots = [sqrt_minus_one(q) for q in moduli]
+    """Integer 2M multiplication (Section 2; 3M for the non-2M moduli beyond the 22nd) + CRT over the first `nmod` moduli.
+    Returns a dict of stages."""
+    moduli = hybrid_moduli(nmod)
+    roots = roots_of(moduli)
     M = product(moduli)
     Ar, Ai, Br, Bi = (np.asarray(x).astype(object) for x in (Ar, Ai, Br, Bi))
     Apl = _residue_planes(Ar, Ai, moduli, roots)
     Bpl = _residue_planes(Br, Bi, moduli, roots)
-    Cpm, res_r, res_i = [], [], []
-    for (Ap, Am), (Bp, Bm), ml, sl in zip(Apl, Bpl, moduli, roots):
-        Cp, Cm = mul_2m(Ap, Bp, ml), mul_2m(Am, Bm, ml)
-        Cpm.append((Cp, Cm))
-        r, i = post_2m(Cp, Cm, ml, sl)
-        res_r.append(r)
-        res_i.append(i)
+    Cpm, res_r, res_i = _multiply_and_post(Apl, Bpl, moduli, roots)
     Xr, Xi = lift(crt(res_r, moduli), M), lift(crt(res_i, moduli), M)
     return dict(moduli=moduli, roots=roots, M=M, Apm=Apl, Bpm=Bpl, Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi)
 
@@ -253,27 +304,21 @@ def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto
     A = np.asarray(A)
     B = np.asarray(B)
     k = A.shape[1]
-    moduli = greedy_2m_moduli()[:nmod]                            # step 1
-    roots = [sqrt_minus_one(q) for q in moduli]
+    moduli = hybrid_moduli(nmod)                                   # step 1 (2M moduli only while nmod <= 22)
+    roots = roots_of(moduli)
     M = product(moduli)
     Pt, PA, PB, ck = scaling_targets(M, k, herk)
     eA = scaling_exponents(A, 1, PA, ck)                           # step 2
     eB = scaling_exponents(B, 0, PB, ck)
     Aq = quantise(A, eA, 1)                                        # step 3
     Bq = quantise(B, eB, 0)
-    Apl = _residue_planes(Aq[0], Aq[1], moduli, roots)             # step 4: (2a)
+    Apl = _residue_planes(Aq[0], Aq[1], moduli, roots)             # step 4: (2a), or the 3M sums
     Bpl = _residue_planes(Bq[0], Bq[1], moduli, roots)
     st = dict(moduli=moduli, roots=roots, M=M, Pt=Pt, PA=PA, PB=PB, ck=ck, eA=eA, eB=eB, Aq=Aq, Bq=Bq,
               Apm=Apl, Bpm=Bpl)
     if upto == "pre":
         return st
-    Cpm, res_r, res_i = [], [], []
-    for (Ap, Am), (Bp, Bm), ml, sl in zip(Apl, Bpl, moduli, roots):
-        Cp, Cm = mul_2m(Ap, Bp, ml), mul_2m(Am, Bm, ml)            # (2b)
-        Cpm.append((Cp, Cm))
-        r, i = post_2m(Cp, Cm, ml, sl)                             # (2c)
-        res_r.append(r)
-        res_i.append(i)
+    Cpm, res_r, res_i = _multiply_and_post(Apl, Bpl, moduli, roots)      # (2b), (2c) / Eq. (1)
     Xr, Xi = lift(crt(res_r, moduli), M), lift(crt(res_i, moduli), M)   # steps 5, 6
     C = unscale(Xr, eA, eB, out_bits) + 1j * unscale(Xi, eA, eB, out_bits)   # step 7
     st.update(Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi, C=C)

@@ -344,3 +344,100 @@ def test_her2k_staged_symmetry_exactness_and_error():
     assert (st["Xr"] == Xr).all() and (st["Xi"] == Xi).all()
     Cref, D = direct.zher2k_dd(A, B)
     assert direct.componentwise_error(st["C"], Cref, D) <= 1e-14
+
+
+# ------------------------------------------------------------------ hybrid 2M/3M (Section 3 remark, Section 4)
+def test_hybrid_moduli_extend_the_2m_set_with_coprime_non_2m_moduli(printed):
+    h = staged.hybrid_moduli(26)
+    assert h[:22] == staged.greedy_2m_moduli()
+    assert h[22:] == [256, 253, 251, 249]
+    assert all(not staged.is_2m_modulus(q) for q in h[22:])
+    assert all(math.gcd(a, b) == 1 for i, a in enumerate(h) for b in h[:i])
+    # greedy: every number between two consecutive extras shares a factor with something kept before it
+    for hi, lo in zip([257] + h[22:-1], h[22:]):
+        for cand in range(lo + 1, hi):
+            kept_before = h[:h.index(lo)]
+            assert any(math.gcd(cand, q) != 1 for q in kept_before), cand
+    # 256, 253 and 251 are printed in the paper's real-modulus list; 255 and 247 clash with the 2M moduli 205/221
+    real = set(printed["mreal_prefix"])
+    assert {256, 253, 251} <= real and math.gcd(255, 205) == 5 and math.gcd(247, 221) == 13
+    assert staged.hybrid_moduli(16) == staged.greedy_2m_moduli()[:16]
+    assert staged.roots_of(h)[:22] == [staged.sqrt_minus_one(q) for q in h[:22]] and staged.roots_of(h)[22:] == [None] * 4
+
+
+def test_symmetric_range_for_even_modulus_and_even_product():
+    x = np.arange(-1000, 1000)
+    r = staged.sym(x, 256)
+    assert r.min() == -128 and r.max() == 127 and ((r - x) % 256 == 0).all()
+    assert staged.sym(128, 256) == -128 and staged.sym(127, 256) == 127 and staged.sym(-128, 256) == -128
+    M = 256 * 253
+    for X in (0, 1, M // 2 - 1, M // 2, M - 1, -M // 2):
+        L = staged.lift(X % M, M)
+        assert -M // 2 <= L < M // 2 and (L - X) % M == 0        # Algorithm 1 step 6: [-M/2, M/2)
+    assert staged.lift(M // 2, M) == -M // 2
+
+
+def test_3m_identity_brute_force():
+    # Eq. (1) after the reduction modulo m equals the complex product mod m, for every small Gaussian integer pair
+    # and for entries across the whole residue range
+    for m in staged.hybrid_moduli(26)[22:]:
+        vals = list(range(-3, 4)) + [m // 2 - 1, -(m // 2), 77, -101]
+        for ar in vals:
+            for ai in vals:
+                a3 = staged.pre_3m(ar, ai, m)
+                assert (a3[0] - ar) % m == 0 and (a3[1] - ai) % m == 0 and (a3[2] - ar - ai) % m == 0
+                assert all(-(m // 2) <= v <= (m - 1) // 2 for v in a3)
+                for br in (-2, 0, 1, 5, m // 2 - 1):
+                    for bi in (-7, 0, 3, -(m // 2)):
+                        b3 = staged.pre_3m(br, bi, m)
+                        P = [staged.sym(x * y, m) for x, y in zip(a3, b3)]
+                        cr, ci = staged.post_3m(P[0], P[1], P[2], m)
+                        assert (cr - (ar * br - ai * bi)) % m == 0
+                        assert (ci - (ar * bi + ai * br)) % m == 0
+                        assert -(m // 2) <= cr <= (m - 1) // 2 and -(m // 2) <= ci <= (m - 1) // 2
+
+
+def test_3m_hand_example():
+    # m = 253 (no square root of -1: 253 = 11 * 23), a = 3 + 2i, b = 1 - 4i, ab = 11 - 10i:
+    # P1 = 3, P2 = -8, P3 = (3 + 2)(1 - 4) = -15; real = P1 - P2 = 11, imaginary = P3 - P1 - P2 = -10
+    a3, b3 = staged.pre_3m(3, 2, 253), staged.pre_3m(1, -4, 253)
+    assert a3 == (3, 2, 5) and b3 == (1, -4, -3)
+    P = [staged.sym(x * y, 253) for x, y in zip(a3, b3)]
+    assert P == [3, -8, -15] and staged.post_3m(*P, 253) == (11, -10)
+    with pytest.raises(ValueError):
+        staged.sqrt_minus_one(253)
+
+
+@pytest.mark.parametrize("nmod", [23, 24, 26])
+def test_hybrid_integer_path_equals_exact_product(nmod):
+    # entries large enough that the result needs the moduli beyond the 22nd: |c| < 2 k 2^(2 b) must stay below M/2
+    rng = np.random.default_rng(nmod)
+    m, n, k, bits = 6, 5, 9, 75
+    big = lambda shape: np.array([int(rng.integers(-2 ** 62, 2 ** 62)) * 2 ** (bits - 62) + int(rng.integers(0, 2 ** 13))
+                                  for _ in range(int(np.prod(shape)))], dtype=object).reshape(shape)
+    Ar, Ai, Br, Bi = big((m, k)), big((m, k)), big((k, n)), big((k, n))
+    st = staged.gemm2m_int_staged(Ar, Ai, Br, Bi, nmod)
+    cr = Ar.dot(Br) - Ai.dot(Bi)          # exact: Python integers
+    ci = Ar.dot(Bi) + Ai.dot(Br)
+    assert max(abs(int(v)) for v in np.concatenate([cr.ravel(), ci.ravel()])) > staged.product(staged.greedy_2m_moduli()) // 2
+    assert (st["Xr"] == cr).all() and (st["Xi"] == ci).all()
+    assert len(st["Cpm"][22]) == 3 and len(st["Cpm"][0]) == 2
+    # a wrong sign in the 3M post-processing, or 3M residues fed to the 2M formulas, cannot survive this: the last
+    # modulus alone decides the top bits of the result
+
+
+@pytest.mark.parametrize("nmod", [23, 26])
+def test_hybrid_float_path_bound_and_error(nmod):
+    A, B = inputs.complex_inputs(10, 7, 60, seed=3 + nmod, dist="phi", phi=4.0)     # wide exponent span
+    st = staged.zgemm2m_staged(A, B, nmod)
+    assert st["moduli"][22:] == [256, 253, 251, 249][: nmod - 22]
+    assert st["PA"] + st["PB"] == st["Pt"] and 2 ** st["Pt"] <= (st["M"] - 1) // 2 < 2 ** (st["Pt"] + 1)
+    assert all(abs(int(v)) <= 2 ** st["Pt"] for v in np.concatenate([st["Xr"].ravel(), st["Xi"].ravel()]))
+    pairs = np.array([(i, j) for i in range(10) for j in range(7)])
+    Xs, vals = staged.staged_samples(st, pairs)       # plain integer product of the quantised matrices
+    assert all(int(st["Xr"][i, j]) == xr and int(st["Xi"][i, j]) == xi for (i, j), (xr, xi) in zip(pairs.tolist(), Xs))
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(st["C"], Cref, D) <= 2.0 ** -52
+    # more moduli than 22 must not be worse than 22
+    e22 = direct.componentwise_error(staged.zgemm2m_staged(A, B, 22)["C"], Cref, D)
+    assert direct.componentwise_error(st["C"], Cref, D) <= e22
