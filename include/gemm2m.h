@@ -25,6 +25,12 @@
  *   - `nmod` selects the first nmod moduli of the set of Section 4 (241, 233, 229, 221, 205, ... , 37, 29; 22 in
  *     all).  More moduli = larger M = more accuracy and proportionally more work.  16 gives about double
  *     precision accuracy for zgemm2m/zherk2m, 7 about single precision for cgemm2m.
+ *   - Hybrid 2M/3M (remark after Algorithm 1; Section 4, last paragraph but one): zgemm2m and cgemm2m also accept
+ *     nmod = 23 ... 26.  The moduli beyond the 22nd are the non-2M moduli 256, 253, 251, 249 (the next numbers of the
+ *     greedy walk down from 256 that are coprime to everything chosen before); each of them takes 3M multiplication,
+ *     Eq. (1), applied after the reduction modulo m: three real int8 GEMMs A_r B_r, A_i B_i, (A_r + A_i)(B_r + B_i).
+ *     M reaches about 2^184; useful when a row of A or a column of B spans many binary orders of magnitude.  The
+ *     rank-k family and gemm2m_gaussian_int take 2M moduli only.
  *   - One call at a time per workspace: calls that share a workspace must be ordered on the GPU (same stream).
  *   - Non-finite inputs: a row of A (column of B) that contains an Inf or NaN yields NaN in the whole
  *     corresponding row (column) of C; no error is reported.
@@ -42,7 +48,7 @@ extern "C" {
 typedef enum {
     GEMM2M_OK = 0,
     GEMM2M_ERR_ARG = 1,            /* negative size, leading dimension too small, null pointer with non-empty matrix */
-    GEMM2M_ERR_NMOD = 2,           /* nmod outside [1, 22], or > 8 for the int64 result of gemm2m_gaussian_int */
+    GEMM2M_ERR_NMOD = 2,           /* nmod outside [1, 26] (zgemm2m, cgemm2m) or [1, 22] (rank-k family), or > 8 for gemm2m_gaussian_int */
     GEMM2M_ERR_WORKSPACE = 3,      /* no workspace registered or too small; nothing was launched */
     GEMM2M_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (see gemm2m_last_cuda_error) */
     GEMM2M_ERR_ARCH = 5,           /* current device is not compute capability 10.0 */
@@ -59,9 +65,12 @@ const char* gemm2m_status_string(int status);
 /* Text of the last CUDA error seen by this thread's calls (static/thread-local string, never NULL). */
 const char* gemm2m_last_cuda_error(void);
 
-/* Number of 2M moduli available (22): the greedy coprime set in [1, 256] of Section 4. */
+/* Number of moduli available to zgemm2m / cgemm2m (26): the 2M moduli followed by the 3M moduli of the hybrid. */
 int gemm2m_max_moduli(void);
-/* j-th modulus (0-based, descending) and its smallest positive square root of -1 (Section 2).  Host pointers. */
+/* Number of 2M moduli available (22): the greedy coprime set in [1, 256] of Section 4. */
+int gemm2m_max_2m_moduli(void);
+/* j-th modulus (0-based; the 2M moduli in descending order, then the 3M moduli) and its smallest positive square root
+ * of -1 (Section 2), 0 for a 3M modulus.  Host pointers. */
 int gemm2m_modulus(int j, int* m, int* s);
 
 /* Bytes of device workspace a call of `op` with these sizes needs (for the rank-k family pass m = n).  0 on bad arguments. */
@@ -172,7 +181,7 @@ int gemm2m_debug_set_panels(int max_panels);
 /* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host
  * pointers, any may be NULL), so that CPU tests can check them against an independent computation:
  *   scale[4]        = P_t, P_A, P_B, c_k of the scaling rule (herk != 0: P_A = P_B)
- *   crt_gr/gi[nmod*4] = signed base-2^40 digits of the folded CRT weights (real / imaginary part), crt_m[4] = digits of M
+ *   crt_gr/gi[nmod*5] = signed base-2^40 digits of the folded CRT weights (real / imaginary part), crt_m[5] = digits of M
  *   nchunks         = number of digits in use
  *   res_w[nmod*16]  = int8 byte weights of the residue kernels: 8 for the real part, then 8 for the imaginary part */
 int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,

@@ -46,6 +46,7 @@ def lib():
     L.gemm2m_status_string.argtypes = [i32]
     L.gemm2m_last_cuda_error.restype = ctypes.c_char_p
     L.gemm2m_max_moduli.restype = i32
+    L.gemm2m_max_2m_moduli.restype = i32
     L.gemm2m_modulus.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.gemm2m_workspace_bytes.restype = sz
     L.gemm2m_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
@@ -98,6 +99,10 @@ def _colmajor(t, name):
 
 def max_moduli():
     return int(lib().gemm2m_max_moduli())
+
+
+def max_2m_moduli():
+    return int(lib().gemm2m_max_2m_moduli())
 
 
 def modulus(j):
@@ -241,9 +246,9 @@ def debug_tables(nmod, k, herk=False):
     """Host-side constants of the library for `nmod` moduli (see gemm2m_debug_tables)."""
     import numpy as np
     scale = np.zeros(4, dtype=np.int32)
-    gr = np.zeros((nmod, 4), dtype=np.float64)
-    gi = np.zeros((nmod, 4), dtype=np.float64)
-    mc = np.zeros(4, dtype=np.float64)
+    gr = np.zeros((nmod, 5), dtype=np.float64)
+    gi = np.zeros((nmod, 5), dtype=np.float64)
+    mc = np.zeros(5, dtype=np.float64)
     nch = np.zeros(1, dtype=np.int32)
     w = np.zeros((nmod, 16), dtype=np.int8)
     ptr = lambda a: ctypes.c_void_p(a.ctypes.data)

@@ -69,6 +69,7 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     const bool herk = op >= GEMM2M_OP_ZHERK;                                   // the rank-k family: one scale vector, C+ only
     const bool two = op == GEMM2M_OP_ZHER2K || op == GEMM2M_OP_DSYR2K;         // rank-2k: two operands
     const bool real_in = op == GEMM2M_OP_DSYRK || op == GEMM2M_OP_DSYR2K;      // real input, packed as Z = X1 + i X2
+    if (herk && nmod > kMax2M) return false;                                   // the hybrid moduli serve the complex GEMMs only
     if (herk) m = n;
     if (real_in) k = (k + 1) / 2;
     const int64_t kp = round_up(k > 0 ? k : 1, 128), ldp = round_up(m > 0 ? m : 1, 16);
@@ -81,9 +82,10 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_exp_b = take(herk ? 0 : 4 * n);
     c->off_pack_a = take(real_in ? 16 * n * k : 0);
     c->off_pack_b = take(real_in && two ? 16 * n * k : 0);
-    c->off_apm = take(2 * (int64_t)nmod * m * kp);
-    c->off_bpm = take((herk && !two) ? 0 : 2 * (int64_t)nmod * n * kp);
-    c->off_cpm = take((herk ? 1 : 2) * (int64_t)nmod * n * ldp);
+    const int64_t planes = plane_count(nmod);                                  // 2 per 2M modulus, 3 per 3M modulus
+    c->off_apm = take(planes * m * kp);
+    c->off_bpm = take((herk && !two) ? 0 : planes * n * kp);
+    c->off_cpm = take((herk ? (int64_t)nmod : planes) * n * ldp);
     c->kp = kp;
     c->ldp = ldp;
     c->total = off;
@@ -187,18 +189,18 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     CK(launch_residues_fp<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
     CK(launch_residues_fp<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
     CK(ph.end(st));
-    // Eq. (2b): 2 nmod real int8 GEMMs; TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
+    // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
     // panel p run on the library's side stream, on the SM resources the GEMM kernel leaves free.  (Forming the residues of
     // later panels of B beside the GEMMs as well was measured and brought nothing: the GEMMs slow down by what is hidden.)
     GemmArgs ga;
     ga.rowop = bpm; ga.colop = apm;
     ga.R = n; ga.Cn = m; ga.Kp = c.kp;
-    ga.row_planes = ga.col_planes = 2 * nmod;
+    ga.row_planes = ga.col_planes = plane_count(nmod);
     ga.row_plane0 = ga.col_plane0 = 0;
-    ga.nbatch = 2 * nmod;
+    ga.nbatch = plane_count(nmod);
     ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
-    build_mod_table(nmod, &ga.mods);
+    build_mod_table(nmod, true, &ga.mods);
     ga.dev_status = dev_status;
     int panels = (int)(n / 1024);
     panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
@@ -250,6 +252,8 @@ const char* gemm2m_status_string(int status) {
 const char* gemm2m_last_cuda_error(void) { return g_cuda_err; }
 
 int gemm2m_max_moduli(void) { return kMaxMod; }
+
+int gemm2m_max_2m_moduli(void) { return kMax2M; }
 
 int gemm2m_modulus(int j, int* m, int* s) {
     if (j < 0 || j >= kMaxMod) return GEMM2M_ERR_ARG;
@@ -329,7 +333,7 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     ga.row_plane0 = ga.col_plane0 = 0;
     ga.nbatch = 2 * nmod;
     ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
-    build_mod_table(nmod, &ga.mods);
+    build_mod_table(nmod, true, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
     ga.row_begin = 0; ga.row_end = n;
     CK(ph.begin(2, st));
@@ -361,7 +365,7 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     const bool real_in = op == GEMM2M_OP_DSYRK || op == GEMM2M_OP_DSYR2K;
     if (n < 0 || k < 0) return GEMM2M_ERR_ARG;
     if (lda < (n > 1 ? n : 1) || ldc < (n > 1 ? n : 1) || (two && ldb < (n > 1 ? n : 1))) return GEMM2M_ERR_ARG;
-    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
+    if (nmod < 1 || nmod > kMax2M) return GEMM2M_ERR_NMOD;    // 2M moduli only: the hybrid serves the complex GEMMs
     if (n > kMaxRows) return GEMM2M_ERR_ARG;
     if (n == 0) return GEMM2M_OK;
     if (!C || (k > 0 && (!A || (two && !B)))) return GEMM2M_ERR_ARG;
@@ -425,7 +429,7 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     ga.col_plane0 = 0;       // "+" planes
     ga.nbatch = nmod;
     ga.out = cp; ga.ldp = c.ldp;
-    build_mod_table(nmod, &ga.mods);
+    build_mod_table(nmod, false, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
     ga.row_begin = 0; ga.row_end = n;
     CK(ph.begin(2, st));

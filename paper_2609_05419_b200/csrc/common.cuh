@@ -1,20 +1,29 @@
 // Shared declarations of the gemm2m CUDA library: constant tables passed to kernels by value,
 // launch wrappers of each phase, and small device helpers.  Notation follows the paper:
-// m_j = 2M modulus, s_j = its square root of -1, M = product of the moduli in use.
+// m_j = modulus (the first 22 are 2M moduli with s_j = their square root of -1; the hybrid of Section 3 appends up to four
+// non-2M moduli that take 3M multiplication, Eq. (1)), M = product of the moduli in use.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace gemm2m {
 
-constexpr int kMaxMod = 22;        // size of the greedy 2M modulus set in [1, 256] (Section 4)
-constexpr int kMaxChunks = 4;      // 40-bit digits needed for M/2 < 2^152
+constexpr int kMax2M = 22;         // size of the greedy 2M modulus set in [1, 256] (Section 4)
+constexpr int kMax3M = 4;          // non-2M moduli of the hybrid: 256, 253, 251, 249 (quantised values then still fit 96 bits)
+constexpr int kMaxMod = kMax2M + kMax3M;
+constexpr int kMaxPlanes = 2 * kMax2M + 3 * kMax3M;   // residue planes per operand: two per 2M modulus, three per 3M modulus
+constexpr int kMaxChunks = 5;      // 40-bit digits needed for M/2 < 2^184
 constexpr int kChunkBits = 40;
 constexpr int kExpNonFinite = INT32_MIN;   // scale-exponent sentinel: row/column holds an Inf or NaN
 
 // Device status word values (written by kernels whose bounded waits give up).
 constexpr int kDevOk = 0;
 constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilogue = 103;
+
+// Number of 2M moduli among the first nmod, and of residue planes per operand.  Plane order: X+ of the 2M moduli, X- of the
+// 2M moduli, then for the 3M moduli X_r, X_i, X_r + X_i (each group in modulus order).
+__host__ __device__ inline int count_2m(int nmod) { return nmod < kMax2M ? nmod : kMax2M; }
+__host__ __device__ inline int plane_count(int nmod) { return 2 * count_2m(nmod) + 3 * (nmod - count_2m(nmod)); }
 
 // Per-modulus constants for the residue kernels, Eq. (2a).
 // A quantised part x (two's complement, 64 bits; 96 bits in the wide mode used from 19-20 moduli on) is written as 4
@@ -31,20 +40,22 @@ struct ResidueTable {
     uint32_t w_top[kMaxMod], ws_top[kMaxMod];  // b = 8..11: only used when quantised values exceed 62 bits
     int32_t s[kMaxMod];
     int32_t xmax[kMaxMod];                     // bound on |real dp4a sum| + |imaginary dp4a sum| (host side only)
-    int nmod;
+    int nmod, n2;                              // moduli in use; the first n2 are 2M moduli, the rest (ws = w) take 3M
 };
 
-// Moduli for the GEMM epilogue (reduction of the int32 accumulators mod m_j).
+// Modulus of every batch entry of a GEMM launch, for the epilogue (reduction of the int32 accumulators).
 struct ModTable {
-    int32_t m[kMaxMod];
-    float inv_m[kMaxMod];
-    int nmod;
+    int32_t m[kMaxPlanes];
+    float inv_m[kMaxPlanes];
+    int nplanes;
 };
 
 // CRT constants for the floating-point post-processing (Eq. (2c) folded into the CRT weights):
 //   X_r = sum_j (c-_j + c+_j) Gr_j  (mod M),  Gr_j = sym(2^-1 q_j mod m_j) (M/m_j)
 //   X_i = sum_j (c-_j - c+_j) Gi_j  (mod M),  Gi_j = sym(s_j 2^-1 q_j mod m_j) (M/m_j)
-// with q_j = (M/m_j)^-1 mod m_j.  Each weight is stored as signed base-2^40 digits held in doubles, so
+// with q_j = (M/m_j)^-1 mod m_j.  For a 3M modulus (j >= n2) the planes hold P1, P2, P3 of Eq. (1) and
+//   X_r += (P1 - P2) G_j,  X_i += (P3 - P1 - P2) G_j,  G_j = sym(q_j mod m_j) (M/m_j)   (stored in both gr and gi).
+// Each weight is stored as signed base-2^40 digits held in doubles, so
 // that every digit-column sum is an exact integer below 2^53.  The multiple of M to remove is estimated from the
 // two leading digit-column sums: t = rint(S_top q_hi + S_(top-1) q_lo), q_hi = 2^(40 top)/M, q_lo = q_hi 2^-40.
 struct CrtTable {
@@ -52,7 +63,7 @@ struct CrtTable {
     double gi[kMaxMod][kMaxChunks];
     double Mc[kMaxChunks];                     // digits of M
     double q_hi, q_lo;
-    int nmod, nchunks;
+    int nmod, n2, nchunks;
 };
 
 // CRT constants for the exact int64 result (nmod <= 8, M < 2^62).
@@ -71,11 +82,12 @@ int modulus_value(int j);
 int modulus_root(int j);
 void build_residue_table(int nmod, ResidueTable* t);
 double residue_reduction_margin(const ResidueTable& t, int j);
-void build_mod_table(int nmod, ModTable* t);
+// per_plane: one entry per residue plane in plane order (complex GEMM); otherwise one entry per modulus (rank-k family).
+void build_mod_table(int nmod, bool per_plane, ModTable* t);
 void build_crt_table(int nmod, CrtTable* t);
 void build_crt_table_int(int nmod, CrtTableInt* t);
 ScaleTargets scale_targets(int nmod, int64_t k, bool herk);
-int64_t gemm_k_limit(int nmod);     // largest K for which k ((m_1-1)/2)^2 fits int32
+int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
 
 // ---- phase launchers (prepost.cu) ----
 // Exponent scan: largest |Re|,|Im| bit pattern per row of a column-major matrix (rows x cols, ld).
@@ -102,7 +114,7 @@ cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n
                             int64_t ldc, cudaStream_t st, int* launches);
 
 // ---- int8 GEMM (gemm_i8.cu) ----
-// For each batch b in [0, nbatch): out[b][r][c] = sym( sum_k rowop[b + row_plane0][r][k] * colop[b + col_plane0][c][k]  mod m_{b % nmod} ),
+// For each batch b in [0, nbatch): out[b][r][c] = sym( sum_k rowop[b + row_plane0][r][k] * colop[b + col_plane0][c][k]  mod (modulus of batch entry b) ),
 // r < R, c < Cn, k < Kp (zero padded); planes are [*][rows][Kp] int8; out planes are [R][ldp] int8.
 struct GemmArgs {
     const int8_t* rowop; const int8_t* colop;

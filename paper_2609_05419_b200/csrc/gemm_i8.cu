@@ -132,7 +132,7 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
             const int acc = it & 1;
             int b, tr, tc;
             decode_tile(p, tile, &b, &tr, &tc);
-            const int jm = b % p.mods.nmod;
+            const int jm = b;                             // the modulus table has one entry per batch entry
             const int m = p.mods.m[jm];
             const float inv_m = p.mods.inv_m[jm];
             if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase[acc], abort_flag, p.dev_status, kDevTimeoutEpilogue))) break;
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __rest
     const int64_t r = row_begin + (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
     const int b = blockIdx.z;
     if (r >= R || r >= row_end || c >= Cn) return;
-    const int jm = b % mods.nmod;
+    const int jm = b;
     const int m = mods.m[jm];
     const int* pr = reinterpret_cast<const int*>(rowop + ((int64_t)(row_plane0 + b) * R + r) * Kp);
     const int* pc = reinterpret_cast<const int*>(colop + ((int64_t)(col_plane0 + b) * Cn + c) * Kp);
@@ -237,8 +237,7 @@ __global__ void __launch_bounds__(256) gemm_i8_check_kernel(const int8_t* __rest
         for (int64_t k = k0 / 4; k < k1 / 4; ++k) acc = __dp4a(pr[k], pc[k], acc);
         res = (res + acc % m) % m;
     }
-    const int h = (m - 1) / 2;
-    if (res > h) res -= m; else if (res < -h) res += m;
+    if (res > (m - 1) / 2) res -= m; else if (res < -(m / 2)) res += m;   // [-(m-1)/2, (m-1)/2]; even m: [-m/2, m/2 - 1]
     out[(int64_t)b * R * ldp + r * ldp + c] = (int8_t)res;
 }
 

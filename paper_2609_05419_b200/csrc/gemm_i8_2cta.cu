@@ -177,7 +177,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
             const int acc = it & 1;
             int b, tr, tc;
             decode_tile(p, tile, &b, &tr, &tc);
-            const int jm = b % p.mods.nmod;
+            const int jm = b;                             // the modulus table has one entry per batch entry
             const int m = p.mods.m[jm];
             const float inv_m = p.mods.inv_m[jm];
             if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase[acc], abort_flag, p.dev_status, kDevTimeoutEpilogue))) break;

@@ -126,9 +126,8 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 __device__ __forceinline__ int sym_reduce_acc(int x, int m, float inv_m) {
     const int q = __float2int_rn(__int2float_rn(x) * inv_m);
     int r = x - q * m;
-    const int h = (m - 1) >> 1;
-    if (r > h) r -= m;
-    if (r < -h) r += m;
+    if (r > ((m - 1) >> 1)) r -= m;
+    if (r < -(m >> 1)) r += m;        // even m (256, hybrid only): the range is [-m/2, m/2 - 1]
     return r;
 }
 

@@ -148,8 +148,8 @@ __device__ __forceinline__ long long quantise_part(T v, int e) {
     return neg ? -(long long)q : (long long)q;
 }
 
-// Wide mode: |result| < 2^76 (19 or more moduli); returned as the low 32 bits and the signed upper 64 bits of the 96-bit
-// two's complement value.
+// Wide mode: |result| < 2^92 (19 or more moduli; 2^76 without the hybrid's 3M moduli); returned as the low 32 bits and the
+// signed upper 64 bits of the 96-bit two's complement value.
 template <typename T>
 __device__ __forceinline__ void quantise_part_wide(T v, int e, uint32_t* lo, long long* upper) {
     using F = FpBits<T>;
@@ -160,7 +160,7 @@ __device__ __forceinline__ void quantise_part_wide(T v, int e, uint32_t* lo, lon
     const int sh = max(E, 1) - (F::kBias + F::kMantBits) - e;
     const bool neg = (sizeof(T) == 8) ? (__double_as_longlong((double)v) < 0) : (__float_as_int((float)v) < 0);
     unsigned __int128 q;
-    if (sh >= 0) q = (unsigned __int128)mant << min(sh, 64);
+    if (sh >= 0) q = (unsigned __int128)mant << min(sh, 74);   // a legitimate shift stays below 92 - 23; the clamp only keeps the shift defined
     else q = (-sh > 63) ? 0 : (mant >> (-sh));
     const __int128 sq = neg ? -(__int128)q : (__int128)q;
     *lo = (uint32_t)(unsigned __int128)sq;
@@ -209,15 +209,33 @@ __device__ __forceinline__ Digits split_digits_wide(uint32_t lo, long long upper
     return d;
 }
 
-// Residues of NE consecutive elements of one operand row for every modulus, written as NE-byte vectors into both sign
-// planes.  dst points at plane 0, this row, first k of the run; tr / ti (wide mode) hold the four top digits of each part.
+// One symmetric residue from y = bits(Y0) + x (see sym_reduce_pm).
+__device__ __forceinline__ uint32_t sym_reduce_one(int y, int neg_m, float inv_m, float cq) {
+    const int t = __float_as_int(fmaf(__int_as_float(y), inv_m, cq));
+    return (uint32_t)(t * neg_m + y);
+}
+
+__device__ __forceinline__ uint32_t pack4(const uint32_t (&b)[4]) {   // low bytes of four words -> one word
+    return __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+}
+
+template <int NE>
+__device__ __forceinline__ void store_run(int8_t* dst, const uint32_t (&w)[NE / 4]) {
+    if (NE == 16) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2 % (NE / 4)], w[3 % (NE / 4)]);
+    else *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+}
+
+// Residues of NE consecutive elements of one operand row for every modulus, written as NE-byte vectors into the planes of
+// that modulus: X+ and X- (Eq. 2a) for the 2M moduli, then X_r, X_i and X_r + X_i (Eq. 1 after the reduction) for the 3M
+// moduli of the hybrid.  dst points at plane 0, this row, first k of the run; tr / ti (wide mode) hold the four top digits
+// of each part.
 template <int NE, bool WIDE>
 __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tr, const uint32_t* ti,
                                          const ResidueTable& tab, int8_t* dst, int64_t plane_stride) {
     static_assert(NE == 8 || NE == 16, "runs of 8 or 16 elements");
-    const int nmod = tab.nmod;
+    const int nmod = tab.nmod, n2 = tab.n2;
 #pragma unroll 1
-    for (int j = 0; j < nmod; ++j) {
+    for (int j = 0; j < n2; ++j) {
         const int neg_m = -tab.m[j], y0 = tab.magic[j];
         const float inv_m = tab.inv_m[j], cq = tab.cq[j];
         const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
@@ -238,18 +256,43 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
                 const int ym = (int)(2u * (uint32_t)Ry - (uint32_t)yp);     // the doubled bit pattern wraps, the difference does not
                 sym_reduce_pm(yp, ym, neg_m, inv_m, cq, &bp[b], &bm[b]);
             }
-            pw[w] = __byte_perm(__byte_perm(bp[0], bp[1], 0x0040), __byte_perm(bp[2], bp[3], 0x0040), 0x5410);
-            mw[w] = __byte_perm(__byte_perm(bm[0], bm[1], 0x0040), __byte_perm(bm[2], bm[3], 0x0040), 0x5410);
+            pw[w] = pack4(bp);
+            mw[w] = pack4(bm);
         }
-        int8_t* dp = dst + (int64_t)j * plane_stride;
-        int8_t* dm = dst + (int64_t)(nmod + j) * plane_stride;
-        if (NE == 16) {
-            *reinterpret_cast<uint4*>(dp) = make_uint4(pw[0], pw[1], pw[2 % (NE / 4)], pw[3 % (NE / 4)]);
-            *reinterpret_cast<uint4*>(dm) = make_uint4(mw[0], mw[1], mw[2 % (NE / 4)], mw[3 % (NE / 4)]);
-        } else {
-            *reinterpret_cast<uint2*>(dp) = make_uint2(pw[0], pw[1]);
-            *reinterpret_cast<uint2*>(dm) = make_uint2(mw[0], mw[1]);
+        store_run<NE>(dst + (int64_t)j * plane_stride, pw);
+        store_run<NE>(dst + (int64_t)(n2 + j) * plane_stride, mw);
+    }
+    const int n3 = nmod - n2;
+    int8_t* dst3 = dst + (int64_t)(2 * n2) * plane_stride;
+#pragma unroll 1
+    for (int j3 = 0; j3 < n3; ++j3) {
+        const int j = n2 + j3;
+        const int neg_m = -tab.m[j], y0 = tab.magic[j];
+        const float inv_m = tab.inv_m[j], cq = tab.cq[j];
+        const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], wt = WIDE ? tab.w_top[j] : 0u;
+        uint32_t rw[NE / 4], iw[NE / 4], sw[NE / 4];
+#pragma unroll
+        for (int w = 0; w < NE / 4; ++w) {
+            uint32_t br[4], bi[4], bs[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = 4 * w + b;
+                int Ry = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
+                if (WIDE) Ry = dp4a_ss(tr[i], wt, Ry);
+                int ys = dp4a_ss(di[i].hi, wh, dp4a_us(di[i].lo, wl, Ry));  // A_r + A_i: the same weights for both parts
+                if (WIDE) ys = dp4a_ss(ti[i], wt, ys);
+                const int Iy = ys - Ry + y0;                                // A_i alone
+                br[b] = sym_reduce_one(Ry, neg_m, inv_m, cq);
+                bi[b] = sym_reduce_one(Iy, neg_m, inv_m, cq);
+                bs[b] = sym_reduce_one(ys, neg_m, inv_m, cq);
+            }
+            rw[w] = pack4(br);
+            iw[w] = pack4(bi);
+            sw[w] = pack4(bs);
         }
+        store_run<NE>(dst3 + (int64_t)j3 * plane_stride, rw);
+        store_run<NE>(dst3 + (int64_t)(n3 + j3) * plane_stride, iw);
+        store_run<NE>(dst3 + (int64_t)(2 * n3 + j3) * plane_stride, sw);
     }
 }
 
@@ -526,21 +569,21 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// cpm: [2 nmod][n][ldp] int8 (row index i contiguous).  A block handles 512 consecutive i of one column j: it first pulls
-// the 2 nmod x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
+// cpm: [planes][n][ldp] int8 (row index i contiguous), planes = C+ and C- of the 2M moduli, then P1, P2, P3 of the 3M
+// moduli.  A block handles 512 consecutive i of one column j: it first pulls the planes x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
 // thread combines 4 consecutive i.
 template <typename T, int NCH>
 __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
                                                                const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
                                                                const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc) {
-    __shared__ __align__(16) uint32_t stage[2 * kMaxMod][kPostThreads];
+    __shared__ __align__(16) uint32_t stage[kMaxPlanes][kPostThreads];
     const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
     const int64_t j = blockIdx.y;
-    const int nmod = tab.nmod;
+    const int nmod = tab.nmod, n2 = tab.n2, n3 = nmod - n2;
     const int64_t plane = n * ldp;
     const int8_t* src = cpm + j * ldp + ib;
     const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);   // ldp is a multiple of 16
-    for (int idx = threadIdx.x; idx < 2 * nmod * (kPostSpan / 16); idx += kPostThreads) {
+    for (int idx = threadIdx.x; idx < (2 * n2 + 3 * n3) * (kPostSpan / 16); idx += kPostThreads) {
         const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
         if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
     }
@@ -555,9 +598,9 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
         for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
     }
 #pragma unroll 2
-    for (int jm = 0; jm < nmod; ++jm) {
+    for (int jm = 0; jm < n2; ++jm) {
         const uint32_t wp = stage[jm][threadIdx.x];            // c+ of 4 elements
-        const uint32_t wm = stage[nmod + jm][threadIdx.x];     // c-
+        const uint32_t wm = stage[n2 + jm][threadIdx.x];       // c-
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int cp = (int)(int8_t)(wp >> (8 * e));
@@ -568,6 +611,23 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
             for (int c = 0; c < NCH; ++c) {
                 Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
                 Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
+            }
+        }
+    }
+#pragma unroll 1
+    for (int j3 = 0; j3 < n3; ++j3) {                      // 3M moduli of the hybrid, Eq. (1)
+        const uint32_t w1 = stage[2 * n2 + j3][threadIdx.x];
+        const uint32_t w2 = stage[2 * n2 + n3 + j3][threadIdx.x];
+        const uint32_t w3 = stage[2 * n2 + 2 * n3 + j3][threadIdx.x];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int p1 = (int)(int8_t)(w1 >> (8 * e)), p2 = (int)(int8_t)(w2 >> (8 * e)), p3 = (int)(int8_t)(w3 >> (8 * e));
+            const double vr = int_to_double(p1 - p2);
+            const double vi = int_to_double(p3 - p1 - p2);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[e][c] = fma(vr, tab.gr[n2 + j3][c], Sr[e][c]);
+                Si[e][c] = fma(vi, tab.gr[n2 + j3][c], Si[e][c]);
             }
         }
     }
@@ -608,7 +668,8 @@ cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n,
             case 1: post_fp_kernel<T, 1><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
             case 2: post_fp_kernel<T, 2><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
             case 3: post_fp_kernel<T, 3><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
-            default: post_fp_kernel<T, 4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 4: post_fp_kernel<T, 4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            default: post_fp_kernel<T, 5><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
         }
         ++*launches;
     }

@@ -9,27 +9,29 @@
 
 namespace gemm2m {
 
-// Greedy coprime set of 2M moduli in [1, 256], descending (Section 4).
-static const int kModuli[kMaxMod] = {241, 233, 229, 221, 205, 197, 193, 181, 173, 157, 149,
-                                     137, 113, 109, 101, 97,  89,  73,  61,  53,  37,  29};
+// Greedy coprime set of 2M moduli in [1, 256], descending (Section 4), followed by the first non-2M moduli of the same
+// greedy walk that are coprime to all of them (hybrid 2M/3M, Sections 3 and 4).
+static const int kModuli[kMaxMod] = {241, 233, 229, 221, 205, 197, 193, 181, 173, 157, 149, 137, 113,
+                                     109, 101, 97,  89,  73,  61,  53,  37,  29,  256, 253, 251, 249};
 
 int modulus_value(int j) { return kModuli[j]; }
 
-int modulus_root(int j) {   // smallest positive s with s^2 = -1 (mod m)
+int modulus_root(int j) {   // smallest positive s with s^2 = -1 (mod m); 0 for a non-2M modulus
+    if (j >= kMax2M) return 0;
     const int m = kModuli[j];
     for (int s = 1; s < m; ++s)
         if ((s * s + 1) % m == 0) return s;
     return 0;
 }
 
-static inline int sym_mod(int64_t x, int m) {   // representative in [-(m-1)/2, (m-1)/2]
+static inline int sym_mod(int64_t x, int m) {   // representative in [-(m-1)/2, (m-1)/2]; even m: [-m/2, m/2 - 1]
     int r = (int)(x % m);
     if (r < 0) r += m;
     if (r > (m - 1) / 2) r -= m;
     return r;
 }
 
-static int inv_mod(int a, int m) {   // a^-1 mod m by search (m <= 241)
+static int inv_mod(int a, int m) {   // a^-1 mod m by search (m <= 256)
     a %= m;
     if (a < 0) a += m;
     for (int x = 1; x < m; ++x)
@@ -83,8 +85,9 @@ static Big product_of(int nmod) {
 void build_residue_table(int nmod, ResidueTable* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
+    t->n2 = count_2m(nmod);
     for (int j = 0; j < nmod; ++j) {
-        const int m = kModuli[j], s = modulus_root(j);
+        const int m = kModuli[j], s = j < kMax2M ? modulus_root(j) : 1;   // 3M modulus: both parts take the plain weights
         t->m[j] = m;
         t->s[j] = s;
         t->inv_m[j] = 1.0f / (float)m;
@@ -135,10 +138,20 @@ double residue_reduction_margin(const ResidueTable& t, int j) {
     return (double)(1LL << e) / (2.0 * (double)(y0 + t.xmax[j]) * (double)dev);
 }
 
-void build_mod_table(int nmod, ModTable* t) {
+void build_mod_table(int nmod, bool per_plane, ModTable* t) {
     std::memset(t, 0, sizeof(*t));
-    t->nmod = nmod;
-    for (int j = 0; j < nmod; ++j) { t->m[j] = kModuli[j]; t->inv_m[j] = 1.0f / (float)kModuli[j]; }
+    const int n2 = count_2m(nmod);
+    int p = 0;
+    auto put = [&](int j) { t->m[p] = kModuli[j]; t->inv_m[p] = 1.0f / (float)kModuli[j]; ++p; };
+    if (!per_plane) {
+        for (int j = 0; j < nmod; ++j) put(j);
+    } else {
+        for (int rep = 0; rep < 2; ++rep)
+            for (int j = 0; j < n2; ++j) put(j);
+        for (int rep = 0; rep < 3; ++rep)
+            for (int j = n2; j < nmod; ++j) put(j);
+    }
+    t->nplanes = p;
 }
 
 // Folded CRT weights: g_j = sym(2^-1 q_j mod m_j), h_j = sym(s_j 2^-1 q_j mod m_j), q_j = (M/m_j)^-1 mod m_j.
@@ -147,6 +160,10 @@ static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h
     *W = M;
     W->divmod_small((uint32_t)m);
     const int q = inv_mod((int)W->mod_small((uint32_t)m), m);
+    if (j >= kMax2M) {              // 3M modulus: Eq. (1) needs no factor besides q_j
+        *g = *h = sym_mod(q, m);
+        return;
+    }
     const int half = (m + 1) / 2;   // 2^-1 mod m (Section 2)
     *g = sym_mod((int64_t)half * q, m);
     *h = sym_mod((int64_t)modulus_root(j) * half % m * q, m);
@@ -156,13 +173,16 @@ static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h
 void build_crt_table(int nmod, CrtTable* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
+    t->n2 = count_2m(nmod);
     const Big M = product_of(nmod);
     Big half = M;   // (M-1)/2 bounds every |G_j|
     half.sub_one();
     half.shr1();
     t->nchunks = (half.bit_length() + kChunkBits - 1) / kChunkBits;
     if (t->nchunks < 1) t->nchunks = 1;
-    for (int c = 0; c < kMaxChunks; ++c) t->Mc[c] = (double)M.bits(c * kChunkBits, kChunkBits);
+    // digits of M; the top digit in use takes every remaining bit (M may be one bit longer than (M-1)/2: 41 bits there)
+    for (int c = 0; c < t->nchunks; ++c)
+        t->Mc[c] = (double)M.bits(c * kChunkBits, c + 1 < t->nchunks ? kChunkBits : 60);
     for (int j = 0; j < nmod; ++j) {
         Big W;
         int g, h;
@@ -212,8 +232,8 @@ ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
 }
 
 int64_t gemm_k_limit(int nmod) {
-    (void)nmod;
-    const int64_t h = (kModuli[0] - 1) / 2;   // the largest modulus comes first
+    // largest |residue|: 120 for the 2M moduli (241 comes first), 128 once the hybrid adds the modulus 256
+    const int64_t h = nmod > kMax2M ? 128 : (kModuli[0] - 1) / 2;
     return (int64_t)INT32_MAX / (h * h);
 }
 

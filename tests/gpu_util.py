@@ -50,12 +50,22 @@ class Workspace:
         kp, ldp = lay["kp"], lay["ldp"]
         out = dict(layout=lay)
         out["eA"] = raw[lay["off_exp_a"]: lay["off_exp_a"] + 4 * rows_a].view(np.int32).copy()
-        out["Apm"] = raw[lay["off_apm"]: lay["off_apm"] + 2 * nmod * rows_a * kp].view(np.int8).reshape(2, nmod, rows_a, kp)
+        n2 = min(nmod, 22)                      # 2M moduli: planes X+ then X-; 3M moduli (hybrid): X_r, X_i, X_r + X_i
+        n3 = nmod - n2
+
+        def split(off, rows, ld):
+            flat = raw[off: off + (2 * n2 + 3 * n3) * rows * ld].view(np.int8)
+            two = flat[: 2 * n2 * rows * ld].reshape(2, n2, rows, ld)
+            three = flat[2 * n2 * rows * ld:].reshape(3, n3, rows, ld)
+            return two, three
+
         if not herk:
+            out["Apm"], out["A3"] = split(lay["off_apm"], rows_a, kp)
             out["eB"] = raw[lay["off_exp_b"]: lay["off_exp_b"] + 4 * n].view(np.int32).copy()
-            out["Bpm"] = raw[lay["off_bpm"]: lay["off_bpm"] + 2 * nmod * n * kp].view(np.int8).reshape(2, nmod, n, kp)
-            out["Cpm"] = raw[lay["off_cpm"]: lay["off_cpm"] + 2 * nmod * n * ldp].view(np.int8).reshape(2, nmod, n, ldp)
+            out["Bpm"], out["B3"] = split(lay["off_bpm"], n, kp)
+            out["Cpm"], out["C3"] = split(lay["off_cpm"], n, ldp)
         else:
+            out["Apm"] = raw[lay["off_apm"]: lay["off_apm"] + 2 * nmod * rows_a * kp].view(np.int8).reshape(2, nmod, rows_a, kp)
             out["Cpm"] = raw[lay["off_cpm"]: lay["off_cpm"] + nmod * n * ldp].view(np.int8).reshape(1, nmod, n, ldp)
         return out
 

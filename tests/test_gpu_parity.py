@@ -128,6 +128,50 @@ def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
         assert direct.componentwise_error(C, Cref, D) <= TOL_Z
 
 
+@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])
+@pytest.mark.parametrize("shape,nmod,phi", [((70, 90, 200), 23, 4.0), ((129, 257, 128), 26, 6.0), ((33, 19, 50), 24, 1.0),
+                                            ((40, 300, 520), 25, 8.0)])
+def test_zgemm_hybrid_every_stage_against_staged_oracle(shape, nmod, phi, kernel):
+    """Hybrid 2M/3M (Section 3 remark): the moduli beyond the 22nd take Eq. (1) with three planes each."""
+    m, n, k = shape
+    A, B = inputs.complex_inputs(m, n, k, seed=17, dist="phi", phi=phi)       # wide exponent span: what the hybrid is for
+    C, st = run_z(A, B, nmod, kernel)
+    ref = staged.zgemm2m_staged(A, B, nmod)
+    assert (st["eA"] == ref["eA"]).all() and (st["eB"] == ref["eB"]).all()
+    for j in range(22):
+        for sgn in range(2):
+            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all(), ("Apm", sgn, j)
+            assert (st["Bpm"][sgn, j, :, :k] == ref["Bpm"][j][sgn].T).all(), ("Bpm", sgn, j)
+            assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j)
+    for j3 in range(nmod - 22):
+        for part in range(3):                                                  # X_r, X_i, X_r + X_i  /  P1, P2, P3
+            assert (st["A3"][part, j3, :, :k] == ref["Apm"][22 + j3][part]).all(), ("A3", part, j3)
+            assert (st["B3"][part, j3, :, :k] == ref["Bpm"][22 + j3][part].T).all(), ("B3", part, j3)
+            assert (st["C3"][part, j3, :, :m] == ref["Cpm"][22 + j3][part].T).all(), ("C3", part, j3)
+    assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
+    assert (C == ref["C"]).mean() > 0.999
+    Cref, D = direct.zgemm4m_dd(A, B)
+    err = direct.componentwise_error(C, Cref, D)
+    if phi <= 4.0:
+        assert err <= TOL_Z
+    else:       # the spread of exponents inside a row exceeds what any M <= 2^184 resolves: the method's own limit, which
+        assert err <= 1.01 * direct.componentwise_error(ref["C"], Cref, D)      # the staged oracle shares
+
+
+def test_hybrid_beats_the_2m_set_on_a_wide_exponent_span_and_cgemm_accepts_it():
+    m, n, k = 48, 40, 160
+    A, B = inputs.complex_inputs(m, n, k, seed=23, dist="phi", phi=6.0)    # all 22 2M moduli fall short of double precision here
+    Cref, D = direct.zgemm4m_dd(A, B)
+    e22 = direct.componentwise_error(run_z(A, B, 22)[0], Cref, D)
+    e26 = direct.componentwise_error(run_z(A, B, 26)[0], Cref, D)
+    assert e22 > 1e-13 and e26 <= TOL_Z
+    A32, B32 = A.astype(np.complex64), B.astype(np.complex64)
+    C32, _ = run_z(A32, B32, 23, cplx=torch.complex64)
+    ref = staged.zgemm2m_staged(A32, B32, 23, out_bits=24)
+    for got, want in ((C32.real, ref["C"].real), (C32.imag, ref["C"].imag)):   # 53 then 24 bits: within one float ulp
+        assert (np.abs(got.astype(np.float64) - want) <= np.spacing(np.abs(want).astype(np.float32)).astype(np.float64)).all()
+
+
 @pytest.mark.parametrize("nmod,tol", [(16, TOL_Z), (15, TOL_Z), (14, 1e-13)])
 def test_zgemm_1024_full_oracle(nmod, tol):
     A, B = inputs.complex_inputs(1024, 1024, 1024, seed=1)

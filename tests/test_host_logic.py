@@ -25,11 +25,15 @@ def test_library_exports_every_declared_symbol():
 
 def test_moduli_and_roots_match_oracle():
     mods = staged.greedy_2m_moduli()
-    assert b.max_moduli() == len(mods)
+    assert b.max_2m_moduli() == len(mods)
     for j, m in enumerate(mods):
         assert b.modulus(j) == (m, staged.sqrt_minus_one(m))
+    hyb = staged.hybrid_moduli(b.max_moduli())
+    assert b.max_moduli() == 26 and hyb[:22] == mods
+    for j in range(22, 26):
+        assert b.modulus(j) == (hyb[j], 0)                # 3M modulus: no root
     with pytest.raises(b.Gemm2mError):
-        b.modulus(22)
+        b.modulus(26)
 
 
 @pytest.mark.parametrize("nmod", [1, 2, 3, 7, 8, 16, 17, 20, 22])
@@ -41,16 +45,16 @@ def test_crt_and_scaling_constants_match_oracle(nmod):
         assert (t["Pt"], t["PA"], t["PB"], t["ck"]) == staged.scaling_targets(M, k, herk)
     t = b.debug_tables(nmod, 8192)
     B = 2 ** 40
-    assert sum(int(t["Mc"][c]) * B ** c for c in range(4)) == M
+    assert sum(int(t["Mc"][c]) * B ** c for c in range(t["nchunks"])) == M       # the digits the kernel reads
     assert (t["nchunks"] - 1) * 40 < ((M - 1) // 2).bit_length() <= t["nchunks"] * 40
     for j, (m, s) in enumerate(zip(mods, [staged.sqrt_minus_one(q) for q in mods])):
         W = M // m
         q = pow(W % m, -1, m)
-        Gr = sum(int(t["gr"][j, c]) * B ** c for c in range(4))
-        Gi = sum(int(t["gi"][j, c]) * B ** c for c in range(4))
+        Gr = sum(int(t["gr"][j, c]) * B ** c for c in range(5))
+        Gi = sum(int(t["gi"][j, c]) * B ** c for c in range(5))
         assert Gr == staged.sym(staged.inv2(m) * q, m) * W          # Eq. (2c) real part folded into the CRT weight
         assert Gi == staged.sym(s * staged.inv2(m) * q, m) * W      # imaginary part
-        assert all(abs(t["gr"][j, c]) < B and abs(t["gi"][j, c]) < B for c in range(4))
+        assert all(abs(t["gr"][j, c]) < B and abs(t["gi"][j, c]) < B for c in range(5))
         for bb in range(8):                                          # byte weights of the residue kernels
             assert int(t["res_w"][j, bb]) == staged.sym(256 ** bb, m)
             assert int(t["res_w"][j, 8 + bb]) == staged.sym(s * 256 ** bb, m)
@@ -60,13 +64,13 @@ def test_residue_reduction_constants_are_exact_for_every_reachable_sum():
     """The residue kernels reduce x (a sum of byte-weight products) modulo m with one FP32 FMA and one integer
     multiply-add.  Emulate that FMA in exact integer arithmetic (float operands are dyadic rationals; round to nearest
     even at unit spacing) for EVERY integer x the kernels can reach and require the symmetric residue in the low byte."""
-    r = b.debug_residue_reduction(22)
-    mods = staged.greedy_2m_moduli()
+    r = b.debug_residue_reduction(26)
+    mods = staged.hybrid_moduli(26)
     for j, m in enumerate(mods):
         y0_bits, xmax = int(r["y0_bits"][j]), int(r["xmax"][j])
         y0 = (y0_bits - 0x4B000000) + 2 ** 23                 # value of the float with that bit pattern (exponent 2^23)
         assert y0 % (256 * m) == 0 and y0 - xmax >= 2 ** 23 and y0 + xmax < 2 ** 24
-        s = staged.sqrt_minus_one(m)
+        s = staged.sqrt_minus_one(m) if j < 22 else 1          # a 3M modulus takes the plain weights for both parts
         w = [abs(staged.sym(256 ** bb, m)) + abs(staged.sym(s * 256 ** bb, m)) for bb in range(12)]
         assert xmax == 255 * sum(w[:4]) + 128 * sum(w[4:])    # four unsigned bytes, eight balanced digits, both parts
         assert float(r["margin"][j]) > 1.0
@@ -86,7 +90,7 @@ def test_residue_reduction_constants_are_exact_for_every_reachable_sum():
         y_bits = y0_bits + x
         low = (y_bits - t_bits * m) & 0xFF
         res = np.where(low >= 128, low - 256, low)
-        want = ((x + (m - 1) // 2) % m) - (m - 1) // 2
+        want = ((x + m // 2) % m) - m // 2                     # symmetric range; [-m/2, m/2 - 1] for the even modulus
         assert np.array_equal(res, want), m
 
 
@@ -105,9 +109,58 @@ def test_folded_crt_weights_reproduce_eq_2c_and_crt():
             post = [staged.post_2m(p, q, m, s) for p, q, m, s in zip(cp, cm, mods, roots)]
             xr = staged.lift(staged.crt([r for r, _ in post], mods), M)
             xi = staged.lift(staged.crt([i for _, i in post], mods), M)
-            Sr = sum((q + p) * sum(int(t["gr"][j, c]) * B ** c for c in range(4)) for j, (p, q) in enumerate(zip(cp, cm)))
-            Si = sum((q - p) * sum(int(t["gi"][j, c]) * B ** c for c in range(4)) for j, (p, q) in enumerate(zip(cp, cm)))
+            Sr = sum((q + p) * sum(int(t["gr"][j, c]) * B ** c for c in range(5)) for j, (p, q) in enumerate(zip(cp, cm)))
+            Si = sum((q - p) * sum(int(t["gi"][j, c]) * B ** c for c in range(5)) for j, (p, q) in enumerate(zip(cp, cm)))
             assert staged.lift(Sr, M) == xr and staged.lift(Si, M) == xi
+
+
+@pytest.mark.parametrize("nmod", [23, 24, 26])
+def test_hybrid_crt_and_scaling_constants_match_oracle(nmod):
+    mods = staged.hybrid_moduli(nmod)
+    roots = staged.roots_of(mods)
+    M = staged.product(mods)
+    for k, herk in ((1, False), (300, False), (8192, False), (131000, False)):
+        t = b.debug_tables(nmod, k, herk)
+        assert (t["Pt"], t["PA"], t["PB"], t["ck"]) == staged.scaling_targets(M, k, herk)
+    t = b.debug_tables(nmod, 64)
+    B = 2 ** 40
+    val = lambda row: sum(int(row[c]) * B ** c for c in range(5))
+    assert val(t["Mc"]) == M and all(t["Mc"][c] == 0 for c in range(t["nchunks"], 5))   # only the digits in use: the kernel reads no others
+    assert (t["nchunks"] - 1) * 40 < ((M - 1) // 2).bit_length() <= t["nchunks"] * 40
+    for j, (m, s) in enumerate(zip(mods, roots)):
+        W = M // m
+        q = pow(W % m, -1, m)
+        if s is not None:
+            assert val(t["gr"][j]) == staged.sym(staged.inv2(m) * q, m) * W
+            assert val(t["gi"][j]) == staged.sym(s * staged.inv2(m) * q, m) * W
+        else:                                                         # Eq. (1) needs no factor besides q_j
+            assert val(t["gr"][j]) == staged.sym(q, m) * W == val(t["gi"][j])
+        for bb in range(8):
+            assert int(t["res_w"][j, bb]) == staged.sym(256 ** bb, m)
+            assert int(t["res_w"][j, 8 + bb]) == staged.sym((s or 1) * 256 ** bb, m)
+    # the folded sums reproduce post-processing + CRT + lift for random residues of every plane
+    rng = np.random.default_rng(nmod)
+    for _ in range(20):
+        Sr = Si = 0
+        res_r, res_i = [], []
+        for j, (m, s) in enumerate(zip(mods, roots)):
+            draw = lambda: int(rng.integers(-(m // 2), (m - 1) // 2 + 1))
+            if s is not None:
+                cp, cm = draw(), draw()
+                r, i = staged.post_2m(cp, cm, m, s)
+                Sr += (cm + cp) * val(t["gr"][j])
+                Si += (cm - cp) * val(t["gi"][j])
+            else:
+                p1, p2, p3 = draw(), draw(), draw()
+                r, i = staged.post_3m(p1, p2, p3, m)
+                Sr += (p1 - p2) * val(t["gr"][j])
+                Si += (p3 - p1 - p2) * val(t["gr"][j])
+            res_r.append(r)
+            res_i.append(i)
+        assert staged.lift(Sr % M, M) == staged.lift(staged.crt(res_r, mods), M)
+        assert staged.lift(Si % M, M) == staged.lift(staged.crt(res_i, mods), M)
+        assert abs(Sr) < 2 ** 12 * M and abs(Si) < 2 ** 12 * M        # the multiple of M to remove stays below 2^12
+    assert 2 ** t["Pt"] / M < 0.494                                   # margin of the quotient estimate in the post kernel
 
 
 def test_workspace_layout_is_ordered_and_sized():
@@ -122,7 +175,13 @@ def test_workspace_layout_is_ordered_and_sized():
         for key in ("off_exp_a", "off_exp_b", "off_apm", "off_bpm", "off_cpm"):
             assert lay[key] % 256 == 0
     assert b.workspace_bytes(b.OP_GAUSSIAN_INT, 8, 8, 8, 9) == 0      # int64 result needs M < 2^63
-    assert b.workspace_bytes(b.OP_ZGEMM, 8, 8, 8, 23) == 0
+    assert b.workspace_bytes(b.OP_ZGEMM, 8, 8, 8, 27) == 0
+    assert b.workspace_bytes(b.OP_ZHERK, 8, 8, 8, 23) == 0            # the hybrid moduli serve the complex GEMMs only
+    # hybrid: two planes per 2M modulus, three per 3M modulus
+    lay = b.workspace_layout(b.OP_ZGEMM, 100, 60, 200, 25)
+    planes = 2 * 22 + 3 * 3
+    assert lay["off_apm"] + planes * 100 * lay["kp"] <= lay["off_bpm"] and lay["off_bpm"] + planes * 60 * lay["kp"] <= lay["off_cpm"]
+    assert lay["off_cpm"] + planes * 60 * lay["ldp"] <= lay["total_bytes"]
     assert b.workspace_bytes(b.OP_ZGEMM, -1, 8, 8, 3) == 0
 
 
@@ -136,7 +195,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.zgemm2m(4, 4, 4, one, 4, one, 3, one, 4, 16, null) == ARG          # ldb < k
     assert L.zgemm2m(4, 4, 4, one, 4, one, 4, one, 3, 16, null) == ARG          # ldc < m
     assert L.zgemm2m(4, 4, 4, one, 4, one, 4, one, 4, 0, null) == NMOD
-    assert L.zgemm2m(4, 4, 4, one, 4, one, 4, one, 4, 23, null) == NMOD
+    assert L.zgemm2m(4, 4, 4, one, 4, one, 4, one, 4, 27, null) == NMOD
     assert L.zgemm2m(4, 4, 4, null, 4, one, 4, one, 4, 16, null) == ARG         # null A with k > 0
     assert L.zgemm2m(0, 4, 4, null, 1, null, 4, null, 1, 16, null) == 0         # empty: valid no-op
     assert L.cgemm2m(4, 0, 4, null, 4, null, 4, null, 4, 7, null) == 0
@@ -144,6 +203,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.gemm2m_gaussian_int(4, 4, 4, one, one, 2, one, one, 4, one, one, 4, 3, null) == ARG
     assert L.zherk2m(4, 4, one, 3, one, 4, 16, null) == ARG
     assert L.zherk2m(0, 4, null, 1, null, 1, 16, null) == 0
+    assert L.zherk2m(4, 4, one, 4, one, 4, 23, null) == NMOD                    # rank-k family: 2M moduli only
     assert L.gemm2m_set_workspace(one, 0) == ARG
     assert L.gemm2m_set_workspace(ctypes.c_void_p(8), 1024) == ARG              # not 256-byte aligned
     assert b.lib().gemm2m_status_string(WS) == b"GEMM2M_ERR_WORKSPACE"
