@@ -174,6 +174,10 @@ int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, g
  * kernel kept only so that tests can tell a fault in a tensor-core kernel from one in the pre/post kernels, 2 = the
  * tcgen05 kernel with one CTA per tile. */
 int gemm2m_debug_set_gemm_kernel(int which);
+/* Which kernel forms the residues of floating-point operands: 0 = the dp4a kernel (default), 1 = the tensor-core kernel
+ * (the digit-weight contraction of Eq. (2a) as an int8 MMA with the planes along the TMEM lanes; same planes, bit for
+ * bit; measured slower than the default and kept as a selectable variant). */
+int gemm2m_debug_set_residue_kernel(int which);
 /* Largest number of column panels zgemm2m/cgemm2m cut C into (default 4).  With 1 the phases run strictly one after the
  * other on the caller's stream, which is what per-phase bandwidth figures should be measured with. */
 int gemm2m_debug_set_panels(int max_panels);

@@ -66,6 +66,7 @@ def lib():
     L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
     L.gemm2m_debug_set_panels.argtypes = [i32]
+    L.gemm2m_debug_set_residue_kernel.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
     L.gemm2m_debug_residue_reduction.argtypes = [i32, vp, vp, vp, vp, vp]
     _lib = L
@@ -236,6 +237,11 @@ def last_launch_count():
 
 def debug_set_gemm_kernel(which):
     _check(lib().gemm2m_debug_set_gemm_kernel(which), "gemm2m_debug_set_gemm_kernel")
+
+
+def debug_set_residue_kernel(which):
+    """0 = dp4a residue kernel (default), 1 = tensor-core residue kernel."""
+    _check(lib().gemm2m_debug_set_residue_kernel(int(which)), "gemm2m_debug_set_residue_kernel")
 
 
 def debug_set_panels(max_panels):

@@ -29,6 +29,7 @@ struct State {
     int max_panels = 4;           // column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
+    int residue_kernel = 0;       // 0 = dp4a residue kernel, 1 = tensor-core residue kernel (measured slower; kept selectable)
     int sm_count = 0;
     int arch_ok = -1;
 };
@@ -130,6 +131,14 @@ int ensure_side_stream() {
 
 constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kernels
 
+template <typename T>
+int run_residues(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e, const ResidueTable& tab,
+                 bool wide, int8_t* planes, int* dev_status, cudaStream_t st) {
+    if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
+    else CK(launch_residues_tc<T>(X, ld, k_contiguous, R, K, Kp, e, tab, wide, planes, dev_status, g.sm_count, st, &g.launches[1]));
+    return GEMM2M_OK;
+}
+
 int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
     const int64_t klim = gemm_k_limit(nmod);
     if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
@@ -186,8 +195,8 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
-    CK(launch_residues_fp<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
-    CK(launch_residues_fp<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
+    if (int s = run_residues<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
+    if (int s = run_residues<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
@@ -415,8 +424,9 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
         CK(cudaMemsetAsync(apm, 0, (size_t)2 * nmod * n * c.kp, st));
         if (two) CK(cudaMemsetAsync(bpm, 0, (size_t)2 * nmod * n * c.kp, st));
     } else {
-        CK(launch_residues_fp<double>(ZA, ldza, false, n, kc, c.kp, eA, rtab, wide, apm, st, &g.launches[1]));
-        if (two) CK(launch_residues_fp<double>(ZB, ldzb, false, n, kc, c.kp, eA, rtab, wide, bpm, st, &g.launches[1]));
+        int* dev_status = (int*)(ws + c.off_status);
+        if (int s = run_residues<double>(ZA, ldza, false, n, kc, c.kp, eA, rtab, wide, apm, dev_status, st)) return s;
+        if (two) { if (int s = run_residues<double>(ZB, ldzb, false, n, kc, c.kp, eA, rtab, wide, bpm, dev_status, st)) return s; }
     }
     CK(ph.end(st));
     // Section 5.  HERK: C+ = A+ A-^T.  HER2K: C+ = A+ B-^T + B+ A-^T (second product accumulated mod m_j).  C- = C+^T in both.
@@ -524,6 +534,13 @@ int gemm2m_debug_set_gemm_kernel(int which) {
     std::lock_guard<std::mutex> lock(g.mu);
     if (which < 0 || which > 2) return GEMM2M_ERR_ARG;
     g.gemm_kernel = which;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_set_residue_kernel(int which) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (which < 0 || which > 1) return GEMM2M_ERR_ARG;
+    g.residue_kernel = which;
     return GEMM2M_OK;
 }
 

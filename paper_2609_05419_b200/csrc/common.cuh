@@ -100,6 +100,10 @@ template <typename T> cudaError_t launch_exponents(const uint64_t* absmax, int64
 // wide = quantised values may need more than 62 bits (P - c_k > 62): they are carried as mantissa x 2^t.
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+// The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.
+template <typename T> cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status,
+                                                     int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).

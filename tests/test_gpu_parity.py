@@ -18,8 +18,10 @@ TOL_C = 2e-6       # complex64
 @pytest.fixture(autouse=True)
 def _default_kernel():
     b.debug_set_gemm_kernel(0)
+    b.debug_set_residue_kernel(0)
     yield
     b.debug_set_gemm_kernel(0)
+    b.debug_set_residue_kernel(0)
 
 
 def run_int(Ar, Ai, Br, Bi, nmod, kernel=0, ldc=None):
@@ -170,6 +172,31 @@ def test_hybrid_beats_the_2m_set_on_a_wide_exponent_span_and_cgemm_accepts_it():
     ref = staged.zgemm2m_staged(A32, B32, 23, out_bits=24)
     for got, want in ((C32.real, ref["C"].real), (C32.imag, ref["C"].imag)):   # 53 then 24 bits: within one float ulp
         assert (np.abs(got.astype(np.float64) - want) <= np.spacing(np.abs(want).astype(np.float32)).astype(np.float64)).all()
+
+
+@pytest.mark.parametrize("shape,nmod,dist,dtype", [((200, 150, 300), 16, "phi", np.complex128), ((129, 257, 128), 14, "uniform", np.complex128),
+                                                   ((33, 19, 50), 22, "phi", np.complex128), ((70, 90, 200), 25, "phi", np.complex128),
+                                                   ((257, 300, 1000), 7, "uniform", np.complex64), ((64, 40, 130), 23, "phi", np.complex64)])
+def test_tensor_core_residue_kernel_gives_the_same_planes(shape, nmod, dist, dtype):
+    """The selectable residue kernel (digit-weight contraction as an int8 MMA): every plane bit-exact against the staged
+    oracle, narrow and wide quantised values, four and two element blocks per instruction, 2M and 3M moduli, ragged tiles."""
+    m, n, k = shape
+    A, B = inputs.complex_inputs(m, n, k, seed=31, dist=dist, phi=2.0, dtype=dtype)
+    b.debug_set_residue_kernel(1)
+    C, st = run_z(A, B, nmod, kernel=1, cplx=torch.complex128 if dtype == np.complex128 else torch.complex64)
+    ref = staged.zgemm2m_staged(A, B, nmod, out_bits=53 if dtype == np.complex128 else 24)
+    n2 = min(nmod, 22)
+    for j in range(n2):
+        for sgn in range(2):
+            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all(), ("Apm", sgn, j)
+            assert (st["Bpm"][sgn, j, :, :k] == ref["Bpm"][j][sgn].T).all(), ("Bpm", sgn, j)
+            assert (st["Apm"][sgn, j, :, k:] == 0).all() and (st["Bpm"][sgn, j, :, k:] == 0).all()     # K padding
+    for j3 in range(nmod - n2):
+        for part in range(3):
+            assert (st["A3"][part, j3, :, :k] == ref["Apm"][22 + j3][part]).all(), ("A3", part, j3)
+            assert (st["B3"][part, j3, :, :k] == ref["Bpm"][22 + j3][part].T).all(), ("B3", part, j3)
+    if dtype == np.complex128:
+        assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
 
 
 @pytest.mark.parametrize("nmod,tol", [(16, TOL_Z), (15, TOL_Z), (14, 1e-13)])
