@@ -97,6 +97,19 @@ int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const
 int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb,
             float* C, int64_t ldc, int nmod, void* stream);
 
+/* BLAS-style extended forms (the paper fixes alpha = 1, beta = 0 and untransposed operands, Section 6; these follow
+ * the ZGEMM / CGEMM conventions beyond that): C = alpha op(A) op(B) + beta C with op(X) = X ('N'), X^T ('T') or X^H ('C'),
+ * op(A) m x k, op(B) k x n.  A is stored m x k ('N', lda >= m) or k x m (lda >= k); B is stored k x n ('N', ldb >= k) or
+ * n x k (ldb >= n).  alpha, beta: HOST pointers to one complex number (re, im); NULL means alpha = 1 / beta = 0.
+ * The product op(A) op(B) is formed exactly as by zgemm2m (a transposed operand is only read in the other orientation; a
+ * conjugated one changes the sign of its imaginary parts before quantisation), rounded once, and then combined with
+ * alpha, beta and the old C in working precision with fused multiply-adds.  beta = 0: C is not read; alpha = 0: A and B
+ * are not read and C = beta C.  A bad trans character returns GEMM2M_ERR_ARG. */
+int zgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A, int64_t lda,
+               const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc, int nmod, void* stream);
+int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const float* alpha, const float* A, int64_t lda,
+               const float* B, int64_t ldb, const float* beta, float* C, int64_t ldc, int nmod, void* stream);
+
 /* Hermitian rank-k update C = A A^H (Section 5, HERK) with ONE real int8 GEMM per modulus: C+ = A+ A-^T and
  * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
  * diagonal is written; diagonal imaginary parts are exactly 0; the strict upper triangle is not touched. */

@@ -146,6 +146,44 @@ def zgemm4m_dd2(A1, B1, A2, B2):
     return C, D
 
 
+def apply_op(X, trans):
+    """op(X) of the BLAS interface: 'N' -> X, 'T' -> X^T, 'C' -> X^H."""
+    X = np.asarray(X)
+    t = trans.upper()
+    if t == "N":
+        return X
+    if t == "T":
+        return X.T
+    if t == "C":
+        return X.conj().T
+    raise ValueError(trans)
+
+
+def zgemm_ex_dd(transa, transb, alpha, A, B, beta, C0):
+    """The ZGEMM definition alpha op(A) op(B) + beta C0 (the paper's Section 6 fixes alpha = 1, beta = 0, no transposes;
+    this is the BLAS convention beyond that).  The product is the double-double 4M product rounded once; the combination
+    with alpha, beta is evaluated in extended precision (64-bit significand) and rounded once.
+    Returns the result and the error scale D = |alpha| |op(A)||op(B)| + |beta| |C0|."""
+    alpha, beta = complex(alpha), complex(beta)
+    L = np.longdouble
+    opA, opB = apply_op(A, transa), apply_op(B, transb)
+    shape = (opA.shape[0], opB.shape[1])
+    re, im, scale = np.zeros(shape, dtype=L), np.zeros(shape, dtype=L), np.zeros(shape)
+    if alpha != 0:                      # alpha = 0: A and B are not referenced
+        P, D = zgemm4m_dd(opA, opB)
+        pr, pi = P.real.astype(L), P.imag.astype(L)
+        re = L(alpha.real) * pr - L(alpha.imag) * pi
+        im = L(alpha.real) * pi + L(alpha.imag) * pr
+        scale = abs(alpha) * D
+    if beta != 0:                       # beta = 0: C0 is not referenced (it may hold NaNs)
+        C0 = _as_z(C0)
+        cr, ci = C0.real.astype(L), C0.imag.astype(L)
+        re = re + L(beta.real) * cr - L(beta.imag) * ci
+        im = im + L(beta.real) * ci + L(beta.imag) * cr
+        scale = scale + abs(beta) * np.abs(C0)
+    return np.asfortranarray(re.astype(np.float64) + 1j * im.astype(np.float64)), np.asfortranarray(scale)
+
+
 def zherk_dd(A):
     """Section 5, HERK: C = A A^H."""
     A = _as_z(A)

@@ -54,6 +54,9 @@ def lib():
     L.gemm2m_gaussian_int.argtypes = [i64, i64, i64, vp, vp, i64, vp, vp, i64, vp, vp, i64, i32, vp]
     L.zgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.cgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    ex = [ctypes.c_char, ctypes.c_char, i64, i64, i64, vp, vp, i64, vp, i64, vp, vp, i64, i32, vp]
+    L.zgemm2m_ex.argtypes = ex
+    L.cgemm2m_ex.argtypes = ex
     L.zherk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
     L.dsyrk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
     L.zher2k2m.argtypes = [i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
@@ -161,6 +164,29 @@ def zgemm2m(A, B, C, nmod=16, stream=None):
 
 def cgemm2m(A, B, C, nmod=7, stream=None):
     _xgemm(lib().cgemm2m, "cgemm2m", A, B, C, nmod, stream)
+
+
+def _xgemm_ex(fn, name, ctype, transa, transb, alpha, A, B, beta, C, nmod, stream):
+    """C = alpha op(A) op(B) + beta C; A, B as stored (column-major views), trans in 'N', 'T', 'C'."""
+    pa, ra, ca, lda = _colmajor(A, "A")
+    pb, rb, cb, ldb = _colmajor(B, "B")
+    pc, m, n, ldc = _colmajor(C, "C")
+    ma, ka = (ra, ca) if transa in "Nn" else (ca, ra)
+    kb, nb = (rb, cb) if transb in "Nn" else (cb, rb)
+    if ka != kb or (ma, nb) != (m, n):
+        raise ValueError("shape mismatch")
+    pair = lambda z: None if z is None else (ctype * 2)(complex(z).real, complex(z).imag)
+    al, be = pair(alpha), pair(beta)
+    ptr = lambda a: None if a is None else ctypes.cast(a, ctypes.c_void_p)
+    _check(fn(transa.encode(), transb.encode(), m, n, ka, ptr(al), pa, lda, pb, ldb, ptr(be), pc, ldc, nmod, _stream_ptr(stream)), name)
+
+
+def zgemm2m_ex(transa, transb, alpha, A, B, beta, C, nmod=16, stream=None):
+    _xgemm_ex(lib().zgemm2m_ex, "zgemm2m_ex", ctypes.c_double, transa, transb, alpha, A, B, beta, C, nmod, stream)
+
+
+def cgemm2m_ex(transa, transb, alpha, A, B, beta, C, nmod=7, stream=None):
+    _xgemm_ex(lib().cgemm2m_ex, "cgemm2m_ex", ctypes.c_float, transa, transb, alpha, A, B, beta, C, nmod, stream)
 
 
 def zherk2m(A, C, nmod=16, stream=None):

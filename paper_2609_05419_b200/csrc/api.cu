@@ -132,10 +132,10 @@ int ensure_side_stream() {
 constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kernels
 
 template <typename T>
-int run_residues(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e, const ResidueTable& tab,
-                 bool wide, int8_t* planes, int* dev_status, cudaStream_t st) {
-    if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
-    else CK(launch_residues_tc<T>(X, ld, k_contiguous, R, K, Kp, e, tab, wide, planes, dev_status, g.sm_count, st, &g.launches[1]));
+int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st) {
+    if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
+    else CK(launch_residues_tc<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, dev_status, g.sm_count, st, &g.launches[1]));
     return GEMM2M_OK;
 }
 
@@ -147,20 +147,31 @@ int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
     return GEMM2M_OK;
 }
 
+// transa / transb: 'N' (as stored), 'T' (transposed) or 'C' (conjugate transposed) operand, BLAS style; alpha, beta: host
+// pointers to (re, im) pairs or null for 1 and 0.  C = alpha op(A) op(B) + beta C with op(A) m x k and op(B) k x n.
 template <typename T>
-int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, const T* B, int64_t ldb, T* C, int64_t ldc, int nmod,
-            void* stream) {
+int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const T* A, int64_t lda, const T* B,
+            int64_t ldb, const double* beta, T* C, int64_t ldc, int nmod, void* stream) {
     std::lock_guard<std::mutex> lock(g.mu);
+    auto norm = [](char c) { return (c == 'n' || c == 'N') ? 'N' : (c == 't' || c == 'T') ? 'T' : (c == 'c' || c == 'C') ? 'C' : '?'; };
+    const char ta = norm(transa), tb = norm(transb);
+    if (ta == '?' || tb == '?') return GEMM2M_ERR_ARG;
     if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
-    if (lda < (m > 1 ? m : 1) || ldb < (k > 1 ? k : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
+    const int64_t rows_a = ta == 'N' ? m : k, rows_b = tb == 'N' ? k : n;      // rows of the matrices as stored
+    if (lda < (rows_a > 1 ? rows_a : 1) || ldb < (rows_b > 1 ? rows_b : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
     if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
     if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
     if (m == 0 || n == 0) return GEMM2M_OK;
-    if (!C || (k > 0 && (!A || !B))) return GEMM2M_ERR_ARG;
+    const bool alpha_zero = alpha && alpha[0] == 0.0 && alpha[1] == 0.0;
+    if (!C || (k > 0 && !alpha_zero && (!A || !B))) return GEMM2M_ERR_ARG;
     if (int s = check_device()) return s;
     cudaStream_t st = (cudaStream_t)stream;
-    if (k == 0) {
-        CK(cudaMemset2DAsync(C, (size_t)ldc * 2 * sizeof(T), 0, (size_t)m * 2 * sizeof(T), (size_t)n, st));
+    if (k == 0 || alpha_zero) {          // nothing to multiply: C = beta C (A and B are not referenced)
+        std::memset(g.launches, 0, sizeof(g.launches));
+        if (!beta || (beta[0] == 0.0 && beta[1] == 0.0))
+            CK(cudaMemset2DAsync(C, (size_t)ldc * 2 * sizeof(T), 0, (size_t)m * 2 * sizeof(T), (size_t)n, st));
+        else if (!(beta[0] == 1.0 && beta[1] == 0.0))
+            CK(launch_scale_c<T>(C, m, n, ldc, beta, st, &g.launches[3]));
         return GEMM2M_OK;
     }
     Carve c;
@@ -188,15 +199,18 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
     // step 2: scale factors
     CK(ph.begin(0, st));
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
-    CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
-    CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
+    // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C'); columns of op(B) are columns of B or its rows
+    if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
+    else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0]));
+    if (tb == 'N') CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
+    else CK(launch_scan_rows<T>(B, n, k, ldb, absB, st, &g.launches[0]));
     CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
     CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
-    if (int s = run_residues<T>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
-    if (int s = run_residues<T>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
+    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
+    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
@@ -230,7 +244,7 @@ int xgemm2m(int op, int64_t m, int64_t n, int64_t k, const T* A, int64_t lda, co
             CK(cudaStreamWaitEvent(g.side, g.panel_done[pnl], 0));
         }
         CK(ph.begin(3, ps));
-        CK(launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]));
+        CK(launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]));
         CK(ph.end(ps));
     }
     if (panels > 1) {   // join: the call is complete on the caller's stream only when the side stream has finished
@@ -357,12 +371,12 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
 
 int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
             int nmod, void* stream) {
-    return xgemm2m<double>(GEMM2M_OP_ZGEMM, m, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
+    return xgemm2m<double>(GEMM2M_OP_ZGEMM, 'N', 'N', m, n, k, nullptr, A, lda, B, ldb, nullptr, C, ldc, nmod, stream);
 }
 
 int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc, int nmod,
             void* stream) {
-    return xgemm2m<float>(GEMM2M_OP_CGEMM, m, n, k, A, lda, B, ldb, C, ldc, nmod, stream);
+    return xgemm2m<float>(GEMM2M_OP_CGEMM, 'N', 'N', m, n, k, nullptr, A, lda, B, ldb, nullptr, C, ldc, nmod, stream);
 }
 
 // The rank-k family of Section 5: HERK (B == nullptr) and HER2K on complex inputs; SYRK / SYR2K on real inputs through
@@ -425,8 +439,8 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
         if (two) CK(cudaMemsetAsync(bpm, 0, (size_t)2 * nmod * n * c.kp, st));
     } else {
         int* dev_status = (int*)(ws + c.off_status);
-        if (int s = run_residues<double>(ZA, ldza, false, n, kc, c.kp, eA, rtab, wide, apm, dev_status, st)) return s;
-        if (two) { if (int s = run_residues<double>(ZB, ldzb, false, n, kc, c.kp, eA, rtab, wide, bpm, dev_status, st)) return s; }
+        if (int s = run_residues<double>(ZA, ldza, false, false, n, kc, c.kp, eA, rtab, wide, apm, dev_status, st)) return s;
+        if (two) { if (int s = run_residues<double>(ZB, ldzb, false, false, n, kc, c.kp, eA, rtab, wide, bpm, dev_status, st)) return s; }
     }
     CK(ph.end(st));
     // Section 5.  HERK: C+ = A+ A-^T.  HER2K: C+ = A+ B-^T + B+ A-^T (second product accumulated mod m_j).  C- = C+^T in both.
@@ -455,6 +469,19 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     CK(ph.end(st));
     ph.done();
     return GEMM2M_OK;
+}
+
+int zgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A, int64_t lda,
+               const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc, int nmod, void* stream) {
+    return xgemm2m<double>(GEMM2M_OP_ZGEMM, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, nmod, stream);
+}
+
+int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const float* alpha, const float* A, int64_t lda,
+               const float* B, int64_t ldb, const float* beta, float* C, int64_t ldc, int nmod, void* stream) {
+    double a[2] = {1.0, 0.0}, b[2] = {0.0, 0.0};
+    if (alpha) { a[0] = alpha[0]; a[1] = alpha[1]; }
+    if (beta) { b[0] = beta[0]; b[1] = beta[1]; }
+    return xgemm2m<float>(GEMM2M_OP_CGEMM, transa, transb, m, n, k, a, A, lda, B, ldb, b, C, ldc, nmod, stream);
 }
 
 int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {

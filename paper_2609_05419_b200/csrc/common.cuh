@@ -97,18 +97,21 @@ template <typename T> cudaError_t launch_scan_cols(const T* X, int64_t rows, int
 template <typename T> cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int ck, int32_t* e, cudaStream_t st, int* launches);
 // Quantise + residues.  k_contiguous = false: operand row r is row r of the column-major matrix X (A: m x k);
 // true: operand row r is column r of X (B: k x n).
-// wide = quantised values may need more than 62 bits (P - c_k > 62): they are carried as mantissa x 2^t.
-template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+// conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
+template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
 // The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.
-template <typename T> cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+template <typename T> cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status,
                                                      int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).
+// alpha, beta: host pointers to (re, im) pairs, or null for alpha = 1 / beta = 0: C = alpha X + beta C.
 template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
-                                                 const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches);
+                                                 const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta, cudaStream_t st, int* launches);
+// C = beta C (the alpha = 0 case of the extended interface); beta = host pointer to (re, im) or null for 0.
+template <typename T> cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches);
 // real_out: C is a real matrix (SYRK / SYR2K through Z = A1 + i A2): only the real part is formed and stored.
 cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
                              bool real_out, cudaStream_t st, int* launches);

@@ -320,7 +320,7 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <typename T, bool WIDE>
-__global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K,
+__global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K,
                                                                      int64_t Kp, const int32_t* __restrict__ e,
                                                                      const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
     using Raw = typename RawCplx<T>::type;
@@ -379,7 +379,8 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
             uint32_t tr[WIDE ? kResRun : 1], ti[WIDE ? kResRun : 1];
 #pragma unroll
             for (int i = 0; i < kResRun; ++i) {
-                const Raw v = src[r * kResRowStride + kResRun * g + g + i];
+                Raw v = src[r * kResRowStride + kResRun * g + g + i];
+                if (conj) v.y = -v.y;                         // conjugated operand: the imaginary part changes sign before quantisation
                 if (WIDE) {
                     uint32_t lr = 0, li = 0;
                     long long ur = 0, ui = 0;
@@ -421,7 +422,7 @@ static int cached_sm_count() {
 }
 
 template <typename T>
-cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
@@ -435,8 +436,8 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, int64_
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
     const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
-    if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
-    else residues_fp_kernel<T, false><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    if (wide) residues_fp_kernel<T, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+    else residues_fp_kernel<T, false><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
     ++*launches;
     return cudaGetLastError();
 }
@@ -572,10 +573,15 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 // cpm: [planes][n][ldp] int8 (row index i contiguous), planes = C+ and C- of the 2M moduli, then P1, P2, P3 of the 3M
 // moduli.  A block handles 512 consecutive i of one column j: it first pulls the planes x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
 // thread combines 4 consecutive i.
-template <typename T, int NCH>
+// AXPBY: C = alpha X + beta C (alpha, beta complex, given as re/im pairs) instead of C = X; the product X is formed
+// exactly as before, then combined in FP64 with fused multiply-adds.  beta = 0 does not read C.
+struct PostScalars { double ar, ai, br, bi; };
+
+template <typename T, int NCH, bool AXPBY>
 __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
                                                                const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
-                                                               const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc) {
+                                                               const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc,
+                                                               const PostScalars sc) {
     __shared__ __align__(16) uint32_t stage[kMaxPlanes][kPostThreads];
     const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
     const int64_t j = blockIdx.y;
@@ -650,13 +656,28 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
             }
         }
     }
+    if (AXPBY) {
+        const bool use_c = sc.br != 0.0 || sc.bi != 0.0;
+        for (int e = 0; e < count; ++e) {
+            const double xr = re[e], xi = im[e];
+            double yr = fma(sc.ar, xr, -sc.ai * xi), yi = fma(sc.ar, xi, sc.ai * xr);
+            if (use_c) {
+                const T* old = C + 2 * (i0 + e + j * ldc);
+                const double cr = (double)old[0], ci = (double)old[1];
+                yr += fma(sc.br, cr, -sc.bi * ci);
+                yi += fma(sc.br, ci, sc.bi * cr);
+            }
+            re[e] = yr;
+            im[e] = yi;
+        }
+    }
     store4<T>(C + 2 * (i0 + j * ldc), re, im, count);
 }
 
-template <typename T>
-cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
-                           const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, cudaStream_t st, int* launches) {
-    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+template <typename T, bool AXPBY>
+static cudaError_t launch_post_fp_t(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                                    const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const PostScalars& sc, cudaStream_t st,
+                                    int* launches) {
     const int64_t per_block = kPostSpan;
     for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {      // grid.y limit
         const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
@@ -665,16 +686,60 @@ cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n,
         T* dst = C + 2 * j0 * ldc;
         // the plane stride is n * ldp for the whole matrix, so pass the full n and offset pointers
         switch (tab.nchunks) {
-            case 1: post_fp_kernel<T, 1><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
-            case 2: post_fp_kernel<T, 2><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
-            case 3: post_fp_kernel<T, 3><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
-            case 4: post_fp_kernel<T, 4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
-            default: post_fp_kernel<T, 5><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 1: post_fp_kernel<T, 1, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 2: post_fp_kernel<T, 2, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 3: post_fp_kernel<T, 3, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 4: post_fp_kernel<T, 4, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            default: post_fp_kernel<T, 5, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
         }
         ++*launches;
     }
     return cudaGetLastError();
 }
+
+template <typename T>
+cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                           const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta,
+                           cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+    PostScalars sc{1.0, 0.0, 0.0, 0.0};
+    if (alpha) { sc.ar = alpha[0]; sc.ai = alpha[1]; }
+    if (beta) { sc.br = beta[0]; sc.bi = beta[1]; }
+    const bool plain = sc.ar == 1.0 && sc.ai == 0.0 && sc.br == 0.0 && sc.bi == 0.0;
+    if (plain) return launch_post_fp_t<T, false>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
+    return launch_post_fp_t<T, true>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
+}
+
+// C = beta C (C = 0 for beta = 0, without reading C): the alpha = 0 case of the extended interface.
+template <typename T>
+__global__ void __launch_bounds__(256) scale_c_kernel(T* __restrict__ C, int64_t m, int64_t n, int64_t ldc, double br, double bi) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x, j = blockIdx.y;
+    if (i >= m) return;
+    T* c = C + 2 * (i + j * ldc);
+    double yr = 0.0, yi = 0.0;
+    if (br != 0.0 || bi != 0.0) {
+        const double cr = (double)c[0], ci = (double)c[1];
+        yr = fma(br, cr, -bi * ci);
+        yi = fma(br, ci, bi * cr);
+    }
+    c[0] = (T)yr;
+    c[1] = (T)yi;
+}
+
+template <typename T>
+cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches) {
+    if (m <= 0 || n <= 0) return cudaSuccess;
+    const double br = beta ? beta[0] : 0.0, bi = beta ? beta[1] : 0.0;
+    for (int64_t j0 = 0; j0 < n; j0 += 65535) {
+        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+        dim3 grid((unsigned)((m + 255) / 256), (unsigned)nj);
+        scale_c_kernel<T><<<grid, 256, 0, st>>>(C + 2 * j0 * ldc, m, nj, ldc, br, bi);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+template cudaError_t launch_scale_c<double>(double*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
+template cudaError_t launch_scale_c<float>(float*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
 
 // HERK (Section 5): only C+ = A+ A-^T was computed; C- = C+^T.  cp: [nmod][n][ldp] with cp[j][col][row] = C+_j[row, col].
 // A block handles 64 rows i x 16 columns j of the lower triangle.  It needs C+[i, j] (rows of cp along i: 16 runs of 64
@@ -864,9 +929,9 @@ template cudaError_t launch_scan_cols<double>(const double*, int64_t, int64_t, i
 template cudaError_t launch_scan_cols<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
 template cudaError_t launch_exponents<double>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
 template cudaError_t launch_exponents<float>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
-template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
-template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
-template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, cudaStream_t, int*);
-template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, cudaStream_t, int*);
+template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, const double*, const double*, cudaStream_t, int*);
+template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, const double*, const double*, cudaStream_t, int*);
 
 }  // namespace gemm2m

@@ -169,7 +169,7 @@ __device__ __forceinline__ bool mbar_wait_short(uint32_t bar, uint32_t parity, v
 // writes does not wait for anything slow.
 template <typename T, bool WIDE, int NB>
 __global__ void __launch_bounds__(rtc::THREADS, 2)
-residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
+residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                    const int32_t* __restrict__ e, const __grid_constant__ TcPlaneTable tab, int8_t* __restrict__ planes,
                    int* dev_status) {
     using namespace rtc;
@@ -324,7 +324,8 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64
                 uint4 dr = make_uint4(0, 0, 0, 0), di = dr;
                 if (row < R) {
                     const int ex = __ldg(e + row);
-                    const Raw v = src[step * 128];
+                    Raw v = src[step * 128];
+                    if (conj) v.y = -v.y;                     // conjugated operand
                     if (ex != kExpNonFinite) {
                         if (!WIDE && ex > -1000 && ex < 1000) {
                             // x 2^-e is an exact FP64 product (or underflows towards zero, where the truncation is zero
@@ -378,7 +379,7 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64
 }
 
 template <typename T>
-cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
                                const ResidueTable& rtab, bool wide, int8_t* planes, int* dev_status, int sm_count, cudaStream_t st,
                                int* launches) {
     using namespace rtc;
@@ -393,7 +394,7 @@ cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, int64_
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
-        kernel<<<grid, THREADS, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes, dev_status);
+        kernel<<<grid, THREADS, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, dev_status);
         return cudaGetLastError();
     };
     cudaError_t err;
@@ -403,9 +404,9 @@ cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, int64_
     return err;
 }
 
-template cudaError_t launch_residues_tc<double>(const double*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&,
+template cudaError_t launch_residues_tc<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&,
                                                 bool, int8_t*, int*, int, cudaStream_t, int*);
-template cudaError_t launch_residues_tc<float>(const float*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&,
+template cudaError_t launch_residues_tc<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&,
                                                bool, int8_t*, int*, int, cudaStream_t, int*);
 
 }  // namespace gemm2m

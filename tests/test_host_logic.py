@@ -16,8 +16,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def test_library_exports_every_declared_symbol():
     text = open(os.path.join(ROOT, "include", "gemm2m.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = set(re.findall(r"\b((?:gemm2m_\w+|zgemm2m|cgemm2m|zherk2m))\s*\(", text))
-    assert {"gemm2m_gaussian_int", "zgemm2m", "cgemm2m", "zherk2m", "gemm2m_set_workspace", "gemm2m_workspace_bytes"} <= names
+    names = set(re.findall(r"^(?:int|size_t|const char\*)\s+(\w+)\s*\(", text, flags=re.M))      # every declared function
+    assert {"gemm2m_gaussian_int", "zgemm2m", "cgemm2m", "zherk2m", "zher2k2m", "dsyrk2m", "dsyr2k2m", "zgemm2m_ex", "cgemm2m_ex",
+            "gemm2m_set_workspace", "gemm2m_workspace_bytes", "gemm2m_zscale_exponents_static"} <= names
+    assert len(names) >= 25
     L = b.lib()
     for name in names:
         assert hasattr(L, name), name

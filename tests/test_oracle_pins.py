@@ -441,3 +441,38 @@ def test_hybrid_float_path_bound_and_error(nmod):
     # more moduli than 22 must not be worse than 22
     e22 = direct.componentwise_error(staged.zgemm2m_staged(A, B, 22)["C"], Cref, D)
     assert direct.componentwise_error(st["C"], Cref, D) <= e22
+
+
+# ------------------------------------------------------------------ extended interface (alpha, beta, op)
+def test_extended_definition_vs_exact_rationals_and_special_cases():
+    rng = np.random.default_rng(5)
+    m, n, k = 4, 3, 5
+    C0 = rng.standard_normal((m, n)) + 1j * rng.standard_normal((m, n))
+    alpha, beta = 0.75 - 1.5j, -0.5 + 0.25j
+    F = Fraction
+    cf = lambda z: (F(float(np.real(z))), F(float(np.imag(z))))
+    for ta, tb in (("N", "N"), ("T", "N"), ("N", "C"), ("C", "T"), ("C", "C")):
+        A = rng.standard_normal((m, k) if ta == "N" else (k, m)) + 1j * rng.standard_normal((m, k) if ta == "N" else (k, m))
+        B = rng.standard_normal((k, n) if tb == "N" else (n, k)) + 1j * rng.standard_normal((k, n) if tb == "N" else (n, k))
+        got, D = direct.zgemm_ex_dd(ta, tb, alpha, A, B, beta, C0)
+        for i in range(m):
+            for j in range(n):
+                sr = si = F(0)
+                for p in range(k):          # the definition, entry by entry, with op() spelled out by index
+                    a = A[i, p] if ta == "N" else (A[p, i] if ta == "T" else np.conj(A[p, i]))
+                    b_ = B[p, j] if tb == "N" else (B[j, p] if tb == "T" else np.conj(B[j, p]))
+                    (ar, ai), (br, bi) = cf(a), cf(b_)
+                    sr += ar * br - ai * bi
+                    si += ar * bi + ai * br
+                (alr, ali), (ber, bei), (cr, ci) = cf(alpha), cf(beta), cf(C0[i, j])
+                er = alr * sr - ali * si + ber * cr - bei * ci
+                ei = alr * si + ali * sr + ber * ci + bei * cr
+                assert abs(F(float(got[i, j].real)) - er) <= F(float(D[i, j])) * F(1, 2 ** 50)
+                assert abs(F(float(got[i, j].imag)) - ei) <= F(float(D[i, j])) * F(1, 2 ** 50)
+    A = rng.standard_normal((m, k)) + 0j
+    B = rng.standard_normal((k, n)) + 0j
+    nanC = np.full((m, n), np.nan + 0j)
+    P, _ = direct.zgemm4m_dd(A, B)
+    assert (direct.zgemm_ex_dd("N", "N", 1, A, B, 0, nanC)[0] == P).all()              # beta = 0: C0 not referenced
+    assert (direct.zgemm_ex_dd("N", "N", 0, A * np.nan, B, 2, C0)[0] == 2 * C0).all()   # alpha = 0: A, B not referenced
+    assert (direct.zgemm_ex_dd("T", "T", 1, A.T.copy(), B.T.copy(), 0, None)[0] == P).all()        # stored transposed
