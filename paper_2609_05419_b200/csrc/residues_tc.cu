@@ -16,7 +16,7 @@
 // The bytes go to a shared-memory buffer and leave as full 128-byte lines with the lanes of a warp along one plane: a store
 // with one plane per lane touches 32 pages 16 to 64 MiB apart per instruction and ran five times slower.
 //
-// One CTA = 288 threads, 256 TMEM columns (two accumulator buffers), two CTAs per SM; a tile is 8 operand rows x 128 k,
+// One CTA = 416 threads, 256 TMEM columns (two accumulator buffers), two CTAs per SM; a tile is 8 operand rows x 128 k,
 // consumed in 8 steps of 128 elements.
 #include "gemm_ptx.cuh"
 
@@ -25,7 +25,7 @@
 namespace gemm2m {
 
 namespace rtc {
-constexpr int ROWS = 8, KT = 128, THREADS = 288;
+constexpr int ROWS = 8, KT = 128, THREADS = 416;   // 8 reducing warps, 4 quantising warps, 1 issuing warp
 constexpr int RING = 4;                         // tiles of raw elements in flight per CTA
 constexpr int STEP = 128;                       // elements per MMA step = TMEM columns per accumulator buffer
 constexpr int TMEM_COLS = 256;                  // two accumulator buffers
@@ -161,11 +161,11 @@ __device__ __forceinline__ bool mbar_wait_short(uint32_t bar, uint32_t parity, v
     }
 }
 
-// Roles: warps 0-3 reduce and store (warp w reads TMEM lanes 32 w ..), warps 4-7 quantise (one element per thread and
+// Roles: warps 0-7 reduce and store (warps w and w + 4 read TMEM lanes 32 w ..), warps 8-11 quantise (one element per thread and
 // step, fetched by the same thread with cp.async into slots nobody else reads, so no block-wide barrier is needed),
-// warp 8 allocates TMEM and issues the MMAs.  Digits and accumulators are double buffered; four mbarrier pairs hand them
-// round: digits_full (128 quantising threads) -> MMA -> digits_empty and tmem_full (tcgen05.commit) -> reduce ->
-// tmem_empty (4 warps).  The quantising warps never store to global memory, so the proxy fence after their shared-memory
+// warp 12 allocates TMEM and issues the MMAs.  Digits and accumulators are double buffered; four mbarrier pairs hand them
+// round: digits_full (4 quantising warps) -> MMA -> digits_empty and tmem_full (tcgen05.commit) -> reduce ->
+// tmem_empty (8 warps).  The quantising warps never store to global memory, so the proxy fence after their shared-memory
 // writes does not wait for anything slow.
 template <typename T, bool WIDE, int NB>
 __global__ void __launch_bounds__(rtc::THREADS, 2)
@@ -191,15 +191,15 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
 
     if (t == 0) {
         for (int a = 0; a < 2; ++a) {
-            mbar_init(bar_dfull + 8 * a, 128);
+            mbar_init(bar_dfull + 8 * a, 4);
             mbar_init(bar_dempty + 8 * a, 1);
             mbar_init(bar_tfull + 8 * a, 1);
-            mbar_init(bar_tempty + 8 * a, 4);
+            mbar_init(bar_tempty + 8 * a, 8);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8) {
+    if (warp == 12) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -222,16 +222,19 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
     const int64_t total = ((R + ROWS - 1) / ROWS) * ktiles;
     bool ok = true;
 
-    if (warp < 4) {
-        // ------------------------------------------------------------------ reduce + store: one TMEM lane = one plane of one block
-        const int my_lane = 32 * warp + lane;
+    if (warp < 8) {
+        // ------------------------------------------------------------------ reduce + store: one TMEM lane = one plane of one block;
+        // warps w and w + 4 share lane quarter w and take one half each of the block's columns
+        const int quarter = warp & 3, half = warp >> 2;
+        constexpr int CW = CPB / 2;                                // columns per warp and step
+        const int my_lane = 32 * quarter + lane;
         const int my_block = my_lane / RPB, my_plane = my_lane % RPB;
         const bool plane_ok = my_plane < tab.nplanes;
         const int pp = plane_ok ? my_plane : 0;
         const int y0 = tab.y0[pp], neg_m = tab.neg_m[pp];
         const float inv_m = tab.inv_m[pp], cq = tab.cq[pp];
-        const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(my_block * CPB);
-        unsigned char* my_out = outbuf + my_lane * OUT_STRIDE;
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)(my_block * CPB + half * CW);
+        unsigned char* my_out = outbuf + my_lane * OUT_STRIDE + half * CW;
         const int64_t plane_stride = R * Kp;
         uint32_t g = 0;
         for (int64_t tile = blockIdx.x; ok && tile < total; tile += gridDim.x) {
@@ -242,38 +245,36 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
                 if (!(ok = mbar_wait_short(bar_tfull + 8 * buf, ph, abort_flag, dev_status, kDevTimeoutEpilogue))) break;
                 tcgen05_fence_after();
                 const int rg = step / NB, kb = step % NB;
-                uint32_t v[CPB / 32][32];
-#pragma unroll
-                for (int c = 0; c < CPB / 32; ++c) tmem_ld32(taddr + buf * STEP + (uint32_t)(32 * c), v[c]);
+                uint32_t v[CW];
+                if constexpr (CW == 16) tmem_ld16(taddr + buf * STEP, v);
+                else tmem_ld32(taddr + buf * STEP, v);
                 tmem_ld_wait();
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);      // the accumulators are in registers: the MMA may go on
 #pragma unroll
-                for (int c = 0; c < CPB / 32; ++c) {
-                    uint32_t w[8];
+                for (int c = 0; c < CW / 16; ++c) {
+                    uint32_t w[4];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
+                    for (int q = 0; q < 4; ++q) {
                         uint32_t b4[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const int y = (int)v[c][4 * q + i] + y0;                               // bits of the float Y0 + x
+                            const int y = (int)v[16 * c + 4 * q + i] + y0;                          // bits of the float Y0 + x
                             const int tq = __float_as_int(fmaf(__int_as_float(y), inv_m, cq));      // bits of 1.5 2^23 + rint(x/m)
                             b4[i] = (uint32_t)(tq * neg_m + y);                                     // low byte: x - rint(x/m) m
                         }
                         w[q] = __byte_perm(__byte_perm(b4[0], b4[1], 0x0040), __byte_perm(b4[2], b4[3], 0x0040), 0x5410);
                     }
-                    uint4* so = reinterpret_cast<uint4*>(my_out + CPB * kb + 32 * c);
-                    so[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                    so[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    *reinterpret_cast<uint4*>(my_out + CPB * kb + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
                 if (kb == NB - 1) {
                     // The 128 k of this row group are complete for every plane: write them out with the lanes of a warp along
                     // the bytes of a plane (full 128-byte lines, one or two planes per instruction) instead of one plane per lane.
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int run = j * 16 + (t >> 3);                  // plane-major: run = plane * NB + block
+                    for (int j = 0; j < 4; ++j) {
+                        const int run = j * 32 + (t >> 3);                  // plane-major: run = plane * NB + block
                         const int p = run / NB, b = run % NB;
                         const int64_t orow = row0 + NB * rg + b;
                         if (p < tab.nplanes && orow < R) {
@@ -281,13 +282,13 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
                             *reinterpret_cast<uint4*>(planes + (int64_t)p * plane_stride + orow * Kp + k0 + 16 * (t & 7)) = val;
                         }
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
             }
         }
-    } else if (warp < 8) {
+    } else if (warp < 12) {
         // ------------------------------------------------------------------ quantise: thread-private ring of raw elements
-        const int pt = t - 128;                                  // 0..127
+        const int pt = t - 256;                                  // 0..127
         // element of this thread within a step: block (= operand row within the step) and k within the block.
         // Consecutive threads take consecutive k when k is contiguous in memory, consecutive rows otherwise.
         const int el_block = k_contiguous ? pt / CPB : pt % NB;
@@ -346,7 +347,8 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
                 *reinterpret_cast<uint4*>(my_digits + buf * DIGIT_BYTES) = dr;
                 *reinterpret_cast<uint4*>(my_digits + buf * DIGIT_BYTES + 128) = di;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(bar_dfull + 8 * buf);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dfull + 8 * buf);      // one arrival per warp: 128 arrivals on one barrier serialise
             }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -371,7 +373,7 @@ residues_tc_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool 
 
     tcgen05_fence_before();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == 12) {
         __syncwarp();
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
