@@ -86,7 +86,8 @@ def main():
     b.set_profiling(False)
     b.device_status()
     total, per = b.last_launch_count()
-    gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod}.get(a.op, 2 * nmod)
+    planes = 2 * min(nmod, 22) + 3 * max(nmod - 22, 0)       # complex GEMM: 2 real GEMMs per 2M modulus, 3 per 3M modulus
+    gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod}.get(a.op, planes)
     kin = (k + 1) // 2 if a.op in ("dsyrk", "dsyr2k") else k
     print(json.dumps({"op": a.op, "m": m, "n": n, "k": k, "nmod": nmod, "ms_per_call": ms, "effective_tflops": flops / ms / 1e9,
                       "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3],

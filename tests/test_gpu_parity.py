@@ -160,6 +160,26 @@ def test_zgemm_hybrid_every_stage_against_staged_oracle(shape, nmod, phi, kernel
         assert err <= 1.01 * direct.componentwise_error(ref["C"], Cref, D)      # the staged oracle shares
 
 
+def test_hybrid_k_split_with_the_even_modulus():
+    """k 128^2 > 2^31 once the modulus 256 is in use: the split point moves to 130 944 and the second K chunk is added to
+    the stored residues in the epilogue, for the 3M planes and the even modulus too.  Rows whose quantised entries are
+    all +-2^j make every residue of 256 equal to 0 or -128 (the corner of its range) where the digit weight allows."""
+    m, n, k, nmod = 24, 40, 131072 + 300, 23
+    A, B = inputs.complex_inputs(m, n, k, seed=61, dist="phi", phi=1.5)
+    A[3, :] = (2.0 ** 40) * (1 + 1j)                   # constant rows / columns: quantise to the same integer everywhere
+    B[:, 5] = -(2.0 ** -17) * (1 - 1j)
+    ref = staged.zgemm2m_staged(A, B, nmod)
+    for kernel in (1, 0):
+        C, st = run_z(A, B, nmod, kernel)
+        for j3 in range(nmod - 22):
+            for part in range(3):
+                assert (st["C3"][part, j3, :, :m] == ref["Cpm"][22 + j3][part].T).all(), ("C3", part, j3, kernel)
+        for j in (0, 21):
+            for sgn in range(2):
+                assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j, kernel)
+        assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
+
+
 def test_hybrid_beats_the_2m_set_on_a_wide_exponent_span_and_cgemm_accepts_it():
     m, n, k = 48, 40, 160
     A, B = inputs.complex_inputs(m, n, k, seed=23, dist="phi", phi=6.0)    # all 22 2M moduli fall short of double precision here
