@@ -20,6 +20,9 @@
  *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  zgemm2m and cgemm2m
  *     additionally use one library-owned stream, forked from and joined back into `stream` with events: work enqueued
  *     on `stream` after the call still sees the finished result.
+ *   - Because a call only enqueues (kernels, memsets, event records and waits), it can be captured into a CUDA graph
+ *     and replayed; the library-owned stream joins the capture through its fork/join events.  Make one call outside any
+ *     capture first: it creates that stream and its events.  (gemm2m_set_profiling must be off during a capture.)
  *   - Argument errors are detected on the host before anything is launched.  m, n or k equal to 0 is valid:
  *     nothing is computed for m = 0 or n = 0, and C is set to zero for k = 0.
  *   - `nmod` selects the first nmod moduli of the set of Section 4 (241, 233, 229, 221, 205, ... , 37, 29; 22 in
