@@ -251,7 +251,7 @@ def run_ours(a):
         step()
     serial, _ = b.phase_ms()
     b.set_profiling(False)
-    b.debug_set_panels(4)
+    b.debug_set_panels(8)
     b.device_status()
 
     # ---- end to end: every step copies its inputs from pinned host memory, calls the library and reads C back.

@@ -194,7 +194,7 @@ int gemm2m_debug_set_gemm_kernel(int which);
  * (the digit-weight contraction of Eq. (2a) as an int8 MMA with the planes along the TMEM lanes; same planes, bit for
  * bit; measured slower than the default and kept as a selectable variant). */
 int gemm2m_debug_set_residue_kernel(int which);
-/* Largest number of column panels zgemm2m/cgemm2m cut C into (default 4).  With 1 the phases run strictly one after the
+/* Largest number of column panels zgemm2m/cgemm2m cut C into (default 8; panels are about 1024 to 2048 columns wide).  With 1 the phases run strictly one after the
  * other on the caller's stream, which is what per-phase bandwidth figures should be measured with. */
 int gemm2m_debug_set_panels(int max_panels);
 

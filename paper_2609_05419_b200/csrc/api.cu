@@ -26,7 +26,7 @@ struct State {
     cudaStream_t side = nullptr;  // library-owned stream on which the post-processing of a column panel overlaps the next panel's GEMMs
     cudaEvent_t panel_done[kMaxPanels] = {};
     cudaEvent_t side_done = nullptr;
-    int max_panels = 4;           // column panels per zgemm2m/cgemm2m call (1 = no overlap)
+    int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
     int residue_kernel = 0;       // 0 = dp4a residue kernel, 1 = tensor-core residue kernel (measured slower; kept selectable)
@@ -225,7 +225,10 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
     build_mod_table(nmod, true, &ga.mods);
     ga.dev_status = dev_status;
+    // panels of about 1024 columns up to four of them, then of 2048 columns (more, narrower panels also keep the operand
+    // slices of a launch inside the L2: 16384 columns in 8 panels measured 6-8 % faster than in 4)
     int panels = (int)(n / 1024);
+    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
     panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
     const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
     if (panels > 1) { if (int s = ensure_side_stream()) return s; }

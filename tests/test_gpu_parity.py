@@ -19,9 +19,11 @@ TOL_C = 2e-6       # complex64
 def _default_kernel():
     b.debug_set_gemm_kernel(0)
     b.debug_set_residue_kernel(0)
+    b.debug_set_panels(8)
     yield
     b.debug_set_gemm_kernel(0)
     b.debug_set_residue_kernel(0)
+    b.debug_set_panels(8)
 
 
 def run_int(Ar, Ai, Br, Bi, nmod, kernel=0, ldc=None):
@@ -366,11 +368,30 @@ def test_panel_pipeline_is_bitwise_identical_and_joins_the_callers_stream():
             side.synchronize()
             b.device_status(side)
             outs.append((to_host(C), to_host(snap)))
-        b.debug_set_panels(4)
+        b.debug_set_panels(8)
     ref = staged.zgemm2m_staged(A, B, 16)["C"]
     for C, snap in outs:
         assert (C == outs[0][0]).all() and (snap == C).all()
     assert ulp_distance(outs[0][0].real, ref.real).max() <= 1 and ulp_distance(outs[0][0].imag, ref.imag).max() <= 1
+
+
+def test_wide_c_in_more_than_four_panels():
+    m, n, k = 70, 10368, 128                      # 10368 columns -> 5 panels of 2304 / 2048 / ... / 1152 columns
+    A, B = inputs.complex_inputs(m, n, k, seed=19)
+    dA, dB = to_dev(A), to_dev(B)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, 16)):
+        outs = []
+        for panels in (8, 1):
+            b.debug_set_panels(panels)
+            C = empty_dev(m, n, torch.complex128, fill=7.0)
+            b.zgemm2m(dA, dB, C, 16)
+            b.device_status()
+            outs.append(to_host(C))
+            if panels == 8:
+                assert b.last_launch_count()[1][2] == 5          # one GEMM launch per panel
+    assert (outs[0] == outs[1]).all()
+    Cref, D = direct.zgemm4m_dd(A, B)
+    assert direct.componentwise_error(outs[0], Cref, D) <= TOL_Z
 
 
 def test_back_to_back_calls_of_different_sizes_share_a_workspace():
