@@ -188,6 +188,44 @@ def scaling_exponents(Z, axis: int, P: int, ck: int):
     return np.where(mu > 0, e, 0).astype(np.int64)
 
 
+TIGHT_FRAC_BITS = 20      # resolution of the fixed-point magnitudes of the 2-norm scaling rule
+
+
+def scaling_exponents_2norm(Z, axis: int, P: int):
+    """The tighter choice of sigma / tau the paper points to the literature for (Algorithm 1 step 2): bound the row's
+    2-norm itself instead of sqrt(2k) times its largest part.  All-integer so that it is reproducible bit for bit:
+    with mu, x as in `scaling_exponents`, every part v of the row is rounded UP to the fixed-point magnitude
+    u = ceil(|v| 2^(20 - (x+1))) (an integer <= 2^20), Q = sum u^2 over the 2k parts, t = the smallest integer with
+    4^t >= Q, and e = x + 1 - P + (t - 20).  Then |v| <= u 2^(x+1-20), so the row's 2-norm is at most
+    2^(x+1-20) sqrt(Q) <= 2^(x+1-20+t) = 2^(P+e): the scaled row has 2-norm <= 2^P, which is all the overflow proof needs.
+    The largest part has u >= 2^19, so t >= 19; and Q <= 2k 4^20, so t - 20 <= c_k: the exponent is never above the
+    max-based rule's."""
+    from fractions import Fraction
+    Z = np.asarray(Z)
+    if axis == 0:
+        Z = Z.T
+    rows = Z.shape[0]
+    e = np.zeros(rows, dtype=np.int64)
+    for i in range(rows):
+        parts = np.concatenate([np.abs(Z[i].real), np.abs(Z[i].imag)]).astype(np.float64)
+        mu = parts.max(initial=0.0)
+        if not mu > 0:
+            continue
+        x = int(np.frexp(mu)[1]) - 1
+        scale = Fraction(2) ** (TIGHT_FRAC_BITS - (x + 1))
+        Q = 0
+        for v in parts:
+            if v != 0:
+                f = Fraction(float(v)) * scale
+                u = -((-f.numerator) // f.denominator)          # ceil
+                Q += u * u
+        t = 0
+        while 4 ** t < Q:
+            t += 1
+        e[i] = x + 1 - P + (t - TIGHT_FRAC_BITS)
+    return e
+
+
 def _quantise_part(x, e):
     """trunc(x 2^-e) exactly, elementwise; x float array, e broadcastable integer array.  Object array of ints."""
     x = np.asarray(x, dtype=np.float64)
@@ -298,9 +336,10 @@ def gemm2m_int_staged(Ar, Ai, Br, Bi, nmod: int):
     return dict(moduli=moduli, roots=roots, M=M, Apm=Apl, Bpm=Bpl, Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi)
 
 
-def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto: str = "all"):
+def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto: str = "all", scaling: str = "max"):
     """Algorithm 1 on floating-point A (m x k), B (k x n).  For herk=True pass B = A^H.
-    upto = "pre" stops after the residue planes (cheap at large sizes)."""
+    upto = "pre" stops after the residue planes (cheap at large sizes).  scaling = "max" (largest part times sqrt(2k))
+    or "2norm" (`scaling_exponents_2norm`)."""
     A = np.asarray(A)
     B = np.asarray(B)
     k = A.shape[1]
@@ -308,8 +347,12 @@ def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto
     roots = roots_of(moduli)
     M = product(moduli)
     Pt, PA, PB, ck = scaling_targets(M, k, herk)
-    eA = scaling_exponents(A, 1, PA, ck)                           # step 2
-    eB = scaling_exponents(B, 0, PB, ck)
+    if scaling == "2norm":
+        eA = scaling_exponents_2norm(A, 1, PA)                     # step 2
+        eB = scaling_exponents_2norm(B, 0, PB)
+    else:
+        eA = scaling_exponents(A, 1, PA, ck)
+        eB = scaling_exponents(B, 0, PB, ck)
     Aq = quantise(A, eA, 1)                                        # step 3
     Bq = quantise(B, eB, 0)
     Apl = _residue_planes(Aq[0], Aq[1], moduli, roots)             # step 4: (2a), or the 3M sums

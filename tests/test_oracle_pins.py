@@ -476,3 +476,39 @@ def test_extended_definition_vs_exact_rationals_and_special_cases():
     assert (direct.zgemm_ex_dd("N", "N", 1, A, B, 0, nanC)[0] == P).all()              # beta = 0: C0 not referenced
     assert (direct.zgemm_ex_dd("N", "N", 0, A * np.nan, B, 2, C0)[0] == 2 * C0).all()   # alpha = 0: A, B not referenced
     assert (direct.zgemm_ex_dd("T", "T", 1, A.T.copy(), B.T.copy(), 0, None)[0] == P).all()        # stored transposed
+
+
+# ------------------------------------------------------------------ 2-norm scaling rule
+def test_2norm_scaling_keeps_the_overflow_bound_and_is_never_looser():
+    A, B = inputs.complex_inputs(19, 11, 700, seed=12, dist="phi", phi=1.5)
+    A[4, :] = 0
+    A[7, :] = 0
+    A[7, 13] = 3.0 - 4.0j                       # a single entry: the 2-norm is 5, the max-based rule budgets sqrt(2k) 4
+    for nmod in (7, 16, 22, 25):
+        st_max = staged.zgemm2m_staged(A, B, nmod, upto="pre")
+        st = staged.zgemm2m_staged(A, B, nmod, upto="pre", scaling="2norm")
+        assert st["eA"][4] == 0
+        assert (st["eA"] <= st_max["eA"]).all() and (st["eB"] <= st_max["eB"]).all()
+        assert (st_max["eA"] - st["eA"]).max() <= st["ck"] + 1
+        assert st_max["eA"][7] - st["eA"][7] >= st["ck"] - 2          # nearly the whole sqrt(2k) factor comes back
+        for (qr, qi), axis, P in ((st["Aq"], 1, st["PA"]), (st["Bq"], 0, st["PB"])):
+            sq = (qr.astype(object) ** 2 + qi.astype(object) ** 2).sum(axis=axis)
+            assert all(int(v) <= 4 ** P for v in sq)                  # what Cauchy-Schwarz needs
+            # and tight: one more bit would break the bound for at least one row (the rule wastes < 2 bits: ceil to a
+            # power of 4 and the 2^-20 rounding up)
+            assert any(16 * int(v) > 4 ** P for v in sq if v)
+
+
+def test_2norm_scaling_gains_accuracy_and_equals_the_integer_product():
+    A, B = inputs.complex_inputs(12, 9, 2048, seed=9, dist="phi", phi=0.5)
+    Cref, D = direct.zgemm4m_dd(A, B)
+    err = {}
+    for scaling in ("max", "2norm"):
+        st = staged.zgemm2m_staged(A, B, 14, scaling=scaling)
+        assert all(abs(int(v)) <= 2 ** st["Pt"] for v in np.concatenate([st["Xr"].ravel(), st["Xi"].ravel()]))
+        pairs = np.array([(i, j) for i in range(12) for j in range(9)])
+        Xs, _ = staged.staged_samples(st, pairs)                      # no wrap-around: equals the plain integer product
+        assert all(int(st["Xr"][i, j]) == xr and int(st["Xi"][i, j]) == xi for (i, j), (xr, xi) in zip(pairs.tolist(), Xs))
+        err[scaling] = direct.componentwise_error(st["C"], Cref, D)
+    assert err["2norm"] * 4 <= err["max"]          # k = 2048: c_k = 6; about three bits per operand come back, and the error is
+    # proportional to 2^e of each operand (truncation of one factor times the other factor), not to their product
