@@ -113,6 +113,17 @@ int zgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const 
 int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const float* alpha, const float* A, int64_t lda,
                const float* B, int64_t ldb, const float* beta, float* C, int64_t ldc, int nmod, void* stream);
 
+/* Choice of the scale factors sigma_i, tau_j of zgemm2m / cgemm2m and their _ex forms (Algorithm 1 step 2; the paper
+ * leaves it to the literature).  Both choices are powers of two that make the 2-norm of every scaled row of A at most
+ * 2^P_A and of every scaled column of B at most 2^P_B, P_A + P_B = floor(log2((M-1)/2)), which by Cauchy-Schwarz keeps every
+ * entry of the integer product inside the range the CRT can represent.
+ *   0 (default): from the largest |Re| or |Im| of the row, times sqrt(2k): one pass over the operands;
+ *   1: from an upper bound of the row's 2-norm itself (sum of the squares of the parts, each rounded up to 20 fractional
+ *      bits below the largest one's binade, in 64-bit integers): a second pass over A and B, and in return 3 to 6 more
+ *      bits of each operand survive the truncation, about what one more modulus buys.  Falls back to 0 for k > 2^22.
+ * Process-wide; takes effect with the next call.  The rank-k family always uses 0. */
+int gemm2m_set_scaling(int mode);
+
 /* Hermitian rank-k update C = A A^H (Section 5, HERK) with ONE real int8 GEMM per modulus: C+ = A+ A-^T and
  * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
  * diagonal is written; diagonal imaginary parts are exactly 0; the strict upper triangle is not touched. */

@@ -69,6 +69,7 @@ def lib():
     L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
     L.gemm2m_debug_set_panels.argtypes = [i32]
+    L.gemm2m_set_scaling.argtypes = [i32]
     L.gemm2m_debug_set_residue_kernel.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
     L.gemm2m_debug_residue_reduction.argtypes = [i32, vp, vp, vp, vp, vp]
@@ -263,6 +264,11 @@ def last_launch_count():
 
 def debug_set_gemm_kernel(which):
     _check(lib().gemm2m_debug_set_gemm_kernel(which), "gemm2m_debug_set_gemm_kernel")
+
+
+def set_scaling(mode):
+    """0 = scale factors from the largest part of each row / column (default), 1 = from a bound of its 2-norm."""
+    _check(lib().gemm2m_set_scaling(int(mode)), "gemm2m_set_scaling")
 
 
 def debug_set_residue_kernel(which):

@@ -29,6 +29,7 @@ struct State {
     int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
+    int scaling = 0;              // 0 = largest part times sqrt(2k), 1 = 2-norm rule (zgemm2m / cgemm2m)
     int residue_kernel = 0;       // 0 = dp4a residue kernel, 1 = tensor-core residue kernel (measured slower; kept selectable)
     int sm_count = 0;
     int arch_ok = -1;
@@ -59,9 +60,10 @@ int check_device() {
     return g.arch_ok ? GEMM2M_OK : GEMM2M_ERR_ARCH;
 }
 
-// Workspace: [status 256 B][absmax A u64][absmax B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each 256-byte aligned.
+// Workspace: [status 256 B][absmax A u64][absmax B u64][sumsq A u64][sumsq B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each
+// 256-byte aligned.
 struct Carve {
-    int64_t off_status, off_abs_a, off_abs_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
+    int64_t off_status, off_abs_a, off_abs_b, off_q_a, off_q_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
 };
 
 bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
@@ -79,6 +81,8 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_status = take(256);
     c->off_abs_a = take(8 * m);
     c->off_abs_b = take(herk ? 0 : 8 * n);
+    c->off_q_a = take(herk ? 0 : 8 * m);        // sums of squares of the 2-norm scaling rule (zeroed together with the maxima)
+    c->off_q_b = take(herk ? 0 : 8 * n);
     c->off_exp_a = take(4 * m);
     c->off_exp_b = take(herk ? 0 : 4 * n);
     c->off_pack_a = take(real_in ? 16 * n * k : 0);
@@ -192,7 +196,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     build_residue_table(nmod, &rtab);
     CrtTable ctab;
     build_crt_table(nmod, &ctab);
-    const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
+    // quantised parts stay below 2^(P - c_k) with the max-based rule and below 2^P with the 2-norm rule
+    const bool two_norm_mode = g.scaling == 1 && k <= (1ll << 22);
+    const bool wideA = two_norm_mode ? sc.PA > 61 : sc.PA - sc.ck > 62, wideB = two_norm_mode ? sc.PB > 61 : sc.PB - sc.ck > 62;
 
     Phases ph;
     if (int s = begin_call(&ph)) return s;
@@ -204,8 +210,17 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0]));
     if (tb == 'N') CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
     else CK(launch_scan_rows<T>(B, n, k, ldb, absB, st, &g.launches[0]));
-    CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
-    CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
+    if (!two_norm_mode) {                                          // (k > 2^22: the sums of 2k squares below 2^40 would not fit 64 bits)
+        CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
+        CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
+    } else {
+        uint64_t* qA = (uint64_t*)(ws + c.off_q_a);
+        uint64_t* qB = (uint64_t*)(ws + c.off_q_b);
+        if (ta == 'N') CK(launch_exponents_2norm<T>(A, m, k, lda, true, absA, qA, sc.PA, eA, st, &g.launches[0]));
+        else CK(launch_exponents_2norm<T>(A, k, m, lda, false, absA, qA, sc.PA, eA, st, &g.launches[0]));
+        if (tb == 'N') CK(launch_exponents_2norm<T>(B, k, n, ldb, false, absB, qB, sc.PB, eB, st, &g.launches[0]));
+        else CK(launch_exponents_2norm<T>(B, n, k, ldb, true, absB, qB, sc.PB, eB, st, &g.launches[0]));
+    }
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
@@ -564,6 +579,13 @@ int gemm2m_debug_set_gemm_kernel(int which) {
     std::lock_guard<std::mutex> lock(g.mu);
     if (which < 0 || which > 2) return GEMM2M_ERR_ARG;
     g.gemm_kernel = which;
+    return GEMM2M_OK;
+}
+
+int gemm2m_set_scaling(int mode) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (mode < 0 || mode > 1) return GEMM2M_ERR_ARG;
+    g.scaling = mode;
     return GEMM2M_OK;
 }
 

@@ -95,6 +95,10 @@ template <typename T> cudaError_t launch_scan_rows(const T* X, int64_t rows, int
 // The same per column.
 template <typename T> cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches);
 template <typename T> cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int ck, int32_t* e, cudaStream_t st, int* launches);
+// 2-norm scaling rule: second pass over X (rows x cols, ld) summing the squared fixed-point magnitudes per row (per_row) or
+// per column into qsum (zeroed by the caller), then e = x + 1 - P + ceil(log4 Q) - 20 with x from absmax.
+template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t rows, int64_t cols, int64_t ld, bool per_row, const uint64_t* absmax,
+                                                         uint64_t* qsum, int P, int32_t* e, cudaStream_t st, int* launches);
 // Quantise + residues.  k_contiguous = false: operand row r is row r of the column-major matrix X (A: m x k);
 // true: operand row r is column r of X (B: k x n).
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
