@@ -202,29 +202,39 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
 
     Phases ph;
     if (int s = begin_call(&ph)) return s;
-    // step 2: scale factors
-    CK(ph.begin(0, st));
+    // step 2: scale factors.  The scan of B (bandwidth-bound) runs on the library's side stream beside the scan and the
+    // residues of A (which are bound by arithmetic); the residues of B wait for it.  (With the panel overlap switched off
+    // everything stays on the caller's stream, one phase after the other.)
+    if (int s = ensure_side_stream()) return s;
+    cudaStream_t sb = g.max_panels > 1 ? g.side : st;
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
-    // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C'); columns of op(B) are columns of B or its rows
+    if (sb != st) {
+        CK(cudaEventRecord(g.panel_done[0], st));
+        CK(cudaStreamWaitEvent(sb, g.panel_done[0], 0));
+    }
+    uint64_t* qA = (uint64_t*)(ws + c.off_q_a);
+    uint64_t* qB = (uint64_t*)(ws + c.off_q_b);
+    CK(ph.begin(0, sb));
+    // columns of op(B) are columns of B as stored ('N') or its rows ('T', 'C')
+    if (tb == 'N') CK(launch_scan_cols<T>(B, k, n, ldb, absB, sb, &g.launches[0]));
+    else CK(launch_scan_rows<T>(B, n, k, ldb, absB, sb, &g.launches[0]));
+    if (!two_norm_mode) CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, sb, &g.launches[0]));
+    else if (tb == 'N') CK(launch_exponents_2norm<T>(B, k, n, ldb, false, absB, qB, sc.PB, eB, sb, &g.launches[0]));
+    else CK(launch_exponents_2norm<T>(B, n, k, ldb, true, absB, qB, sc.PB, eB, sb, &g.launches[0]));
+    CK(ph.end(sb));
+    if (sb != st) CK(cudaEventRecord(g.side_done, sb));
+    CK(ph.begin(0, st));
+    // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C')
     if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
     else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0]));
-    if (tb == 'N') CK(launch_scan_cols<T>(B, k, n, ldb, absB, st, &g.launches[0]));
-    else CK(launch_scan_rows<T>(B, n, k, ldb, absB, st, &g.launches[0]));
-    if (!two_norm_mode) {                                          // (k > 2^22: the sums of 2k squares below 2^40 would not fit 64 bits)
-        CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
-        CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
-    } else {
-        uint64_t* qA = (uint64_t*)(ws + c.off_q_a);
-        uint64_t* qB = (uint64_t*)(ws + c.off_q_b);
-        if (ta == 'N') CK(launch_exponents_2norm<T>(A, m, k, lda, true, absA, qA, sc.PA, eA, st, &g.launches[0]));
-        else CK(launch_exponents_2norm<T>(A, k, m, lda, false, absA, qA, sc.PA, eA, st, &g.launches[0]));
-        if (tb == 'N') CK(launch_exponents_2norm<T>(B, k, n, ldb, false, absB, qB, sc.PB, eB, st, &g.launches[0]));
-        else CK(launch_exponents_2norm<T>(B, n, k, ldb, true, absB, qB, sc.PB, eB, st, &g.launches[0]));
-    }
+    if (!two_norm_mode) CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));     // (2-norm rule: not for k > 2^22,
+    else if (ta == 'N') CK(launch_exponents_2norm<T>(A, m, k, lda, true, absA, qA, sc.PA, eA, st, &g.launches[0]));   // where the sums
+    else CK(launch_exponents_2norm<T>(A, k, m, lda, false, absA, qA, sc.PA, eA, st, &g.launches[0]));   // of squares would not fit 64 bits)
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
     if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
+    if (sb != st) CK(cudaStreamWaitEvent(st, g.side_done, 0));
     if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
@@ -246,7 +256,6 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
     panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
     const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
-    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
     for (int pnl = 0; pnl < panels; ++pnl) {
         const int64_t j0 = pnl * panel_cols, j1 = (j0 + panel_cols < n) ? j0 + panel_cols : n;
         if (j0 >= j1) break;
