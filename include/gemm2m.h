@@ -78,8 +78,9 @@ int gemm2m_modulus(int j, int* m, int* s);
 
 /* Bytes of device workspace a call of `op` with these sizes needs (for the rank-k family pass m = n).  0 on bad arguments. */
 size_t gemm2m_workspace_bytes(int op, int64_t m, int64_t n, int64_t k, int nmod);
-/* Register a caller-owned device buffer (256-byte aligned) used by later calls of this host thread's current
- * device.  Passing (NULL, 0) unregisters.  The buffer must stay valid until the last call using it has finished. */
+/* Register a caller-owned device buffer (256-byte aligned) of the CURRENT device; later calls made while that device is
+ * current use it (one workspace per device; the library's side stream and events are per device too).  Passing (NULL, 0)
+ * unregisters.  The buffer must stay valid until the last call using it has finished. */
 int gemm2m_set_workspace(void* dev_ptr, size_t bytes);
 
 /* Gaussian-integer product by 2M multiplication (Section 2, Eq. (2a)-(2c)) and CRT over nmod <= 8 moduli.

@@ -12,29 +12,38 @@ using namespace gemm2m;
 
 namespace {
 
-struct State {
-    std::mutex mu;
+// Per-device part of the library state: the registered workspace, the side stream with its ordering events, and what was
+// learnt about the device.
+struct DevState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
+    cudaStream_t side = nullptr;  // library-owned stream on which the post-processing of a column panel overlaps the next panel's GEMMs
+    cudaEvent_t panel_done[8] = {};
+    cudaEvent_t side_done = nullptr;
+    int sm_count = 0;
+    int arch_ok = -1;
+};
+
+struct State {
+    std::mutex mu;
+    static constexpr int kMaxDevices = 64;
+    DevState dev[kMaxDevices];
+    int cur = 0;                  // device of the call being served (set by use_current_device)
     int profiling = 0;
     static constexpr int kProfSlots = 64, kMaxIntervals = 24, kMaxPanels = 8;
     struct Interval { cudaEvent_t a = nullptr, b = nullptr; int phase = 0; };
     struct Slot { Interval iv[kMaxIntervals]; int n = 0; };
     Slot slots[kProfSlots];       // timed intervals (phase, start, end) of the profiled calls
     int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
-    Slot* cur = nullptr;          // slot of the call being enqueued
-    cudaStream_t side = nullptr;  // library-owned stream on which the post-processing of a column panel overlaps the next panel's GEMMs
-    cudaEvent_t panel_done[kMaxPanels] = {};
-    cudaEvent_t side_done = nullptr;
+    Slot* cur_slot = nullptr;     // slot of the call being enqueued
     int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
     int scaling = 0;              // 0 = largest part times sqrt(2k), 1 = 2-norm rule (zgemm2m / cgemm2m)
     int residue_kernel = 0;       // 0 = dp4a residue kernel, 1 = tensor-core residue kernel (measured slower; kept selectable)
-    int sm_count = 0;
-    int arch_ok = -1;
 };
 State g;
+DevState& D() { return g.dev[g.cur]; }
 thread_local char g_cuda_err[256] = "no error";
 
 int cuda_fail(cudaError_t e) {
@@ -49,15 +58,24 @@ int cuda_fail(cudaError_t e) {
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
+// Points D() at the state of the calling thread's current device (the caller holds g.mu).
+void select_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < State::kMaxDevices) g.cur = dev;
+}
+
+// The same, and checks the device's architecture once.
 int check_device() {
-    if (g.arch_ok < 0) {
-        int dev = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= State::kMaxDevices) return GEMM2M_ERR_CUDA;
+    g.cur = dev;
+    if (D().arch_ok < 0) {
         cudaDeviceProp prop;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return GEMM2M_ERR_CUDA;
-        g.arch_ok = (prop.major == 10 && prop.minor == 0) ? 1 : 0;
-        g.sm_count = prop.multiProcessorCount;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return GEMM2M_ERR_CUDA;
+        D().arch_ok = (prop.major == 10 && prop.minor == 0) ? 1 : 0;
+        D().sm_count = prop.multiProcessorCount;
     }
-    return g.arch_ok ? GEMM2M_OK : GEMM2M_ERR_ARCH;
+    return D().arch_ok ? GEMM2M_OK : GEMM2M_ERR_ARCH;
 }
 
 // Workspace: [status 256 B][absmax A u64][absmax B u64][sumsq A u64][sumsq B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each
@@ -100,16 +118,16 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
 struct Phases {   // event bookkeeping of one call: every phase is a set of intervals, each on the stream its kernels run on
     bool on = false;
     cudaError_t begin(int phase, cudaStream_t st) {
-        if (!on || g.cur->n >= State::kMaxIntervals) return cudaSuccess;
-        State::Interval& iv = g.cur->iv[g.cur->n];
+        if (!on || g.cur_slot->n >= State::kMaxIntervals) return cudaSuccess;
+        State::Interval& iv = g.cur_slot->iv[g.cur_slot->n];
         iv.phase = phase;
         if (!iv.a) { cudaError_t e = cudaEventCreate(&iv.a); if (e != cudaSuccess) return e; }
         if (!iv.b) { cudaError_t e = cudaEventCreate(&iv.b); if (e != cudaSuccess) return e; }
         return cudaEventRecord(iv.a, st);
     }
     cudaError_t end(cudaStream_t st) {
-        if (!on || g.cur->n >= State::kMaxIntervals) return cudaSuccess;
-        return cudaEventRecord(g.cur->iv[g.cur->n++].b, st);
+        if (!on || g.cur_slot->n >= State::kMaxIntervals) return cudaSuccess;
+        return cudaEventRecord(g.cur_slot->iv[g.cur_slot->n++].b, st);
     }
     void done() { if (on) ++g.prof_calls; }
 };
@@ -118,18 +136,18 @@ int begin_call(Phases* ph) {
     ph->on = g.profiling != 0;
     std::memset(g.launches, 0, sizeof(g.launches));
     if (ph->on) {
-        g.cur = &g.slots[g.prof_calls % State::kProfSlots];
-        g.cur->n = 0;
+        g.cur_slot = &g.slots[g.prof_calls % State::kProfSlots];
+        g.cur_slot->n = 0;
     }
     return GEMM2M_OK;
 }
 
 // Side stream and ordering events, created on first use (no device memory involved).
 int ensure_side_stream() {
-    if (!g.side) CK(cudaStreamCreateWithFlags(&g.side, cudaStreamNonBlocking));
-    for (auto& e : g.panel_done)
+    if (!D().side) CK(cudaStreamCreateWithFlags(&D().side, cudaStreamNonBlocking));
+    for (auto& e : D().panel_done)
         if (!e) CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-    if (!g.side_done) CK(cudaEventCreateWithFlags(&g.side_done, cudaEventDisableTiming));
+    if (!D().side_done) CK(cudaEventCreateWithFlags(&D().side_done, cudaEventDisableTiming));
     return GEMM2M_OK;
 }
 
@@ -139,15 +157,15 @@ template <typename T>
 int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
                  const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st) {
     if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
-    else CK(launch_residues_tc<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, dev_status, g.sm_count, st, &g.launches[1]));
+    else CK(launch_residues_tc<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, dev_status, D().sm_count, st, &g.launches[1]));
     return GEMM2M_OK;
 }
 
 int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
     const int64_t klim = gemm_k_limit(nmod);
     if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
-    else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(a, klim, g.sm_count, st, &g.launches[2]));
-    else CK(launch_gemm_tcgen05_pair(a, klim, g.sm_count, st, &g.launches[2]));
+    else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(a, klim, D().sm_count, st, &g.launches[2]));
+    else CK(launch_gemm_tcgen05_pair(a, klim, D().sm_count, st, &g.launches[2]));
     return GEMM2M_OK;
 }
 
@@ -180,8 +198,8 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     }
     Carve c;
     if (!carve(op, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
-    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
-    char* ws = (char*)g.ws;
+    if (!D().ws || D().ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)D().ws;
     int* dev_status = (int*)(ws + c.off_status);
     uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
     uint64_t* absB = (uint64_t*)(ws + c.off_abs_b);
@@ -206,11 +224,11 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // residues of A (which are bound by arithmetic); the residues of B wait for it.  (With the panel overlap switched off
     // everything stays on the caller's stream, one phase after the other.)
     if (int s = ensure_side_stream()) return s;
-    cudaStream_t sb = g.max_panels > 1 ? g.side : st;
+    cudaStream_t sb = g.max_panels > 1 ? D().side : st;
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
     if (sb != st) {
-        CK(cudaEventRecord(g.panel_done[0], st));
-        CK(cudaStreamWaitEvent(sb, g.panel_done[0], 0));
+        CK(cudaEventRecord(D().panel_done[0], st));
+        CK(cudaStreamWaitEvent(sb, D().panel_done[0], 0));
     }
     uint64_t* qA = (uint64_t*)(ws + c.off_q_a);
     uint64_t* qB = (uint64_t*)(ws + c.off_q_b);
@@ -222,7 +240,7 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     else if (tb == 'N') CK(launch_exponents_2norm<T>(B, k, n, ldb, false, absB, qB, sc.PB, eB, sb, &g.launches[0]));
     else CK(launch_exponents_2norm<T>(B, n, k, ldb, true, absB, qB, sc.PB, eB, sb, &g.launches[0]));
     CK(ph.end(sb));
-    if (sb != st) CK(cudaEventRecord(g.side_done, sb));
+    if (sb != st) CK(cudaEventRecord(D().side_done, sb));
     CK(ph.begin(0, st));
     // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C')
     if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
@@ -234,7 +252,7 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
     if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
-    if (sb != st) CK(cudaStreamWaitEvent(st, g.side_done, 0));
+    if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
     if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
@@ -265,18 +283,18 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
         if (int s = run_gemm(ga, nmod, st)) return s;
         CK(ph.end(st));
         const bool last = j1 >= n;
-        cudaStream_t ps = last ? st : g.side;
+        cudaStream_t ps = last ? st : D().side;
         if (!last) {
-            CK(cudaEventRecord(g.panel_done[pnl], st));
-            CK(cudaStreamWaitEvent(g.side, g.panel_done[pnl], 0));
+            CK(cudaEventRecord(D().panel_done[pnl], st));
+            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
         }
         CK(ph.begin(3, ps));
         CK(launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]));
         CK(ph.end(ps));
     }
     if (panels > 1) {   // join: the call is complete on the caller's stream only when the side stream has finished
-        CK(cudaEventRecord(g.side_done, g.side));
-        CK(cudaStreamWaitEvent(st, g.side_done, 0));
+        CK(cudaEventRecord(D().side_done, D().side));
+        CK(cudaStreamWaitEvent(st, D().side_done, 0));
     }
     ph.done();
     return GEMM2M_OK;
@@ -337,8 +355,9 @@ int gemm2m_set_workspace(void* dev_ptr, size_t bytes) {
     std::lock_guard<std::mutex> lock(g.mu);
     if ((dev_ptr == nullptr) != (bytes == 0)) return GEMM2M_ERR_ARG;
     if (((uintptr_t)dev_ptr & 255) != 0) return GEMM2M_ERR_ARG;
-    g.ws = dev_ptr;
-    g.ws_bytes = bytes;
+    select_device();
+    D().ws = dev_ptr;
+    D().ws_bytes = bytes;
     if (dev_ptr) CK(cudaMemset(dev_ptr, 0, 256));   // device status word
     return GEMM2M_OK;
 }
@@ -361,8 +380,8 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     }
     Carve c;
     if (!carve(GEMM2M_OP_GAUSSIAN_INT, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
-    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
-    char* ws = (char*)g.ws;
+    if (!D().ws || D().ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)D().ws;
     int8_t* apm = (int8_t*)(ws + c.off_apm);
     int8_t* bpm = (int8_t*)(ws + c.off_bpm);
     int8_t* cpm = (int8_t*)(ws + c.off_cpm);
@@ -423,8 +442,8 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     cudaStream_t st = (cudaStream_t)stream;
     Carve c;
     if (!carve(op, n, n, k > 0 ? k : 1, nmod, &c)) return GEMM2M_ERR_ARG;
-    if (!g.ws || g.ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
-    char* ws = (char*)g.ws;
+    if (!D().ws || D().ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)D().ws;
     uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
     int32_t* eA = (int32_t*)(ws + c.off_exp_a);
     int8_t* apm = (int8_t*)(ws + c.off_apm);
@@ -532,11 +551,12 @@ int dsyr2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B
 int gemm2m_device_status(void* stream) {
     std::lock_guard<std::mutex> lock(g.mu);
     CK(cudaStreamSynchronize((cudaStream_t)stream));
-    if (!g.ws) return GEMM2M_OK;
+    select_device();
+    if (!D().ws) return GEMM2M_OK;
     int code = 0;
-    CK(cudaMemcpy(&code, g.ws, sizeof(int), cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(&code, D().ws, sizeof(int), cudaMemcpyDeviceToHost));
     if (code != kDevOk) {
-        CK(cudaMemset(g.ws, 0, sizeof(int)));
+        CK(cudaMemset(D().ws, 0, sizeof(int)));
         return GEMM2M_ERR_DEVICE_TIMEOUT;
     }
     return GEMM2M_OK;
