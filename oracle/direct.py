@@ -196,6 +196,13 @@ def zher2k_dd(A, B):
     return zgemm4m_dd2(A, B.conj().T, B, A.conj().T)
 
 
+def dgemm_dd(A, B):
+    """Real C = A B with every dot product in double-double, rounded once, and D = |A||B|."""
+    A, B = np.asarray(A, dtype=np.float64), np.asarray(B, dtype=np.float64)
+    C, D = zgemm4m_dd(A.astype(np.complex128), B.astype(np.complex128))
+    return np.asfortranarray(C.real), D
+
+
 def dsyrk_dd(A):
     """Section 5, SYRK: C = A A^T for real A (returned real)."""
     A = np.asarray(A, dtype=np.float64)

@@ -5,6 +5,7 @@ Every function follows one passage of the paper, in its notation, with no blocki
   is_2m_modulus, greedy_2m_moduli   Section 2 (definition of a 2M modulus) and Section 4 (greedy coprime set in [1, 256])
   sqrt_minus_one, inv2              Section 2: s^2 = -1 (mod m); 2^-1 = (m+1)/2
   pre_2m, mul_2m, post_2m           Eq. (2a), (2b), (2c)
+  greedy_real_moduli, dgemm_o2_staged      Section 3.1 (the real Ozaki-II scheme) with the real modulus set of Section 4
   hybrid_moduli, pre_3m, mul_3m, post_3m   Section 3 (hybrid 2M/3M remark) and Section 4 (non-2M moduli once the 2M set is
                                     exhausted); Eq. (1) applied after the reduction modulo m
   crt, lift                         Section 3.1 (CRT formula) and Algorithm 1 steps 5-6
@@ -52,6 +53,15 @@ def greedy_2m_moduli(limit: int = 256):
     kept = []
     for cand in range(limit, 1, -1):
         if is_2m_modulus(cand) and all(math.gcd(cand, q) == 1 for q in kept):
+            kept.append(cand)
+    return kept
+
+
+def greedy_real_moduli(limit: int = 256):
+    """Section 4, the set available to real Ozaki-II GEMMs: the same greedy walk without the 2M condition."""
+    kept = []
+    for cand in range(limit, 1, -1):
+        if all(math.gcd(cand, q) == 1 for q in kept):
             kept.append(cand)
     return kept
 
@@ -366,6 +376,37 @@ def zgemm2m_staged(A, B, nmod: int, herk: bool = False, out_bits: int = 53, upto
     C = unscale(Xr, eA, eB, out_bits) + 1j * unscale(Xi, eA, eB, out_bits)   # step 7
     st.update(Cpm=Cpm, res_r=res_r, res_i=res_i, Xr=Xr, Xi=Xi, C=C)
     return st
+
+
+def scaling_targets_real(M: int, k: int):
+    """Real scheme: a row has k real terms, so c_k = ceil(log2(k)/2); P_t, P_A, P_B as in `scaling_targets`."""
+    Pt = ((M - 1) // 2).bit_length() - 1
+    ck = 0
+    while 4 ** ck < max(k, 1):
+        ck += 1
+    return Pt, -((-Pt) // 2), Pt // 2, ck
+
+
+def dgemm_o2_staged(A, B, nmod: int, out_bits: int = 53):
+    """Section 3.1: the real Ozaki-II scheme C = A B for real A (m x k), B (k x n): scale and truncate, one real integer
+    GEMM per modulus of the real set, CRT, lift, unscale.  The same readings as for Algorithm 1 (power-of-two scale
+    factors from the largest magnitude of a row times sqrt(k), truncation, symmetric residues, single rounding)."""
+    A = np.asarray(A, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    k = A.shape[1]
+    moduli = greedy_real_moduli()[:nmod]
+    M = product(moduli)
+    Pt, PA, PB, ck = scaling_targets_real(M, k)
+    eA = scaling_exponents(A + 0j, 1, PA, ck)
+    eB = scaling_exponents(B + 0j, 0, PB, ck)
+    Aq = _quantise_part(A, eA[:, None])
+    Bq = _quantise_part(B, eB[None, :])
+    Apl = [np.asarray(sym(_small(Aq) % ml, ml)).astype(np.int64) for ml in moduli]
+    Bpl = [np.asarray(sym(_small(Bq) % ml, ml)).astype(np.int64) for ml in moduli]
+    Cpl = [sym(_exact_matmul(a, b_), ml) for a, b_, ml in zip(Apl, Bpl, moduli)]
+    X = lift(crt(Cpl, moduli), M)
+    C = unscale(X, eA, eB, out_bits)
+    return dict(moduli=moduli, M=M, Pt=Pt, PA=PA, PB=PB, ck=ck, eA=eA, eB=eB, Aq=Aq, Bq=Bq, Apl=Apl, Bpl=Bpl, Cpl=Cpl, X=X, C=C)
 
 
 def syrk_complexify(X):

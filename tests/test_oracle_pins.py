@@ -512,3 +512,37 @@ def test_2norm_scaling_gains_accuracy_and_equals_the_integer_product():
         err[scaling] = direct.componentwise_error(st["C"], Cref, D)
     assert err["2norm"] * 4 <= err["max"]          # k = 2048: c_k = 6; about three bits per operand come back, and the error is
     # proportional to 2^e of each operand (truncation of one factor times the other factor), not to their product
+
+
+# ------------------------------------------------------------------ real Ozaki-II scheme (Section 3.1)
+def test_real_scheme_moduli_and_integer_exactness(printed):
+    mods = staged.greedy_real_moduli()
+    assert mods[:10] == printed["mreal_prefix"]
+    assert all(math.gcd(a, c) == 1 for i, a in enumerate(mods) for c in mods[:i])
+    rng = np.random.default_rng(8)
+    # integer-valued inputs whose product fits M/2: the scheme must return the exact product (every step is exact)
+    A = rng.integers(-1000, 1000, size=(7, 33)).astype(np.float64)
+    B = rng.integers(-1000, 1000, size=(33, 5)).astype(np.float64)
+    st = staged.dgemm_o2_staged(A, B, 15)
+    assert (st["C"] == A @ B).all()
+    assert all(abs(int(v)) <= 2 ** st["Pt"] for v in st["X"].ravel())
+    exact = st["Aq"].astype(object).dot(st["Bq"].astype(object))             # no wrap-around: plain integer product
+    assert (st["X"] == exact).all()
+    sq = (st["Aq"].astype(object) ** 2).sum(axis=1)
+    assert all(int(v) <= 4 ** st["PA"] for v in sq)                           # the row 2-norm bound of the scaling rule
+
+
+def test_real_scheme_error_vs_modulus_count():
+    rng = np.random.default_rng(9)
+    A = (rng.random((10, 300)) - 0.5) * np.exp(0.5 * rng.standard_normal((10, 300)))
+    B = (rng.random((300, 8)) - 0.5) * np.exp(0.5 * rng.standard_normal((300, 8)))
+    Cref, D = direct.dgemm_dd(A, B)
+    errs = [direct.componentwise_error(staged.dgemm_o2_staged(A, B, n)["C"], Cref, D) for n in (8, 12, 15)]
+    assert errs[0] > 100 * errs[1] > 100 * errs[2] and errs[2] <= 1e-14      # 15 real moduli ~ 16 2M moduli (Section 4)
+    # against exact rationals on a tiny case
+    F = Fraction
+    got, _ = direct.dgemm_dd(A[:3, :20], B[:20, :2])
+    for i in range(3):
+        for j in range(2):
+            ex = sum(F(float(A[i, p])) * F(float(B[p, j])) for p in range(20))
+            assert abs(F(float(got[i, j])) - ex) <= abs(ex) * F(1, 2 ** 52)
