@@ -60,7 +60,7 @@ typedef enum {
 
 typedef enum {
     GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3,
-    GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6
+    GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6, GEMM2M_OP_DGEMM_OZAKI2 = 7
 } gemm2m_op;
 
 /* Human-readable name of a status code (static string). */
@@ -124,6 +124,15 @@ int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const 
  *      bits of each operand survive the truncation, about what one more modulus buys.  Falls back to 0 for k > 2^22.
  * Process-wide; takes effect with the next call.  The rank-k family always uses 0. */
 int gemm2m_set_scaling(int mode);
+
+/* The real Ozaki-II scheme the paper builds on and compares with (Section 3.1; "1 ZGEMM costs about 2.16 DGEMMs",
+ * Section 6): C = A B for REAL double matrices (A: m x k, lda >= m; B: k x n, ldb >= k; C: m x n, ldc >= m, real doubles),
+ * with ONE real int8 GEMM per modulus of the real modulus set of Section 4 (256, 255, 253, 251, 247, 241, ...; every
+ * coprime number qualifies, nmod <= 20, 15 give M ~ 2^117).  Same readings as zgemm2m: power-of-two scale factors from
+ * the largest magnitude of a row / column times sqrt(k), truncation, symmetric residues, one rounding.  Workspace:
+ * gemm2m_workspace_bytes(GEMM2M_OP_DGEMM_OZAKI2, ...). */
+int dgemm_ozaki2(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
+                 int nmod, void* stream);
 
 /* Hermitian rank-k update C = A A^H (Section 5, HERK) with ONE real int8 GEMM per modulus: C+ = A+ A-^T and
  * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
@@ -225,6 +234,10 @@ int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_g
  *   inv_m    = the float reciprocal in use
  *   xmax     = bound on the magnitude of the reduced sums
  *   margin   = (1/(2 m_j)) / ((Y0 + xmax) |inv_m - 1/m_j|): the quotient estimate is exact while this exceeds 1 */
+/* The same constants for the real scheme of dgemm_ozaki2 (tests only; host pointers, any may be NULL): moduli[nmod],
+ * scale[4] = P_t, P_A, P_B, c_k, crt_g[nmod*5] = digits of sym(q_j)(M/m_j), crt_m[5], nchunks, and the reduction constants. */
+int gemm2m_debug_tables_real(int nmod, int64_t k, int* moduli, int* scale, double* crt_g, double* crt_m, int* nchunks, int32_t* y0_bits, float* cq,
+                             float* inv_m, int32_t* xmax, double* margin);
 int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin);
 
 #ifdef __cplusplus

@@ -10,7 +10,7 @@ from __future__ import annotations
 import ctypes
 import os
 
-OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K = 0, 1, 2, 3, 4, 5, 6
+OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K, OP_DGEMM_OZAKI2 = 0, 1, 2, 3, 4, 5, 6, 7
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -69,6 +69,8 @@ def lib():
     L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
     L.gemm2m_debug_set_panels.argtypes = [i32]
+    L.dgemm_ozaki2.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.gemm2m_debug_tables_real.argtypes = [i32, i64] + [vp] * 10
     L.gemm2m_set_scaling.argtypes = [i32]
     L.gemm2m_debug_set_residue_kernel.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
@@ -190,6 +192,11 @@ def cgemm2m_ex(transa, transb, alpha, A, B, beta, C, nmod=7, stream=None):
     _xgemm_ex(lib().cgemm2m_ex, "cgemm2m_ex", ctypes.c_float, transa, transb, alpha, A, B, beta, C, nmod, stream)
 
 
+def dgemm_ozaki2(A, B, C, nmod=15, stream=None):
+    """Real C = A B by the real Ozaki-II scheme (float64 CUDA tensors, column-major views)."""
+    _xgemm(lib().dgemm_ozaki2, "dgemm_ozaki2", A, B, C, nmod, stream)
+
+
 def zherk2m(A, C, nmod=16, stream=None):
     pa, n, k, lda = _colmajor(A, "A")
     pc, n1, n2, ldc = _colmajor(C, "C")
@@ -308,3 +315,23 @@ def debug_residue_reduction(nmod):
     _check(lib().gemm2m_debug_residue_reduction(nmod, ptr(y0), ptr(cq), ptr(inv), ptr(xmax), ptr(margin)),
            "gemm2m_debug_residue_reduction")
     return dict(y0_bits=y0, cq=cq, inv_m=inv, xmax=xmax, margin=margin)
+
+
+def debug_tables_real(nmod, k):
+    """Host-side constants of the real scheme (see gemm2m_debug_tables_real)."""
+    import numpy as np
+    mods = np.zeros(nmod, dtype=np.int32)
+    scale = np.zeros(4, dtype=np.int32)
+    g = np.zeros((nmod, 5), dtype=np.float64)
+    mc = np.zeros(5, dtype=np.float64)
+    nch = np.zeros(1, dtype=np.int32)
+    y0 = np.zeros(nmod, dtype=np.int32)
+    cq = np.zeros(nmod, dtype=np.float32)
+    inv = np.zeros(nmod, dtype=np.float32)
+    xmax = np.zeros(nmod, dtype=np.int32)
+    margin = np.zeros(nmod, dtype=np.float64)
+    ptr = lambda a: ctypes.c_void_p(a.ctypes.data)
+    _check(lib().gemm2m_debug_tables_real(nmod, k, ptr(mods), ptr(scale), ptr(g), ptr(mc), ptr(nch), ptr(y0), ptr(cq), ptr(inv),
+                                          ptr(xmax), ptr(margin)), "gemm2m_debug_tables_real")
+    return dict(moduli=mods, Pt=int(scale[0]), PA=int(scale[1]), PB=int(scale[2]), ck=int(scale[3]), g=g, Mc=mc, nchunks=int(nch[0]),
+                y0_bits=y0, cq=cq, inv_m=inv, xmax=xmax, margin=margin)

@@ -86,8 +86,10 @@ struct Carve {
 
 bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     if (m < 0 || n < 0 || k < 0 || nmod < 1 || nmod > kMaxMod) return false;
-    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_DSYR2K) return false;
-    const bool herk = op >= GEMM2M_OP_ZHERK;                                   // the rank-k family: one scale vector, C+ only
+    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_DGEMM_OZAKI2) return false;
+    const bool real_scheme = op == GEMM2M_OP_DGEMM_OZAKI2;                      // one plane per modulus of the real set
+    if (real_scheme && nmod > kMaxReal) return false;
+    const bool herk = op >= GEMM2M_OP_ZHERK && op <= GEMM2M_OP_DSYR2K;         // the rank-k family: one scale vector, C+ only
     const bool two = op == GEMM2M_OP_ZHER2K || op == GEMM2M_OP_DSYR2K;         // rank-2k: two operands
     const bool real_in = op == GEMM2M_OP_DSYRK || op == GEMM2M_OP_DSYR2K;      // real input, packed as Z = X1 + i X2
     if (herk && nmod > kMax2M) return false;                                   // the hybrid moduli serve the complex GEMMs only
@@ -105,7 +107,7 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_exp_b = take(herk ? 0 : 4 * n);
     c->off_pack_a = take(real_in ? 16 * n * k : 0);
     c->off_pack_b = take(real_in && two ? 16 * n * k : 0);
-    const int64_t planes = plane_count(nmod);                                  // 2 per 2M modulus, 3 per 3M modulus
+    const int64_t planes = real_scheme ? nmod : plane_count(nmod);             // 2 per 2M modulus, 3 per 3M modulus
     c->off_apm = take(planes * m * kp);
     c->off_bpm = take((herk && !two) ? 0 : planes * n * kp);
     c->off_cpm = take((herk ? (int64_t)nmod : planes) * n * ldp);
@@ -530,6 +532,95 @@ int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const 
     return xgemm2m<float>(GEMM2M_OP_CGEMM, transa, transb, m, n, k, a, A, lda, B, ldb, b, C, ldc, nmod, stream);
 }
 
+int dgemm_ozaki2(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
+                 int nmod, void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
+    if (lda < (m > 1 ? m : 1) || ldb < (k > 1 ? k : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
+    if (nmod < 1 || nmod > kMaxReal) return GEMM2M_ERR_NMOD;
+    if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
+    if (m == 0 || n == 0) return GEMM2M_OK;
+    if (!C || (k > 0 && (!A || !B))) return GEMM2M_ERR_ARG;
+    if (int s = check_device()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (k == 0) {
+        CK(cudaMemset2DAsync(C, (size_t)ldc * sizeof(double), 0, (size_t)m * sizeof(double), (size_t)n, st));
+        return GEMM2M_OK;
+    }
+    Carve c;
+    if (!carve(GEMM2M_OP_DGEMM_OZAKI2, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!D().ws || D().ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)D().ws;
+    uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
+    uint64_t* absB = (uint64_t*)(ws + c.off_abs_b);
+    int32_t* eA = (int32_t*)(ws + c.off_exp_a);
+    int32_t* eB = (int32_t*)(ws + c.off_exp_b);
+    int8_t* apl = (int8_t*)(ws + c.off_apm);
+    int8_t* bpl = (int8_t*)(ws + c.off_bpm);
+    int8_t* cpl = (int8_t*)(ws + c.off_cpm);
+    const ScaleTargets sc = scale_targets_real(nmod, k);
+    ResidueTable rtab;
+    build_residue_table_real(nmod, &rtab);
+    CrtTable ctab;
+    build_crt_table_real(nmod, &ctab);
+    const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
+    Phases ph;
+    if (int s = begin_call(&ph)) return s;
+    // Section 3.1: scale factors, truncation, residues for every modulus, one real int8 GEMM per modulus, CRT, unscale
+    CK(ph.begin(0, st));
+    CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
+    CK(launch_scan_real<double>(A, m, k, lda, true, absA, st, &g.launches[0]));
+    CK(launch_scan_real<double>(B, k, n, ldb, false, absB, st, &g.launches[0]));
+    CK(launch_exponents<double>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
+    CK(launch_exponents<double>(absB, n, sc.PB, sc.ck, eB, st, &g.launches[0]));
+    CK(ph.end(st));
+    CK(ph.begin(1, st));
+    CK(launch_residues_real<double>(A, lda, false, m, k, c.kp, eA, rtab, wideA, apl, st, &g.launches[1]));
+    CK(launch_residues_real<double>(B, ldb, true, n, k, c.kp, eB, rtab, wideB, bpl, st, &g.launches[1]));
+    CK(ph.end(st));
+    GemmArgs ga;
+    ga.rowop = bpl; ga.colop = apl;
+    ga.R = n; ga.Cn = m; ga.Kp = c.kp;
+    ga.row_planes = ga.col_planes = nmod;
+    ga.row_plane0 = ga.col_plane0 = 0;
+    ga.nbatch = nmod;
+    ga.out = cpl; ga.ldp = c.ldp; ga.accumulate = 0;
+    build_mod_table_real(nmod, &ga.mods);
+    ga.dev_status = (int*)(ws + c.off_status);
+    int panels = (int)(n / 1024);
+    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
+    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
+    const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
+    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
+    const int64_t klim = gemm_k_limit_real();
+    for (int pnl = 0; pnl < panels; ++pnl) {
+        const int64_t j0 = pnl * panel_cols, j1 = (j0 + panel_cols < n) ? j0 + panel_cols : n;
+        if (j0 >= j1) break;
+        ga.row_begin = j0;
+        ga.row_end = j1;
+        CK(ph.begin(2, st));
+        if (g.gemm_kernel == 1) CK(launch_gemm_check(ga, klim, st, &g.launches[2]));
+        else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(ga, klim, D().sm_count, st, &g.launches[2]));
+        else CK(launch_gemm_tcgen05_pair(ga, klim, D().sm_count, st, &g.launches[2]));
+        CK(ph.end(st));
+        const bool last = j1 >= n;
+        cudaStream_t ps = last ? st : D().side;
+        if (!last) {
+            CK(cudaEventRecord(D().panel_done[pnl], st));
+            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
+        }
+        CK(ph.begin(3, ps));
+        CK(launch_post_real(cpl, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]));
+        CK(ph.end(ps));
+    }
+    if (panels > 1) {
+        CK(cudaEventRecord(D().side_done, D().side));
+        CK(cudaStreamWaitEvent(st, D().side_done, 0));
+    }
+    ph.done();
+    return GEMM2M_OK;
+}
+
 int zherk2m(int64_t n, int64_t k, const double* A, int64_t lda, double* C, int64_t ldc, int nmod, void* stream) {
     return rank_update(GEMM2M_OP_ZHERK, n, k, A, lda, nullptr, 0, C, ldc, nmod, stream);
 }
@@ -622,6 +713,30 @@ int gemm2m_debug_set_residue_kernel(int which) {
     std::lock_guard<std::mutex> lock(g.mu);
     if (which < 0 || which > 1) return GEMM2M_ERR_ARG;
     g.residue_kernel = which;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_tables_real(int nmod, int64_t k, int* moduli, int* scale, double* crt_g, double* crt_m, int* nchunks, int32_t* y0_bits, float* cq,
+                             float* inv_m, int32_t* xmax, double* margin) {
+    if (nmod < 1 || nmod > kMaxReal || k < 0) return GEMM2M_ERR_ARG;
+    const ScaleTargets sc = scale_targets_real(nmod, k);
+    if (scale) { scale[0] = sc.Pt; scale[1] = sc.PA; scale[2] = sc.PB; scale[3] = sc.ck; }
+    CrtTable ct;
+    build_crt_table_real(nmod, &ct);
+    ResidueTable rt;
+    build_residue_table_real(nmod, &rt);
+    for (int j = 0; j < nmod; ++j) {
+        if (moduli) moduli[j] = real_modulus_value(j);
+        for (int c = 0; c < kMaxChunks; ++c)
+            if (crt_g) crt_g[j * kMaxChunks + c] = ct.gr[j][c];
+        if (y0_bits) y0_bits[j] = rt.magic[j];
+        if (cq) cq[j] = rt.cq[j];
+        if (inv_m) inv_m[j] = rt.inv_m[j];
+        if (xmax) xmax[j] = rt.xmax[j];
+        if (margin) margin[j] = residue_reduction_margin(rt, j);
+    }
+    if (crt_m) for (int c = 0; c < kMaxChunks; ++c) crt_m[c] = ct.Mc[c];
+    if (nchunks) *nchunks = ct.nchunks;
     return GEMM2M_OK;
 }
 

@@ -11,6 +11,7 @@ namespace gemm2m {
 constexpr int kMax2M = 22;         // size of the greedy 2M modulus set in [1, 256] (Section 4)
 constexpr int kMax3M = 4;          // non-2M moduli of the hybrid: 256, 253, 251, 249 (quantised values then still fit 96 bits)
 constexpr int kMaxMod = kMax2M + kMax3M;
+constexpr int kMaxReal = 20;       // moduli of the real Ozaki-II scheme (Section 3.1; set of Section 4): M up to 2^155
 constexpr int kMaxPlanes = 2 * kMax2M + 3 * kMax3M;   // residue planes per operand: two per 2M modulus, three per 3M modulus
 constexpr int kMaxChunks = 5;      // 40-bit digits needed for M/2 < 2^184
 constexpr int kChunkBits = 40;
@@ -87,6 +88,13 @@ void build_mod_table(int nmod, bool per_plane, ModTable* t);
 void build_crt_table(int nmod, CrtTable* t);
 void build_crt_table_int(int nmod, CrtTableInt* t);
 ScaleTargets scale_targets(int nmod, int64_t k, bool herk);
+// The same for the real Ozaki-II scheme (dgemm_ozaki2): moduli 256, 255, 253, ..., one residue plane per modulus.
+int real_modulus_value(int j);
+void build_residue_table_real(int nmod, ResidueTable* t);
+void build_mod_table_real(int nmod, ModTable* t);
+void build_crt_table_real(int nmod, CrtTable* t);
+ScaleTargets scale_targets_real(int nmod, int64_t k);
+int64_t gemm_k_limit_real();
 int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
 
 // ---- phase launchers (prepost.cu) ----
@@ -114,6 +122,12 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
 // alpha, beta: host pointers to (re, im) pairs, or null for alpha = 1 / beta = 0: C = alpha X + beta C.
 template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
                                                  const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta, cudaStream_t st, int* launches);
+// Real Ozaki-II scheme (Section 3.1): scans, residues (one plane per modulus) and post-processing of real matrices.
+template <typename T> cudaError_t launch_scan_real(const T* X, int64_t rows, int64_t cols, int64_t ld, bool per_row, uint64_t* absmax, cudaStream_t st, int* launches);
+template <typename T> cudaError_t launch_residues_real(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                                                       const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+cudaError_t launch_post_real(const int8_t* cp, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
+                             const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches);
 // C = beta C (the alpha = 0 case of the extended interface); beta = host pointer to (re, im) or null for 0.
 template <typename T> cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches);
 // real_out: C is a real matrix (SYRK / SYR2K through Z = A1 + i A2): only the real part is formed and stored.

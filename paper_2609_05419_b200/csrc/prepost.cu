@@ -95,6 +95,57 @@ __global__ void exponents_kernel(const unsigned long long* __restrict__ absmax, 
     e[i] = out;
 }
 
+// ---- real matrices (real Ozaki-II scheme, Section 3.1): the same scans over scalar elements ----------------
+template <typename T>
+__global__ void __launch_bounds__(kScanThreads) scan_rows_real_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
+                                                                      unsigned long long* __restrict__ absmax) {
+    const int64_t r = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
+    if (r >= rows) return;
+    const int64_t c0 = (int64_t)blockIdx.y * span;
+    const int64_t c1 = min(cols, c0 + span);
+    unsigned long long mx = 0;
+    const T* p = X + (r + c0 * ld);
+#pragma unroll 8
+    for (int64_t c = c0; c < c1; ++c, p += ld) mx = max(mx, FpBits<T>::mag(__ldg(p)));
+    if (mx) atomicMax(absmax + r, mx);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kScanThreads) scan_cols_real_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
+                                                                      unsigned long long* __restrict__ absmax) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c = (int64_t)blockIdx.x * (kScanThreads / 32) + warp;
+    if (c >= cols) return;
+    const int64_t r0 = (int64_t)blockIdx.y * span;
+    const int64_t r1 = min(rows, r0 + span);
+    unsigned long long mx = 0;
+    const T* base = X + c * ld;
+#pragma unroll 4
+    for (int64_t r = r0 + lane; r < r1; r += 32) mx = max(mx, FpBits<T>::mag(__ldg(base + r)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if (lane == 0 && mx) atomicMax(absmax + c, mx);
+}
+
+template <typename T>
+cudaError_t launch_scan_real(const T* X, int64_t rows, int64_t cols, int64_t ld, bool per_row, uint64_t* absmax, cudaStream_t st, int* launches) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    if (per_row) {
+        int64_t span = kScanRowsSpan;
+        while ((cols + span - 1) / span > 65535) span *= 2;
+        dim3 grid((unsigned)((rows + kScanThreads - 1) / kScanThreads), (unsigned)((cols + span - 1) / span));
+        scan_rows_real_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    } else {
+        int64_t span = 2 * kScanColsSpan;
+        while ((rows + span - 1) / span > 65535) span *= 2;
+        dim3 grid((unsigned)((cols + kScanThreads / 32 - 1) / (kScanThreads / 32)), (unsigned)((rows + span - 1) / span));
+        scan_cols_real_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+template cudaError_t launch_scan_real<double>(const double*, int64_t, int64_t, int64_t, bool, uint64_t*, cudaStream_t, int*);
+
 // ---- 2-norm scaling rule: second pass over the operand --------------------------------------------------
 // floor(log2) of the finite non-zero magnitude with bit pattern b.
 template <typename T>
@@ -555,6 +606,123 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
     return cudaGetLastError();
 }
 
+// ---- real floating-point inputs (real Ozaki-II scheme): one plane per modulus ---------------------------------------
+template <int NE, bool WIDE>
+__device__ __forceinline__ void emit_run_real(const Digits (&dr)[NE], const uint32_t* tr, const ResidueTable& tab, int8_t* dst, int64_t plane_stride) {
+    const int nmod = tab.nmod;
+#pragma unroll 1
+    for (int j = 0; j < nmod; ++j) {
+        const int neg_m = -tab.m[j], y0 = tab.magic[j];
+        const float inv_m = tab.inv_m[j], cq = tab.cq[j];
+        const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], wt = WIDE ? tab.w_top[j] : 0u;
+        uint32_t rw[NE / 4];
+#pragma unroll
+        for (int w = 0; w < NE / 4; ++w) {
+            uint32_t br[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = 4 * w + b;
+                int Ry = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));
+                if (WIDE) Ry = dp4a_ss(tr[i], wt, Ry);
+                br[b] = sym_reduce_one(Ry, neg_m, inv_m, cq);
+            }
+            rw[w] = pack4(br);
+        }
+        store_run<NE>(dst + (int64_t)j * plane_stride, rw);
+    }
+}
+
+template <typename T, bool WIDE>
+__global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_real_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, int64_t R,
+                                                                                   int64_t K, int64_t Kp, const int32_t* __restrict__ e,
+                                                                                   const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T* ring = reinterpret_cast<T*>(smem_raw);
+    constexpr int kStageElems = kResRows * kResRowStride;
+    const int t = threadIdx.x;
+    const int64_t ktiles = Kp / kResK;
+    const int64_t total = ((R + kResRows - 1) / kResRows) * ktiles;
+    const int64_t plane_stride = R * Kp;
+
+    auto issue = [&](int64_t tile, int stage) {
+        const int64_t row0 = (tile / ktiles) * kResRows, k0 = (tile % ktiles) * kResK;
+        T* dst = ring + stage * kStageElems;
+        if (!k_contiguous) {
+            const int r = t & (kResRows - 1);
+            const int64_t row = row0 + r;
+#pragma unroll
+            for (int kk = t / kResRows; kk < kResK; kk += kResThreads / kResRows) {
+                const int64_t k = k0 + kk;
+                const bool ok = row < R && k < K;
+                cp_async_zfill<sizeof(T)>(dst + r * kResRowStride + kk + (kk >> 3), ok ? X + (row + k * ld) : X, ok);
+            }
+        } else {
+            const int kk = t & (kResK - 1);
+            const int64_t k = k0 + kk;
+#pragma unroll
+            for (int r = t / kResK; r < kResRows; r += kResThreads / kResK) {
+                const int64_t row = row0 + r;
+                const bool ok = row < R && k < K;
+                cp_async_zfill<sizeof(T)>(dst + r * kResRowStride + kk + (kk >> 3), ok ? X + (k + row * ld) : X, ok);
+            }
+        }
+        cp_async_commit();
+    };
+
+    int64_t tile = blockIdx.x;
+    if (tile >= total) return;
+    issue(tile, 0);
+    for (int it = 0; tile < total; tile += gridDim.x, ++it) {
+        const int64_t next = tile + gridDim.x;
+        if (next < total) { issue(next, (it + 1) & 1); cp_async_wait_group<1>(); }
+        else cp_async_wait_group<0>();
+        __syncthreads();
+        const T* src = ring + (it & 1) * kStageElems;
+        const int64_t row0 = (tile / ktiles) * kResRows, k0 = (tile % ktiles) * kResK;
+        const int g = t & (kResK / kResRun - 1), r = t / (kResK / kResRun);
+        const int64_t row = row0 + r;
+        if (row < R) {
+            const int ex = __ldg(e + row);
+            const bool fast = !WIDE && ex > -1000 && ex < 1000;
+            const double scale = __longlong_as_double((long long)(1023 - (fast ? ex : 0)) << 52);
+            Digits dr[kResRun];
+            uint32_t tr[WIDE ? kResRun : 1];
+#pragma unroll
+            for (int i = 0; i < kResRun; ++i) {
+                const T v = src[r * kResRowStride + kResRun * g + g + i];
+                if (WIDE) {
+                    uint32_t lr = 0;
+                    long long ur = 0;
+                    if (ex != kExpNonFinite) quantise_part_wide<T>(v, ex, &lr, &ur);
+                    dr[i] = split_digits_wide(lr, ur, &tr[i]);
+                } else {
+                    long long qr = 0;
+                    if (fast) qr = __double2ll_rz((double)v * scale);
+                    else if (ex != kExpNonFinite) qr = quantise_part<T>(v, ex);
+                    dr[i] = split_digits(qr);
+                }
+            }
+            emit_run_real<kResRun, WIDE>(dr, tr, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T>
+cudaError_t launch_residues_real(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                                 const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
+    if (R <= 0 || Kp <= 0) return cudaSuccess;
+    constexpr size_t smem = kResSmemBytes(sizeof(T));
+    const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
+    const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
+    const unsigned grid = (unsigned)(total < resident ? total : resident);
+    if (wide) residues_real_kernel<T, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    else residues_real_kernel<T, false><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, R, K, Kp, e, tab, planes);
+    ++*launches;
+    return cudaGetLastError();
+}
+template cudaError_t launch_residues_real<double>(const double*, int64_t, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+
 // ---- int8 Gaussian-integer inputs (no scaling): one 32 x 128 tile per block, loaded synchronously ---------------------
 constexpr int kResIRows = 32, kResIRun = 16;
 constexpr int kResIRowStride = kResK + kResK / kResIRun + 1;
@@ -821,6 +989,79 @@ cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n,
     const bool plain = sc.ar == 1.0 && sc.ai == 0.0 && sc.br == 0.0 && sc.bi == 0.0;
     if (plain) return launch_post_fp_t<T, false>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
     return launch_post_fp_t<T, true>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
+}
+
+// Real Ozaki-II scheme (Section 3.1): cp: [nmod][n][ldp] int8, one plane per modulus; X = sum_j c_j G_j (mod M) with
+// G_j = sym(q_j)(M/m_j) in tab.gr; real double output.  Same staging and finish as post_fp_kernel.
+template <int NCH>
+__global__ void __launch_bounds__(kPostThreads) post_real_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t m, int64_t n,
+                                                                 const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
+                                                                 const __grid_constant__ CrtTable tab, double* __restrict__ C, int64_t ldc) {
+    __shared__ __align__(16) uint32_t stage[kMaxMod][kPostThreads];
+    const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
+    const int64_t j = blockIdx.y;
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cp + j * ldp + ib;
+    const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);
+    for (int idx = threadIdx.x; idx < nmod * (kPostSpan / 16); idx += kPostThreads) {
+        const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
+        if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    const int64_t i0 = ib + 4 * threadIdx.x;
+    if (i0 >= m) return;
+    double S[4][NCH];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) S[e][c] = 0.0;
+    }
+#pragma unroll 2
+    for (int jm = 0; jm < nmod; ++jm) {
+        const uint32_t w = stage[jm][threadIdx.x];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const double v = int_to_double((int)(int8_t)(w >> (8 * e)));
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) S[e][c] = fma(v, tab.gr[jm][c], S[e][c]);
+        }
+    }
+    const int fb = __ldg(eB + j);
+    for (int e = 0; e < 4; ++e) {
+        if (i0 + e < m) {
+            const int ea = __ldg(eA + i0 + e);
+            double out;
+            if (ea == kExpNonFinite || fb == kExpNonFinite) {
+                out = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(S[e], tab, &h, &l);
+                out = scale_pow2(h + l, ea + fb);
+            }
+            C[i0 + e + j * ldc] = out;
+        }
+    }
+}
+
+cudaError_t launch_post_real(const int8_t* cp, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                             const int32_t* eB, const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+    for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {
+        const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
+        dim3 grid((unsigned)((m + kPostSpan - 1) / kPostSpan), (unsigned)nj);
+        const int8_t* src = cp + j0 * ldp;
+        double* dst = C + j0 * ldc;
+        switch (tab.nchunks) {
+            case 1: post_real_kernel<1><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 2: post_real_kernel<2><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 3: post_real_kernel<3><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            default: post_real_kernel<4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+        }
+        ++*launches;
+    }
+    return cudaGetLastError();
 }
 
 // C = beta C (C = 0 for beta = 0, without reading C): the alpha = 0 case of the extended interface.

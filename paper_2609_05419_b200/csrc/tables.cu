@@ -14,7 +14,12 @@ namespace gemm2m {
 static const int kModuli[kMaxMod] = {241, 233, 229, 221, 205, 197, 193, 181, 173, 157, 149, 137, 113,
                                      109, 101, 97,  89,  73,  61,  53,  37,  29,  256, 253, 251, 249};
 
+// The set available to the real Ozaki-II scheme (Section 4): the same greedy walk without the 2M condition.
+static const int kRealModuli[kMaxReal] = {256, 255, 253, 251, 247, 241, 239, 233, 229, 227,
+                                          223, 217, 211, 199, 197, 193, 191, 181, 179, 173};
+
 int modulus_value(int j) { return kModuli[j]; }
+int real_modulus_value(int j) { return kRealModuli[j]; }
 
 int modulus_root(int j) {   // smallest positive s with s^2 = -1 (mod m); 0 for a non-2M modulus
     if (j >= kMax2M) return 0;
@@ -76,18 +81,19 @@ struct Big {
     double to_double() const { double v = 0; for (size_t i = w.size(); i-- > 0;) v = v * 4294967296.0 + w[i]; return v; }
 };
 
-static Big product_of(int nmod) {
+static Big product_of(int nmod, const int* mods = kModuli) {
     Big M = Big::from(1);
-    for (int j = 0; j < nmod; ++j) M.mul_small((uint32_t)kModuli[j]);
+    for (int j = 0; j < nmod; ++j) M.mul_small((uint32_t)mods[j]);
     return M;
 }
 
-void build_residue_table(int nmod, ResidueTable* t) {
+// mods: the modulus list; n2: how many of the first nmod are 2M moduli (the others take the plain weights for both parts).
+static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTable* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
-    t->n2 = count_2m(nmod);
+    t->n2 = n2;
     for (int j = 0; j < nmod; ++j) {
-        const int m = kModuli[j], s = j < kMax2M ? modulus_root(j) : 1;   // 3M modulus: both parts take the plain weights
+        const int m = mods[j], s = j < n2 ? modulus_root(j) : 1;
         t->m[j] = m;
         t->s[j] = s;
         t->inv_m[j] = 1.0f / (float)m;
@@ -125,6 +131,9 @@ void build_residue_table(int nmod, ResidueTable* t) {
     }
 }
 
+void build_residue_table(int nmod, ResidueTable* t) { build_residue_table_for(kModuli, nmod, count_2m(nmod), t); }
+void build_residue_table_real(int nmod, ResidueTable* t) { build_residue_table_for(kRealModuli, nmod, 0, t); }
+
 // 2^e / (2 (Y0 + xmax) |n m - 2^e|) for inv_m = n 2^-e: the factor by which the error term of the residue kernels'
 // quotient estimate stays below the distance 1/(2m) of x/m from the nearest rounding boundary (must exceed 1).
 double residue_reduction_margin(const ResidueTable& t, int j) {
@@ -154,13 +163,19 @@ void build_mod_table(int nmod, bool per_plane, ModTable* t) {
     t->nplanes = p;
 }
 
+void build_mod_table_real(int nmod, ModTable* t) {
+    std::memset(t, 0, sizeof(*t));
+    for (int j = 0; j < nmod; ++j) { t->m[j] = kRealModuli[j]; t->inv_m[j] = 1.0f / (float)kRealModuli[j]; }
+    t->nplanes = nmod;
+}
+
 // Folded CRT weights: g_j = sym(2^-1 q_j mod m_j), h_j = sym(s_j 2^-1 q_j mod m_j), q_j = (M/m_j)^-1 mod m_j.
-static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h) {
-    const int m = kModuli[j];
+static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h, const int* mods = kModuli, int n2 = kMax2M) {
+    const int m = mods[j];
     *W = M;
     W->divmod_small((uint32_t)m);
     const int q = inv_mod((int)W->mod_small((uint32_t)m), m);
-    if (j >= kMax2M) {              // 3M modulus: Eq. (1) needs no factor besides q_j
+    if (j >= n2) {                  // 3M modulus (Eq. (1)) or real scheme (Section 3.1): no factor besides q_j
         *g = *h = sym_mod(q, m);
         return;
     }
@@ -170,11 +185,11 @@ static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h
     (void)nmod;
 }
 
-void build_crt_table(int nmod, CrtTable* t) {
+static void build_crt_table_for(const int* mods, int nmod, int n2, CrtTable* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
-    t->n2 = count_2m(nmod);
-    const Big M = product_of(nmod);
+    t->n2 = n2;
+    const Big M = product_of(nmod, mods);
     Big half = M;   // (M-1)/2 bounds every |G_j|
     half.sub_one();
     half.shr1();
@@ -186,7 +201,7 @@ void build_crt_table(int nmod, CrtTable* t) {
     for (int j = 0; j < nmod; ++j) {
         Big W;
         int g, h;
-        folded_weights(nmod, j, M, &W, &g, &h);
+        folded_weights(nmod, j, M, &W, &g, &h, mods, mods == kModuli ? kMax2M : 0);
         Big Gr = W, Gi = W;
         Gr.mul_small((uint32_t)std::abs(g));
         Gi.mul_small((uint32_t)std::abs(h));
@@ -198,6 +213,9 @@ void build_crt_table(int nmod, CrtTable* t) {
     t->q_hi = std::ldexp(1.0, kChunkBits * (t->nchunks - 1)) / M.to_double();
     t->q_lo = t->nchunks > 1 ? std::ldexp(t->q_hi, -kChunkBits) : 0.0;
 }
+
+void build_crt_table(int nmod, CrtTable* t) { build_crt_table_for(kModuli, nmod, count_2m(nmod), t); }
+void build_crt_table_real(int nmod, CrtTable* t) { build_crt_table_for(kRealModuli, nmod, 0, t); }
 
 void build_crt_table_int(int nmod, CrtTableInt* t) {
     std::memset(t, 0, sizeof(*t));
@@ -230,6 +248,23 @@ ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
     while ((1ull << (2 * s.ck)) < (uint64_t)(2 * kk)) ++s.ck;
     return s;
 }
+
+// Real scheme (Section 3.1): a row has k real terms, c_k = ceil(log2(k)/2).
+ScaleTargets scale_targets_real(int nmod, int64_t k) {
+    Big half = product_of(nmod, kRealModuli);
+    half.sub_one();
+    half.shr1();
+    ScaleTargets s;
+    s.Pt = half.bit_length() - 1;
+    s.PA = (s.Pt + 1) / 2;
+    s.PB = s.Pt / 2;
+    s.ck = 0;
+    const int64_t kk = k > 0 ? k : 1;
+    while ((1ull << (2 * s.ck)) < (uint64_t)kk) ++s.ck;
+    return s;
+}
+
+int64_t gemm_k_limit_real() { return (int64_t)INT32_MAX / (128 * 128); }   // the modulus 256 comes first
 
 int64_t gemm_k_limit(int nmod) {
     // largest |residue|: 120 for the 2M moduli (241 comes first), 128 once the hybrid adds the modulus 256

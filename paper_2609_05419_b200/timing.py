@@ -5,6 +5,7 @@
   python -m paper_2609_05419_b200.timing --op zherk --n 8192 --k 8192 --nmod 16
 
   python -m paper_2609_05419_b200.timing --op dsyrk --n 8192 --k 8192 --nmod 16      (also zher2k, dsyr2k)
+  python -m paper_2609_05419_b200.timing --op dgemm --m 8192 --n 8192 --k 8192 --nmod 15     (real Ozaki-II scheme)
 
 Prints one JSON line: effective TFLOP/s (BLAS flop counts: 8mnk for GEMM, 4n^2k HERK, 8n^2k HER2K, n^2k SYRK, 2n^2k SYR2K,
 divided by the time), milliseconds per call and per phase.
@@ -23,7 +24,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k"])
+    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=8192)
@@ -48,6 +49,10 @@ def main():
         opcode = {"zherk": b.OP_ZHERK, "zher2k": b.OP_ZHER2K, "dsyrk": b.OP_DSYRK, "dsyr2k": b.OP_DSYR2K}[a.op]
         flops = {"zherk": 4.0, "zher2k": 8.0, "dsyrk": 1.0, "dsyr2k": 2.0}[a.op] * n * n * k     # BLAS flop counts
         tdtype = torch.float64 if real else torch.complex128
+    elif a.op == "dgemm":              # real Ozaki-II scheme: the real parts of the same synthetic inputs
+        Ah, Bh = inputs.complex_inputs(m, n, k, a.seed, a.dist, a.phi)
+        A, B = dev(np.asfortranarray(Ah.real.copy())), dev(np.asfortranarray(Bh.real.copy()))
+        opcode, flops, tdtype = b.OP_DGEMM_OZAKI2, 2.0 * m * n * k, torch.float64
     else:
         Ah, Bh = inputs.complex_inputs(m, n, k, a.seed, a.dist, a.phi, dtype=dtype)
         A, B = dev(Ah), dev(Bh)
@@ -68,6 +73,8 @@ def main():
             b.dsyr2k2m(A, B, C, nmod, stream)
         elif a.op == "cgemm":
             b.cgemm2m(A, B, C, nmod, stream)
+        elif a.op == "dgemm":
+            b.dgemm_ozaki2(A, B, C, nmod, stream)
         else:
             b.zgemm2m(A, B, C, nmod, stream)
 
@@ -87,7 +94,7 @@ def main():
     b.device_status()
     total, per = b.last_launch_count()
     planes = 2 * min(nmod, 22) + 3 * max(nmod - 22, 0)       # complex GEMM: 2 real GEMMs per 2M modulus, 3 per 3M modulus
-    gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod}.get(a.op, planes)
+    gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod, "dgemm": nmod}.get(a.op, planes)
     kin = (k + 1) // 2 if a.op in ("dsyrk", "dsyr2k") else k
     print(json.dumps({"op": a.op, "m": m, "n": n, "k": k, "nmod": nmod, "ms_per_call": ms, "effective_tflops": flops / ms / 1e9,
                       "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3],

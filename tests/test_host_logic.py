@@ -18,7 +18,7 @@ def test_library_exports_every_declared_symbol():
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = set(re.findall(r"^(?:int|size_t|const char\*)\s+(\w+)\s*\(", text, flags=re.M))      # every declared function
     assert {"gemm2m_gaussian_int", "zgemm2m", "cgemm2m", "zherk2m", "zher2k2m", "dsyrk2m", "dsyr2k2m", "zgemm2m_ex", "cgemm2m_ex",
-            "gemm2m_set_workspace", "gemm2m_workspace_bytes", "gemm2m_zscale_exponents_static"} <= names
+            "gemm2m_set_workspace", "gemm2m_workspace_bytes", "gemm2m_zscale_exponents_static", "dgemm_ozaki2", "gemm2m_set_scaling"} <= names
     assert len(names) >= 25
     L = b.lib()
     for name in names:
@@ -163,6 +163,42 @@ def test_hybrid_crt_and_scaling_constants_match_oracle(nmod):
         assert staged.lift(Si % M, M) == staged.lift(staged.crt(res_i, mods), M)
         assert abs(Sr) < 2 ** 12 * M and abs(Si) < 2 ** 12 * M        # the multiple of M to remove stays below 2^12
     assert 2 ** t["Pt"] / M < 0.494                                   # margin of the quotient estimate in the post kernel
+
+
+@pytest.mark.parametrize("nmod", [1, 8, 15, 20])
+def test_real_scheme_constants_match_oracle(nmod):
+    mods = staged.greedy_real_moduli()[:nmod]
+    M = staged.product(mods)
+    t = b.debug_tables_real(nmod, 8192)
+    assert list(t["moduli"]) == mods
+    assert (t["Pt"], t["PA"], t["PB"], t["ck"]) == staged.scaling_targets_real(M, 8192)
+    B = 2 ** 40
+    val = lambda row: sum(int(row[c]) * B ** c for c in range(5))
+    assert val(t["Mc"]) == M and all(t["Mc"][c] == 0 for c in range(t["nchunks"], 5))
+    assert (t["nchunks"] - 1) * 40 < max(((M - 1) // 2).bit_length(), 1) <= t["nchunks"] * 40
+    for j, m in enumerate(mods):
+        W = M // m
+        assert val(t["g"][j]) == staged.sym(pow(W % m, -1, m) if m > 1 else 0, m) * W
+    assert 2 ** t["Pt"] / M < 0.494 or nmod == 1                      # margin of the quotient estimate in the post kernel
+    # the residue kernels' reduction, exhaustively, as for the 2M moduli
+    assert (t["margin"] > 1.0).all()
+    for j, m in enumerate(mods):
+        y0_bits, xmax = int(t["y0_bits"][j]), int(t["xmax"][j])
+        y0 = (y0_bits - 0x4B000000) + 2 ** 23
+        assert y0 % (256 * m) == 0 and y0 - xmax >= 2 ** 23 and y0 + xmax < 2 ** 24
+        mant, ex = np.frexp(np.float64(t["inv_m"][j]))
+        n, e = int(mant * 2 ** 24), 24 - int(ex)
+        cq = int(t["cq"][j])
+        assert cq == 3 * 2 ** 22 - y0 // m
+        x = np.arange(-xmax, xmax + 1, dtype=np.int64)
+        num = (y0 + x) * n + (cq << e)
+        fl = num >> e
+        rem = num - (fl << e)
+        half = 1 << (e - 1)
+        tq = fl + ((rem > half) | ((rem == half) & (fl & 1 == 1)))
+        low = ((y0_bits + x) - (0x4B000000 + (tq - 2 ** 23)) * m) & 0xFF
+        res = np.where(low >= 128, low - 256, low)
+        assert np.array_equal(res, ((x + m // 2) % m) - m // 2), m
 
 
 def test_workspace_layout_is_ordered_and_sized():
