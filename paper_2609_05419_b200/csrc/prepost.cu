@@ -31,6 +31,16 @@ template <> __device__ __forceinline__ Cplx<float> load_cplx<float>(const float*
     return {v.x, v.y};
 }
 
+static int cached_sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
+    return sms;
+}
+
 constexpr int kScanThreads = 256;
 constexpr int kScanRowsSpan = 64;     // columns handled by one block of scan_rows
 constexpr int kScanColsSpan = 2048;   // rows handled by one warp of scan_cols
@@ -263,8 +273,10 @@ template <typename T>
 cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
     int64_t span = kScanRowsSpan;
+    const int64_t row_blocks = (rows + kScanThreads - 1) / kScanThreads;
+    while (span > 8 && row_blocks * ((cols + span - 1) / span) < 4 * cached_sm_count()) span /= 2;   // small matrices: enough blocks to fill the GPU
     while ((cols + span - 1) / span > 65535) span *= 2;        // grid.y limit
-    dim3 grid((unsigned)((rows + kScanThreads - 1) / kScanThreads), (unsigned)((cols + span - 1) / span));
+    dim3 grid((unsigned)row_blocks, (unsigned)((cols + span - 1) / span));
     scan_rows_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
     ++*launches;
     return cudaGetLastError();
@@ -273,8 +285,10 @@ template <typename T>
 cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
     int64_t span = kScanColsSpan;
+    const int64_t col_blocks = (cols + kScanThreads / 32 - 1) / (kScanThreads / 32);
+    while (span > 256 && col_blocks * ((rows + span - 1) / span) < 4 * cached_sm_count()) span /= 2;
     while ((rows + span - 1) / span > 65535) span *= 2;        // grid.y limit
-    dim3 grid((unsigned)((cols + kScanThreads / 32 - 1) / (kScanThreads / 32)), (unsigned)((rows + span - 1) / span));
+    dim3 grid((unsigned)col_blocks, (unsigned)((rows + span - 1) / span));
     scan_cols_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
     ++*launches;
     return cudaGetLastError();
@@ -575,15 +589,6 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
 
 constexpr size_t kResSmemBytes(size_t elem) { return (size_t)kResStages * kResRows * kResRowStride * elem; }
 
-static int cached_sm_count() {
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            sms = 148;
-    }
-    return sms;
-}
 
 template <typename T>
 cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
