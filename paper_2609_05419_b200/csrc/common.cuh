@@ -45,9 +45,14 @@ struct ResidueTable {
 };
 
 // Modulus of every batch entry of a GEMM launch, for the epilogue (reduction of the int32 accumulators).
+// The accumulator's four balanced base-256 digits are contracted with w (one dp4a starting at the bit pattern y0 of the
+// float Y0), then reduced as in the residue kernels: one FMA with cq, one integer multiply-add (see ResidueTable).
 struct ModTable {
     int32_t m[kMaxPlanes];
     float inv_m[kMaxPlanes];
+    uint32_t w[kMaxPlanes];        // int8 x4: sym(256^b mod m), b = 0..3
+    int32_t y0[kMaxPlanes];
+    float cq[kMaxPlanes];
     int nplanes;
 };
 
@@ -95,7 +100,7 @@ void build_mod_table_real(int nmod, ModTable* t);
 void build_crt_table_real(int nmod, CrtTable* t);
 ScaleTargets scale_targets_real(int nmod, int64_t k);
 int64_t gemm_k_limit_real();
-int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
+int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 (plus a stored residue) stays below 0x7F7F7F7F
 
 // ---- phase launchers (prepost.cu) ----
 // Exponent scan: largest |Re|,|Im| bit pattern per row of a column-major matrix (rows x cols, ld).

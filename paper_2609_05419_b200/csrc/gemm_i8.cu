@@ -133,8 +133,7 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
             int b, tr, tc;
             decode_tile(p, tile, &b, &tr, &tc);
             const int jm = b;                             // the modulus table has one entry per batch entry
-            const int m = p.mods.m[jm];
-            const float inv_m = p.mods.inv_m[jm];
+            const ModConsts mc = load_mod_consts(p.mods, jm);
             if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase[acc], abort_flag, p.dev_status, kDevTimeoutEpilogue))) break;
             acc_phase[acc] ^= 1u;
             tcgen05_fence_after();
@@ -153,8 +152,8 @@ gemm_i8_tcgen05_kernel(const __grid_constant__ CUtensorMap map_row, const __grid
                         const int64_t col = col0 + c * 32 + g * 16;
                         if (col < p.ldp) {
                             uint4* dst = reinterpret_cast<uint4*>(orow + c * 32 + g * 16);
-                            if (p.accumulate) reduce_store16<true>(v + g * 16, dst, m, inv_m);
-                            else reduce_store16<false>(v + g * 16, dst, m, inv_m);
+                            if (p.accumulate) reduce_store16<true>(v + g * 16, dst, mc);
+                            else reduce_store16<false>(v + g * 16, dst, mc);
                         }
                     }
                 }

@@ -131,19 +131,34 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Symmetric residue of an int32 accumulator: float quotient estimate (off by at most one), exact integer remainder, fix-up.
-__device__ __forceinline__ int sym_reduce_acc(int x, int m, float inv_m) {
-    const int q = __float2int_rn(__int2float_rn(x) * inv_m);
-    int r = x - q * m;
-    if (r > ((m - 1) >> 1)) r -= m;
-    if (r < -(m >> 1)) r += m;        // even m (256, hybrid only): the range is [-m/2, m/2 - 1]
-    return r;
+// Constants of the epilogue's reduction modulo the modulus of one batch entry (see ModTable).
+struct ModConsts {
+    uint32_t w;        // int8 x4: sym(256^b mod m), b = 0..3
+    int y0;            // bit pattern of the float Y0
+    int neg_m;
+    float inv_m, cq;
+};
+__device__ __forceinline__ ModConsts load_mod_consts(const ModTable& t, int b) {
+    return ModConsts{t.w[b], t.y0[b], -t.m[b], t.inv_m[b], t.cq[b]};
+}
+
+// Symmetric residue of an int32 accumulator x (|x| + 128 <= 0x7F7F7F7F), in the low byte of the result.  The four balanced
+// base-256 digits of x (add 128 to every byte with carries, flip every byte's top bit) are contracted with 256^b mod m by
+// one dp4a that starts at the bit pattern of the float Y0 (plus `extra`, a residue to be added): the sum is the bit
+// pattern of Y0 + x' with x' = x (mod m) and |x'| small; one FMA gives 1.5 2^23 + rint(x'/m) exactly and one integer
+// multiply-add leaves x' - rint(x'/m) m in the low byte (the proof is the residue kernels').  No conversions, no fix-ups.
+__device__ __forceinline__ uint32_t sym_reduce_acc(uint32_t x, const ModConsts c, int extra) {
+    const uint32_t rec = (x + 0x80808080u) ^ 0x80808080u;
+    int y;
+    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(y) : "r"(rec), "r"(c.w), "r"(c.y0 + extra));
+    const int t = __float_as_int(fmaf(__int_as_float(y), c.inv_m, c.cq));
+    return (uint32_t)(t * c.neg_m + y);
 }
 
 // 16 consecutive accumulators of one TMEM lane -> 16 symmetric residues packed into one 16-byte vector.
 // ACC: add the residues already stored at `dst` first (later K chunks, second product of a rank-2k update).
 template <bool ACC>
-__device__ __forceinline__ void reduce_store16(const uint32_t* v, uint4* dst, int m, float inv_m) {
+__device__ __forceinline__ void reduce_store16(const uint32_t* v, uint4* dst, const ModConsts c) {
     uint32_t old[4] = {0, 0, 0, 0};
     if (ACC) { const uint4 o = *dst; old[0] = o.x; old[1] = o.y; old[2] = o.z; old[3] = o.w; }
     uint32_t w[4];
@@ -151,11 +166,7 @@ __device__ __forceinline__ void reduce_store16(const uint32_t* v, uint4* dst, in
     for (int q = 0; q < 4; ++q) {
         uint32_t b[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            int x = (int)v[q * 4 + e];
-            if (ACC) x += (int)(int8_t)(old[q] >> (8 * e));
-            b[e] = (uint32_t)sym_reduce_acc(x, m, inv_m);
-        }
+        for (int e = 0; e < 4; ++e) b[e] = sym_reduce_acc(v[q * 4 + e], c, ACC ? (int)(int8_t)(old[q] >> (8 * e)) : 0);
         w[q] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
     }
     *dst = make_uint4(w[0], w[1], w[2], w[3]);

@@ -147,11 +147,23 @@ double residue_reduction_margin(const ResidueTable& t, int j) {
     return (double)(1LL << e) / (2.0 * (double)(y0 + t.xmax[j]) * (double)dev);
 }
 
+// Epilogue constants of one batch entry: the reduction constants of the residue kernels for this modulus (the bound used
+// there, twelve digits of both parts, covers the four digits of an accumulator plus one stored residue).
+static void fill_mod_entry(ModTable* t, int p, const int* mods, int j) {
+    ResidueTable r;
+    build_residue_table_for(mods, j + 1, 0, &r);
+    t->m[p] = r.m[j];
+    t->inv_m[p] = r.inv_m[j];
+    t->w[p] = r.w_lo[j];
+    t->y0[p] = r.magic[j];
+    t->cq[p] = r.cq[j];
+}
+
 void build_mod_table(int nmod, bool per_plane, ModTable* t) {
     std::memset(t, 0, sizeof(*t));
     const int n2 = count_2m(nmod);
     int p = 0;
-    auto put = [&](int j) { t->m[p] = kModuli[j]; t->inv_m[p] = 1.0f / (float)kModuli[j]; ++p; };
+    auto put = [&](int j) { fill_mod_entry(t, p, kModuli, j); ++p; };
     if (!per_plane) {
         for (int j = 0; j < nmod; ++j) put(j);
     } else {
@@ -165,7 +177,7 @@ void build_mod_table(int nmod, bool per_plane, ModTable* t) {
 
 void build_mod_table_real(int nmod, ModTable* t) {
     std::memset(t, 0, sizeof(*t));
-    for (int j = 0; j < nmod; ++j) { t->m[j] = kRealModuli[j]; t->inv_m[j] = 1.0f / (float)kRealModuli[j]; }
+    for (int j = 0; j < nmod; ++j) fill_mod_entry(t, j, kRealModuli, j);
     t->nplanes = nmod;
 }
 
@@ -264,12 +276,16 @@ ScaleTargets scale_targets_real(int nmod, int64_t k) {
     return s;
 }
 
-int64_t gemm_k_limit_real() { return (int64_t)INT32_MAX / (128 * 128); }   // the modulus 256 comes first
+// The epilogue recodes an accumulator into four balanced base-256 digits, which represents values up to 0x7F7F7F7F; a later
+// K chunk also adds the stored residue (at most 128 in magnitude) before the reduction.
+static constexpr int64_t kAccLimit = 0x7F7F7F7FLL - 128;
+
+int64_t gemm_k_limit_real() { return kAccLimit / (128 * 128); }   // the modulus 256 comes first
 
 int64_t gemm_k_limit(int nmod) {
     // largest |residue|: 120 for the 2M moduli (241 comes first), 128 once the hybrid adds the modulus 256
     const int64_t h = nmod > kMax2M ? 128 : (kModuli[0] - 1) / 2;
-    return (int64_t)INT32_MAX / (h * h);
+    return kAccLimit / (h * h);
 }
 
 }  // namespace gemm2m
