@@ -45,8 +45,8 @@ struct ResidueTable {
 };
 
 // Modulus of every batch entry of a GEMM launch, for the epilogue (reduction of the int32 accumulators).
-// The accumulator's four balanced base-256 digits are contracted with w (one dp4a starting at the bit pattern y0 of the
-// float Y0), then reduced as in the residue kernels: one FMA with cq, one integer multiply-add (see ResidueTable).
+// The four bytes of the accumulator plus 2^31 are contracted with w (one dp4a starting at y0 = the bit pattern of the float
+// Y0 minus sym(2^31 mod m)), then reduced as in the residue kernels: one FMA with cq, one integer multiply-add.
 struct ModTable {
     int32_t m[kMaxPlanes];
     float inv_m[kMaxPlanes];
@@ -100,7 +100,7 @@ void build_mod_table_real(int nmod, ModTable* t);
 void build_crt_table_real(int nmod, CrtTable* t);
 ScaleTargets scale_targets_real(int nmod, int64_t k);
 int64_t gemm_k_limit_real();
-int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 (plus a stored residue) stays below 0x7F7F7F7F
+int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
 
 // ---- phase launchers (prepost.cu) ----
 // Exponent scan: largest |Re|,|Im| bit pattern per row of a column-major matrix (rows x cols, ld).

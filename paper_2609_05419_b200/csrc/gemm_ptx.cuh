@@ -134,7 +134,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // Constants of the epilogue's reduction modulo the modulus of one batch entry (see ModTable).
 struct ModConsts {
     uint32_t w;        // int8 x4: sym(256^b mod m), b = 0..3
-    int y0;            // bit pattern of the float Y0
+    int y0;            // bit pattern of the float Y0, minus sym(2^31 mod m)
     int neg_m;
     float inv_m, cq;
 };
@@ -142,15 +142,15 @@ __device__ __forceinline__ ModConsts load_mod_consts(const ModTable& t, int b) {
     return ModConsts{t.w[b], t.y0[b], -t.m[b], t.inv_m[b], t.cq[b]};
 }
 
-// Symmetric residue of an int32 accumulator x (|x| + 128 <= 0x7F7F7F7F), in the low byte of the result.  The four balanced
-// base-256 digits of x (add 128 to every byte with carries, flip every byte's top bit) are contracted with 256^b mod m by
-// one dp4a that starts at the bit pattern of the float Y0 (plus `extra`, a residue to be added): the sum is the bit
-// pattern of Y0 + x' with x' = x (mod m) and |x'| small; one FMA gives 1.5 2^23 + rint(x'/m) exactly and one integer
-// multiply-add leaves x' - rint(x'/m) m in the low byte (the proof is the residue kernels').  No conversions, no fix-ups.
+// Symmetric residue of an int32 accumulator x, in the low byte of the result.  x + 2^31 (one XOR) is a non-negative 32-bit
+// number whose four unsigned bytes are contracted with 256^b mod m by one dp4a; the accumulation starts at the bit pattern
+// of the float Y0 minus sym(2^31 mod m) (folded into y0 by the table builder) plus `extra`, a residue to be added.  The sum
+// is the bit pattern of Y0 + x' with x' = x (mod m) and |x'| small; one FMA gives 1.5 2^23 + rint(x'/m) exactly and one
+// integer multiply-add leaves x' - rint(x'/m) m in the low byte (the proof is the residue kernels').  No conversions, no
+// fix-ups.
 __device__ __forceinline__ uint32_t sym_reduce_acc(uint32_t x, const ModConsts c, int extra) {
-    const uint32_t rec = (x + 0x80808080u) ^ 0x80808080u;
     int y;
-    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(y) : "r"(rec), "r"(c.w), "r"(c.y0 + extra));
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(y) : "r"(x ^ 0x80000000u), "r"(c.w), "r"(c.y0 + extra));
     const int t = __float_as_int(fmaf(__int_as_float(y), c.inv_m, c.cq));
     return (uint32_t)(t * c.neg_m + y);
 }

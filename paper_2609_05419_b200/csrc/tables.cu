@@ -148,14 +148,15 @@ double residue_reduction_margin(const ResidueTable& t, int j) {
 }
 
 // Epilogue constants of one batch entry: the reduction constants of the residue kernels for this modulus (the bound used
-// there, twelve digits of both parts, covers the four digits of an accumulator plus one stored residue).
+// there, twelve digits of both parts, covers four unsigned bytes, the 2^31 correction and one stored residue).
 static void fill_mod_entry(ModTable* t, int p, const int* mods, int j) {
     ResidueTable r;
     build_residue_table_for(mods, j + 1, 0, &r);
     t->m[p] = r.m[j];
     t->inv_m[p] = r.inv_m[j];
     t->w[p] = r.w_lo[j];
-    t->y0[p] = r.magic[j];
+    // the epilogue contracts the bytes of x + 2^31: take 2^31 mod m out again
+    t->y0[p] = r.magic[j] - sym_mod(1LL << 31, r.m[j]);
     t->cq[p] = r.cq[j];
 }
 
@@ -276,9 +277,8 @@ ScaleTargets scale_targets_real(int nmod, int64_t k) {
     return s;
 }
 
-// The epilogue recodes an accumulator into four balanced base-256 digits, which represents values up to 0x7F7F7F7F; a later
-// K chunk also adds the stored residue (at most 128 in magnitude) before the reduction.
-static constexpr int64_t kAccLimit = 0x7F7F7F7FLL - 128;
+// The accumulators must stay inside int32 (the epilogue works on x + 2^31 as an unsigned 32-bit number).
+static constexpr int64_t kAccLimit = 0x7FFFFFFFLL;
 
 int64_t gemm_k_limit_real() { return kAccLimit / (128 * 128); }   // the modulus 256 comes first
 
