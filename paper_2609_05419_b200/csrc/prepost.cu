@@ -791,6 +791,11 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
 // weighted residues exactly in 40-bit digit columns (FP64 FMAs on integers below 2^53), remove the multiple
 // of M, and round the lifted integer once to floating point before scaling by 2^(e_i + f_j).
 // =====================================================================================================
+// Byte e (0..3) of w as a signed integer: one byte permute that copies the byte and replicates its sign bit.
+__device__ __forceinline__ int sbyte(uint32_t w, int e) {
+    return (int)__byte_perm(w, 0u, 0x8880u + 0x1111u * (uint32_t)e);
+}
+
 __device__ __forceinline__ double int_to_double(int v) {
     // The conversion instruction: one issue slot on a pipe nothing else here uses.  (Building the double from its bit
     // pattern, 2^52 + 2^31 + v minus the constant, took three slots, one of them on the FP64 pipe the FMAs need; measured
@@ -898,8 +903,8 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
         const uint32_t wm = stage[n2 + jm][threadIdx.x];       // c-
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const int cp = (int)(int8_t)(wp >> (8 * e));
-            const int cm = (int)(int8_t)(wm >> (8 * e));
+            const int cp = sbyte(wp, e);
+            const int cm = sbyte(wm, e);
             const double vr = int_to_double(cm + cp);     // Eq. (2c): real part uses C- + C+
             const double vi = int_to_double(cm - cp);     //           imaginary part uses C- - C+
 #pragma unroll
@@ -916,7 +921,7 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
         const uint32_t w3 = stage[2 * n2 + 2 * n3 + j3][threadIdx.x];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const int p1 = (int)(int8_t)(w1 >> (8 * e)), p2 = (int)(int8_t)(w2 >> (8 * e)), p3 = (int)(int8_t)(w3 >> (8 * e));
+            const int p1 = sbyte(w1, e), p2 = sbyte(w2, e), p3 = sbyte(w3, e);
             const double vr = int_to_double(p1 - p2);
             const double vi = int_to_double(p3 - p1 - p2);
 #pragma unroll
@@ -1031,7 +1036,7 @@ __global__ void __launch_bounds__(kPostThreads) post_real_kernel(const int8_t* _
         const uint32_t w = stage[jm][threadIdx.x];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const double v = int_to_double((int)(int8_t)(w >> (8 * e)));
+            const double v = int_to_double(sbyte(w, e));
 #pragma unroll
             for (int c = 0; c < NCH; ++c) S[e][c] = fma(v, tab.gr[jm][c], S[e][c]);
         }
@@ -1153,7 +1158,7 @@ __global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* _
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int ii = 4 * g + e;
-            const int cpv = (int)(int8_t)(wp >> (8 * e));
+            const int cpv = sbyte(wp, e);
             const int cmv = (int)(int8_t)base[kHerkJ * kHerkI + (ii + (ii >> 3)) * 16 + jj];    // C-[i, j] = C+[j, i]
             const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
 #pragma unroll
