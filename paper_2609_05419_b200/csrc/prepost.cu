@@ -793,7 +793,9 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
 // =====================================================================================================
 // Byte e (0..3) of w as a signed integer: one byte permute that copies the byte and replicates its sign bit.
 __device__ __forceinline__ int sbyte(uint32_t w, int e) {
-    return (int)__byte_perm(w, 0u, 0x8880u + 0x1111u * (uint32_t)e);
+    uint32_t r;       // selector nibble = byte index, + 8 to replicate that byte's sign bit (the __byte_perm intrinsic masks that bit off)
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(w), "r"(0u), "r"(0x8880u + 0x1111u * (uint32_t)e));
+    return (int)r;
 }
 
 __device__ __forceinline__ double int_to_double(int v) {
