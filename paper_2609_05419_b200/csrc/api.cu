@@ -503,18 +503,40 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     ga.out = cp; ga.ldp = c.ldp;
     build_mod_table(nmod, false, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
-    ga.row_begin = 0; ga.row_end = n;
-    CK(ph.begin(2, st));
-    ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
-    if (int s = run_gemm(ga, nmod, st)) return s;
-    if (two) {
-        ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
+    // The output is cut into row panels: entry (i, j) of the lower triangle needs C+[i, j] and C+[j, i], i.e. the GEMM output
+    // rows j and i <= the end of i's panel, so the post-processing of the rows of panel p can run on the library's stream
+    // beside the GEMMs of panel p + 1 (the last, largest panel stays on the caller's stream).
+    int panels = (int)(n / 1024);
+    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
+    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
+    const int64_t panel_rows = round_up((n + panels - 1) / panels, 256);
+    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
+    for (int pnl = 0; pnl < panels; ++pnl) {
+        const int64_t r0 = pnl * panel_rows, r1 = (r0 + panel_rows < n) ? r0 + panel_rows : n;
+        if (r0 >= r1) break;
+        ga.row_begin = r0; ga.row_end = r1;
+        CK(ph.begin(2, st));
+        ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
         if (int s = run_gemm(ga, nmod, st)) return s;
+        if (two) {
+            ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
+            if (int s = run_gemm(ga, nmod, st)) return s;
+        }
+        CK(ph.end(st));
+        const bool last = r1 >= n;
+        cudaStream_t ps = last ? st : D().side;
+        if (!last) {
+            CK(cudaEventRecord(D().panel_done[pnl], st));
+            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
+        }
+        CK(ph.begin(3, ps));
+        CK(launch_post_herk(cp, c.ldp, n, r0, r1, eA, ctab, C, ldc, real_in, ps, &g.launches[3]));
+        CK(ph.end(ps));
     }
-    CK(ph.end(st));
-    CK(ph.begin(3, st));
-    CK(launch_post_herk(cp, c.ldp, n, eA, ctab, C, ldc, real_in, st, &g.launches[3]));
-    CK(ph.end(st));
+    if (panels > 1) {
+        CK(cudaEventRecord(D().side_done, D().side));
+        CK(cudaStreamWaitEvent(st, D().side_done, 0));
+    }
     ph.done();
     return GEMM2M_OK;
 }

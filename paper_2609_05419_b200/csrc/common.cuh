@@ -136,8 +136,9 @@ cudaError_t launch_post_real(const int8_t* cp, int64_t ldp, int64_t m, int64_t n
 // C = beta C (the alpha = 0 case of the extended interface); beta = host pointer to (re, im) or null for 0.
 template <typename T> cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches);
 // real_out: C is a real matrix (SYRK / SYR2K through Z = A1 + i A2): only the real part is formed and stored.
-cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
-                             bool real_out, cudaStream_t st, int* launches);
+// Rows [i_begin, i_end) of the lower triangle only (i_begin a multiple of 64): they need the GEMM output rows below i_end.
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const CrtTable& tab,
+                             double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches);
 // Z[i, p] = X[i, p] + i X[i, p + k2] for p < k2 = ceil(k / 2) (zero beyond column k): the complex matrix whose HERK is the SYRK of X.
 cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_t k, double* Z, cudaStream_t st, int* launches);
 cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,

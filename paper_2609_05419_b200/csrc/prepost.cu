@@ -1120,11 +1120,11 @@ constexpr int kHerkMirrorSlots = kHerkI + kHerkI / 8;                      // 16
 constexpr int kHerkPlaneBytes = kHerkJ * kHerkI + kHerkMirrorSlots * 16;   // direct + mirrored bytes per modulus
 
 template <int NCH, bool REAL_OUT>
-__global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n,
+__global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n, int64_t i_begin,
                                                                  const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
                                                                  double* __restrict__ C, int64_t ldc) {
     extern __shared__ __align__(16) unsigned char herk_smem[];
-    const int64_t ibase = (int64_t)blockIdx.x * kHerkI, jbase = (int64_t)blockIdx.y * kHerkJ;
+    const int64_t ibase = i_begin + (int64_t)blockIdx.x * kHerkI, jbase = (int64_t)blockIdx.y * kHerkJ;
     if (ibase + kHerkI - 1 < jbase) return;                                // tile entirely above the diagonal
     const int nmod = tab.nmod;
     const int64_t plane = n * ldp;
@@ -1217,8 +1217,8 @@ cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_
 }
 
 template <bool REAL_OUT>
-static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
-                                      cudaStream_t st, int* launches) {
+static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA,
+                                      const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
     const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
     static bool attr_set = false;
     if (!attr_set) {
@@ -1230,24 +1230,24 @@ static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, 
         attr_set = true;
     }
     const size_t use = (size_t)tab.nmod * kHerkPlaneBytes;
-    const int64_t tiles_j = (n + kHerkJ - 1) / kHerkJ;
+    const int64_t tiles_j = (i_end + kHerkJ - 1) / kHerkJ;  // lower triangle: columns up to the last row of the range
     if (tiles_j > 65535) return cudaErrorInvalidValue;     // n beyond 65535 * 16 columns: far beyond any workspace
-    dim3 grid((unsigned)((n + kHerkI - 1) / kHerkI), (unsigned)tiles_j);
+    dim3 grid((unsigned)((i_end - i_begin + kHerkI - 1) / kHerkI), (unsigned)tiles_j);
     switch (tab.nchunks) {
-        case 1: post_herk_kernel<1, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        case 2: post_herk_kernel<2, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        case 3: post_herk_kernel<3, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
-        default: post_herk_kernel<4, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, eA, tab, C, ldc); break;
+        case 1: post_herk_kernel<1, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        case 2: post_herk_kernel<2, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        case 3: post_herk_kernel<3, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        default: post_herk_kernel<4, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
     }
     ++*launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, const int32_t* eA, const CrtTable& tab, double* C, int64_t ldc,
-                             bool real_out, cudaStream_t st, int* launches) {
-    if (n <= 0) return cudaSuccess;
-    return real_out ? launch_post_herk_t<true>(cp, ldp, n, eA, tab, C, ldc, st, launches)
-                    : launch_post_herk_t<false>(cp, ldp, n, eA, tab, C, ldc, st, launches);
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const CrtTable& tab,
+                             double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches) {
+    if (n <= 0 || i_end <= i_begin) return cudaSuccess;
+    return real_out ? launch_post_herk_t<true>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches)
+                    : launch_post_herk_t<false>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches);
 }
 
 // Exact integer variant for gemm2m_gaussian_int: X = sum_j sym(v_j g_j mod m_j) (M/m_j) mod M in int64 (M < 2^62).

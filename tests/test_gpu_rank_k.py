@@ -112,3 +112,44 @@ def test_rank_k_at_size_sampled():
     Cs, Ds = direct.zgemm4m_dd_samples(Az, np.asfortranarray(Az.T), pairs)
     assert direct.componentwise_error(Ch[pairs[:, 0], pairs[:, 1]], Cs.real, Ds) <= TOL
     assert (np.triu(Ch, 1)[np.triu(np.ones((n, n), dtype=bool), 1)] == -5.0).all()
+
+
+def test_rank_k_row_panels_are_bitwise_identical():
+    """The rank-k family cuts the output into row panels and post-processes panel p beside the GEMMs of panel p + 1: the
+    result must not depend on the number of panels, the upper triangle stays untouched, and work queued on the caller's
+    stream right after the call sees the whole result."""
+    n, k, nmod = 2304, 96, 16                      # 2304 rows -> 2 panels of 1280 / 1024
+    A = inputs.herk_input(n, k, seed=51, dist="phi", phi=1.0)
+    B = inputs.herk_input(n, k, seed=52, dist="phi", phi=1.0)
+    X = real_input(n, k, seed=53)
+    dA, dB, dX = to_dev(A), to_dev(B), to_dev(X)
+    results = {}
+    try:
+        with Workspace(max(b.workspace_bytes(b.OP_ZHER2K, n, n, k, nmod), b.workspace_bytes(b.OP_DSYRK, n, n, k, nmod))):
+            for panels in (1, 8):
+                b.debug_set_panels(panels)
+                C1 = empty_dev(n, n, torch.complex128, fill=-5.0)
+                C2 = empty_dev(n, n, torch.complex128, fill=-5.0)
+                C3 = empty_dev(n, n, torch.float64, fill=-5.0)
+                b.zherk2m(dA, C1, nmod)
+                snap = C1.clone()                  # same stream, no synchronisation in between
+                if panels == 8:
+                    assert b.last_launch_count()[1][2:] == [2, 2]      # one GEMM and one post launch per panel
+                b.zher2k2m(dA, dB, C2, nmod)
+                b.dsyrk2m(dX, C3, nmod)
+                b.device_status()
+                assert (to_host(snap) == to_host(C1)).all()
+                results[panels] = (to_host(C1), to_host(C2), to_host(C3))
+    finally:
+        b.debug_set_panels(8)
+    for a, c in zip(results[1], results[8]):
+        assert (a == c).all()
+    C1, C2, C3 = results[8]
+    iu = np.triu_indices(n, 1)
+    assert (C1[iu] == -5.0).all() and (C2[iu] == -5.0).all() and (C3[iu] == -5.0).all()
+    il = np.tril_indices(n)
+    pairs = np.stack([il[0], il[1]], axis=1)[:: 997]                            # a sample of the lower triangle, all panels
+    Cs, Ds = direct.zgemm4m_dd_samples(A, A.conj().T, pairs)
+    assert direct.componentwise_error(C1[pairs[:, 0], pairs[:, 1]], Cs, Ds) <= TOL
+    Cs, Ds = direct.zgemm4m_dd_samples(X.astype(np.complex128), X.T.astype(np.complex128), pairs)
+    assert direct.componentwise_error(C3[pairs[:, 0], pairs[:, 1]] + 0j, Cs, Ds) <= TOL
