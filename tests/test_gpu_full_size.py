@@ -87,3 +87,62 @@ def test_zherk_8192_sampled():
     AH = np.asfortranarray(A.conj().T)
     Cs, Ds = direct.zgemm4m_dd_samples(A, AH, pairs)
     assert direct.componentwise_error(got, Cs, Ds) <= 1e-14
+
+
+def test_extensions_4096_sampled():
+    """The later entry points at a size that spans many tiles, panels and waves: hybrid moduli, transposed / conjugated
+    operands with alpha and beta, the 2-norm scaling rule and the real scheme, each on sampled entries against the
+    double-double definition (and, for the hybrid, against the exact staged integers)."""
+    m = n = k = 4096
+    A, B = inputs.complex_inputs(m, n, k, seed=5, dist="phi", phi=2.0)
+    pairs = inputs.sample_indices(m, n, 2048, seed=6, tile=128)
+    idx = torch.from_numpy(pairs).cuda()
+    Cs, Ds = direct.zgemm4m_dd_samples(A, B, pairs)
+    dA, dB = to_dev(A), to_dev(B)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, 24)):
+        C = empty_dev(m, n, torch.complex128)
+        # hybrid 2M/3M, 24 moduli: 50 planes per operand
+        b.zgemm2m(dA, dB, C, 24)
+        b.device_status()
+        got = C[idx[:, 0], idx[:, 1]].cpu().numpy()
+        assert direct.componentwise_error(got, Cs, Ds) <= 1e-14
+        sub = pairs[:128]
+        rows, ri = np.unique(sub[:, 0], return_inverse=True)
+        cols, ci = np.unique(sub[:, 1], return_inverse=True)
+        st = staged.zgemm2m_staged(A[rows, :], B[:, cols], 24, upto="pre")
+        _, vals = staged.staged_samples(st, np.stack([ri, ci], axis=1))
+        g = got[:128]
+        assert ulp_distance(g.real, vals.real).max() <= 1 and ulp_distance(g.imag, vals.imag).max() <= 1
+        # C = alpha A^H^H B^T^T + beta C with the operands stored conjugate-transposed / transposed
+        alpha, beta = 0.5 - 2.0j, 1.5 + 0.25j
+        C0 = C.clone()
+        c0 = C0[idx[:, 0], idx[:, 1]].cpu().numpy()
+        dAh = to_dev(np.asfortranarray(A.conj().T))
+        dBt = to_dev(np.asfortranarray(B.T))
+        b.zgemm2m_ex("C", "T", alpha, dAh, dBt, beta, C, 18)
+        b.device_status()
+        got = C[idx[:, 0], idx[:, 1]].cpu().numpy()
+        want = alpha * Cs.astype(np.clongdouble) + beta * c0.astype(np.clongdouble)
+        scale = abs(alpha) * Ds + abs(beta) * np.abs(c0)
+        assert (np.abs(got - want.astype(np.complex128)) <= 1e-14 * scale).all()
+        # 2-norm scaling rule: 16 moduli reach 1e-14 for this exponent spread, where the max-based rule needs 18
+        b.set_scaling(1)
+        try:
+            b.zgemm2m(dA, dB, C, 16)
+            b.device_status()
+        finally:
+            b.set_scaling(0)
+        e2 = direct.componentwise_error(C[idx[:, 0], idx[:, 1]].cpu().numpy(), Cs, Ds)
+        b.zgemm2m(dA, dB, C, 16)
+        b.device_status()
+        e0 = direct.componentwise_error(C[idx[:, 0], idx[:, 1]].cpu().numpy(), Cs, Ds)
+        assert e2 < e0 and e2 <= 1e-14
+    # real Ozaki-II scheme
+    Ar, Br = np.asfortranarray(A.real.copy()), np.asfortranarray(B.real.copy())
+    with Workspace(b.workspace_bytes(b.OP_DGEMM_OZAKI2, m, n, k, 17)):
+        Cr = empty_dev(m, n, torch.float64)
+        b.dgemm_ozaki2(to_dev(Ar), to_dev(Br), Cr, 17)
+        b.device_status()
+        got = Cr[idx[:, 0], idx[:, 1]].cpu().numpy()
+    Cd, Dd = direct.zgemm4m_dd_samples(Ar.astype(np.complex128), Br.astype(np.complex128), pairs)
+    assert direct.componentwise_error(got + 0j, Cd, Dd) <= 1e-14
