@@ -102,7 +102,7 @@ ScaleTargets scale_targets_real(int nmod, int64_t k);
 int64_t gemm_k_limit_real();
 int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
 
-// ---- phase launchers (prepost.cu) ----
+// ---- phase launchers (scan.cu, residues.cu, post.cu) ----
 // Exponent scan: largest |Re|,|Im| bit pattern per row of a column-major matrix (rows x cols, ld).
 template <typename T> cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches);
 // The same per column.

@@ -1,0 +1,516 @@
+// Algorithm 1 steps 4 (Eq. 2c), 5, 6, 7: post-processing of the residue planes of the products (complex GEMM, rank-k family,
+// real scheme, exact int64 result), plus the small packing and scaling kernels of the rank-k and extended interfaces.
+#include "prepost_common.cuh"
+
+namespace gemm2m {
+
+// =====================================================================================================
+// Steps 4 (Eq. 2c), 5, 6, 7: per output element, fold the 2M post-processing into the CRT weights, sum the
+// weighted residues exactly in 40-bit digit columns (FP64 FMAs on integers below 2^53), remove the multiple
+// of M, and round the lifted integer once to floating point before scaling by 2^(e_i + f_j).
+// =====================================================================================================
+// Byte e (0..3) of w as a signed integer: one byte permute that copies the byte and replicates its sign bit.
+__device__ __forceinline__ int sbyte(uint32_t w, int e) {
+    uint32_t r;       // selector nibble = byte index, + 8 to replicate that byte's sign bit (the __byte_perm intrinsic masks that bit off)
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(w), "r"(0u), "r"(0x8880u + 0x1111u * (uint32_t)e));
+    return (int)r;
+}
+
+__device__ __forceinline__ double int_to_double(int v) {
+    // The conversion instruction: one issue slot on a pipe nothing else here uses.  (Building the double from its bit
+    // pattern, 2^52 + 2^31 + v minus the constant, took three slots, one of them on the FP64 pipe the FMAs need; measured
+    // 7 % slower for the whole kernel.)
+    return (double)v;
+}
+
+// Lifted X (exact integer, |X| <= (M-1)/2) from the digit-column sums S[c], returned as an unevaluated sum hi + lo with
+// |lo| <= ulp(hi)/2.  The weighted sum X' = sum_c S[c] 2^(40c) is X + t M with |t| < 2^12; |X/M| stays below 0.494 by the
+// scaling rule, so rounding X'/M (from the two leading sums; the rest is below 2^-60 M) gives t exactly.
+template <int NCH>
+__device__ __forceinline__ void crt_finish(double (&S)[NCH], const CrtTable& tab, double* hi, double* lo) {
+    const double t = rint(NCH > 1 ? fma(S[NCH - 1], tab.q_hi, S[NCH > 1 ? NCH - 2 : 0] * tab.q_lo) : S[0] * tab.q_hi);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) S[c] = fma(-t, tab.Mc[c], S[c]);          // exact: |t| < 2^12, digits < 2^40
+    const double two40 = 1099511627776.0, inv40 = 1.0 / 1099511627776.0;
+#pragma unroll
+    for (int c = 0; c + 1 < NCH; ++c) {                                     // carry into canonical digits [0, 2^40)
+        const double carry = floor(S[c] * inv40);
+        S[c] = fma(-carry, two40, S[c]);
+        S[c + 1] += carry;
+    }
+    double h = S[NCH - 1], l = 0.0;                                          // top digit keeps the sign
+#pragma unroll
+    for (int c = NCH - 2; c >= 0; --c) {
+        h *= two40;
+        l *= two40;
+        const double s = h + S[c];                                           // TwoSum
+        const double bb = s - h;
+        const double err = (h - (s - bb)) + (S[c] - bb);
+        h = s;
+        l += err;
+    }
+    *hi = h;
+    *lo = l;
+}
+
+__device__ __forceinline__ double scale_pow2(double x, int e) {   // x 2^e with e split so that both factors are normal
+    const int e1 = max(-1000, min(1000, e));
+    const int e2 = max(-1000, min(1000, e - e1));
+    const int e3 = e - e1 - e2;
+    double y = x * __longlong_as_double((long long)(e1 + 1023) << 52);
+    if (e2) y *= __longlong_as_double((long long)(e2 + 1023) << 52);
+    if (e3) y = ldexp(y, e3);
+    return y;
+}
+
+template <typename T> __device__ __forceinline__ void store4(T* dst, const double (&re)[4], const double (&im)[4], int count);
+template <> __device__ __forceinline__ void store4<double>(double* dst, const double (&re)[4], const double (&im)[4], int count) {
+    for (int i = 0; i < count; ++i) *reinterpret_cast<double2*>(dst + 2 * i) = make_double2(re[i], im[i]);
+}
+template <> __device__ __forceinline__ void store4<float>(float* dst, const double (&re)[4], const double (&im)[4], int count) {
+    if (count == 4 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        *reinterpret_cast<float4*>(dst) = make_float4((float)re[0], (float)im[0], (float)re[1], (float)im[1]);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4((float)re[2], (float)im[2], (float)re[3], (float)im[3]);
+    } else {
+        for (int i = 0; i < count; ++i) *reinterpret_cast<float2*>(dst + 2 * i) = make_float2((float)re[i], (float)im[i]);
+    }
+}
+
+constexpr int kPostThreads = 128;
+constexpr int kPostSpan = kPostThreads * 4;   // consecutive row indices i handled by one block
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// cpm: [planes][n][ldp] int8 (row index i contiguous), planes = C+ and C- of the 2M moduli, then P1, P2, P3 of the 3M
+// moduli.  A block handles 512 consecutive i of one column j: it first pulls the planes x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
+// thread combines 4 consecutive i.
+// AXPBY: C = alpha X + beta C (alpha, beta complex, given as re/im pairs) instead of C = X; the product X is formed
+// exactly as before, then combined in FP64 with fused multiply-adds.  beta = 0 does not read C.
+struct PostScalars { double ar, ai, br, bi; };
+
+template <typename T, int NCH, bool AXPBY>
+__global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
+                                                               const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
+                                                               const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc,
+                                                               const PostScalars sc) {
+    __shared__ __align__(16) uint32_t stage[kMaxPlanes][kPostThreads];
+    const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
+    const int64_t j = blockIdx.y;
+    const int nmod = tab.nmod, n2 = tab.n2, n3 = nmod - n2;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cpm + j * ldp + ib;
+    const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);   // ldp is a multiple of 16
+    for (int idx = threadIdx.x; idx < (2 * n2 + 3 * n3) * (kPostSpan / 16); idx += kPostThreads) {
+        const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
+        if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    const int64_t i0 = ib + 4 * threadIdx.x;
+    if (i0 >= m) return;
+    double Sr[4][NCH], Si[4][NCH];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
+    }
+#pragma unroll 2
+    for (int jm = 0; jm < n2; ++jm) {
+        const uint32_t wp = stage[jm][threadIdx.x];            // c+ of 4 elements
+        const uint32_t wm = stage[n2 + jm][threadIdx.x];       // c-
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int cp = sbyte(wp, e);
+            const int cm = sbyte(wm, e);
+            const double vr = int_to_double(cm + cp);     // Eq. (2c): real part uses C- + C+
+            const double vi = int_to_double(cm - cp);     //           imaginary part uses C- - C+
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
+                Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
+            }
+        }
+    }
+#pragma unroll 1
+    for (int j3 = 0; j3 < n3; ++j3) {                      // 3M moduli of the hybrid, Eq. (1)
+        const uint32_t w1 = stage[2 * n2 + j3][threadIdx.x];
+        const uint32_t w2 = stage[2 * n2 + n3 + j3][threadIdx.x];
+        const uint32_t w3 = stage[2 * n2 + 2 * n3 + j3][threadIdx.x];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int p1 = sbyte(w1, e), p2 = sbyte(w2, e), p3 = sbyte(w3, e);
+            const double vr = int_to_double(p1 - p2);
+            const double vi = int_to_double(p3 - p1 - p2);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[e][c] = fma(vr, tab.gr[n2 + j3][c], Sr[e][c]);
+                Si[e][c] = fma(vi, tab.gr[n2 + j3][c], Si[e][c]);
+            }
+        }
+    }
+    const int fb = __ldg(eB + j);
+    double re[4], im[4];
+    int count = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        if (i0 + e < m) {
+            ++count;
+            const int ea = __ldg(eA + i0 + e);
+            if (ea == kExpNonFinite || fb == kExpNonFinite) {
+                re[e] = im[e] = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(Sr[e], tab, &h, &l);
+                re[e] = scale_pow2(h + l, ea + fb);
+                crt_finish<NCH>(Si[e], tab, &h, &l);
+                im[e] = scale_pow2(h + l, ea + fb);
+            }
+        }
+    }
+    if (AXPBY) {
+        const bool use_c = sc.br != 0.0 || sc.bi != 0.0;
+        for (int e = 0; e < count; ++e) {
+            const double xr = re[e], xi = im[e];
+            double yr = fma(sc.ar, xr, -sc.ai * xi), yi = fma(sc.ar, xi, sc.ai * xr);
+            if (use_c) {
+                const T* old = C + 2 * (i0 + e + j * ldc);
+                const double cr = (double)old[0], ci = (double)old[1];
+                yr += fma(sc.br, cr, -sc.bi * ci);
+                yi += fma(sc.br, ci, sc.bi * cr);
+            }
+            re[e] = yr;
+            im[e] = yi;
+        }
+    }
+    store4<T>(C + 2 * (i0 + j * ldc), re, im, count);
+}
+
+template <typename T, bool AXPBY>
+static cudaError_t launch_post_fp_t(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                                    const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const PostScalars& sc, cudaStream_t st,
+                                    int* launches) {
+    const int64_t per_block = kPostSpan;
+    for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {      // grid.y limit
+        const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
+        dim3 grid((unsigned)((m + per_block - 1) / per_block), (unsigned)nj);
+        const int8_t* src = cpm + j0 * ldp;
+        T* dst = C + 2 * j0 * ldc;
+        // the plane stride is n * ldp for the whole matrix, so pass the full n and offset pointers
+        switch (tab.nchunks) {
+            case 1: post_fp_kernel<T, 1, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 2: post_fp_kernel<T, 2, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 3: post_fp_kernel<T, 3, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            case 4: post_fp_kernel<T, 4, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+            default: post_fp_kernel<T, 5, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
+        }
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                           const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta,
+                           cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+    PostScalars sc{1.0, 0.0, 0.0, 0.0};
+    if (alpha) { sc.ar = alpha[0]; sc.ai = alpha[1]; }
+    if (beta) { sc.br = beta[0]; sc.bi = beta[1]; }
+    const bool plain = sc.ar == 1.0 && sc.ai == 0.0 && sc.br == 0.0 && sc.bi == 0.0;
+    if (plain) return launch_post_fp_t<T, false>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
+    return launch_post_fp_t<T, true>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
+}
+
+// Real Ozaki-II scheme (Section 3.1): cp: [nmod][n][ldp] int8, one plane per modulus; X = sum_j c_j G_j (mod M) with
+// G_j = sym(q_j)(M/m_j) in tab.gr; real double output.  Same staging and finish as post_fp_kernel.
+template <int NCH>
+__global__ void __launch_bounds__(kPostThreads) post_real_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t m, int64_t n,
+                                                                 const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
+                                                                 const __grid_constant__ CrtTable tab, double* __restrict__ C, int64_t ldc) {
+    __shared__ __align__(16) uint32_t stage[kMaxMod][kPostThreads];
+    const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
+    const int64_t j = blockIdx.y;
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cp + j * ldp + ib;
+    const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);
+    for (int idx = threadIdx.x; idx < nmod * (kPostSpan / 16); idx += kPostThreads) {
+        const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
+        if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    const int64_t i0 = ib + 4 * threadIdx.x;
+    if (i0 >= m) return;
+    double S[4][NCH];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) S[e][c] = 0.0;
+    }
+#pragma unroll 2
+    for (int jm = 0; jm < nmod; ++jm) {
+        const uint32_t w = stage[jm][threadIdx.x];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const double v = int_to_double(sbyte(w, e));
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) S[e][c] = fma(v, tab.gr[jm][c], S[e][c]);
+        }
+    }
+    const int fb = __ldg(eB + j);
+    for (int e = 0; e < 4; ++e) {
+        if (i0 + e < m) {
+            const int ea = __ldg(eA + i0 + e);
+            double out;
+            if (ea == kExpNonFinite || fb == kExpNonFinite) {
+                out = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(S[e], tab, &h, &l);
+                out = scale_pow2(h + l, ea + fb);
+            }
+            C[i0 + e + j * ldc] = out;
+        }
+    }
+}
+
+cudaError_t launch_post_real(const int8_t* cp, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                             const int32_t* eB, const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+    for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {
+        const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
+        dim3 grid((unsigned)((m + kPostSpan - 1) / kPostSpan), (unsigned)nj);
+        const int8_t* src = cp + j0 * ldp;
+        double* dst = C + j0 * ldc;
+        switch (tab.nchunks) {
+            case 1: post_real_kernel<1><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 2: post_real_kernel<2><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            case 3: post_real_kernel<3><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+            default: post_real_kernel<4><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc); break;
+        }
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+// C = beta C (C = 0 for beta = 0, without reading C): the alpha = 0 case of the extended interface.
+template <typename T>
+__global__ void __launch_bounds__(256) scale_c_kernel(T* __restrict__ C, int64_t m, int64_t n, int64_t ldc, double br, double bi) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x, j = blockIdx.y;
+    if (i >= m) return;
+    T* c = C + 2 * (i + j * ldc);
+    double yr = 0.0, yi = 0.0;
+    if (br != 0.0 || bi != 0.0) {
+        const double cr = (double)c[0], ci = (double)c[1];
+        yr = fma(br, cr, -bi * ci);
+        yi = fma(br, ci, bi * cr);
+    }
+    c[0] = (T)yr;
+    c[1] = (T)yi;
+}
+
+template <typename T>
+cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches) {
+    if (m <= 0 || n <= 0) return cudaSuccess;
+    const double br = beta ? beta[0] : 0.0, bi = beta ? beta[1] : 0.0;
+    for (int64_t j0 = 0; j0 < n; j0 += 65535) {
+        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+        dim3 grid((unsigned)((m + 255) / 256), (unsigned)nj);
+        scale_c_kernel<T><<<grid, 256, 0, st>>>(C + 2 * j0 * ldc, m, nj, ldc, br, bi);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+template cudaError_t launch_scale_c<double>(double*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
+template cudaError_t launch_scale_c<float>(float*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
+
+// HERK (Section 5): only C+ = A+ A-^T was computed; C- = C+^T.  cp: [nmod][n][ldp] with cp[j][col][row] = C+_j[row, col].
+// A block handles 64 rows i x 16 columns j of the lower triangle.  It needs C+[i, j] (rows of cp along i: 16 runs of 64
+// bytes per modulus) and C-[i, j] = C+[j, i] (rows of cp along j: 64 runs of 16 bytes per modulus); both are pulled into
+// shared memory with asynchronous 16-byte copies, then each thread combines 4 consecutive i of one column.
+// Lower triangle only; on the diagonal C- - C+ = 0, so the imaginary part is exactly zero.
+constexpr int kHerkI = 64, kHerkJ = 16, kHerkThreads = 256;
+constexpr int kHerkMirrorSlots = kHerkI + kHerkI / 8;                      // 16-byte slots, one pad slot per 8 rows (bank spread)
+constexpr int kHerkPlaneBytes = kHerkJ * kHerkI + kHerkMirrorSlots * 16;   // direct + mirrored bytes per modulus
+
+template <int NCH, bool REAL_OUT>
+__global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n, int64_t i_begin,
+                                                                 const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
+                                                                 double* __restrict__ C, int64_t ldc) {
+    extern __shared__ __align__(16) unsigned char herk_smem[];
+    const int64_t ibase = i_begin + (int64_t)blockIdx.x * kHerkI, jbase = (int64_t)blockIdx.y * kHerkJ;
+    if (ibase + kHerkI - 1 < jbase) return;                                // tile entirely above the diagonal
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int t = threadIdx.x;
+    // direct part: for each modulus and each column j of the tile, 64 bytes along i (4 copies of 16 bytes)
+    for (int idx = t; idx < nmod * kHerkJ * (kHerkI / 16); idx += kHerkThreads) {
+        const int v = idx & 3, jj = (idx >> 2) & (kHerkJ - 1), jm = idx / (kHerkJ * 4);
+        const int64_t i = ibase + 16 * v, j = jbase + jj;
+        if (j < n && i < ldp) cp_async16(herk_smem + jm * kHerkPlaneBytes + jj * kHerkI + 16 * v, cp + (int64_t)jm * plane + j * ldp + i);
+    }
+    // mirrored part: for each modulus and each row i of the tile, the 16 bytes C+[jbase .. jbase+15, i]
+    for (int idx = t; idx < nmod * kHerkI; idx += kHerkThreads) {
+        const int ii = idx & (kHerkI - 1), jm = idx / kHerkI;
+        const int64_t i = ibase + ii;
+        if (i < n && jbase < ldp)
+            cp_async16(herk_smem + jm * kHerkPlaneBytes + kHerkJ * kHerkI + (ii + (ii >> 3)) * 16, cp + (int64_t)jm * plane + i * ldp + jbase);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    const int g = t & 15, jj = t >> 4;                                     // 4 consecutive rows i0 .. i0+3 of column j
+    const int64_t i0 = ibase + 4 * g, j = jbase + jj;
+    if (j >= n || i0 >= n || i0 + 3 < j) return;
+    double Sr[4][NCH], Si[4][NCH];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
+    }
+#pragma unroll 2
+    for (int jm = 0; jm < nmod; ++jm) {
+        const unsigned char* base = herk_smem + jm * kHerkPlaneBytes;
+        const uint32_t wp = *reinterpret_cast<const uint32_t*>(base + jj * kHerkI + 4 * g);      // C+[i0..i0+3, j]
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int ii = 4 * g + e;
+            const int cpv = sbyte(wp, e);
+            const int cmv = (int)(int8_t)base[kHerkJ * kHerkI + (ii + (ii >> 3)) * 16 + jj];    // C-[i, j] = C+[j, i]
+            const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
+                if (!REAL_OUT) Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
+            }
+        }
+    }
+    const int ej = __ldg(eA + j);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int64_t i = i0 + e;
+        if (i < n && i >= j) {
+            const int ei = __ldg(eA + i);
+            double re, im = 0.0;
+            if (ei == kExpNonFinite || ej == kExpNonFinite) {
+                re = im = __longlong_as_double(0x7FF8000000000000ll);
+            } else {
+                double h, l;
+                crt_finish<NCH>(Sr[e], tab, &h, &l);
+                re = scale_pow2(h + l, ei + ej);
+                if (!REAL_OUT) {
+                    crt_finish<NCH>(Si[e], tab, &h, &l);
+                    im = scale_pow2(h + l, ei + ej);
+                }
+            }
+            if (REAL_OUT) C[i + j * ldc] = re;
+            else *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) pack_real_pair_kernel(const double* __restrict__ X, int64_t ld, int64_t n, int64_t k, int64_t k2,
+                                                             double* __restrict__ Z) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t p = blockIdx.y;
+    if (i >= n) return;
+    const double re = __ldg(X + i + p * ld);
+    const double im = (p + k2 < k) ? __ldg(X + i + (p + k2) * ld) : 0.0;
+    *reinterpret_cast<double2*>(Z + 2 * (i + p * n)) = make_double2(re, im);
+}
+
+cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_t k, double* Z, cudaStream_t st, int* launches) {
+    const int64_t k2 = (k + 1) / 2;
+    if (n <= 0 || k2 <= 0) return cudaSuccess;
+    for (int64_t p0 = 0; p0 < k2; p0 += 65535) {      // grid.y limit
+        const int64_t np = (k2 - p0 < 65535) ? k2 - p0 : 65535;
+        dim3 grid((unsigned)((n + 255) / 256), (unsigned)np);
+        pack_real_pair_kernel<<<grid, 256, 0, st>>>(X + p0 * ld, ld, n, k - p0, k2, Z + 2 * p0 * n);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+template <bool REAL_OUT>
+static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA,
+                                      const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
+    const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<3, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<4, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
+    }
+    const size_t use = (size_t)tab.nmod * kHerkPlaneBytes;
+    const int64_t tiles_j = (i_end + kHerkJ - 1) / kHerkJ;  // lower triangle: columns up to the last row of the range
+    if (tiles_j > 65535) return cudaErrorInvalidValue;     // n beyond 65535 * 16 columns: far beyond any workspace
+    dim3 grid((unsigned)((i_end - i_begin + kHerkI - 1) / kHerkI), (unsigned)tiles_j);
+    switch (tab.nchunks) {
+        case 1: post_herk_kernel<1, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        case 2: post_herk_kernel<2, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        case 3: post_herk_kernel<3, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+        default: post_herk_kernel<4, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const CrtTable& tab,
+                             double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches) {
+    if (n <= 0 || i_end <= i_begin) return cudaSuccess;
+    return real_out ? launch_post_herk_t<true>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches)
+                    : launch_post_herk_t<false>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches);
+}
+
+// Exact integer variant for gemm2m_gaussian_int: X = sum_j sym(v_j g_j mod m_j) (M/m_j) mod M in int64 (M < 2^62).
+__global__ void __launch_bounds__(256) post_int_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
+                                                       const __grid_constant__ CrtTableInt tab, int64_t* __restrict__ Cr,
+                                                       int64_t* __restrict__ Ci, int64_t ldc) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t j = blockIdx.y;
+    if (i >= m) return;
+    const int nmod = tab.nmod;
+    const int64_t plane = n * ldp;
+    const int8_t* src = cpm + j * ldp + i;
+    long long xr = 0, xi = 0;
+    const long long M = tab.M;
+    for (int jm = 0; jm < nmod; ++jm) {
+        const int cp = src[(int64_t)jm * plane], cm = src[(int64_t)(nmod + jm) * plane];
+        const int mj = tab.m[jm], half = (mj - 1) / 2;
+        int ur = ((cm + cp) * tab.gr[jm]) % mj;       // Eq. (2c) and the CRT factor q_j, folded
+        int ui = ((cm - cp) * tab.gi[jm]) % mj;
+        if (ur > half) ur -= mj; else if (ur < -half) ur += mj;
+        if (ui > half) ui -= mj; else if (ui < -half) ui += mj;
+        xr = (xr + (long long)ur * tab.W[jm]) % M;    // |term| < 2^62, |xr| < M < 2^62: no overflow
+        xi = (xi + (long long)ui * tab.W[jm]) % M;
+    }
+    const long long h = (M - 1) / 2;                  // lift to [-(M-1)/2, (M-1)/2]
+    if (xr > h) xr -= M; else if (xr < -h) xr += M;
+    if (xi > h) xi -= M; else if (xi < -h) xi += M;
+    Cr[i + j * ldc] = xr;
+    Ci[i + j * ldc] = xi;
+}
+
+cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,
+                            int64_t ldc, cudaStream_t st, int* launches) {
+    if (m <= 0 || n <= 0) return cudaSuccess;
+    for (int64_t j0 = 0; j0 < n; j0 += 65535) {
+        const int64_t nj = (n - j0 < 65535) ? n - j0 : 65535;
+        dim3 grid((unsigned)((m + 255) / 256), (unsigned)nj);
+        post_int_kernel<<<grid, 256, 0, st>>>(cpm + j0 * ldp, ldp, m, n, tab, Cr + j0 * ldc, Ci + j0 * ldc, ldc);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+
+template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, const double*, const double*, cudaStream_t, int*);
+template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, const double*, const double*, cudaStream_t, int*);
+
+}  // namespace gemm2m
