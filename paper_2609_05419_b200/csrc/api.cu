@@ -171,6 +171,42 @@ int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
     return GEMM2M_OK;
 }
 
+// Panel pipeline shared by every entry point: the rows [0, n) of the GEMM's row operand (columns of C for the GEMMs, rows of the
+// lower triangle for the rank-k family) are cut into panels of about 1024 rows up to four of them, then of about 2048 rows
+// (more, narrower panels also keep the operand slices of a launch inside the L2: 16384 columns in 8 panels measured 6-8 %
+// faster than in 4).  gemm(r0, r1) enqueues the GEMMs of a panel on the caller's stream; post(r0, r1, stream) its
+// post-processing, which runs on the library's stream beside the GEMMs of the next panel, except for the last panel.  The
+// call is complete on the caller's stream only when the library's stream has been joined back.
+template <typename GemmFn, typename PostFn>
+int panel_pipeline(int64_t n, cudaStream_t st, Phases& ph, GemmFn gemm, PostFn post) {
+    int panels = (int)(n / 1024);
+    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
+    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
+    const int64_t panel_rows = round_up((n + panels - 1) / panels, 256);
+    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
+    for (int pnl = 0; pnl < panels; ++pnl) {
+        const int64_t r0 = pnl * panel_rows, r1 = (r0 + panel_rows < n) ? r0 + panel_rows : n;
+        if (r0 >= r1) break;
+        CK(ph.begin(2, st));
+        if (int s = gemm(r0, r1)) return s;
+        CK(ph.end(st));
+        const bool last = r1 >= n;
+        cudaStream_t ps = last ? st : D().side;
+        if (!last) {
+            CK(cudaEventRecord(D().panel_done[pnl], st));
+            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
+        }
+        CK(ph.begin(3, ps));
+        CK(post(r0, r1, ps));
+        CK(ph.end(ps));
+    }
+    if (panels > 1) {
+        CK(cudaEventRecord(D().side_done, D().side));
+        CK(cudaStreamWaitEvent(st, D().side_done, 0));
+    }
+    return GEMM2M_OK;
+}
+
 // transa / transb: 'N' (as stored), 'T' (transposed) or 'C' (conjugate transposed) operand, BLAS style; alpha, beta: host
 // pointers to (re, im) pairs or null for 1 and 0.  C = alpha op(A) op(B) + beta C with op(A) m x k and op(B) k x n.
 template <typename T>
@@ -270,34 +306,11 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
     build_mod_table(nmod, true, &ga.mods);
     ga.dev_status = dev_status;
-    // panels of about 1024 columns up to four of them, then of 2048 columns (more, narrower panels also keep the operand
-    // slices of a launch inside the L2: 16384 columns in 8 panels measured 6-8 % faster than in 4)
-    int panels = (int)(n / 1024);
-    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
-    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
-    const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
-    for (int pnl = 0; pnl < panels; ++pnl) {
-        const int64_t j0 = pnl * panel_cols, j1 = (j0 + panel_cols < n) ? j0 + panel_cols : n;
-        if (j0 >= j1) break;
-        ga.row_begin = j0;
-        ga.row_end = j1;
-        CK(ph.begin(2, st));
-        if (int s = run_gemm(ga, nmod, st)) return s;
-        CK(ph.end(st));
-        const bool last = j1 >= n;
-        cudaStream_t ps = last ? st : D().side;
-        if (!last) {
-            CK(cudaEventRecord(D().panel_done[pnl], st));
-            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
-        }
-        CK(ph.begin(3, ps));
-        CK(launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]));
-        CK(ph.end(ps));
-    }
-    if (panels > 1) {   // join: the call is complete on the caller's stream only when the side stream has finished
-        CK(cudaEventRecord(D().side_done, D().side));
-        CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    }
+    if (int s = panel_pipeline(n, st, ph,
+            [&](int64_t j0, int64_t j1) { ga.row_begin = j0; ga.row_end = j1; return run_gemm(ga, nmod, st); },
+            [&](int64_t j0, int64_t j1, cudaStream_t ps) {
+                return launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]);
+            })) return s;
     ph.done();
     return GEMM2M_OK;
 }
@@ -506,37 +519,20 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     // The output is cut into row panels: entry (i, j) of the lower triangle needs C+[i, j] and C+[j, i], i.e. the GEMM output
     // rows j and i <= the end of i's panel, so the post-processing of the rows of panel p can run on the library's stream
     // beside the GEMMs of panel p + 1 (the last, largest panel stays on the caller's stream).
-    int panels = (int)(n / 1024);
-    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
-    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
-    const int64_t panel_rows = round_up((n + panels - 1) / panels, 256);
-    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
-    for (int pnl = 0; pnl < panels; ++pnl) {
-        const int64_t r0 = pnl * panel_rows, r1 = (r0 + panel_rows < n) ? r0 + panel_rows : n;
-        if (r0 >= r1) break;
-        ga.row_begin = r0; ga.row_end = r1;
-        CK(ph.begin(2, st));
-        ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
-        if (int s = run_gemm(ga, nmod, st)) return s;
-        if (two) {
-            ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
-            if (int s = run_gemm(ga, nmod, st)) return s;
-        }
-        CK(ph.end(st));
-        const bool last = r1 >= n;
-        cudaStream_t ps = last ? st : D().side;
-        if (!last) {
-            CK(cudaEventRecord(D().panel_done[pnl], st));
-            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
-        }
-        CK(ph.begin(3, ps));
-        CK(launch_post_herk(cp, c.ldp, n, r0, r1, eA, ctab, C, ldc, real_in, ps, &g.launches[3]));
-        CK(ph.end(ps));
-    }
-    if (panels > 1) {
-        CK(cudaEventRecord(D().side_done, D().side));
-        CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    }
+    if (int s = panel_pipeline(n, st, ph,
+            [&](int64_t r0, int64_t r1) {
+                ga.row_begin = r0; ga.row_end = r1;
+                ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
+                if (int s = run_gemm(ga, nmod, st)) return s;
+                if (two) {
+                    ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
+                    if (int s = run_gemm(ga, nmod, st)) return s;
+                }
+                return (int)GEMM2M_OK;
+            },
+            [&](int64_t r0, int64_t r1, cudaStream_t ps) {
+                return launch_post_herk(cp, c.ldp, n, r0, r1, eA, ctab, C, ldc, real_in, ps, &g.launches[3]);
+            })) return s;
     ph.done();
     return GEMM2M_OK;
 }
@@ -609,36 +605,18 @@ int dgemm_ozaki2(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, 
     ga.out = cpl; ga.ldp = c.ldp; ga.accumulate = 0;
     build_mod_table_real(nmod, &ga.mods);
     ga.dev_status = (int*)(ws + c.off_status);
-    int panels = (int)(n / 1024);
-    if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
-    panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
-    const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
-    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
     const int64_t klim = gemm_k_limit_real();
-    for (int pnl = 0; pnl < panels; ++pnl) {
-        const int64_t j0 = pnl * panel_cols, j1 = (j0 + panel_cols < n) ? j0 + panel_cols : n;
-        if (j0 >= j1) break;
-        ga.row_begin = j0;
-        ga.row_end = j1;
-        CK(ph.begin(2, st));
-        if (g.gemm_kernel == 1) CK(launch_gemm_check(ga, klim, st, &g.launches[2]));
-        else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(ga, klim, D().sm_count, st, &g.launches[2]));
-        else CK(launch_gemm_tcgen05_pair(ga, klim, D().sm_count, st, &g.launches[2]));
-        CK(ph.end(st));
-        const bool last = j1 >= n;
-        cudaStream_t ps = last ? st : D().side;
-        if (!last) {
-            CK(cudaEventRecord(D().panel_done[pnl], st));
-            CK(cudaStreamWaitEvent(D().side, D().panel_done[pnl], 0));
-        }
-        CK(ph.begin(3, ps));
-        CK(launch_post_real(cpl, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]));
-        CK(ph.end(ps));
-    }
-    if (panels > 1) {
-        CK(cudaEventRecord(D().side_done, D().side));
-        CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    }
+    if (int s = panel_pipeline(n, st, ph,
+            [&](int64_t j0, int64_t j1) {
+                ga.row_begin = j0; ga.row_end = j1;
+                if (g.gemm_kernel == 1) CK(launch_gemm_check(ga, klim, st, &g.launches[2]));
+                else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(ga, klim, D().sm_count, st, &g.launches[2]));
+                else CK(launch_gemm_tcgen05_pair(ga, klim, D().sm_count, st, &g.launches[2]));
+                return (int)GEMM2M_OK;
+            },
+            [&](int64_t j0, int64_t j1, cudaStream_t ps) {
+                return launch_post_real(cpl, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]);
+            })) return s;
     ph.done();
     return GEMM2M_OK;
 }
