@@ -26,7 +26,6 @@ struct DevState {
 
 struct State {
     std::mutex mu;
-    static constexpr int kMaxDevices = 64;
     DevState dev[kMaxDevices];
     int cur = 0;                  // device of the call being served (set by use_current_device)
     int profiling = 0;
@@ -61,13 +60,13 @@ inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 // Points D() at the state of the calling thread's current device (the caller holds g.mu).
 void select_device() {
     int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < State::kMaxDevices) g.cur = dev;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) g.cur = dev;
 }
 
 // The same, and checks the device's architecture once.
 int check_device() {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= State::kMaxDevices) return GEMM2M_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GEMM2M_ERR_CUDA;
     g.cur = dev;
     if (D().arch_ok < 0) {
         cudaDeviceProp prop;

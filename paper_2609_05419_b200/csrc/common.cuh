@@ -83,6 +83,14 @@ struct CrtTableInt {
 
 struct ScaleTargets { int Pt, PA, PB, ck; };
 
+// Function attributes (dynamic shared memory size, cluster occupancy) belong to a device: launchers cache "done" per device.
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+    return dev;
+}
+
 // ---- host-side table builders (tables.cu) ----
 int modulus_value(int j);
 int modulus_root(int j);

@@ -225,8 +225,10 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
 cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches) {
     using namespace cfg2;
     if (a.R <= 0 || a.Cn <= 0 || a.nbatch <= 0 || a.row_end <= a.row_begin) return cudaSuccess;
-    static bool attr_set = false;
-    static int max_pairs = 0;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[current_device_slot()];
+    static int max_pairs_dev[kMaxDevices] = {};
+    int& max_pairs = max_pairs_dev[current_device_slot()];
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(gemm_i8_tcgen05_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         if (err != cudaSuccess) return err;

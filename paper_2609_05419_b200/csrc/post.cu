@@ -438,7 +438,8 @@ template <bool REAL_OUT>
 static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA,
                                       const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
     const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
-    static bool attr_set = false;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[current_device_slot()];
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -28,7 +28,8 @@ template <> __device__ __forceinline__ Cplx<float> load_cplx<float>(const float*
 }
 
 inline int cached_sm_count() {
-    static int sms = 0;
+    static int sms_dev[kMaxDevices] = {};
+    int& sms = sms_dev[current_device_slot()];
     if (!sms) {
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)

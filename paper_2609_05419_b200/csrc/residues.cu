@@ -309,7 +309,8 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
-    static bool attr_set = false;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[current_device_slot()];
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<T, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -501,7 +502,8 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = (size_t)kResIRows * kResIRowStride * sizeof(QPair);
-    static bool attr_set = false;
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[current_device_slot()];
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(residues_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
