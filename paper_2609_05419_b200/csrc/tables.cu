@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 namespace gemm2m {
@@ -88,6 +89,16 @@ static Big product_of(int nmod, const int* mods = kModuli) {
 }
 
 // mods: the modulus list; n2: how many of the first nmod are 2M moduli (the others take the plain weights for both parts).
+// The tables are functions of the modulus count alone: each is built once per process and copied out afterwards, so that a
+// call's host cost is its launches, not multi-word arithmetic.
+template <class T, int N, class F>
+static void memoised(int nmod, T* out, F&& build) {
+    static T cache[N + 1];
+    static std::once_flag once[N + 1];
+    std::call_once(once[nmod], [&] { build(&cache[nmod]); });
+    *out = cache[nmod];
+}
+
 static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTable* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
@@ -131,8 +142,12 @@ static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTa
     }
 }
 
-void build_residue_table(int nmod, ResidueTable* t) { build_residue_table_for(kModuli, nmod, count_2m(nmod), t); }
-void build_residue_table_real(int nmod, ResidueTable* t) { build_residue_table_for(kRealModuli, nmod, 0, t); }
+void build_residue_table(int nmod, ResidueTable* t) {
+    memoised<ResidueTable, kMaxMod>(nmod, t, [&](ResidueTable* c) { build_residue_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_residue_table_real(int nmod, ResidueTable* t) {
+    memoised<ResidueTable, kMaxReal>(nmod, t, [&](ResidueTable* c) { build_residue_table_for(kRealModuli, nmod, 0, c); });
+}
 
 // 2^e / (2 (Y0 + xmax) |n m - 2^e|) for inv_m = n 2^-e: the factor by which the error term of the residue kernels'
 // quotient estimate stays below the distance 1/(2m) of x/m from the nearest rounding boundary (must exceed 1).
@@ -160,7 +175,7 @@ static void fill_mod_entry(ModTable* t, int p, const int* mods, int j) {
     t->cq[p] = r.cq[j];
 }
 
-void build_mod_table(int nmod, bool per_plane, ModTable* t) {
+static void build_mod_table_for(int nmod, bool per_plane, ModTable* t) {
     std::memset(t, 0, sizeof(*t));
     const int n2 = count_2m(nmod);
     int p = 0;
@@ -176,10 +191,17 @@ void build_mod_table(int nmod, bool per_plane, ModTable* t) {
     t->nplanes = p;
 }
 
+void build_mod_table(int nmod, bool per_plane, ModTable* t) {
+    if (per_plane) memoised<ModTable, kMaxMod>(nmod, t, [&](ModTable* c) { build_mod_table_for(nmod, true, c); });
+    else memoised<ModTable, kMaxMod>(nmod, t, [&](ModTable* c) { build_mod_table_for(nmod, false, c); });
+}
+
 void build_mod_table_real(int nmod, ModTable* t) {
-    std::memset(t, 0, sizeof(*t));
-    for (int j = 0; j < nmod; ++j) fill_mod_entry(t, j, kRealModuli, j);
-    t->nplanes = nmod;
+    memoised<ModTable, kMaxReal>(nmod, t, [&](ModTable* c) {
+        std::memset(c, 0, sizeof(*c));
+        for (int j = 0; j < nmod; ++j) fill_mod_entry(c, j, kRealModuli, j);
+        c->nplanes = nmod;
+    });
 }
 
 // Folded CRT weights: g_j = sym(2^-1 q_j mod m_j), h_j = sym(s_j 2^-1 q_j mod m_j), q_j = (M/m_j)^-1 mod m_j.
@@ -227,10 +249,14 @@ static void build_crt_table_for(const int* mods, int nmod, int n2, CrtTable* t) 
     t->q_lo = t->nchunks > 1 ? std::ldexp(t->q_hi, -kChunkBits) : 0.0;
 }
 
-void build_crt_table(int nmod, CrtTable* t) { build_crt_table_for(kModuli, nmod, count_2m(nmod), t); }
-void build_crt_table_real(int nmod, CrtTable* t) { build_crt_table_for(kRealModuli, nmod, 0, t); }
+void build_crt_table(int nmod, CrtTable* t) {
+    memoised<CrtTable, kMaxMod>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_crt_table_real(int nmod, CrtTable* t) {
+    memoised<CrtTable, kMaxReal>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kRealModuli, nmod, 0, c); });
+}
 
-void build_crt_table_int(int nmod, CrtTableInt* t) {
+static void build_crt_table_int_for(int nmod, CrtTableInt* t) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
     const Big M = product_of(nmod);
@@ -246,13 +272,22 @@ void build_crt_table_int(int nmod, CrtTableInt* t) {
     }
 }
 
-// Scaling budget: P_t = floor(log2((M-1)/2)) split between rows of A and columns of B; c_k = ceil(log2(2k)/2).
-ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
-    Big half = product_of(nmod);
+void build_crt_table_int(int nmod, CrtTableInt* t) {
+    memoised<CrtTableInt, kMaxMod>(nmod, t, [&](CrtTableInt* c) { build_crt_table_int_for(nmod, c); });
+}
+
+// floor(log2((M-1)/2)) for the first nmod moduli of a list.
+static int budget_bits(int nmod, const int* mods) {
+    Big half = product_of(nmod, mods);
     half.sub_one();
     half.shr1();
+    return half.bit_length() - 1;
+}
+
+// Scaling budget: P_t = floor(log2((M-1)/2)) split between rows of A and columns of B; c_k = ceil(log2(2k)/2).
+ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
     ScaleTargets s;
-    s.Pt = half.bit_length() - 1;
+    memoised<int, kMaxMod>(nmod, &s.Pt, [&](int* c) { *c = budget_bits(nmod, kModuli); });
     s.PA = (s.Pt + 1) / 2;
     s.PB = s.Pt / 2;
     if (herk) s.PA = s.PB = s.Pt / 2;
@@ -264,11 +299,8 @@ ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
 
 // Real scheme (Section 3.1): a row has k real terms, c_k = ceil(log2(k)/2).
 ScaleTargets scale_targets_real(int nmod, int64_t k) {
-    Big half = product_of(nmod, kRealModuli);
-    half.sub_one();
-    half.shr1();
     ScaleTargets s;
-    s.Pt = half.bit_length() - 1;
+    memoised<int, kMaxReal>(nmod, &s.Pt, [&](int* c) { *c = budget_bits(nmod, kRealModuli); });
     s.PA = (s.Pt + 1) / 2;
     s.PB = s.Pt / 2;
     s.ck = 0;
