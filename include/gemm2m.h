@@ -65,7 +65,8 @@ typedef enum {
 
 typedef enum {
     GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3,
-    GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6, GEMM2M_OP_DGEMM_OZAKI2 = 7
+    GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6, GEMM2M_OP_DGEMM_OZAKI2 = 7,
+    GEMM2M_OP_ZGEMM_EISENSTEIN = 8
 } gemm2m_op;
 
 /* Human-readable name of a status code (static string). */
@@ -138,6 +139,30 @@ int gemm2m_set_scaling(int mode);
  * gemm2m_workspace_bytes(GEMM2M_OP_DGEMM_OZAKI2, ...). */
 int dgemm_ozaki2(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
                  int nmod, void* stream);
+
+/* The Eisenstein-integer analogue of zgemm2m that Sections 3.2 and 4 point out: the Gaussian integers are replaced by
+ * Z[w], w = exp(2 pi i/3), whose 2M moduli are the products of primes congruent to 1 mod 3 (greedy coprime set below 256:
+ * 247, 241, 229, 223, 217, 211, 199, ..., 43, 37; nmod <= 23, M up to 2^160.9 against 2^152 for the Gaussian set).
+ * Same interface, layout, workspace rules and GEMMs as zgemm2m / zgemm2m_ex (two real int8 GEMMs per modulus); different:
+ *   - quantisation rounds each scaled entry to the NEAREST point of the hexagonal lattice, held as (u + v sqrt(-3))/2 with
+ *     u = v (mod 2).  The decision is taken in fixed point (32 fraction bits, 2/sqrt(3) as a 128-bit constant), so that it is
+ *     reproducible bit for bit; it differs from the exact nearest point only within 2^-30 of a cell boundary;
+ *   - the residues are u +- d_j v with d_j = 2 s_j + 1 a square root of -3 modulo m_j (s_j^2 + s_j + 1 = 0), twice the images
+ *     of the entry under w -> s_j and w -> s_j^2; the factor 4 this leaves in the products is folded into the CRT weights;
+ *   - the scale factors use c_k = ceil(log2(5k)/2) (lattice rounding can move a point outwards; the coordinates of a
+ *     product are bounded by twice its modulus), and P_B - c_k >= 2 is required: too few moduli for k give GEMM2M_ERR_NMOD;
+ *   - the lifted result (U + V sqrt(-3))/2 is converted with one rounding per part: Re = U/2, Im = V sqrt(3)/2 (the
+ *     irrational factor as a double-double).
+ * The always-on max-based scaling rule is used (gemm2m_set_scaling does not apply).  Workspace:
+ * gemm2m_workspace_bytes(GEMM2M_OP_ZGEMM_EISENSTEIN, ...). */
+int zgemm2m_eisenstein(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C,
+                       int64_t ldc, int nmod, void* stream);
+int zgemm2m_eisenstein_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A,
+                          int64_t lda, const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc, int nmod,
+                          void* stream);
+/* Size of the Eisenstein modulus set (23) and its j-th modulus with the smallest s_j > 1, s_j^2 + s_j + 1 = 0 (mod m_j). */
+int gemm2m_max_eisenstein_moduli(void);
+int gemm2m_eisenstein_modulus(int j, int* m, int* s);
 
 /* Hermitian rank-k update C = A A^H (Section 5, HERK) with ONE real int8 GEMM per modulus: C+ = A+ A-^T and
  * C- = C+^T.  A: n x k complex128 (lda >= n).  Only the lower triangle of C (n x n, ldc >= n) including the
@@ -244,6 +269,10 @@ int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_g
 int gemm2m_debug_tables_real(int nmod, int64_t k, int* moduli, int* scale, double* crt_g, double* crt_m, int* nchunks, int32_t* y0_bits, float* cq,
                              float* inv_m, int32_t* xmax, double* margin);
 int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin);
+/* The same for the Eisenstein set (tests only): scale[4], crt_gr / crt_gi[nmod*5] = digits of sym(4^-1 q_j)(M/m_j) and of
+ * sym(-(4 d_j)^-1 q_j)(M/m_j), crt_m[5], nchunks, and the reduction constants. */
+int gemm2m_debug_tables_eisenstein(int nmod, int64_t k, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,
+                                   int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin);
 
 #ifdef __cplusplus
 }

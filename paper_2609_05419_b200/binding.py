@@ -11,6 +11,7 @@ import ctypes
 import os
 
 OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K, OP_DGEMM_OZAKI2 = 0, 1, 2, 3, 4, 5, 6, 7
+OP_ZGEMM_EISENSTEIN = 8
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -57,6 +58,11 @@ def lib():
     ex = [ctypes.c_char, ctypes.c_char, i64, i64, i64, vp, vp, i64, vp, i64, vp, vp, i64, i32, vp]
     L.zgemm2m_ex.argtypes = ex
     L.cgemm2m_ex.argtypes = ex
+    L.zgemm2m_eisenstein.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.zgemm2m_eisenstein_ex.argtypes = ex
+    L.gemm2m_max_eisenstein_moduli.restype = i32
+    L.gemm2m_eisenstein_modulus.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.gemm2m_debug_tables_eisenstein.argtypes = [i32, i64] + [vp] * 10
     L.zherk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
     L.dsyrk2m.argtypes = [i64, i64, vp, i64, vp, i64, i32, vp]
     L.zher2k2m.argtypes = [i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
@@ -190,6 +196,45 @@ def zgemm2m_ex(transa, transb, alpha, A, B, beta, C, nmod=16, stream=None):
 
 def cgemm2m_ex(transa, transb, alpha, A, B, beta, C, nmod=7, stream=None):
     _xgemm_ex(lib().cgemm2m_ex, "cgemm2m_ex", ctypes.c_float, transa, transb, alpha, A, B, beta, C, nmod, stream)
+
+
+def zgemm2m_eisenstein(A, B, C, nmod=16, stream=None):
+    """C = A B through the Eisenstein-integer variant (complex128 CUDA tensors, column-major views)."""
+    _xgemm(lib().zgemm2m_eisenstein, "zgemm2m_eisenstein", A, B, C, nmod, stream)
+
+
+def zgemm2m_eisenstein_ex(transa, transb, alpha, A, B, beta, C, nmod=16, stream=None):
+    _xgemm_ex(lib().zgemm2m_eisenstein_ex, "zgemm2m_eisenstein_ex", ctypes.c_double, transa, transb, alpha, A, B, beta, C, nmod, stream)
+
+
+def max_eisenstein_moduli():
+    return int(lib().gemm2m_max_eisenstein_moduli())
+
+
+def eisenstein_modulus(j):
+    m, s = ctypes.c_int(0), ctypes.c_int(0)
+    _check(lib().gemm2m_eisenstein_modulus(j, ctypes.byref(m), ctypes.byref(s)), "gemm2m_eisenstein_modulus")
+    return m.value, s.value
+
+
+def debug_tables_eisenstein(nmod, k):
+    """Host-side constants of the Eisenstein variant (see gemm2m_debug_tables_eisenstein)."""
+    import numpy as np
+    scale = np.zeros(4, dtype=np.int32)
+    gr = np.zeros((nmod, 5), dtype=np.float64)
+    gi = np.zeros((nmod, 5), dtype=np.float64)
+    mc = np.zeros(5, dtype=np.float64)
+    nch = np.zeros(1, dtype=np.int32)
+    y0 = np.zeros(nmod, dtype=np.int32)
+    cq = np.zeros(nmod, dtype=np.float32)
+    inv = np.zeros(nmod, dtype=np.float32)
+    xmax = np.zeros(nmod, dtype=np.int32)
+    margin = np.zeros(nmod, dtype=np.float64)
+    ptr = lambda a: ctypes.c_void_p(a.ctypes.data)
+    _check(lib().gemm2m_debug_tables_eisenstein(nmod, k, ptr(scale), ptr(gr), ptr(gi), ptr(mc), ptr(nch), ptr(y0), ptr(cq), ptr(inv),
+                                                ptr(xmax), ptr(margin)), "gemm2m_debug_tables_eisenstein")
+    return dict(Pt=int(scale[0]), PA=int(scale[1]), PB=int(scale[2]), ck=int(scale[3]), gr=gr, gi=gi, Mc=mc, nchunks=int(nch[0]),
+                y0_bits=y0, cq=cq, inv_m=inv, xmax=xmax, margin=margin)
 
 
 def dgemm_ozaki2(A, B, C, nmod=15, stream=None):

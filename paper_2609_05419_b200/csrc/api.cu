@@ -85,7 +85,9 @@ struct Carve {
 
 bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     if (m < 0 || n < 0 || k < 0 || nmod < 1 || nmod > kMaxMod) return false;
-    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_DGEMM_OZAKI2) return false;
+    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_ZGEMM_EISENSTEIN) return false;
+    const bool eis = op == GEMM2M_OP_ZGEMM_EISENSTEIN;                          // two planes per modulus of the Eisenstein set
+    if (eis && nmod > kMaxEis) return false;
     const bool real_scheme = op == GEMM2M_OP_DGEMM_OZAKI2;                      // one plane per modulus of the real set
     if (real_scheme && nmod > kMaxReal) return false;
     const bool herk = op >= GEMM2M_OP_ZHERK && op <= GEMM2M_OP_DSYR2K;         // the rank-k family: one scale vector, C+ only
@@ -106,7 +108,7 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_exp_b = take(herk ? 0 : 4 * n);
     c->off_pack_a = take(real_in ? 16 * n * k : 0);
     c->off_pack_b = take(real_in && two ? 16 * n * k : 0);
-    const int64_t planes = real_scheme ? nmod : plane_count(nmod);             // 2 per 2M modulus, 3 per 3M modulus
+    const int64_t planes = real_scheme ? nmod : eis ? 2 * nmod : plane_count(nmod);   // 2 per 2M modulus, 3 per 3M modulus
     c->off_apm = take(planes * m * kp);
     c->off_bpm = take((herk && !two) ? 0 : planes * n * kp);
     c->off_cpm = take((herk ? (int64_t)nmod : planes) * n * ldp);
@@ -162,8 +164,7 @@ int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R
     return GEMM2M_OK;
 }
 
-int run_gemm(const GemmArgs& a, int nmod, cudaStream_t st) {
-    const int64_t klim = gemm_k_limit(nmod);
+int run_gemm(const GemmArgs& a, int64_t klim, cudaStream_t st) {
     if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
     else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(a, klim, D().sm_count, st, &g.launches[2]));
     else CK(launch_gemm_tcgen05_pair(a, klim, D().sm_count, st, &g.launches[2]));
@@ -218,7 +219,8 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
     const int64_t rows_a = ta == 'N' ? m : k, rows_b = tb == 'N' ? k : n;      // rows of the matrices as stored
     if (lda < (rows_a > 1 ? rows_a : 1) || ldb < (rows_b > 1 ? rows_b : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
-    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
+    const bool eis = op == GEMM2M_OP_ZGEMM_EISENSTEIN;
+    if (nmod < 1 || nmod > (eis ? kMaxEis : kMaxMod)) return GEMM2M_ERR_NMOD;
     if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
     if (m == 0 || n == 0) return GEMM2M_OK;
     const bool alpha_zero = alpha && alpha[0] == 0.0 && alpha[1] == 0.0;
@@ -246,13 +248,14 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     int8_t* bpm = (int8_t*)(ws + c.off_bpm);
     int8_t* cpm = (int8_t*)(ws + c.off_cpm);
 
-    const ScaleTargets sc = scale_targets(nmod, k, false);
+    const ScaleTargets sc = eis ? scale_targets_eis(nmod, k) : scale_targets(nmod, k, false);
+    if (eis && sc.PB - sc.ck < 2) return GEMM2M_ERR_NMOD;          // the lattice rounding needs scaled parts of 4 or more
     ResidueTable rtab;
-    build_residue_table(nmod, &rtab);
     CrtTable ctab;
-    build_crt_table(nmod, &ctab);
+    if (eis) { build_residue_table_eis(nmod, &rtab); build_crt_table_eis(nmod, &ctab); }
+    else { build_residue_table(nmod, &rtab); build_crt_table(nmod, &ctab); }
     // quantised parts stay below 2^(P - c_k) with the max-based rule and below 2^P with the 2-norm rule
-    const bool two_norm_mode = g.scaling == 1 && k <= (1ll << 22);
+    const bool two_norm_mode = !eis && g.scaling == 1 && k <= (1ll << 22);
     const bool wideA = two_norm_mode ? sc.PA > 61 : sc.PA - sc.ck > 62, wideB = two_norm_mode ? sc.PB > 61 : sc.PB - sc.ck > 62;
 
     Phases ph;
@@ -288,9 +291,15 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
-    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s;
+    if constexpr (sizeof(T) == 8) {
+        if (eis) CK(launch_residues_hex(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, apm, st, &g.launches[1]));
+    }
+    if (!eis) { if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s; }
     if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s;
+    if constexpr (sizeof(T) == 8) {
+        if (eis) CK(launch_residues_hex(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, bpm, st, &g.launches[1]));
+    }
+    if (!eis) { if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s; }
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
@@ -299,14 +308,17 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     GemmArgs ga;
     ga.rowop = bpm; ga.colop = apm;
     ga.R = n; ga.Cn = m; ga.Kp = c.kp;
-    ga.row_planes = ga.col_planes = plane_count(nmod);
+    const int nplanes = eis ? 2 * nmod : plane_count(nmod);
+    ga.row_planes = ga.col_planes = nplanes;
     ga.row_plane0 = ga.col_plane0 = 0;
-    ga.nbatch = plane_count(nmod);
+    ga.nbatch = nplanes;
     ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
-    build_mod_table(nmod, true, &ga.mods);
+    if (eis) build_mod_table_eis(nmod, &ga.mods);
+    else build_mod_table(nmod, true, &ga.mods);
     ga.dev_status = dev_status;
+    const int64_t klim = eis ? gemm_k_limit_eis() : gemm_k_limit(nmod);
     if (int s = panel_pipeline(n, st, ph,
-            [&](int64_t j0, int64_t j1) { ga.row_begin = j0; ga.row_end = j1; return run_gemm(ga, nmod, st); },
+            [&](int64_t j0, int64_t j1) { ga.row_begin = j0; ga.row_end = j1; return run_gemm(ga, klim, st); },
             [&](int64_t j0, int64_t j1, cudaStream_t ps) {
                 return launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]);
             })) return s;
@@ -420,7 +432,7 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
     ga.dev_status = (int*)(ws + c.off_status);
     ga.row_begin = 0; ga.row_end = n;
     CK(ph.begin(2, st));
-    if (int s = run_gemm(ga, nmod, st)) return s;
+    if (int s = run_gemm(ga, gemm_k_limit(nmod), st)) return s;
     CK(ph.end(st));
     CK(ph.begin(3, st));
     CK(launch_post_int(cpm, c.ldp, m, n, ctab, Cr, Ci, ldc, st, &g.launches[3]));
@@ -437,6 +449,25 @@ int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const
 int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc, int nmod,
             void* stream) {
     return xgemm2m<float>(GEMM2M_OP_CGEMM, 'N', 'N', m, n, k, nullptr, A, lda, B, ldb, nullptr, C, ldc, nmod, stream);
+}
+
+int zgemm2m_eisenstein(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
+                       int nmod, void* stream) {
+    return xgemm2m<double>(GEMM2M_OP_ZGEMM_EISENSTEIN, 'N', 'N', m, n, k, nullptr, A, lda, B, ldb, nullptr, C, ldc, nmod, stream);
+}
+
+int zgemm2m_eisenstein_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const double* alpha, const double* A, int64_t lda,
+                          const double* B, int64_t ldb, const double* beta, double* C, int64_t ldc, int nmod, void* stream) {
+    return xgemm2m<double>(GEMM2M_OP_ZGEMM_EISENSTEIN, transa, transb, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, nmod, stream);
+}
+
+int gemm2m_max_eisenstein_moduli(void) { return kMaxEis; }
+
+int gemm2m_eisenstein_modulus(int j, int* m, int* s) {
+    if (j < 0 || j >= kMaxEis) return GEMM2M_ERR_ARG;
+    if (m) *m = eis_modulus_value(j);
+    if (s) *s = eis_cube_root(j);
+    return GEMM2M_OK;
 }
 
 // The rank-k family of Section 5: HERK (B == nullptr) and HER2K on complex inputs; SYRK / SYR2K on real inputs through
@@ -522,10 +553,10 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
             [&](int64_t r0, int64_t r1) {
                 ga.row_begin = r0; ga.row_end = r1;
                 ga.colop = apm; ga.rowop = two ? bpm : apm; ga.accumulate = 0;
-                if (int s = run_gemm(ga, nmod, st)) return s;
+                if (int s = run_gemm(ga, gemm_k_limit(nmod), st)) return s;
                 if (two) {
                     ga.colop = bpm; ga.rowop = apm; ga.accumulate = 1;
-                    if (int s = run_gemm(ga, nmod, st)) return s;
+                    if (int s = run_gemm(ga, gemm_k_limit(nmod), st)) return s;
                 }
                 return (int)GEMM2M_OK;
             },
@@ -728,6 +759,31 @@ int gemm2m_debug_tables_real(int nmod, int64_t k, int* moduli, int* scale, doubl
         if (moduli) moduli[j] = real_modulus_value(j);
         for (int c = 0; c < kMaxChunks; ++c)
             if (crt_g) crt_g[j * kMaxChunks + c] = ct.gr[j][c];
+        if (y0_bits) y0_bits[j] = rt.magic[j];
+        if (cq) cq[j] = rt.cq[j];
+        if (inv_m) inv_m[j] = rt.inv_m[j];
+        if (xmax) xmax[j] = rt.xmax[j];
+        if (margin) margin[j] = residue_reduction_margin(rt, j);
+    }
+    if (crt_m) for (int c = 0; c < kMaxChunks; ++c) crt_m[c] = ct.Mc[c];
+    if (nchunks) *nchunks = ct.nchunks;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_tables_eisenstein(int nmod, int64_t k, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks, int32_t* y0_bits,
+                                   float* cq, float* inv_m, int32_t* xmax, double* margin) {
+    if (nmod < 1 || nmod > kMaxEis || k < 0) return GEMM2M_ERR_ARG;
+    const ScaleTargets sc = scale_targets_eis(nmod, k);
+    if (scale) { scale[0] = sc.Pt; scale[1] = sc.PA; scale[2] = sc.PB; scale[3] = sc.ck; }
+    CrtTable ct;
+    build_crt_table_eis(nmod, &ct);
+    ResidueTable rt;
+    build_residue_table_eis(nmod, &rt);
+    for (int j = 0; j < nmod; ++j) {
+        for (int c = 0; c < kMaxChunks; ++c) {
+            if (crt_gr) crt_gr[j * kMaxChunks + c] = ct.gr[j][c];
+            if (crt_gi) crt_gi[j * kMaxChunks + c] = ct.gi[j][c];
+        }
         if (y0_bits) y0_bits[j] = rt.magic[j];
         if (cq) cq[j] = rt.cq[j];
         if (inv_m) inv_m[j] = rt.inv_m[j];

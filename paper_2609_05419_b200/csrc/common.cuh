@@ -11,6 +11,7 @@ namespace gemm2m {
 constexpr int kMax2M = 22;         // size of the greedy 2M modulus set in [1, 256] (Section 4)
 constexpr int kMax3M = 4;          // non-2M moduli of the hybrid: 256, 253, 251, 249 (quantised values then still fit 96 bits)
 constexpr int kMaxMod = kMax2M + kMax3M;
+constexpr int kMaxEis = 23;        // moduli of the Eisenstein-integer variant (Sections 3.2, 4): M up to 2^160.9
 constexpr int kMaxReal = 20;       // moduli of the real Ozaki-II scheme (Section 3.1; set of Section 4): M up to 2^155
 constexpr int kMaxPlanes = 2 * kMax2M + 3 * kMax3M;   // residue planes per operand: two per 2M modulus, three per 3M modulus
 constexpr int kMaxChunks = 5;      // 40-bit digits needed for M/2 < 2^184
@@ -69,7 +70,9 @@ struct CrtTable {
     double gi[kMaxMod][kMaxChunks];
     double Mc[kMaxChunks];                     // digits of M
     double q_hi, q_lo;
+    double im_hi, im_lo;                       // Eisenstein variant: the imaginary part is V (im_hi + im_lo); 0 = no factor
     int nmod, n2, nchunks;
+    int re_shift;                              // Eisenstein variant: the real part is U 2^re_shift
 };
 
 // CRT constants for the exact int64 result (nmod <= 8, M < 2^62).
@@ -107,6 +110,13 @@ void build_residue_table_real(int nmod, ResidueTable* t);
 void build_mod_table_real(int nmod, ModTable* t);
 void build_crt_table_real(int nmod, CrtTable* t);
 ScaleTargets scale_targets_real(int nmod, int64_t k);
+int eis_modulus_value(int j);
+int eis_cube_root(int j);
+void build_residue_table_eis(int nmod, ResidueTable* t);
+void build_mod_table_eis(int nmod, ModTable* t);
+void build_crt_table_eis(int nmod, CrtTable* t);
+ScaleTargets scale_targets_eis(int nmod, int64_t k);
+int64_t gemm_k_limit_eis();
 int64_t gemm_k_limit_real();
 int64_t gemm_k_limit(int nmod);     // largest K for which K max|residue|^2 fits int32
 
@@ -123,6 +133,8 @@ template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t row
 // Quantise + residues.  k_contiguous = false: operand row r is row r of the column-major matrix X (A: m x k);
 // true: operand row r is column r of X (B: k x n).
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
+cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                                const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
 // The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.

@@ -164,8 +164,13 @@ __global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __r
             } else {
                 double h, l;
                 crt_finish<NCH>(Sr[e], tab, &h, &l);
-                re[e] = scale_pow2(h + l, ea + fb);
+                re[e] = scale_pow2(h + l, ea + fb + tab.re_shift);
                 crt_finish<NCH>(Si[e], tab, &h, &l);
+                if (tab.im_hi != 0.0) {          // Eisenstein variant: V sqrt(3)/2 as a double-double product, rounded once below
+                    const double p = h * tab.im_hi;
+                    l = fma(h, tab.im_lo, fma(l, tab.im_hi, fma(h, tab.im_hi, -p)));
+                    h = p;
+                }
                 im[e] = scale_pow2(h + l, ea + fb);
             }
         }

@@ -48,6 +48,54 @@ __device__ __forceinline__ void quantise_part_wide(T v, int e, uint32_t* lo, lon
     *upper = (long long)(sq >> 32);
 }
 
+// Eisenstein variant (Sections 3.2, 4): the lattice point (u + v sqrt(-3))/2, u = v (mod 2), nearest to (x + iy) 2^-e.
+// X = |x| 2^-e and t = |y| 2^-e (2/sqrt 3) are formed as fixed-point numbers with 32 fraction bits (floor; the factor as
+// the 128-bit constant floor(2^127 2/sqrt 3), the product exact in 192 bits before the shift).  The nearest point with
+// u, v even is (2 rn(X), 2 rn(t/2)); it is at least as near as the nearest point with u, v odd, (2 floor(X) + 1,
+// 2 floor(t/2) + 1), exactly when |X - rn(X)| + (3/2) |t - 2 rn(t/2)| <= 1.  The signs of x and y carry over to u and v.
+// |u|, |v| < 2^82 by the scaling rule; returned like quantise_part_wide.
+__device__ __forceinline__ void quantise_hex(double x, double y, int e, uint32_t* ulo, long long* uup, uint32_t* vlo, long long* vup) {
+    using F = FpBits<double>;
+    typedef unsigned __int128 u128;
+    auto split = [](double v, int e, unsigned long long* mant, int* sh) {
+        const unsigned long long mag = F::mag(v);
+        const int E = (int)(mag >> F::kMantBits);
+        *mant = mag & ((1ull << F::kMantBits) - 1);
+        if (E) *mant |= (1ull << F::kMantBits);
+        *sh = max(E, 1) - (F::kBias + F::kMantBits) - e + 32;      // |v| 2^(32 - e) = mant 2^sh
+    };
+    unsigned long long mx, my;
+    int shx, shy;
+    split(x, e, &mx, &shx);
+    split(y, e, &my, &shy);
+    u128 Xf;
+    if (shx >= 0) Xf = (u128)mx << min(shx, 74);                     // a legitimate shift is below 60; the clamp keeps it defined
+    else Xf = (-shx > 63) ? 0 : (mx >> (-shx));
+    constexpr unsigned long long kK3hi = 0x93CD3A2C8198E269ull, kK3lo = 0x0C7C0F257D92BE83ull;   // floor(2^127 2/sqrt 3)
+    const u128 p0 = (u128)my * kK3lo, p1 = (u128)my * kK3hi;
+    const u128 top = p1 + (p0 >> 64);                                // bits 64.. of the 181-bit product
+    const int r = 127 - shy - 64;                                    // t 2^32 = product >> (127 - shy), and 127 - shy >= 64
+    const u128 Tf = r >= 128 ? 0 : (r <= 0 ? top : (top >> r));
+    const uint32_t fx = (uint32_t)Xf;
+    const unsigned long long ft = (unsigned long long)Tf & 0x1FFFFFFFFull;
+    const unsigned long long dx0 = fx < 0x80000000u ? fx : 0x100000000ull - fx;
+    const unsigned long long dt0 = ft < 0x100000000ull ? ft : 0x200000000ull - ft;
+    u128 u, v;
+    if (2 * dx0 + 3 * dt0 <= 0x200000000ull) {
+        u = ((Xf + 0x80000000ull) >> 32) << 1;
+        v = ((Tf + 0x100000000ull) >> 33) << 1;
+    } else {
+        u = ((Xf >> 32) << 1) | 1;
+        v = ((Tf >> 33) << 1) | 1;
+    }
+    const __int128 su = __double_as_longlong(x) < 0 ? -(__int128)u : (__int128)u;
+    const __int128 sv = __double_as_longlong(y) < 0 ? -(__int128)v : (__int128)v;
+    *ulo = (uint32_t)(u128)su;
+    *uup = (long long)(su >> 32);
+    *vlo = (uint32_t)(u128)sv;
+    *vup = (long long)(sv >> 32);
+}
+
 __device__ __forceinline__ int dp4a_us(uint32_t a_unsigned, uint32_t b_signed, int c) {
     int d;
     asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a_unsigned), "r"(b_signed), "r"(c));
@@ -211,7 +259,7 @@ __device__ __forceinline__ void cp_async_zfill(void* smem_dst, const void* gmem_
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <typename T, bool WIDE, int NMOD>
+template <typename T, bool WIDE, int NMOD, bool HEX = false>
 __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K,
                                                                      int64_t Kp, const int32_t* __restrict__ e,
                                                                      const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
@@ -277,8 +325,12 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
                     uint32_t lr = 0, li = 0;
                     long long ur = 0, ui = 0;
                     if (ex != kExpNonFinite) {
-                        quantise_part_wide<T>(v.x, ex, &lr, &ur);
-                        quantise_part_wide<T>(v.y, ex, &li, &ui);
+                        if (HEX) {
+                            quantise_hex((double)v.x, (double)v.y, ex, &lr, &ur, &li, &ui);
+                        } else {
+                            quantise_part_wide<T>(v.x, ex, &lr, &ur);
+                            quantise_part_wide<T>(v.y, ex, &li, &ui);
+                        }
                     }
                     dr[i] = split_digits_wide(lr, ur, &tr[i]);
                     di[i] = split_digits_wide(li, ui, &ti[i]);
@@ -335,6 +387,26 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
             if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
             else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
     }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// Eisenstein variant: the same kernel with the lattice rounding in front (complex double operands, 96-bit coordinates).
+cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
+                                const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches) {
+    if (R <= 0 || Kp <= 0) return cudaSuccess;
+    constexpr size_t smem = kResSmemBytes(2 * sizeof(double));
+    static bool attr_set_dev[kMaxDevices] = {};
+    bool& attr_set = attr_set_dev[current_device_slot()];
+    if (!attr_set) {
+        cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<double, true, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attr_set = true;
+    }
+    const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
+    const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
+    const unsigned grid = (unsigned)(total < resident ? total : resident);
+    residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
     ++*launches;
     return cudaGetLastError();
 }

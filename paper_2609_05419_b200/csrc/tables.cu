@@ -19,7 +19,22 @@ static const int kModuli[kMaxMod] = {241, 233, 229, 221, 205, 197, 193, 181, 173
 static const int kRealModuli[kMaxReal] = {256, 255, 253, 251, 247, 241, 239, 233, 229, 227,
                                           223, 217, 211, 199, 197, 193, 191, 181, 179, 173};
 
+// The analogous set for the Eisenstein integers (Sections 3.2 and 4): coprime products of primes congruent to 1 mod 3.
+static const int kEisModuli[kMaxEis] = {247, 241, 229, 223, 217, 211, 199, 193, 181, 163, 157, 151,
+                                        139, 127, 109, 103, 97,  79,  73,  67,  61,  43,  37};
+
 int modulus_value(int j) { return kModuli[j]; }
+int eis_modulus_value(int j) { return kEisModuli[j]; }
+
+int eis_cube_root(int j) {   // smallest s > 1 with s^2 + s + 1 = 0 (mod m)
+    const int m = kEisModuli[j];
+    for (int s = 2; s < m; ++s)
+        if ((s * s + s + 1) % m == 0) return s;
+    return 0;
+}
+// d = 2s + 1 = s - s^2 is a square root of -3: in the coordinates (u + v sqrt(-3))/2 of the Eisenstein integers the two ring
+// homomorphisms are u +- d v (up to the unit 2), which is Eq. (2a) with d in the place of s.
+static int eis_sqrt_minus3(int j) { return (2 * eis_cube_root(j) + 1) % kEisModuli[j]; }
 int real_modulus_value(int j) { return kRealModuli[j]; }
 
 int modulus_root(int j) {   // smallest positive s with s^2 = -1 (mod m); 0 for a non-2M modulus
@@ -99,12 +114,12 @@ static void memoised(int nmod, T* out, F&& build) {
     *out = cache[nmod];
 }
 
-static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTable* t) {
+static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTable* t, int (*root)(int) = modulus_root) {
     std::memset(t, 0, sizeof(*t));
     t->nmod = nmod;
     t->n2 = n2;
     for (int j = 0; j < nmod; ++j) {
-        const int m = mods[j], s = j < n2 ? modulus_root(j) : 1;
+        const int m = mods[j], s = j < n2 ? root(j) : 1;
         t->m[j] = m;
         t->s[j] = s;
         t->inv_m[j] = 1.0f / (float)m;
@@ -144,6 +159,9 @@ static void build_residue_table_for(const int* mods, int nmod, int n2, ResidueTa
 
 void build_residue_table(int nmod, ResidueTable* t) {
     memoised<ResidueTable, kMaxMod>(nmod, t, [&](ResidueTable* c) { build_residue_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_residue_table_eis(int nmod, ResidueTable* t) {
+    memoised<ResidueTable, kMaxEis>(nmod, t, [&](ResidueTable* c) { build_residue_table_for(kEisModuli, nmod, nmod, c, eis_sqrt_minus3); });
 }
 void build_residue_table_real(int nmod, ResidueTable* t) {
     memoised<ResidueTable, kMaxReal>(nmod, t, [&](ResidueTable* c) { build_residue_table_for(kRealModuli, nmod, 0, c); });
@@ -196,6 +214,14 @@ void build_mod_table(int nmod, bool per_plane, ModTable* t) {
     else memoised<ModTable, kMaxMod>(nmod, t, [&](ModTable* c) { build_mod_table_for(nmod, false, c); });
 }
 
+void build_mod_table_eis(int nmod, ModTable* t) {   // one entry per plane: the + planes, then the - planes
+    memoised<ModTable, kMaxEis>(nmod, t, [&](ModTable* c) {
+        std::memset(c, 0, sizeof(*c));
+        for (int p = 0; p < 2 * nmod; ++p) fill_mod_entry(c, p, kEisModuli, p % nmod);
+        c->nplanes = 2 * nmod;
+    });
+}
+
 void build_mod_table_real(int nmod, ModTable* t) {
     memoised<ModTable, kMaxReal>(nmod, t, [&](ModTable* c) {
         std::memset(c, 0, sizeof(*c));
@@ -210,6 +236,14 @@ static void folded_weights(int nmod, int j, const Big& M, Big* W, int* g, int* h
     *W = M;
     W->divmod_small((uint32_t)m);
     const int q = inv_mod((int)W->mod_small((uint32_t)m), m);
+    if (mods == kEisModuli) {
+        // The residue planes hold u +- d v = 2 (a + s b), 2 (a + s^2 b), so the products are 4 C+, 4 C-.  With
+        // C = (U + V sqrt(-3))/2:  U = C+ + C- = 4^-1 (sum of the planes), V = (C+ - C-)/d = -(4d)^-1 (minus plane - plus plane).
+        const int quarter = inv_mod(4, m);
+        *g = sym_mod((int64_t)quarter * q, m);
+        *h = sym_mod(-(int64_t)inv_mod(4 * eis_sqrt_minus3(j) % m, m) * q, m);
+        return;
+    }
     if (j >= n2) {                  // 3M modulus (Eq. (1)) or real scheme (Section 3.1): no factor besides q_j
         *g = *h = sym_mod(q, m);
         return;
@@ -236,7 +270,7 @@ static void build_crt_table_for(const int* mods, int nmod, int n2, CrtTable* t) 
     for (int j = 0; j < nmod; ++j) {
         Big W;
         int g, h;
-        folded_weights(nmod, j, M, &W, &g, &h, mods, mods == kModuli ? kMax2M : 0);
+        folded_weights(nmod, j, M, &W, &g, &h, mods, mods == kModuli ? kMax2M : mods == kEisModuli ? kMaxEis : 0);
         Big Gr = W, Gi = W;
         Gr.mul_small((uint32_t)std::abs(g));
         Gi.mul_small((uint32_t)std::abs(h));
@@ -251,6 +285,15 @@ static void build_crt_table_for(const int* mods, int nmod, int n2, CrtTable* t) 
 
 void build_crt_table(int nmod, CrtTable* t) {
     memoised<CrtTable, kMaxMod>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_crt_table_eis(int nmod, CrtTable* t) {
+    memoised<CrtTable, kMaxEis>(nmod, t, [&](CrtTable* c) {
+        build_crt_table_for(kEisModuli, nmod, nmod, c);
+        // result = (U + V sqrt(-3))/2: the real part is U/2, the imaginary part V sqrt(3)/2 with the factor as a double-double
+        c->re_shift = -1;
+        c->im_hi = 0x1.bb67ae8584caap-1;
+        c->im_lo = 0x1.cec95d0b5c1e3p-55;
+    });
 }
 void build_crt_table_real(int nmod, CrtTable* t) {
     memoised<CrtTable, kMaxReal>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kRealModuli, nmod, 0, c); });
@@ -297,6 +340,19 @@ ScaleTargets scale_targets(int nmod, int64_t k, bool herk) {
     return s;
 }
 
+// Eisenstein variant: lattice rounding moves a point by up to 0.578 and the coordinates U, V of an entry c of the product are
+// bounded by 2|c|: c_k = ceil(log2(5k)/2) keeps them below 2^P_t as long as the scaled parts reach 4 (P_B - c_k >= 2).
+ScaleTargets scale_targets_eis(int nmod, int64_t k) {
+    ScaleTargets s;
+    memoised<int, kMaxEis>(nmod, &s.Pt, [&](int* c) { *c = budget_bits(nmod, kEisModuli); });
+    s.PA = (s.Pt + 1) / 2;
+    s.PB = s.Pt / 2;
+    s.ck = 0;
+    const int64_t kk = k > 0 ? k : 1;
+    while ((1ull << (2 * s.ck)) < (uint64_t)(5 * kk)) ++s.ck;
+    return s;
+}
+
 // Real scheme (Section 3.1): a row has k real terms, c_k = ceil(log2(k)/2).
 ScaleTargets scale_targets_real(int nmod, int64_t k) {
     ScaleTargets s;
@@ -313,6 +369,8 @@ ScaleTargets scale_targets_real(int nmod, int64_t k) {
 static constexpr int64_t kAccLimit = 0x7FFFFFFFLL;
 
 int64_t gemm_k_limit_real() { return kAccLimit / (128 * 128); }   // the modulus 256 comes first
+
+int64_t gemm_k_limit_eis() { const int64_t h = (kEisModuli[0] - 1) / 2; return kAccLimit / (h * h); }
 
 int64_t gemm_k_limit(int nmod) {
     // largest |residue|: 120 for the 2M moduli (241 comes first), 128 once the hybrid adds the modulus 256

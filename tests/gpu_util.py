@@ -51,6 +51,8 @@ class Workspace:
         out = dict(layout=lay)
         out["eA"] = raw[lay["off_exp_a"]: lay["off_exp_a"] + 4 * rows_a].view(np.int32).copy()
         n2 = min(nmod, 22)                      # 2M moduli: planes X+ then X-; 3M moduli (hybrid): X_r, X_i, X_r + X_i
+        if op == b.OP_ZGEMM_EISENSTEIN:         # two planes for every modulus of the Eisenstein set
+            n2 = nmod
         n3 = nmod - n2
 
         def split(off, rows, ld):

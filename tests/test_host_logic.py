@@ -245,3 +245,52 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.gemm2m_set_workspace(one, 0) == ARG
     assert L.gemm2m_set_workspace(ctypes.c_void_p(8), 1024) == ARG              # not 256-byte aligned
     assert b.lib().gemm2m_status_string(WS) == b"GEMM2M_ERR_WORKSPACE"
+
+
+@pytest.mark.parametrize("nmod", [1, 2, 8, 16, 23])
+def test_eisenstein_constants_match_oracle(nmod):
+    from oracle import eisenstein as E
+    mods = E.greedy_eisenstein_moduli()[:nmod]
+    assert b.max_eisenstein_moduli() == len(E.greedy_eisenstein_moduli()) == 23
+    assert [b.eisenstein_modulus(j) for j in range(nmod)] == [(m, E.cube_root_of_unity(m)) for m in mods]
+    M = staged.product(mods)
+    for k in (1, 64, 8192, 10 ** 6):
+        t = b.debug_tables_eisenstein(nmod, k)
+        assert (t["Pt"], t["PA"], t["PB"], t["ck"]) == E.scaling_targets_e(M, k)
+    B = 2 ** 40
+    val = lambda row: sum(int(row[c]) * B ** c for c in range(5))
+    assert val(t["Mc"]) == M and all(t["Mc"][c] == 0 for c in range(t["nchunks"], 5))
+    assert (t["nchunks"] - 1) * 40 < max(((M - 1) // 2).bit_length(), 1) <= t["nchunks"] * 40
+    # Folded weights: with planes P+ = 2(a + s b), P- = 2(a + s^2 b) of both operands the products are 4 C+, 4 C-; the kernel
+    # forms sum_j gr_j (P-_j + P+_j) and sum_j gi_j (P-_j - P+_j), which must be U = 2 c_a - c_b and V = c_b modulo M.
+    rng = np.random.default_rng(nmod)
+    for _ in range(20):
+        ca, cb = (int(v) for v in rng.integers(-10 ** 9, 10 ** 9, 2))
+        U = V = 0
+        for j, m in enumerate(mods):
+            s = E.cube_root_of_unity(m)
+            cp, cm = staged.sym(4 * (ca + s * cb), m), staged.sym(4 * (ca + s * s * cb), m)
+            U += val(t["gr"][j]) * (cm + cp)
+            V += val(t["gi"][j]) * (cm - cp)
+        assert (U - (2 * ca - cb)) % M == 0 and (V - cb) % M == 0
+    for j, m in enumerate(mods):
+        assert abs(val(t["gr"][j])) <= (m - 1) // 2 * (M // m) and abs(val(t["gi"][j])) <= (m - 1) // 2 * (M // m)
+    # the residue kernels' reduction, exhaustively, as for the 2M moduli
+    assert (t["margin"] > 1.0).all()
+    for j, m in enumerate(mods):
+        y0_bits, xmax = int(t["y0_bits"][j]), int(t["xmax"][j])
+        y0 = (y0_bits - 0x4B000000) + 2 ** 23
+        assert y0 % (256 * m) == 0 and y0 - xmax >= 2 ** 23 and y0 + xmax < 2 ** 24
+        mant, ex = np.frexp(np.float64(t["inv_m"][j]))
+        n, e = int(mant * 2 ** 24), 24 - int(ex)
+        cq = int(t["cq"][j])
+        assert cq == 3 * 2 ** 22 - y0 // m
+        x = np.arange(-xmax, xmax + 1, dtype=np.int64)
+        num = (y0 + x) * n + (cq << e)
+        fl = num >> e
+        rem = num - (fl << e)
+        half = 1 << (e - 1)
+        tq = fl + ((rem > half) | ((rem == half) & (fl & 1 == 1)))
+        low = ((y0_bits + x) - (0x4B000000 + (tq - 2 ** 23)) * m) & 0xFF
+        res = np.where(low >= 128, low - 256, low)
+        assert np.array_equal(res, ((x + m // 2) % m) - m // 2), m
