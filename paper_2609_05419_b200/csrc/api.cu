@@ -256,7 +256,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     else { build_residue_table(nmod, &rtab); build_crt_table(nmod, &ctab); }
     // quantised parts stay below 2^(P - c_k) with the max-based rule and below 2^P with the 2-norm rule
     const bool two_norm_mode = !eis && g.scaling == 1 && k <= (1ll << 22);
-    const bool wideA = two_norm_mode ? sc.PA > 61 : sc.PA - sc.ck > 62, wideB = two_norm_mode ? sc.PB > 61 : sc.PB - sc.ck > 62;
+    // (Eisenstein variant: the coordinate u reaches 2^(P - c_k + 1) + 1)
+    const int head = eis ? 2 : 0;
+    const bool wideA = two_norm_mode ? sc.PA > 61 : sc.PA - sc.ck + head > 62, wideB = two_norm_mode ? sc.PB > 61 : sc.PB - sc.ck + head > 62;
 
     Phases ph;
     if (int s = begin_call(&ph)) return s;
@@ -292,12 +294,12 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
     if constexpr (sizeof(T) == 8) {
-        if (eis) CK(launch_residues_hex(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, apm, st, &g.launches[1]));
+        if (eis) CK(launch_residues_hex(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
     }
     if (!eis) { if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s; }
     if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
     if constexpr (sizeof(T) == 8) {
-        if (eis) CK(launch_residues_hex(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, bpm, st, &g.launches[1]));
+        if (eis) CK(launch_residues_hex(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
     }
     if (!eis) { if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s; }
     CK(ph.end(st));

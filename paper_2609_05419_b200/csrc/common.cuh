@@ -110,6 +110,8 @@ void build_residue_table_real(int nmod, ResidueTable* t);
 void build_mod_table_real(int nmod, ModTable* t);
 void build_crt_table_real(int nmod, CrtTable* t);
 ScaleTargets scale_targets_real(int nmod, int64_t k);
+// The same for the Eisenstein-integer variant (zgemm2m_eisenstein): moduli 247, 241, 229, ..., two planes per modulus, the
+// residue table's s_j = 2 (cube root) + 1, a square root of -3.
 int eis_modulus_value(int j);
 int eis_cube_root(int j);
 void build_residue_table_eis(int nmod, ResidueTable* t);
@@ -134,7 +136,7 @@ template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t row
 // true: operand row r is column r of X (B: k x n).
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
 cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                                const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
+                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
 // The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.

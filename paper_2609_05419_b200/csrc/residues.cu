@@ -53,8 +53,8 @@ __device__ __forceinline__ void quantise_part_wide(T v, int e, uint32_t* lo, lon
 // the 128-bit constant floor(2^127 2/sqrt 3), the product exact in 192 bits before the shift).  The nearest point with
 // u, v even is (2 rn(X), 2 rn(t/2)); it is at least as near as the nearest point with u, v odd, (2 floor(X) + 1,
 // 2 floor(t/2) + 1), exactly when |X - rn(X)| + (3/2) |t - 2 rn(t/2)| <= 1.  The signs of x and y carry over to u and v.
-// |u|, |v| < 2^82 by the scaling rule; returned like quantise_part_wide.
-__device__ __forceinline__ void quantise_hex(double x, double y, int e, uint32_t* ulo, long long* uup, uint32_t* vlo, long long* vup) {
+// |u|, |v| < 2^82 by the scaling rule (below 2^62 in the narrow mode).
+__device__ __forceinline__ void quantise_hex(double x, double y, int e, __int128* su_out, __int128* sv_out) {
     using F = FpBits<double>;
     typedef unsigned __int128 u128;
     auto split = [](double v, int e, unsigned long long* mant, int* sh) {
@@ -88,12 +88,8 @@ __device__ __forceinline__ void quantise_hex(double x, double y, int e, uint32_t
         u = ((Xf >> 32) << 1) | 1;
         v = ((Tf >> 33) << 1) | 1;
     }
-    const __int128 su = __double_as_longlong(x) < 0 ? -(__int128)u : (__int128)u;
-    const __int128 sv = __double_as_longlong(y) < 0 ? -(__int128)v : (__int128)v;
-    *ulo = (uint32_t)(u128)su;
-    *uup = (long long)(su >> 32);
-    *vlo = (uint32_t)(u128)sv;
-    *vup = (long long)(sv >> 32);
+    *su_out = __double_as_longlong(x) < 0 ? -(__int128)u : (__int128)u;
+    *sv_out = __double_as_longlong(y) < 0 ? -(__int128)v : (__int128)v;
 }
 
 __device__ __forceinline__ int dp4a_us(uint32_t a_unsigned, uint32_t b_signed, int c) {
@@ -326,7 +322,10 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
                     long long ur = 0, ui = 0;
                     if (ex != kExpNonFinite) {
                         if (HEX) {
-                            quantise_hex((double)v.x, (double)v.y, ex, &lr, &ur, &li, &ui);
+                            __int128 su, sv;
+                            quantise_hex((double)v.x, (double)v.y, ex, &su, &sv);
+                            lr = (uint32_t)(unsigned __int128)su; ur = (long long)(su >> 32);
+                            li = (uint32_t)(unsigned __int128)sv; ui = (long long)(sv >> 32);
                         } else {
                             quantise_part_wide<T>(v.x, ex, &lr, &ur);
                             quantise_part_wide<T>(v.y, ex, &li, &ui);
@@ -336,7 +335,14 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
                     di[i] = split_digits_wide(li, ui, &ti[i]);
                 } else {
                     long long qr = 0, qi = 0;
-                    if (fast) {
+                    if (HEX) {
+                        if (ex != kExpNonFinite) {
+                            __int128 su, sv;
+                            quantise_hex((double)v.x, (double)v.y, ex, &su, &sv);
+                            qr = (long long)su;
+                            qi = (long long)sv;
+                        }
+                    } else if (fast) {
                         qr = __double2ll_rz((double)v.x * scale);
                         qi = __double2ll_rz((double)v.y * scale);
                     } else if (ex != kExpNonFinite) {
@@ -393,20 +399,24 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
 
 // Eisenstein variant: the same kernel with the lattice rounding in front (complex double operands, 96-bit coordinates).
 cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                                const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches) {
+                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(double));
     static bool attr_set_dev[kMaxDevices] = {};
     bool& attr_set = attr_set_dev[current_device_slot()];
     if (!attr_set) {
         cudaError_t err = cudaFuncSetAttribute(residues_fp_kernel<double, true, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<double, false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<double, false, 16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         attr_set = true;
     }
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
     const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
-    residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
     ++*launches;
     return cudaGetLastError();
 }

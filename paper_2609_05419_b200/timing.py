@@ -6,6 +6,7 @@
 
   python -m paper_2609_05419_b200.timing --op dsyrk --n 8192 --k 8192 --nmod 16      (also zher2k, dsyr2k)
   python -m paper_2609_05419_b200.timing --op dgemm --m 8192 --n 8192 --k 8192 --nmod 15     (real Ozaki-II scheme)
+  python -m paper_2609_05419_b200.timing --op zgemm_eis --m 8192 --n 8192 --k 8192 --nmod 16 (Eisenstein-integer variant)
 
 Prints one JSON line: effective TFLOP/s (BLAS flop counts: 8mnk for GEMM, 4n^2k HERK, 8n^2k HER2K, n^2k SYRK, 2n^2k SYR2K,
 divided by the time), milliseconds per call and per phase.
@@ -24,7 +25,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm"])
+    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm", "zgemm_eis"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=8192)
@@ -56,7 +57,8 @@ def main():
     else:
         Ah, Bh = inputs.complex_inputs(m, n, k, a.seed, a.dist, a.phi, dtype=dtype)
         A, B = dev(Ah), dev(Bh)
-        opcode, flops = (b.OP_CGEMM if a.op == "cgemm" else b.OP_ZGEMM), 8.0 * m * n * k
+        opcode = {"cgemm": b.OP_CGEMM, "zgemm_eis": b.OP_ZGEMM_EISENSTEIN}.get(a.op, b.OP_ZGEMM)
+        flops = 8.0 * m * n * k
     C = torch.empty((n, m), dtype=tdtype, device="cuda").t()
     ws = torch.zeros(b.workspace_bytes(opcode, m, n, k, nmod), dtype=torch.uint8, device="cuda")
     b.set_workspace(ws)
@@ -75,6 +77,8 @@ def main():
             b.cgemm2m(A, B, C, nmod, stream)
         elif a.op == "dgemm":
             b.dgemm_ozaki2(A, B, C, nmod, stream)
+        elif a.op == "zgemm_eis":
+            b.zgemm2m_eisenstein(A, B, C, nmod, stream)
         else:
             b.zgemm2m(A, B, C, nmod, stream)
 
@@ -94,6 +98,8 @@ def main():
     b.device_status()
     total, per = b.last_launch_count()
     planes = 2 * min(nmod, 22) + 3 * max(nmod - 22, 0)       # complex GEMM: 2 real GEMMs per 2M modulus, 3 per 3M modulus
+    if a.op == "zgemm_eis":
+        planes = 2 * nmod
     gemms = {"zherk": nmod, "zher2k": 2 * nmod, "dsyrk": nmod, "dsyr2k": 2 * nmod, "dgemm": nmod}.get(a.op, planes)
     kin = (k + 1) // 2 if a.op in ("dsyrk", "dsyr2k") else k
     print(json.dumps({"op": a.op, "m": m, "n": n, "k": k, "nmod": nmod, "ms_per_call": ms, "effective_tflops": flops / ms / 1e9,
