@@ -12,8 +12,9 @@
  *
  * Beyond that path the library offers, each documented at its declaration: the hybrid 2M/3M moduli (nmod 23..26), the
  * BLAS-style forms with op(A), op(B), alpha, beta (zgemm2m_ex, cgemm2m_ex), the rank-k family of Section 5 (zherk2m,
- * zher2k2m, dsyrk2m, dsyr2k2m), an optional tighter choice of the scale factors (gemm2m_set_scaling) and the real
- * Ozaki-II scheme of Section 3.1 (dgemm_ozaki2).
+ * zher2k2m, dsyrk2m, dsyr2k2m), an optional tighter choice of the scale factors (gemm2m_set_scaling), the real
+ * Ozaki-II scheme of Section 3.1 (dgemm_ozaki2) and the Eisenstein-integer variant of Sections 3.2 and 4
+ * (zgemm2m_eisenstein).
  *
  * Conventions for every entry point
  *   - BLAS-3 style as in the paper's problem statement (Section 1: A in C^{m x k}, B in C^{k x n}; Section 6:
