@@ -156,9 +156,18 @@ int ensure_side_stream() {
 
 constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kernels
 
+// hex: the Eisenstein variant's lattice rounding in front of the same residue arithmetic (complex double only).
 template <typename T>
 int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st) {
+                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st, bool hex = false) {
+    if (hex) {
+        if constexpr (sizeof(T) == 8) {
+            CK(launch_residues_hex(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
+            return GEMM2M_OK;
+        } else {
+            return GEMM2M_ERR_ARG;
+        }
+    }
     if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
     else CK(launch_residues_tc<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, dev_status, D().sm_count, st, &g.launches[1]));
     return GEMM2M_OK;
@@ -293,15 +302,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
-    if constexpr (sizeof(T) == 8) {
-        if (eis) CK(launch_residues_hex(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
-    }
-    if (!eis) { if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st)) return s; }
+    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st, eis)) return s;
     if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    if constexpr (sizeof(T) == 8) {
-        if (eis) CK(launch_residues_hex(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, st, &g.launches[1]));
-    }
-    if (!eis) { if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st)) return s; }
+    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st, eis)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
