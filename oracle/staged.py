@@ -236,8 +236,9 @@ def scaling_exponents_2norm(Z, axis: int, P: int):
     return e
 
 
-def _quantise_part(x, e):
-    """trunc(x 2^-e) exactly, elementwise; x float array, e broadcastable integer array.  Object array of ints."""
+def _quantise_part(x, e, int64_ok: bool = False):
+    """trunc(x 2^-e) exactly, elementwise; x float array, e broadcastable integer array.  Object array of ints
+    (int64_ok: an int64 array instead when no entry needs a left shift -- the same values, for large inputs)."""
     x = np.asarray(x, dtype=np.float64)
     mant, ex = np.frexp(x)
     Mi = np.ldexp(mant, 53).astype(np.int64)             # x = Mi 2^(ex-53), |Mi| < 2^53, exact
@@ -245,9 +246,11 @@ def _quantise_part(x, e):
     sgn = np.sign(Mi)
     mag = np.abs(Mi)
     right = np.minimum(np.maximum(-sh, 0), 63)
-    out = (sgn * (mag >> right)).astype(object)          # truncation toward zero on the magnitude
+    out = sgn * (mag >> right)                           # truncation toward zero on the magnitude
     pos = sh > 0
-    if np.any(pos):
+    if not (int64_ok and not np.any(pos)):
+        out = out.astype(object)
+    if np.any(pos):                                      # left shifts: the value may not fit 64 bits
         flat_out = out.ravel()
         flat_M = Mi.ravel()
         flat_sh = np.broadcast_to(sh, x.shape).ravel()
@@ -257,11 +260,11 @@ def _quantise_part(x, e):
     return out
 
 
-def quantise(Z, e, axis: int):
+def quantise(Z, e, axis: int, int64_ok: bool = False):
     """Algorithm 1 step 3 with truncation: (Zr', Zi') = trunc(parts of Z / 2^e) with e per row (axis=1) or column (axis=0)."""
     Z = np.asarray(Z)
     eb = e[:, None] if axis == 1 else e[None, :]
-    return _quantise_part(Z.real, eb), _quantise_part(Z.imag, eb)
+    return _quantise_part(Z.real, eb, int64_ok), _quantise_part(Z.imag, eb, int64_ok)
 
 
 def round_int_nearest_even(X: int, bits: int):

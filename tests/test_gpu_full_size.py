@@ -146,3 +146,61 @@ def test_extensions_4096_sampled():
         got = Cr[idx[:, 0], idx[:, 1]].cpu().numpy()
     Cd, Dd = direct.zgemm4m_dd_samples(Ar.astype(np.complex128), Br.astype(np.complex128), pairs)
     assert direct.componentwise_error(got + 0j, Cd, Dd) <= 1e-14
+
+
+def test_zgemm_8192_full_coverage_of_the_integer_stages():
+    """Every element of every plane at the benchmark's size: (a) the residue planes of A for two moduli against the oracle's
+    quantiser and Eq. (2a) on all 67 M entries, and for all moduli on sampled rows of A and columns of B; (b) Eq. (2b) on all
+    2N planes by a Freivalds check modulo m_j: Cpm X = Bpm (Apm^T X) (mod m_j) for four random vectors X, computed exactly in
+    float64 (all partial sums stay below 2^31).  A wrong entry of a product plane escapes a vector with probability at most
+    1/p, p the smallest prime factor of m_j."""
+    m = n = k = 8192
+    nmod = 16
+    A, B = inputs.complex_inputs(m, n, k, seed=1, dist="phi", phi=0.5)
+    moduli = staged.greedy_2m_moduli()[:nmod]
+    roots = staged.roots_of(moduli)
+    M = staged.product(moduli)
+    Pt, PA, PB, ck = staged.scaling_targets(M, k)
+    eA, eB = staged.scaling_exponents(A, 1, PA, ck), staged.scaling_exponents(B, 0, PB, ck)
+    rng = np.random.default_rng(5)
+    X = rng.integers(0, 1024, (m, 4)).astype(np.float64)
+    with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, nmod)) as ws:
+        C = empty_dev(m, n, torch.complex128)
+        b.zgemm2m(to_dev(A), to_dev(B), C, nmod)
+        b.device_status()
+        lay = b.workspace_layout(b.OP_ZGEMM, m, n, k, nmod)
+        kp, ldp = lay["kp"], lay["ldp"]
+        assert kp == k and ldp == m
+
+        def plane(off, rows, ld, idx):
+            lo = off + idx * rows * ld
+            return ws.buf[lo: lo + rows * ld].cpu().numpy().view(np.int8).reshape(rows, ld)
+
+        assert (ws.buf[lay["off_exp_a"]: lay["off_exp_a"] + 4 * m].cpu().numpy().view(np.int32) == eA).all()
+        assert (ws.buf[lay["off_exp_b"]: lay["off_exp_b"] + 4 * n].cpu().numpy().view(np.int32) == eB).all()
+        # (b) Eq. (2b), every plane
+        for sgn in range(2):
+            for j, mj in enumerate(moduli):
+                idx = sgn * nmod + j
+                Ap = plane(lay["off_apm"], m, kp, idx).astype(np.float64)
+                Bp = plane(lay["off_bpm"], n, kp, idx).astype(np.float64)
+                Cp = plane(lay["off_cpm"], n, ldp, idx).astype(np.float64)     # Cp[col, row] = C+-[row, col]
+                assert np.abs(Ap).max() <= (mj - 1) // 2 and np.abs(Bp).max() <= (mj - 1) // 2 and np.abs(Cp).max() <= (mj - 1) // 2
+                inner = np.mod(Ap.T @ X, mj)                                    # (k x 4), entries < 2^31 before the reduction
+                assert np.array_equal(np.mod(Cp @ X, mj), np.mod(Bp @ inner, mj)), (sgn, j)
+        # (a) steps 3-4 on every entry of A for the first and the last modulus ...
+        Ar, Ai = staged.quantise(A, eA, 1, int64_ok=True)
+        assert Ar.dtype == np.int64
+        for j in (0, nmod - 1):
+            want = staged.pre_2m(Ar % moduli[j], Ai % moduli[j], moduli[j], roots[j])
+            for sgn in range(2):
+                assert np.array_equal(plane(lay["off_apm"], m, kp, sgn * nmod + j), want[sgn]), (sgn, j)
+        # ... and for every modulus on sampled rows of A and columns of B
+        rows = np.unique(np.concatenate([rng.integers(0, m, 96), [0, 1, 127, 128, m - 1]]))
+        Br, Bi = staged.quantise(B[:, rows], eB[rows], 0, int64_ok=True)
+        for j, mj in enumerate(moduli):
+            wa = staged.pre_2m(Ar[rows] % mj, Ai[rows] % mj, mj, roots[j])
+            wb = staged.pre_2m(Br % mj, Bi % mj, mj, roots[j])
+            for sgn in range(2):
+                assert np.array_equal(plane(lay["off_apm"], m, kp, sgn * nmod + j)[rows], wa[sgn]), ("A", sgn, j)
+                assert np.array_equal(plane(lay["off_bpm"], n, kp, sgn * nmod + j)[rows], wb[sgn].T), ("B", sgn, j)
