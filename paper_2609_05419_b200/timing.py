@@ -8,6 +8,10 @@
   python -m paper_2609_05419_b200.timing --op dgemm --m 8192 --n 8192 --k 8192 --nmod 15     (real Ozaki-II scheme)
   python -m paper_2609_05419_b200.timing --op zgemm_eis --m 8192 --n 8192 --k 8192 --nmod 16 (Eisenstein-integer variant)
 
+  python -m paper_2609_05419_b200.timing --op int8_yardstick --m 8192 --n 8192 --k 8192 --nmod 16
+      (NOT this library: 2 x nmod int8 GEMMs with int32 output by the vendor library through torch._int_mm, back to back,
+       as a yardstick for the tensor-core phase only)
+
 Prints one JSON line: effective TFLOP/s (BLAS flop counts: 8mnk for GEMM, 4n^2k HERK, 8n^2k HER2K, n^2k SYRK, 2n^2k SYR2K,
 divided by the time), milliseconds per call and per phase.
 """
@@ -23,9 +27,29 @@ from . import binding as b
 from . import inputs
 
 
+def yardstick(a):
+    """The vendor library's int8 GEMM (int32 output, no modular reduction) on operands of the residue planes' shape."""
+    g = torch.Generator(device="cuda").manual_seed(a.seed)
+    X = torch.randint(-120, 121, (a.m, a.k), dtype=torch.int8, device="cuda", generator=g)
+    Y = torch.randint(-120, 121, (a.n, a.k), dtype=torch.int8, device="cuda", generator=g).t()     # K-major like the planes
+    count = 2 * a.nmod
+    run = lambda: [torch._int_mm(X, Y) for _ in range(count)]
+    for _ in range(max(a.warmup, 1)):
+        run()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.steps
+    print(json.dumps({"op": a.op, "m": a.m, "n": a.n, "k": a.k, "gemms_per_step": count, "ms_per_step": ms,
+                      "int8_tops": 2.0 * count * a.m * a.n * a.k / ms / 1e9, "output": "int32, no reduction modulo m"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm", "zgemm_eis"])
+    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm", "zgemm_eis", "int8_yardstick"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=8192)
@@ -36,6 +60,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--seed", type=int, default=1)
     a = ap.parse_args()
+    if a.op == "int8_yardstick":
+        return yardstick(a)
     rank = a.op in ("zherk", "zher2k", "dsyrk", "dsyr2k")
     m, n, k, nmod = (a.n if rank else a.m), a.n, a.k, a.nmod
     dtype = np.complex64 if a.op == "cgemm" else np.complex128
