@@ -149,3 +149,57 @@ def test_2048_sampled_against_the_oracle():
     assert ulp_distance(C[np.ix_(rows, cols)].imag, sub["C"].imag).max() <= 1
     Cref, D = direct.zgemm4m_dd_samples(A, B, np.stack([rows, cols], axis=1))
     assert np.max(np.abs(C[rows, cols] - Cref) / D) < 1e-14
+
+
+def test_error_and_time_against_modulus_count_beside_the_gaussian_set():
+    """4096^3, phi = 0.5: the error of the Eisenstein variant falls by about M^-1/2 per modulus (Section 3.1) down to the
+    rounding floor; per modulus it is at least as accurate as zgemm2m from the point where its M is larger (Section 4: the
+    Eisenstein set decreases more slowly).  With GEMM2M_SWEEP_DIR set, the table is also written there as JSON."""
+    import json
+    import math
+    import os
+    m = n = k = 4096
+    A, B = inputs.complex_inputs(m, n, k, seed=2, dist="phi", phi=0.5)
+    pairs = inputs.sample_indices(m, n, 1024, seed=7, tile=128)
+    Cs, Ds = direct.zgemm4m_dd_samples(A, B, pairs)
+    idx = torch.from_numpy(pairs).cuda()
+    dA, dB = to_dev(A), to_dev(B)
+    nmods = list(range(8, 24))
+    rows = []
+    with Workspace(max(b.workspace_bytes(OP, m, n, k, 23), b.workspace_bytes(b.OP_ZGEMM, m, n, k, 22))):
+        C = empty_dev(m, n, torch.complex128)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for nmod in nmods:
+            row = dict(nmod=nmod)
+            for name, fn, mods in (("eis", b.zgemm2m_eisenstein, E.greedy_eisenstein_moduli()),
+                                   ("gauss", b.zgemm2m, staged.greedy_2m_moduli())):
+                if nmod > len(mods):
+                    continue
+                fn(dA, dB, C, nmod)                  # warm
+                e0.record()
+                for _ in range(3):
+                    fn(dA, dB, C, nmod)
+                e1.record()
+                b.device_status()
+                got = C[idx[:, 0], idx[:, 1]].cpu().numpy()
+                row[name] = dict(log2M=round(math.log2(staged.product(mods[:nmod])), 2), ms=e0.elapsed_time(e1) / 3,
+                                 max_err=direct.componentwise_error(got, Cs, Ds))
+            rows.append(row)
+    errs = {r["nmod"]: r["eis"]["max_err"] for r in rows}
+    floor = 4e-16
+    for a, c in zip(nmods, nmods[1:]):
+        assert errs[c] <= max(1.5 * errs[a], floor), (a, c, errs)
+        if errs[c] > 20 * floor:
+            assert errs[c] < errs[a] / 3, (a, c, errs)
+    assert errs[16] <= 1e-14 and all(errs[nm] <= 4 * floor for nm in nmods if nm >= 18)
+    slope = math.log2(errs[8] / errs[12]) / (rows[4]["eis"]["log2M"] - rows[0]["eis"]["log2M"])
+    assert 0.35 < slope < 0.65, slope
+    for r in rows:                                   # same error law for both rings: compare at equal M, not at equal N
+        if "gauss" in r and r["eis"]["max_err"] > 20 * floor and r["gauss"]["max_err"] > 20 * floor:
+            ratio = math.log2(r["gauss"]["max_err"] / r["eis"]["max_err"])
+            gap = 0.5 * (r["eis"]["log2M"] - r["gauss"]["log2M"])
+            assert abs(ratio - gap) < 2.5, (r, ratio, gap)
+    out_dir = os.environ.get("GEMM2M_SWEEP_DIR", "")
+    if out_dir and os.path.isdir(out_dir):
+        with open(os.path.join(out_dir, "sweep_nmod_eisenstein_4096.json"), "w") as f:
+            json.dump(rows, f, indent=1)
