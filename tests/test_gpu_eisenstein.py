@@ -203,3 +203,27 @@ def test_error_and_time_against_modulus_count_beside_the_gaussian_set():
     if out_dir and os.path.isdir(out_dir):
         with open(os.path.join(out_dir, "sweep_nmod_eisenstein_4096.json"), "w") as f:
             json.dump(rows, f, indent=1)
+
+
+def test_k_beyond_the_int32_range_of_one_gemm_and_ragged_padded_operands():
+    # k above 2^31 / 123^2 = 141 944: the GEMM runs in two K chunks whose residues are added modulo m_j
+    m, n, k, nmod = 3, 2, 142200, 4
+    A, B = inputs.complex_inputs(m, n, k, seed=9, dist="uniform")
+    C, st = run_e(A, B, nmod)
+    ref = E.zgemm_eisenstein_staged(A, B, nmod)
+    for j, mj in enumerate(ref["moduli"]):
+        for sgn in range(2):
+            assert (st["Cpm"][sgn, j, :, :m] == staged.sym(4 * ref["Cpm"][j][sgn].T, mj)).all(), (sgn, j)
+    assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
+    # ragged sizes with padded leading dimensions; the padding of C stays untouched
+    m, n, k, nmod = 131, 77, 301, 21
+    A, B = inputs.complex_inputs(m, n, k, seed=10, dist="phi", phi=2.0)
+    pad = lambda a, ld: np.asfortranarray(np.vstack([a, np.full((ld - a.shape[0], a.shape[1]), 99 + 1j, dtype=a.dtype)]))
+    with Workspace(b.workspace_bytes(OP, m, n, k, nmod)):
+        Cf = empty_dev(140, n, torch.complex128, fill=-7)
+        b.zgemm2m_eisenstein(to_dev(pad(A, 136))[:m], to_dev(pad(B, 320))[:k], Cf[:m], nmod)
+        b.device_status()
+        Cf = to_host(Cf)
+    ref = E.zgemm_eisenstein_staged(A, B, nmod)
+    assert (Cf[m:] == -7).all()
+    assert ulp_distance(Cf[:m].real, ref["C"].real).max() <= 1 and ulp_distance(Cf[:m].imag, ref["C"].imag).max() <= 1
