@@ -16,6 +16,11 @@ lattice.  Everything else is Algorithm 1 with the ring changed, written here in 
                                     reproduce bit for bit); pinned against the definition in the tests
   zgemm_eisenstein_staged           the whole path
 
+Parity unpinned: `greedy_eisenstein_moduli` against the paper.  Section 4 prints one figure for this variant, M ~ 2^154.5
+for the 8-bit moduli; the set defined here (every prime congruent to 1 mod 3 below 256 divides exactly one modulus) has
+M = 2^160.9, and no reading of the walk tried reproduces the printed figure.  The set is pinned by its definition and the
+qualitative claim (more bits than the Gaussian set's 2^152) only; everything else in this file is pinned by the tests.
+
 Readings (the paper only sketches this variant):
   * s is the smallest positive root;
   * scale factors as in Algorithm 1 step 2 from the largest |Re|, |Im| of a row / column, with c_k = ceil(log2(5k)/2):
