@@ -242,6 +242,14 @@ def test_argument_errors_are_reported_before_any_launch():
     assert L.zherk2m(4, 4, one, 3, one, 4, 16, null) == ARG
     assert L.zherk2m(0, 4, null, 1, null, 1, 16, null) == 0
     assert L.zherk2m(4, 4, one, 4, one, 4, 23, null) == NMOD                    # rank-k family: 2M moduli only
+    assert L.zgemm2m_eisenstein(4, 4, 4, one, 4, one, 4, one, 4, 24, null) == NMOD      # the Eisenstein set has 23 moduli
+    assert L.zgemm2m_eisenstein(4, 4, 4, one, 3, one, 4, one, 4, 16, null) == ARG
+    assert L.zgemm2m_eisenstein(4, 0, 4, null, 4, null, 4, null, 4, 16, null) == 0
+    assert L.zgemm2m_eisenstein_ex(b"X", b"N", 4, 4, 4, null, one, 4, one, 4, null, one, 4, 16, null) == ARG   # bad trans character
+    assert L.zgemm2m_eisenstein_ex(b"T", b"N", 4, 4, 8, null, one, 4, one, 8, null, one, 4, 16, null) == ARG   # A stored k x m: lda < k
+    assert b.workspace_bytes(b.OP_ZGEMM_EISENSTEIN, 64, 64, 64, 24) == 0 and b.workspace_bytes(b.OP_ZGEMM_EISENSTEIN, 64, 64, 64, 23) > 0
+    lay = b.workspace_layout(b.OP_ZGEMM_EISENSTEIN, 100, 90, 70, 23)
+    assert lay["off_apm"] + 2 * 23 * 100 * lay["kp"] <= lay["off_bpm"] and lay["off_cpm"] + 2 * 23 * 90 * lay["ldp"] <= lay["total_bytes"]
     assert L.gemm2m_set_workspace(one, 0) == ARG
     assert L.gemm2m_set_workspace(ctypes.c_void_p(8), 1024) == ARG              # not 256-byte aligned
     assert b.lib().gemm2m_status_string(WS) == b"GEMM2M_ERR_WORKSPACE"
