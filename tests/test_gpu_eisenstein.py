@@ -74,8 +74,8 @@ def test_lattice_rounding_on_cell_boundaries_and_special_values():
     for nmod in (6, 16):
         M = staged.product(E.greedy_eisenstein_moduli()[:nmod])
         Pt, PA, PB, ck = E.scaling_targets_e(M, k)
-        sigmas = (0, 20, -30)
-        A = np.zeros((3, k), dtype=np.complex128)
+        sigmas = (0, 20, -30, -1005, 900)         # the last two: exponents outside the kernel's fast scaling path
+        A = np.zeros((len(sigmas), k), dtype=np.complex128)
         for i, sg in enumerate(sigmas):
             A[i, 0] = 1.5 * 2.0 ** (sg + PA - ck - 1)
             A[i, 1:] = np.array(vals) * 2.0 ** sg
