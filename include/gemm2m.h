@@ -67,7 +67,7 @@ typedef enum {
 typedef enum {
     GEMM2M_OP_GAUSSIAN_INT = 0, GEMM2M_OP_ZGEMM = 1, GEMM2M_OP_CGEMM = 2, GEMM2M_OP_ZHERK = 3,
     GEMM2M_OP_ZHER2K = 4, GEMM2M_OP_DSYRK = 5, GEMM2M_OP_DSYR2K = 6, GEMM2M_OP_DGEMM_OZAKI2 = 7,
-    GEMM2M_OP_ZGEMM_EISENSTEIN = 8
+    GEMM2M_OP_ZGEMM_EISENSTEIN = 8, GEMM2M_OP_ZGEMM_HOST = 9
 } gemm2m_op;
 
 /* Human-readable name of a status code (static string). */
@@ -103,6 +103,19 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k,
  * complex128, lda >= m, ldb >= k, ldc >= m. */
 int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb,
             double* C, int64_t ldc, int nmod, void* stream);
+
+/* zgemm2m on HOST operands (the end-to-end form): A_host, B_host, C_host are host pointers with the layout of zgemm2m's A,
+ * B, C; the transfers are part of the call and overlap its kernels.  A is uploaded first (every GEMM needs all of its
+ * residue planes); B is uploaded in up to 32 column panels, and each panel is scanned, reduced to residues, multiplied and
+ * post-processed while the next one is on the bus (the scale factor of a column of B depends on that column alone, so the
+ * result is bit for bit zgemm2m's); each finished column panel of C is downloaded beside the next panel's work.  Copies run
+ * on two library-owned streams, one per direction, ordered against `stream` by events; the call is complete on `stream`
+ * when the last panel of C has arrived, and C_host, A_host, B_host must stay valid and unmodified until then.
+ * Page-locked host memory (cudaHostAlloc / cudaHostRegister, torch pin_memory) is needed for the copies to be asynchronous
+ * and to overlap; pageable memory works but serialises.  The workspace additionally holds compact device copies of A, B and
+ * C: gemm2m_workspace_bytes(GEMM2M_OP_ZGEMM_HOST, ...).  Always the max-based scaling rule; nmod up to 26. */
+int zgemm2m_host(int64_t m, int64_t n, int64_t k, const double* A_host, int64_t lda, const double* B_host, int64_t ldb,
+                 double* C_host, int64_t ldc, int nmod, void* stream);
 
 /* The same for complex single precision (interleaved complex64). */
 int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb,

@@ -12,6 +12,7 @@ import os
 
 OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K, OP_DGEMM_OZAKI2 = 0, 1, 2, 3, 4, 5, 6, 7
 OP_ZGEMM_EISENSTEIN = 8
+OP_ZGEMM_HOST = 9
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -55,6 +56,7 @@ def lib():
     L.gemm2m_gaussian_int.argtypes = [i64, i64, i64, vp, vp, i64, vp, vp, i64, vp, vp, i64, i32, vp]
     L.zgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.cgemm2m.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
+    L.zgemm2m_host.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     ex = [ctypes.c_char, ctypes.c_char, i64, i64, i64, vp, vp, i64, vp, i64, vp, vp, i64, i32, vp]
     L.zgemm2m_ex.argtypes = ex
     L.cgemm2m_ex.argtypes = ex
@@ -169,6 +171,28 @@ def _xgemm(fn, name, A, B, C, nmod, stream):
 
 def zgemm2m(A, B, C, nmod=16, stream=None):
     _xgemm(lib().zgemm2m, "zgemm2m", A, B, C, nmod, stream)
+
+
+def _colmajor_host(t, name):
+    """(pointer, rows, cols, leading dimension) of a 2-D CPU tensor stored column-major."""
+    if t.dim() != 2 or t.is_cuda:
+        raise ValueError(f"{name}: need a 2-D CPU tensor")
+    rows, cols = t.shape
+    if rows > 1 and t.stride(0) != 1:
+        raise ValueError(f"{name}: need column-major storage (stride 1 along dim 0), e.g. torch.empty(cols, rows).t()")
+    ld = t.stride(1) if cols > 1 else max(rows, 1)
+    return ctypes.c_void_p(t.data_ptr()), rows, cols, max(ld, 1)
+
+
+def zgemm2m_host(A, B, C, nmod=16, stream=None):
+    """C = A B with A, B, C complex128 CPU tensors (column-major views; pinned memory lets the copies overlap the kernels).
+    Asynchronous on `stream`: C is valid, and A, B may be changed, once the stream has completed."""
+    pa, m, k, lda = _colmajor_host(A, "A")
+    pb, k2, n, ldb = _colmajor_host(B, "B")
+    pc, mc, nc, ldc = _colmajor_host(C, "C")
+    if k != k2 or (mc, nc) != (m, n):
+        raise ValueError("shape mismatch")
+    _check(lib().zgemm2m_host(m, n, k, pa, lda, pb, ldb, pc, ldc, nmod, _stream_ptr(stream)), "zgemm2m_host")
 
 
 def cgemm2m(A, B, C, nmod=7, stream=None):

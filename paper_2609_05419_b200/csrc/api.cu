@@ -14,12 +14,17 @@ namespace {
 
 // Per-device part of the library state: the registered workspace, the side stream with its ordering events, and what was
 // learnt about the device.
+constexpr int kHostPanels = 32;   // most column panels of a zgemm2m_host call
+
 struct DevState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     cudaStream_t side = nullptr;  // library-owned stream on which the post-processing of a column panel overlaps the next panel's GEMMs
     cudaEvent_t panel_done[8] = {};
     cudaEvent_t side_done = nullptr;
+    // zgemm2m_host: one stream per copy direction, and the events that order copies and kernels
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t call_begin = nullptr, a_ready = nullptr, b_ready[kHostPanels] = {}, g_ready[kHostPanels] = {}, c_ready[kHostPanels] = {}, c_done = nullptr;
     int sm_count = 0;
     int arch_ok = -1;
 };
@@ -29,7 +34,7 @@ struct State {
     DevState dev[kMaxDevices];
     int cur = 0;                  // device of the call being served (set by use_current_device)
     int profiling = 0;
-    static constexpr int kProfSlots = 64, kMaxIntervals = 24, kMaxPanels = 8;
+    static constexpr int kProfSlots = 64, kMaxIntervals = 4 + 4 * kHostPanels, kMaxPanels = 8;
     struct Interval { cudaEvent_t a = nullptr, b = nullptr; int phase = 0; };
     struct Slot { Interval iv[kMaxIntervals]; int n = 0; };
     Slot slots[kProfSlots];       // timed intervals (phase, start, end) of the profiled calls
@@ -81,11 +86,14 @@ int check_device() {
 // 256-byte aligned.
 struct Carve {
     int64_t off_status, off_abs_a, off_abs_b, off_q_a, off_q_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
+    int64_t off_dev_a, off_dev_b, off_dev_c;      // zgemm2m_host: device copies of A (m x k), B (k x n) and C (m x n), compact
 };
 
 bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     if (m < 0 || n < 0 || k < 0 || nmod < 1 || nmod > kMaxMod) return false;
-    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_ZGEMM_EISENSTEIN) return false;
+    if (op < GEMM2M_OP_GAUSSIAN_INT || op > GEMM2M_OP_ZGEMM_HOST) return false;
+    const bool host = op == GEMM2M_OP_ZGEMM_HOST;                               // zgemm2m plus device copies of the operands
+    if (host) op = GEMM2M_OP_ZGEMM;
     const bool eis = op == GEMM2M_OP_ZGEMM_EISENSTEIN;                          // two planes per modulus of the Eisenstein set
     if (eis && nmod > kMaxEis) return false;
     const bool real_scheme = op == GEMM2M_OP_DGEMM_OZAKI2;                      // one plane per modulus of the real set
@@ -112,6 +120,9 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     c->off_apm = take(planes * m * kp);
     c->off_bpm = take((herk && !two) ? 0 : planes * n * kp);
     c->off_cpm = take((herk ? (int64_t)nmod : planes) * n * ldp);
+    c->off_dev_a = take(host ? 16 * m * k : 0);
+    c->off_dev_b = take(host ? 16 * k * n : 0);
+    c->off_dev_c = take(host ? 16 * m * n : 0);
     c->kp = kp;
     c->ldp = ldp;
     c->total = off;
@@ -151,6 +162,19 @@ int ensure_side_stream() {
     for (auto& e : D().panel_done)
         if (!e) CK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     if (!D().side_done) CK(cudaEventCreateWithFlags(&D().side_done, cudaEventDisableTiming));
+    return GEMM2M_OK;
+}
+
+int ensure_copy_streams() {
+    if (!D().h2d) CK(cudaStreamCreateWithFlags(&D().h2d, cudaStreamNonBlocking));
+    if (!D().d2h) CK(cudaStreamCreateWithFlags(&D().d2h, cudaStreamNonBlocking));
+    auto make = [](cudaEvent_t& e) { return e ? cudaSuccess : cudaEventCreateWithFlags(&e, cudaEventDisableTiming); };
+    CK(make(D().call_begin));
+    CK(make(D().a_ready));
+    CK(make(D().c_done));
+    for (auto& e : D().b_ready) CK(make(e));
+    for (auto& e : D().g_ready) CK(make(e));
+    for (auto& e : D().c_ready) CK(make(e));
     return GEMM2M_OK;
 }
 
@@ -331,6 +355,127 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     return GEMM2M_OK;
 }
 
+// zgemm2m on HOST operands: the copies are part of the call and overlap its kernels.  A goes up first (every GEMM needs all
+// of its planes); B goes up in column panels, and each panel is scanned, reduced to residues, multiplied and post-processed
+// while the next one is still on the bus; the finished column panel of C goes down beside the next panel's work.  The
+// copies run on two library-owned streams (one per direction), ordered against the caller's stream by events; the call is
+// complete on the caller's stream when the last panel of C has arrived in host memory.
+int zgemm_host(int64_t m, int64_t n, int64_t k, const double* hA, int64_t lda, const double* hB, int64_t ldb, double* hC, int64_t ldc,
+               int nmod, void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (m < 0 || n < 0 || k < 0) return GEMM2M_ERR_ARG;
+    if (lda < (m > 1 ? m : 1) || ldb < (k > 1 ? k : 1) || ldc < (m > 1 ? m : 1)) return GEMM2M_ERR_ARG;
+    if (nmod < 1 || nmod > kMaxMod) return GEMM2M_ERR_NMOD;
+    if (m > kMaxRows || n > kMaxRows) return GEMM2M_ERR_ARG;
+    if (m == 0 || n == 0) return GEMM2M_OK;
+    if (!hC || (k > 0 && (!hA || !hB))) return GEMM2M_ERR_ARG;
+    if (int s = check_device()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    Carve c;
+    if (!carve(GEMM2M_OP_ZGEMM_HOST, m, n, k, nmod, &c)) return GEMM2M_ERR_ARG;
+    if (!D().ws || D().ws_bytes < (size_t)c.total) return GEMM2M_ERR_WORKSPACE;
+    char* ws = (char*)D().ws;
+    double* dA = (double*)(ws + c.off_dev_a);
+    double* dB = (double*)(ws + c.off_dev_b);
+    double* dC = (double*)(ws + c.off_dev_c);
+    const size_t col_a = (size_t)m * 16, col_b = (size_t)k * 16;              // bytes of one column of A / C and of B
+    std::memset(g.launches, 0, sizeof(g.launches));
+    if (k == 0) {                                                              // C = 0
+        CK(cudaMemsetAsync(dC, 0, col_a * (size_t)n, st));
+        CK(cudaMemcpy2DAsync(hC, (size_t)ldc * 16, dC, col_a, col_a, (size_t)n, cudaMemcpyDeviceToHost, st));
+        return GEMM2M_OK;
+    }
+    if (int s = ensure_side_stream()) return s;
+    if (int s = ensure_copy_streams()) return s;
+    int* dev_status = (int*)(ws + c.off_status);
+    uint64_t* absA = (uint64_t*)(ws + c.off_abs_a);
+    uint64_t* absB = (uint64_t*)(ws + c.off_abs_b);
+    int32_t* eA = (int32_t*)(ws + c.off_exp_a);
+    int32_t* eB = (int32_t*)(ws + c.off_exp_b);
+    int8_t* apm = (int8_t*)(ws + c.off_apm);
+    int8_t* bpm = (int8_t*)(ws + c.off_bpm);
+    int8_t* cpm = (int8_t*)(ws + c.off_cpm);
+    const ScaleTargets sc = scale_targets(nmod, k, false);
+    ResidueTable rtab;
+    CrtTable ctab;
+    build_residue_table(nmod, &rtab);
+    build_crt_table(nmod, &ctab);
+    const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
+    Phases ph;
+    if (int s = begin_call(&ph)) return s;
+
+    // column panels of B and C: narrow, so that the last panel's kernels and download, which nothing hides, stay short
+    // (the kernels hide behind the upload of B whatever the panel width; 256-column panels measured 43.4 ms per call at
+    // 8192^3 against 44.4 ms with 512 and 45.3 ms with 1024 columns)
+    int panels = (int)(n / 256);
+    panels = panels < 1 ? 1 : (panels > kHostPanels ? kHostPanels : panels);
+    const int64_t panel_cols = round_up((n + panels - 1) / panels, 256);
+
+    // uploads: after everything the caller's stream holds so far (an earlier call may still read the device copies)
+    cudaStream_t up = D().h2d, down = D().d2h, side = D().side;
+    CK(cudaEventRecord(D().call_begin, st));
+    CK(cudaStreamWaitEvent(up, D().call_begin, 0));
+    CK(cudaMemcpy2DAsync(dA, col_a, hA, (size_t)lda * 16, col_a, (size_t)k, cudaMemcpyHostToDevice, up));
+    CK(cudaEventRecord(D().a_ready, up));
+    int used = 0;
+    for (int p = 0; p < panels; ++p) {
+        const int64_t j0 = p * panel_cols, j1 = (j0 + panel_cols < n && p + 1 < panels) ? j0 + panel_cols : n;
+        if (j0 >= j1) break;
+        CK(cudaMemcpy2DAsync(dB + 2 * j0 * k, col_b, hB + 2 * j0 * ldb, (size_t)ldb * 16, col_b, (size_t)(j1 - j0), cudaMemcpyHostToDevice, up));
+        CK(cudaEventRecord(D().b_ready[p], up));
+        used = p + 1;
+    }
+    // A: steps 2-4 as in zgemm2m
+    CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
+    CK(cudaStreamWaitEvent(st, D().a_ready, 0));
+    CK(ph.begin(0, st));
+    CK(launch_scan_rows<double>(dA, m, k, m, absA, st, &g.launches[0]));
+    CK(launch_exponents<double>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));
+    CK(ph.end(st));
+    CK(ph.begin(1, st));
+    CK(launch_residues_fp<double>(dA, m, false, false, m, k, c.kp, eA, rtab, wideA, apm, st, &g.launches[1]));
+    CK(ph.end(st));
+    GemmArgs ga;
+    ga.rowop = bpm; ga.colop = apm;
+    ga.R = n; ga.Cn = m; ga.Kp = c.kp;
+    ga.row_planes = ga.col_planes = plane_count(nmod);
+    ga.row_plane0 = ga.col_plane0 = 0;
+    ga.nbatch = plane_count(nmod);
+    ga.out = cpm; ga.ldp = c.ldp; ga.accumulate = 0;
+    build_mod_table(nmod, true, &ga.mods);
+    ga.dev_status = dev_status;
+    for (int p = 0; p < used; ++p) {
+        const int64_t j0 = p * panel_cols, j1 = (j0 + panel_cols < n && p + 1 < panels) ? j0 + panel_cols : n;
+        const double* Bp = dB + 2 * j0 * k;
+        // the scale factor of a column of B depends on that column alone: steps 2-4 of this panel's columns
+        CK(cudaStreamWaitEvent(st, D().b_ready[p], 0));
+        CK(ph.begin(0, st));
+        CK(launch_scan_cols<double>(Bp, k, j1 - j0, k, absB + j0, st, &g.launches[0]));
+        CK(launch_exponents<double>(absB + j0, j1 - j0, sc.PB, sc.ck, eB + j0, st, &g.launches[0]));
+        CK(ph.end(st));
+        CK(ph.begin(1, st));
+        CK(launch_residues_fp<double>(Bp, k, true, false, j1 - j0, k, c.kp, eB + j0, rtab, wideB, bpm + j0 * c.kp, st, &g.launches[1], n));
+        CK(ph.end(st));
+        CK(ph.begin(2, st));
+        ga.row_begin = j0; ga.row_end = j1;
+        if (int s = run_gemm(ga, gemm_k_limit(nmod), st)) return s;
+        CK(ph.end(st));
+        // Eq. (2c) + steps 5-7 of the panel on the side stream, then its columns of C go down
+        CK(cudaEventRecord(D().g_ready[p], st));
+        CK(cudaStreamWaitEvent(side, D().g_ready[p], 0));
+        CK(ph.begin(3, side));
+        CK(launch_post_fp<double>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, dC, m, nullptr, nullptr, side, &g.launches[3]));
+        CK(ph.end(side));
+        CK(cudaEventRecord(D().c_ready[p], side));
+        CK(cudaStreamWaitEvent(down, D().c_ready[p], 0));
+        CK(cudaMemcpy2DAsync(hC + 2 * j0 * ldc, (size_t)ldc * 16, dC + 2 * j0 * m, col_a, col_a, (size_t)(j1 - j0), cudaMemcpyDeviceToHost, down));
+    }
+    CK(cudaEventRecord(D().c_done, down));
+    CK(cudaStreamWaitEvent(st, D().c_done, 0));
+    ph.done();
+    return GEMM2M_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -449,6 +594,11 @@ int gemm2m_gaussian_int(int64_t m, int64_t n, int64_t k, const int8_t* Ar, const
 int zgemm2m(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc,
             int nmod, void* stream) {
     return xgemm2m<double>(GEMM2M_OP_ZGEMM, 'N', 'N', m, n, k, nullptr, A, lda, B, ldb, nullptr, C, ldc, nmod, stream);
+}
+
+int zgemm2m_host(int64_t m, int64_t n, int64_t k, const double* A_host, int64_t lda, const double* B_host, int64_t ldb, double* C_host,
+                 int64_t ldc, int nmod, void* stream) {
+    return zgemm_host(m, n, k, A_host, lda, B_host, ldb, C_host, ldc, nmod, stream);
 }
 
 int cgemm2m(int64_t m, int64_t n, int64_t k, const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc, int nmod,

@@ -137,8 +137,11 @@ template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t row
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
 cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
                                 const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+// plane_rows: rows of a whole plane when the launch covers a row range of the operand only (X, e and planes then point at the
+// first row of the range); 0 = R.
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
-                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches,
+                                                     int64_t plane_rows = 0);
 // The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.
 template <typename T> cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status,

@@ -258,7 +258,8 @@ template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm vol
 template <typename T, bool WIDE, int NMOD, bool HEX = false>
 __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K,
                                                                      int64_t Kp, const int32_t* __restrict__ e,
-                                                                     const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes) {
+                                                                     const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes,
+                                                                     int64_t plane_rows) {
     using Raw = typename RawCplx<T>::type;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Raw* ring = reinterpret_cast<Raw*>(smem_raw);
@@ -266,7 +267,7 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
     const int t = threadIdx.x;
     const int64_t ktiles = Kp / kResK;
     const int64_t total = ((R + kResRows - 1) / kResRows) * ktiles;
-    const int64_t plane_stride = R * Kp;
+    const int64_t plane_stride = plane_rows * Kp;     // rows of a whole plane (R when the launch covers the operand, more for a row range)
 
     auto issue = [&](int64_t tile, int stage) {
         const int64_t row0 = (tile / ktiles) * kResRows, k0 = (tile % ktiles) * kResK;
@@ -364,7 +365,7 @@ constexpr size_t kResSmemBytes(size_t elem) { return (size_t)kResStages * kResRo
 
 template <typename T>
 cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
+                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, int64_t plane_rows) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
     static bool attr_set_dev[kMaxDevices] = {};
@@ -386,12 +387,12 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
     // saves two instructions per (element, modulus) -- 13 % of the kernel's time at 16 moduli.
     const int spec = (!wide && tab.n2 == tab.nmod) ? tab.nmod : 0;
     switch (spec) {
-#define GEMM2M_RES_CASE(N) case N: residues_fp_kernel<T, false, N><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes); break;
+#define GEMM2M_RES_CASE(N) case N: residues_fp_kernel<T, false, N><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R); break;
         GEMM2M_RES_CASE(7) GEMM2M_RES_CASE(8) GEMM2M_RES_CASE(14) GEMM2M_RES_CASE(15) GEMM2M_RES_CASE(16)
 #undef GEMM2M_RES_CASE
         default:
-            if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
-            else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+            if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
+            else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
     }
     ++*launches;
     return cudaGetLastError();
@@ -401,6 +402,7 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
 cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
                                 const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
+    constexpr int64_t plane_rows = 0;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(double));
     static bool attr_set_dev[kMaxDevices] = {};
     bool& attr_set = attr_set_dev[current_device_slot()];
@@ -414,9 +416,9 @@ cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, 
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
     const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
-    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
-    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
-    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes);
+    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
+    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
+    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
     ++*launches;
     return cudaGetLastError();
 }
@@ -597,7 +599,7 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
     return cudaGetLastError();
 }
 
-template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
-template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*);
+template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t);
+template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t);
 
 }  // namespace gemm2m

@@ -8,6 +8,7 @@
   python -m paper_2609_05419_b200.timing --op dgemm --m 8192 --n 8192 --k 8192 --nmod 15     (real Ozaki-II scheme)
   python -m paper_2609_05419_b200.timing --op zgemm_eis --m 8192 --n 8192 --k 8192 --nmod 16 (Eisenstein-integer variant)
 
+  python -m paper_2609_05419_b200.timing --op zgemm_host --m 8192 --n 8192 --k 8192 --nmod 16 (host operands, copies inside the call)
   python -m paper_2609_05419_b200.timing --op int8_yardstick --m 8192 --n 8192 --k 8192 --nmod 16
       (NOT this library: 2 x nmod int8 GEMMs with int32 output by the vendor library through torch._int_mm, back to back,
        as a yardstick for the tensor-core phase only)
@@ -47,9 +48,40 @@ def yardstick(a):
                       "int8_tops": 2.0 * count * a.m * a.n * a.k / ms / 1e9, "output": "int32, no reduction modulo m"}))
 
 
+def host_call(a):
+    """zgemm2m_host on pinned host operands: milliseconds per call with the transfers inside."""
+    m, n, k, nmod = a.m, a.n, a.k, a.nmod
+    Ah, Bh = inputs.complex_inputs(m, n, k, a.seed, a.dist, a.phi)
+    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x.T)).pin_memory().t()
+    A, B = pin(Ah), pin(Bh)
+    C = torch.empty((n, m), dtype=torch.complex128).pin_memory().t()
+    ws = torch.zeros(b.workspace_bytes(b.OP_ZGEMM_HOST, m, n, k, nmod), dtype=torch.uint8, device="cuda")
+    b.set_workspace(ws)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(a.warmup, 1)):
+        b.zgemm2m_host(A, B, C, nmod, stream)
+    b.device_status()
+    b.set_profiling(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(a.steps):
+        b.zgemm2m_host(A, B, C, nmod, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.steps
+    phase, _ = b.phase_ms()
+    b.set_profiling(False)
+    b.device_status()
+    print(json.dumps({"op": a.op, "m": m, "n": n, "k": k, "nmod": nmod, "ms_per_call": ms, "effective_tflops": 8.0 * m * n * k / ms / 1e9,
+                      "h2d_bytes": 16 * (m * k + k * n), "d2h_bytes": 16 * m * n,
+                      "bus_gbs_h2d_if_alone": 16 * (m * k + k * n) / ms / 1e6,
+                      "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3]}))
+    b.set_workspace(None)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm", "zgemm_eis", "int8_yardstick"])
+    ap.add_argument("--op", default="zgemm", choices=["zgemm", "cgemm", "zherk", "zher2k", "dsyrk", "dsyr2k", "dgemm", "zgemm_eis", "zgemm_host", "int8_yardstick"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=8192)
@@ -62,6 +94,8 @@ def main():
     a = ap.parse_args()
     if a.op == "int8_yardstick":
         return yardstick(a)
+    if a.op == "zgemm_host":
+        return host_call(a)
     rank = a.op in ("zherk", "zher2k", "dsyrk", "dsyr2k")
     m, n, k, nmod = (a.n if rank else a.m), a.n, a.k, a.nmod
     dtype = np.complex64 if a.op == "cgemm" else np.complex128

@@ -250,6 +250,12 @@ def test_argument_errors_are_reported_before_any_launch():
     assert b.workspace_bytes(b.OP_ZGEMM_EISENSTEIN, 64, 64, 64, 24) == 0 and b.workspace_bytes(b.OP_ZGEMM_EISENSTEIN, 64, 64, 64, 23) > 0
     lay = b.workspace_layout(b.OP_ZGEMM_EISENSTEIN, 100, 90, 70, 23)
     assert lay["off_apm"] + 2 * 23 * 100 * lay["kp"] <= lay["off_bpm"] and lay["off_cpm"] + 2 * 23 * 90 * lay["ldp"] <= lay["total_bytes"]
+    assert L.zgemm2m_host(4, 4, 4, one, 3, one, 4, one, 4, 16, null) == ARG                 # host form: same checks
+    assert L.zgemm2m_host(4, 4, 4, one, 4, one, 4, null, 4, 16, null) == ARG
+    assert L.zgemm2m_host(4, 4, 4, one, 4, one, 4, one, 4, 27, null) == NMOD
+    assert L.zgemm2m_host(0, 4, 4, null, 1, null, 4, null, 1, 16, null) == 0
+    z, h = b.workspace_bytes(b.OP_ZGEMM, 300, 200, 100, 16), b.workspace_bytes(b.OP_ZGEMM_HOST, 300, 200, 100, 16)
+    assert h >= z + 16 * (300 * 100 + 100 * 200 + 300 * 200) and h < z + 16 * (300 * 100 + 100 * 200 + 300 * 200) + 3 * 256
     assert L.gemm2m_set_workspace(one, 0) == ARG
     assert L.gemm2m_set_workspace(ctypes.c_void_p(8), 1024) == ARG              # not 256-byte aligned
     assert b.lib().gemm2m_status_string(WS) == b"GEMM2M_ERR_WORKSPACE"
