@@ -10,7 +10,8 @@
  *   4. C = 2^-1 (C- + C+) + i s_j 2^-1 (C- - C+) (mod m_j), Eq. (2c); CRT over j (Section 3.1; Algorithm 1
  *      step 5); lift to the symmetric range (step 6); multiply by sigma_i tau_j (step 7).
  *
- * Beyond that path the library offers, each documented at its declaration: the hybrid 2M/3M moduli (nmod 23..26), the
+ * Beyond that path the library offers, each documented at its declaration: the same call on host operands with the
+ * transfers overlapped inside it (zgemm2m_host), the hybrid 2M/3M moduli (nmod 23..26), the
  * BLAS-style forms with op(A), op(B), alpha, beta (zgemm2m_ex, cgemm2m_ex), the rank-k family of Section 5 (zherk2m,
  * zher2k2m, dsyrk2m, dsyr2k2m), an optional tighter choice of the scale factors (gemm2m_set_scaling), the real
  * Ozaki-II scheme of Section 3.1 (dgemm_ozaki2) and the Eisenstein-integer variant of Sections 3.2 and 4
