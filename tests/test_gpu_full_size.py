@@ -148,12 +148,12 @@ def test_extensions_4096_sampled():
     assert direct.componentwise_error(got + 0j, Cd, Dd) <= 1e-14
 
 
-def test_zgemm_8192_full_coverage_of_the_integer_stages():
+def test_zgemm_8192_full_coverage_of_every_stage():
     """Every element of every plane at the benchmark's size: (a) the residue planes of A for two moduli against the oracle's
     quantiser and Eq. (2a) on all 67 M entries, and for all moduli on sampled rows of A and columns of B; (b) Eq. (2b) on all
     2N planes by a Freivalds check modulo m_j: Cpm X = Bpm (Apm^T X) (mod m_j) for four random vectors X, computed exactly in
     float64 (all partial sums stay below 2^31).  A wrong entry of a product plane escapes a vector with probability at most
-    1/p, p the smallest prime factor of m_j."""
+    1/p, p the smallest prime factor of m_j; (c) the final C on all entries through C x = A (B x) in extended precision."""
     m = n = k = 8192
     nmod = 16
     A, B = inputs.complex_inputs(m, n, k, seed=1, dist="phi", phi=0.5)
@@ -171,6 +171,7 @@ def test_zgemm_8192_full_coverage_of_the_integer_stages():
         lay = b.workspace_layout(b.OP_ZGEMM, m, n, k, nmod)
         kp, ldp = lay["kp"], lay["ldp"]
         assert kp == k and ldp == m
+        Cfull = to_host(C)
 
         def plane(off, rows, ld, idx):
             lo = off + idx * rows * ld
@@ -204,3 +205,18 @@ def test_zgemm_8192_full_coverage_of_the_integer_stages():
             for sgn in range(2):
                 assert np.array_equal(plane(lay["off_apm"], m, kp, sgn * nmod + j)[rows], wa[sgn]), ("A", sgn, j)
                 assert np.array_equal(plane(lay["off_bpm"], n, kp, sgn * nmod + j)[rows], wb[sgn].T), ("B", sgn, j)
+    # (c) steps 5-7, every entry of C, as a net for gross errors: C x = A (B x) for a random +-1 vector x, the right-hand side in
+    # extended precision.  An entry of C that is off by more than about 1e-10 |A||B| would show in its row.
+    L = np.clongdouble
+    x = rng.choice([-1.0, 1.0], n)
+    y = np.zeros(k, dtype=L)
+    for c0 in range(0, n, 1024):
+        y += B[:, c0:c0 + 1024].astype(L) @ x[c0:c0 + 1024].astype(L)
+    lhs, rhs, scale = np.zeros(m, dtype=L), np.zeros(m, dtype=L), np.zeros(m)
+    absBx = np.abs(B) @ np.ones(n)
+    for c0 in range(0, k, 1024):
+        rhs += A[:, c0:c0 + 1024].astype(L) @ y[c0:c0 + 1024]
+        scale += np.abs(A[:, c0:c0 + 1024]) @ absBx[c0:c0 + 1024]
+    for c0 in range(0, n, 1024):
+        lhs += Cfull[:, c0:c0 + 1024].astype(L) @ x[c0:c0 + 1024].astype(L)
+    assert np.max(np.abs(lhs - rhs).astype(np.float64) / scale) < 1e-14
