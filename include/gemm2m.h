@@ -21,12 +21,12 @@
  *   - BLAS-3 style as in the paper's problem statement (Section 1: A in C^{m x k}, B in C^{k x n}; Section 6:
  *     alpha = 1, beta = 0): column-major, complex numbers interleaved (re, im), leading dimensions counted in
  *     elements (complex elements for complex matrices), no transposition arguments, C is overwritten.
- *   - All matrix pointers are DEVICE pointers owned by the caller.  The library never allocates or frees device
+ *   - All matrix pointers are DEVICE pointers owned by the caller (zgemm2m_host alone takes host pointers).  The library never allocates or frees device
  *     memory inside a call; it uses the caller-provided workspace registered with gemm2m_set_workspace().
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and
  *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  zgemm2m and cgemm2m
  *     additionally use one library-owned stream, forked from and joined back into `stream` with events: work enqueued
- *     on `stream` after the call still sees the finished result.
+ *     on `stream` after the call still sees the finished result.  (zgemm2m_host uses two more, for its copies.)
  *   - Because a call only enqueues (kernels, memsets, event records and waits), it can be captured into a CUDA graph
  *     and replayed; the library-owned stream joins the capture through its fork/join events.  Make one call outside any
  *     capture first: it creates that stream and its events.  (gemm2m_set_profiling must be off during a capture.)
