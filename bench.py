@@ -133,7 +133,13 @@ class ClockSampler:
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        self.index = index
+        self.index = str(index)
+        try:    # nvidia-smi numbers the GPUs it sees, CUDA the ones it was given: name the device by its PCI address instead
+            import torch
+            pr = torch.cuda.get_device_properties(index)
+            self.index = "%08x:%02x:%02x.0" % (pr.pci_domain_id, pr.pci_bus_id, pr.pci_device_id)
+        except Exception:
+            pass
         self.proc = None
         self.path = None
 
