@@ -82,10 +82,10 @@ int check_device() {
     return D().arch_ok ? GEMM2M_OK : GEMM2M_ERR_ARCH;
 }
 
-// Workspace: [status 256 B][absmax A u64][absmax B u64][sumsq A u64][sumsq B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each
+// Workspace: [status 256 B][post-processing operand 3 KB][absmax A u64][absmax B u64][sumsq A u64][sumsq B u64][exp A i32][exp B i32][Apm][Bpm][Cpm], each
 // 256-byte aligned.
 struct Carve {
-    int64_t off_status, off_abs_a, off_abs_b, off_q_a, off_q_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
+    int64_t off_status, off_frags, off_abs_a, off_abs_b, off_q_a, off_q_b, off_exp_a, off_exp_b, off_pack_a, off_pack_b, off_apm, off_bpm, off_cpm, kp, ldp, total;
     int64_t off_dev_a, off_dev_b, off_dev_c;      // zgemm2m_host: device copies of A (m x k), B (k x n) and C (m x n), compact
 };
 
@@ -108,6 +108,7 @@ bool carve(int op, int64_t m, int64_t n, int64_t k, int nmod, Carve* c) {
     int64_t off = 0;
     auto take = [&](int64_t bytes) { int64_t o = off; off = round_up(off + bytes, 256); return o; };
     c->off_status = take(256);
+    c->off_frags = take(4 * kPostFragWords);    // tensor-core operand of the complex GEMMs' post-processing (digits of the CRT weights)
     c->off_abs_a = take(8 * m);
     c->off_abs_b = take(herk ? 0 : 8 * n);
     c->off_q_a = take(herk ? 0 : 8 * m);        // sums of squares of the 2-norm scaling rule (zeroed together with the maxima)
@@ -284,9 +285,10 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     const ScaleTargets sc = eis ? scale_targets_eis(nmod, k) : scale_targets(nmod, k, false);
     if (eis && sc.PB - sc.ck < 2) return GEMM2M_ERR_NMOD;          // the lattice rounding needs scaled parts of 4 or more
     ResidueTable rtab;
-    CrtTable ctab;
-    if (eis) { build_residue_table_eis(nmod, &rtab); build_crt_table_eis(nmod, &ctab); }
-    else { build_residue_table(nmod, &rtab); build_crt_table(nmod, &ctab); }
+    PostMmaTable ptab;
+    if (eis) { build_residue_table_eis(nmod, &rtab); build_post_mma_table_eis(nmod, &ptab); }
+    else { build_residue_table(nmod, &rtab); build_post_mma_table(nmod, &ptab); }
+    uint32_t* frags = (uint32_t*)(ws + c.off_frags);
     // quantised parts stay below 2^(P - c_k) with the max-based rule and below 2^P with the 2-norm rule
     const bool two_norm_mode = !eis && g.scaling == 1 && k <= (1ll << 22);
     // (Eisenstein variant: the coordinate u reaches 2^(P - c_k + 1) + 1)
@@ -301,6 +303,7 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     if (int s = ensure_side_stream()) return s;
     cudaStream_t sb = g.max_panels > 1 ? D().side : st;
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
+    CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
     if (sb != st) {
         CK(cudaEventRecord(D().panel_done[0], st));
         CK(cudaStreamWaitEvent(sb, D().panel_done[0], 0));
@@ -349,7 +352,7 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     if (int s = panel_pipeline(n, st, ph,
             [&](int64_t j0, int64_t j1) { ga.row_begin = j0; ga.row_end = j1; return run_gemm(ga, klim, st); },
             [&](int64_t j0, int64_t j1, cudaStream_t ps) {
-                return launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, alpha, beta, ps, &g.launches[3]);
+                return launch_post_fp<T>(cpm, c.ldp, m, n, j0, j1, eA, eB, ptab, frags, C, ldc, alpha, beta, ps, &g.launches[3]);
             })) return s;
     ph.done();
     return GEMM2M_OK;
@@ -397,9 +400,10 @@ int zgemm_host(int64_t m, int64_t n, int64_t k, const double* hA, int64_t lda, c
     int8_t* cpm = (int8_t*)(ws + c.off_cpm);
     const ScaleTargets sc = scale_targets(nmod, k, false);
     ResidueTable rtab;
-    CrtTable ctab;
+    PostMmaTable ptab;
     build_residue_table(nmod, &rtab);
-    build_crt_table(nmod, &ctab);
+    build_post_mma_table(nmod, &ptab);
+    uint32_t* frags = (uint32_t*)(ws + c.off_frags);
     const bool wideA = sc.PA - sc.ck > 62, wideB = sc.PB - sc.ck > 62;
     Phases ph;
     if (int s = begin_call(&ph)) return s;
@@ -427,6 +431,7 @@ int zgemm_host(int64_t m, int64_t n, int64_t k, const double* hA, int64_t lda, c
     }
     // A: steps 2-4 as in zgemm2m
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
+    CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
     CK(cudaStreamWaitEvent(st, D().a_ready, 0));
     CK(ph.begin(0, st));
     CK(launch_scan_rows<double>(dA, m, k, m, absA, st, &g.launches[0]));
@@ -464,7 +469,7 @@ int zgemm_host(int64_t m, int64_t n, int64_t k, const double* hA, int64_t lda, c
         CK(cudaEventRecord(D().g_ready[p], st));
         CK(cudaStreamWaitEvent(side, D().g_ready[p], 0));
         CK(ph.begin(3, side));
-        CK(launch_post_fp<double>(cpm, c.ldp, m, n, j0, j1, eA, eB, ctab, dC, m, nullptr, nullptr, side, &g.launches[3]));
+        CK(launch_post_fp<double>(cpm, c.ldp, m, n, j0, j1, eA, eB, ptab, frags, dC, m, nullptr, nullptr, side, &g.launches[3]));
         CK(ph.end(side));
         CK(cudaEventRecord(D().c_ready[p], side));
         CK(cudaStreamWaitEvent(down, D().c_ready[p], 0));
@@ -960,6 +965,27 @@ int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float*
         if (inv_m) inv_m[j] = rt.inv_m[j];
         if (xmax) xmax[j] = rt.xmax[j];
         if (margin) margin[j] = residue_reduction_margin(rt, j);
+    }
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_post_operands(int eisenstein, int nmod, uint8_t* digits, int* dims, double* consts) {
+    if (nmod < 1 || nmod > (eisenstein ? kMaxEis : kMaxMod)) return GEMM2M_ERR_ARG;
+    PostMmaTable t;
+    if (eisenstein) build_post_mma_table_eis(nmod, &t);
+    else build_post_mma_table(nmod, &t);
+    if (dims) { dims[0] = t.c.planes; dims[1] = t.c.ks; dims[2] = t.c.nb; }
+    if (digits)
+        for (int part = 0; part < 2; ++part)
+            for (int p = 0; p < t.c.planes; ++p)
+                std::memcpy(digits + ((size_t)part * t.c.planes + p) * 4 * kPostMaxNB, t.digit[part][p], 4 * kPostMaxNB);
+    if (consts) {
+        for (int k = 0; k < kPostMaxNB; ++k) {
+            consts[k] = t.c.Mc[k];
+            consts[kPostMaxNB + k] = t.c.off[0][k];
+            consts[2 * kPostMaxNB + k] = t.c.off[1][k];
+        }
+        consts[3 * kPostMaxNB] = t.c.inv_M;
     }
     return GEMM2M_OK;
 }

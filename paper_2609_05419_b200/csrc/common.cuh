@@ -75,6 +75,31 @@ struct CrtTable {
     int re_shift;                              // Eisenstein variant: the real part is U 2^re_shift
 };
 
+// Operands of the post-processing of the complex GEMMs, where the digit-column sums of the CRT are an 8-bit contraction on
+// the tensor cores: per output element, [residues of all planes, + 128] x [base-256 digits of the folded CRT weights mod M].
+//   X_r = sum_planes c_p Wr_p,  X_i = sum_planes c_p Wi_p  (mod M)
+// with, for a 2M modulus j (planes C+_j and C-_j; Eq. (2c) folded in), Wr = Gr_j for both and Wi = -Gi_j / +Gi_j; for a 3M
+// modulus (planes P1, P2, P3 of Eq. (1)) Wr = +G, -G, 0 and Wi = -G, -G, +G.  Every weight is reduced to [0, M) and written in
+// bytes, W = sum_p d_p 256^p, p < 4 nb (nb even); with the residues moved to [0, 255] as well every digit-column sum is a
+// non-negative integer.  The contraction runs as warp-level m16n8k32 MMAs: ks K-steps of 32 planes, nb blocks of 8 columns;
+// bfrag holds the B-operand registers of every lane, [(s nb + q) 2 + h][lane], so that the digit column sums of one part land
+// in the accumulators of two neighbouring lanes (see post_fp.cu for the column order).
+constexpr int kPostMaxNB = 6, kPostMaxKS = 2;
+constexpr int kPostFragWords = kPostMaxKS * kPostMaxNB * 2 * 32;
+struct PostConsts {
+    double Mc[kPostMaxNB];                     // M = sum_k Mc[k] 2^(32k), lower digits balanced in [-2^31, 2^31), each stored times 2^(32k)
+    double off[2][kPostMaxNB];                 // per part: (1.5 2^52 + digit k of 128 sum_planes W_p) 2^(32k), what comes off chunk k
+    double inv_M;                              // 1 / M
+    double im_hi, im_lo;                       // Eisenstein variant: the imaginary part is V (im_hi + im_lo); 0 = no factor
+    int re_shift;                              // Eisenstein variant: the real part is U 2^re_shift
+    int planes, ks, nb;
+};
+struct PostMmaTable {
+    PostConsts c;
+    uint32_t bfrag[kPostFragWords];            // host copy; launch_post_operands writes it to device memory
+    uint8_t digit[2][kMaxPlanes][4 * kPostMaxNB];  // [part][plane][p]: the digits themselves (host side; for tests)
+};
+
 // CRT constants for the exact int64 result (nmod <= 8, M < 2^62).
 struct CrtTableInt {
     int64_t W[8];          // M / m_j
@@ -103,6 +128,8 @@ double residue_reduction_margin(const ResidueTable& t, int j);
 void build_mod_table(int nmod, bool per_plane, ModTable* t);
 void build_crt_table(int nmod, CrtTable* t);
 void build_crt_table_int(int nmod, CrtTableInt* t);
+void build_post_mma_table(int nmod, PostMmaTable* t);
+void build_post_mma_table_eis(int nmod, PostMmaTable* t);
 ScaleTargets scale_targets(int nmod, int64_t k, bool herk);
 // The same for the real Ozaki-II scheme (dgemm_ozaki2): moduli 256, 255, 253, ..., one residue plane per modulus.
 int real_modulus_value(int j);
@@ -150,8 +177,11 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).
 // alpha, beta: host pointers to (re, im) pairs, or null for alpha = 1 / beta = 0: C = alpha X + beta C.
+// dev_frags: device copy of tab.bfrag, written earlier on an ordered stream by launch_post_operands (kPostFragWords words).
+cudaError_t launch_post_operands(const PostMmaTable& tab, uint32_t* dev_frags, cudaStream_t st, int* launches);
 template <typename T> cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA, const int32_t* eB,
-                                                 const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta, cudaStream_t st, int* launches);
+                                                 const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc, const double* alpha, const double* beta,
+                                                 cudaStream_t st, int* launches);
 // Real Ozaki-II scheme (Section 3.1): scans, residues (one plane per modulus) and post-processing of real matrices.
 template <typename T> cudaError_t launch_scan_real(const T* X, int64_t rows, int64_t cols, int64_t ld, bool per_row, uint64_t* absmax, cudaStream_t st, int* launches);
 template <typename T> cudaError_t launch_residues_real(const T* X, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp, const int32_t* e,

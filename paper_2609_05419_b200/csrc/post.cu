@@ -1,6 +1,6 @@
 // Algorithm 1 steps 4 (Eq. 2c), 5, 6, 7: post-processing of the residue planes of the products (complex GEMM, rank-k family,
 // real scheme, exact int64 result), plus the small packing and scaling kernels of the rank-k and extended interfaces.
-#include "prepost_common.cuh"
+#include "post_common.cuh"
 
 namespace gemm2m {
 
@@ -53,181 +53,8 @@ __device__ __forceinline__ void crt_finish(double (&S)[NCH], const CrtTable& tab
     *lo = l;
 }
 
-__device__ __forceinline__ double scale_pow2(double x, int e) {   // x 2^e with e split so that both factors are normal
-    const int e1 = max(-1000, min(1000, e));
-    const int e2 = max(-1000, min(1000, e - e1));
-    const int e3 = e - e1 - e2;
-    double y = x * __longlong_as_double((long long)(e1 + 1023) << 52);
-    if (e2) y *= __longlong_as_double((long long)(e2 + 1023) << 52);
-    if (e3) y = ldexp(y, e3);
-    return y;
-}
-
-template <typename T> __device__ __forceinline__ void store4(T* dst, const double (&re)[4], const double (&im)[4], int count);
-template <> __device__ __forceinline__ void store4<double>(double* dst, const double (&re)[4], const double (&im)[4], int count) {
-    for (int i = 0; i < count; ++i) *reinterpret_cast<double2*>(dst + 2 * i) = make_double2(re[i], im[i]);
-}
-template <> __device__ __forceinline__ void store4<float>(float* dst, const double (&re)[4], const double (&im)[4], int count) {
-    if (count == 4 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-        *reinterpret_cast<float4*>(dst) = make_float4((float)re[0], (float)im[0], (float)re[1], (float)im[1]);
-        *reinterpret_cast<float4*>(dst + 4) = make_float4((float)re[2], (float)im[2], (float)re[3], (float)im[3]);
-    } else {
-        for (int i = 0; i < count; ++i) *reinterpret_cast<float2*>(dst + 2 * i) = make_float2((float)re[i], (float)im[i]);
-    }
-}
-
 constexpr int kPostThreads = 128;
 constexpr int kPostSpan = kPostThreads * 4;   // consecutive row indices i handled by one block
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
-// cpm: [planes][n][ldp] int8 (row index i contiguous), planes = C+ and C- of the 2M moduli, then P1, P2, P3 of the 3M
-// moduli.  A block handles 512 consecutive i of one column j: it first pulls the planes x 512 residue bytes into shared memory with asynchronous 16-byte copies (all in flight at once), then each
-// thread combines 4 consecutive i.
-// AXPBY: C = alpha X + beta C (alpha, beta complex, given as re/im pairs) instead of C = X; the product X is formed
-// exactly as before, then combined in FP64 with fused multiply-adds.  beta = 0 does not read C.
-struct PostScalars { double ar, ai, br, bi; };
-
-template <typename T, int NCH, bool AXPBY>
-__global__ void __launch_bounds__(kPostThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t n,
-                                                               const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
-                                                               const __grid_constant__ CrtTable tab, T* __restrict__ C, int64_t ldc,
-                                                               const PostScalars sc) {
-    __shared__ __align__(16) uint32_t stage[kMaxPlanes][kPostThreads];
-    const int64_t ib = (int64_t)blockIdx.x * kPostSpan;
-    const int64_t j = blockIdx.y;
-    const int nmod = tab.nmod, n2 = tab.n2, n3 = nmod - n2;
-    const int64_t plane = n * ldp;
-    const int8_t* src = cpm + j * ldp + ib;
-    const int vec_per_plane = (int)min((int64_t)(kPostSpan / 16), (ldp - ib) / 16);   // ldp is a multiple of 16
-    for (int idx = threadIdx.x; idx < (2 * n2 + 3 * n3) * (kPostSpan / 16); idx += kPostThreads) {
-        const int p = idx / (kPostSpan / 16), v = idx - p * (kPostSpan / 16);
-        if (v < vec_per_plane) cp_async16(&stage[p][4 * v], src + (int64_t)p * plane + 16 * v);
-    }
-    cp_async_wait_all();
-    __syncthreads();
-    const int64_t i0 = ib + 4 * threadIdx.x;
-    if (i0 >= m) return;
-    double Sr[4][NCH], Si[4][NCH];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
-    }
-#pragma unroll 2
-    for (int jm = 0; jm < n2; ++jm) {
-        const uint32_t wp = stage[jm][threadIdx.x];            // c+ of 4 elements
-        const uint32_t wm = stage[n2 + jm][threadIdx.x];       // c-
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int cp = sbyte(wp, e);
-            const int cm = sbyte(wm, e);
-            const double vr = int_to_double(cm + cp);     // Eq. (2c): real part uses C- + C+
-            const double vi = int_to_double(cm - cp);     //           imaginary part uses C- - C+
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
-                Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
-            }
-        }
-    }
-#pragma unroll 1
-    for (int j3 = 0; j3 < n3; ++j3) {                      // 3M moduli of the hybrid, Eq. (1)
-        const uint32_t w1 = stage[2 * n2 + j3][threadIdx.x];
-        const uint32_t w2 = stage[2 * n2 + n3 + j3][threadIdx.x];
-        const uint32_t w3 = stage[2 * n2 + 2 * n3 + j3][threadIdx.x];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int p1 = sbyte(w1, e), p2 = sbyte(w2, e), p3 = sbyte(w3, e);
-            const double vr = int_to_double(p1 - p2);
-            const double vi = int_to_double(p3 - p1 - p2);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                Sr[e][c] = fma(vr, tab.gr[n2 + j3][c], Sr[e][c]);
-                Si[e][c] = fma(vi, tab.gr[n2 + j3][c], Si[e][c]);
-            }
-        }
-    }
-    const int fb = __ldg(eB + j);
-    double re[4], im[4];
-    int count = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        if (i0 + e < m) {
-            ++count;
-            const int ea = __ldg(eA + i0 + e);
-            if (ea == kExpNonFinite || fb == kExpNonFinite) {
-                re[e] = im[e] = __longlong_as_double(0x7FF8000000000000ll);
-            } else {
-                double h, l;
-                crt_finish<NCH>(Sr[e], tab, &h, &l);
-                re[e] = scale_pow2(h + l, ea + fb + tab.re_shift);
-                crt_finish<NCH>(Si[e], tab, &h, &l);
-                if (tab.im_hi != 0.0) {          // Eisenstein variant: V sqrt(3)/2 as a double-double product, rounded once below
-                    const double p = h * tab.im_hi;
-                    l = fma(h, tab.im_lo, fma(l, tab.im_hi, fma(h, tab.im_hi, -p)));
-                    h = p;
-                }
-                im[e] = scale_pow2(h + l, ea + fb);
-            }
-        }
-    }
-    if (AXPBY) {
-        const bool use_c = sc.br != 0.0 || sc.bi != 0.0;
-        for (int e = 0; e < count; ++e) {
-            const double xr = re[e], xi = im[e];
-            double yr = fma(sc.ar, xr, -sc.ai * xi), yi = fma(sc.ar, xi, sc.ai * xr);
-            if (use_c) {
-                const T* old = C + 2 * (i0 + e + j * ldc);
-                const double cr = (double)old[0], ci = (double)old[1];
-                yr += fma(sc.br, cr, -sc.bi * ci);
-                yi += fma(sc.br, ci, sc.bi * cr);
-            }
-            re[e] = yr;
-            im[e] = yi;
-        }
-    }
-    store4<T>(C + 2 * (i0 + j * ldc), re, im, count);
-}
-
-template <typename T, bool AXPBY>
-static cudaError_t launch_post_fp_t(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
-                                    const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const PostScalars& sc, cudaStream_t st,
-                                    int* launches) {
-    const int64_t per_block = kPostSpan;
-    for (int64_t j0 = j_begin; j0 < j_end; j0 += 65535) {      // grid.y limit
-        const int64_t nj = (j_end - j0 < 65535) ? j_end - j0 : 65535;
-        dim3 grid((unsigned)((m + per_block - 1) / per_block), (unsigned)nj);
-        const int8_t* src = cpm + j0 * ldp;
-        T* dst = C + 2 * j0 * ldc;
-        // the plane stride is n * ldp for the whole matrix, so pass the full n and offset pointers
-        switch (tab.nchunks) {
-            case 1: post_fp_kernel<T, 1, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
-            case 2: post_fp_kernel<T, 2, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
-            case 3: post_fp_kernel<T, 3, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
-            case 4: post_fp_kernel<T, 4, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
-            default: post_fp_kernel<T, 5, AXPBY><<<grid, kPostThreads, 0, st>>>(src, ldp, m, n, eA, eB + j0, tab, dst, ldc, sc); break;
-        }
-        ++*launches;
-    }
-    return cudaGetLastError();
-}
-
-template <typename T>
-cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
-                           const int32_t* eB, const CrtTable& tab, T* C, int64_t ldc, const double* alpha, const double* beta,
-                           cudaStream_t st, int* launches) {
-    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
-    PostScalars sc{1.0, 0.0, 0.0, 0.0};
-    if (alpha) { sc.ar = alpha[0]; sc.ai = alpha[1]; }
-    if (beta) { sc.br = beta[0]; sc.bi = beta[1]; }
-    const bool plain = sc.ar == 1.0 && sc.ai == 0.0 && sc.br == 0.0 && sc.bi == 0.0;
-    if (plain) return launch_post_fp_t<T, false>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
-    return launch_post_fp_t<T, true>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, C, ldc, sc, st, launches);
-}
 
 // Real Ozaki-II scheme (Section 3.1): cp: [nmod][n][ldp] int8, one plane per modulus; X = sum_j c_j G_j (mod M) with
 // G_j = sym(q_j)(M/m_j) in tab.gr; real double output.  Same staging and finish as post_fp_kernel.
@@ -516,7 +343,5 @@ cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n
 }
 
 
-template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, double*, int64_t, const double*, const double*, cudaStream_t, int*);
-template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const CrtTable&, float*, int64_t, const double*, const double*, cudaStream_t, int*);
 
 }  // namespace gemm2m

@@ -1,0 +1,342 @@
+// Algorithm 1 steps 4 (Eq. 2c; Eq. 1 for the 3M moduli of the hybrid), 5, 6, 7 for the complex GEMMs: from the residue planes of
+// the products to C.  Per output element the work is X = sum over planes of (residue) x (folded CRT weight) mod M for the real
+// and the imaginary part, an exact integer of up to 184 bits.  The weights (reduced to [0, M)) are written in base-256 digits,
+// which turns the sums over the planes into a small 8-bit contraction, [elements x planes] . [planes x digit columns], that
+// runs on the tensor cores (warp-level m16n8k32 MMAs, int32 accumulators; residues moved to [0, 255] so that every column
+// sum is non-negative, at most 56 . 255 . 255 < 2^22).  What is left per element is to add the digit columns up (integer, then
+// FP64 on 32-bit-spaced chunks), remove the multiple of M, round once and scale by 2^(e_i + f_j).
+// Bound by HBM traffic: 1 byte per plane read, 16 (8) bytes written per element.
+#include "post_common.cuh"
+
+namespace gemm2m {
+
+#ifndef GEMM2M_POST_WARPS
+#define GEMM2M_POST_WARPS 4
+#endif
+#ifndef GEMM2M_POST_GROUPS
+#define GEMM2M_POST_GROUPS 4
+#endif
+constexpr int kPfWarps = GEMM2M_POST_WARPS;     // warps per block
+constexpr int kPfGroups = GEMM2M_POST_GROUPS;   // MMA groups of 32 elements per warp and step
+constexpr int kPfThreads = 32 * kPfWarps;
+constexpr int kPfSpan = 32 * kPfGroups * kPfWarps;      // consecutive row indices i per step of a block
+constexpr int kPfStrideW = kPfSpan / 4 + 8;     // words per staged plane: + 8, so that the 32 fragment loads of a warp hit 32 banks
+constexpr int kPfStages = 2;                    // staging ring: the next step is on its way while this one is processed
+static_assert(kPfSpan % 128 == 0, "plane stride = 8 mod 32 words");
+
+// Words per element in the exchange buffer: 2 parts x NB chunks of 8 bytes, plus a pad that keeps the 16-byte accesses of a
+// warp on distinct banks.
+__host__ __device__ constexpr int pf_row_words(int nb) { return 4 * nb + 4; }
+__host__ __device__ constexpr int pf_block_words(int ks, int nb) { return kPfStages * 32 * ks * kPfStrideW + kPfWarps * 32 * pf_row_words(nb); }
+
+// D = A B, A: 16 x 32 bytes (row-major fragments), B: 32 x 8 bytes (column-major fragments), D: 16 x 8 int32; unsigned bytes.
+__device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
+}
+__device__ __forceinline__ void mma_u8_acc(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// hi:lo = b 2^16 + (hi_word 2^32 + a): four digit-column sums s0..s3 packed as a = s0 + 2^8 s1, b = s2 + 2^8 s3 (both below
+// 2^31) under the high word of a double, one wide multiply-add.
+// (two16 holds 65536 in a register: with the constant in the instruction the compiler splits the product into a shift pair.)
+__device__ __forceinline__ unsigned long long pack_chunk(uint32_t a, uint32_t b, uint32_t hi_word, uint32_t two16) {
+    unsigned long long r;
+    asm("{\n\t.reg .b64 c;\n\tmov.b64 c, {%1, %2};\n\tmad.wide.u32 %0, %3, %4, c;\n\t}" : "=l"(r) : "r"(a), "r"(hi_word), "r"(b), "r"(two16));
+    return r;
+}
+
+// Lifted X (exact integer, |X| <= M/2) of one part from its NB chunks, returned as an unevaluated sum hi + lo with
+// |lo| <= ulp(hi)/2.  Chunk k arrives as the bit pattern of the double (1.5 2^52 + V_k) 2^(32k), with
+// V_k = s_4k + 2^8 s_(4k+1) + 2^16 s_(4k+2) + 2^24 s_(4k+3) < 2^46.1 the four digit-column sums it covers; off[k] takes the
+// conversion offset and the chunk's share of 128 sum_planes W_p off again, exactly, which leaves W_k with
+// X' = sum_k W_k 2^(32k) = sum_planes residue_p W_p = X + t M.
+// t = rint(X'/M) from the three leading chunks: M >= 2^(32 NB - 64) (its bytes fill more than NB - 2 chunks), so the
+// rest is below 2^-17 M; |t| < 2^14, and |X/M| stays away from 1/2 by the scaling rule.  W_k - t Mc_k is exact
+// (|t Mc_k| < 2^46 before the weight).  The chunks are then added with error-free transformations, neighbours first, so
+// hi + lo equals X to 2^-105 relative.
+template <int NB>
+__device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const double (&off)[kPostMaxNB], const PostConsts& pc, double* hi, double* lo) {
+    double W[NB];
+#pragma unroll
+    for (int k = 0; k < NB; ++k) W[k] = bits[k] - off[k];
+    double lead = W[NB - 1];
+#pragma unroll
+    for (int k = NB - 2; k >= 0 && k >= NB - 3; --k) lead += W[k];
+    const double t = rint(lead * pc.inv_M);
+#pragma unroll
+    for (int k = 0; k < NB; ++k) W[k] = fma(-t, pc.Mc[k], W[k]);
+    double ph[NB / 2], l = 0.0;
+#pragma unroll
+    for (int k = 0; k < NB / 2; ++k) {
+        const double a = W[2 * k + 1], b = W[2 * k];
+        const double s = a + b;                                              // TwoSum
+        const double bb = s - a;
+        l += (a - (s - bb)) + (b - bb);
+        ph[k] = s;
+    }
+    double h = ph[NB / 2 - 1];
+#pragma unroll
+    for (int k = NB / 2 - 2; k >= 0; --k) {
+        const double s = h + ph[k];
+        const double bb = s - h;
+        l += (h - (s - bb)) + (ph[k] - bb);
+        h = s;
+    }
+    *hi = h;
+    *lo = l;
+}
+
+template <typename T> __device__ __forceinline__ void store_cplx(T* dst, double re, double im);
+template <> __device__ __forceinline__ void store_cplx<double>(double* dst, double re, double im) { *reinterpret_cast<double2*>(dst) = make_double2(re, im); }
+template <> __device__ __forceinline__ void store_cplx<float>(float* dst, double re, double im) { *reinterpret_cast<float2*>(dst) = make_float2((float)re, (float)im); }
+
+// cpm: [planes][n][ldp] int8 (row index i contiguous); plane = n ldp is the plane stride; ncols columns starting at the
+// pointers given.  The work is cut into steps of kPfSpan consecutive i of one column j, numbered column by column within a
+// block of rows; every thread block takes an equal, contiguous share of the steps.  The planes x kPfSpan residue bytes of a step
+// are pulled into shared memory with asynchronous 16-byte copies while the previous step is processed.  A warp owns 32 kPfGroups
+// of the i; for each group of 32 it gathers the MMA operand (rows = elements, K = planes; lane (g, t) takes the word of
+// elements 4g..4g+3 of the planes t, t+4, t+8, t+12 of each half K-step, moves the bytes to [0, 255] and transposes the 4 x 4
+// bytes), multiplies by the digit matrix held in registers, packs each run of four digit-column sums into one 64-bit chunk,
+// and passes the chunks through shared memory so that lane L ends up with all chunks of element L, which it finishes and
+// stores (consecutive lanes, consecutive i).  Many warps per SM matter more here than long steps: the per-element finish is a
+// chain of dependent FP64 operations.
+template <typename T, int KS, int NB, bool AXPBY>
+__global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t plane, int ncols,
+                                                             const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
+                                                             const uint32_t* __restrict__ frags, const __grid_constant__ PostConsts pc,
+                                                             T* __restrict__ C, int64_t ldc, const PostScalars sc) {
+    static_assert(NB % 2 == 0, "whole chunks per lane");
+    extern __shared__ __align__(16) uint32_t pf_smem[];
+    constexpr int kStageWords = 32 * KS * kPfStrideW;
+    constexpr int kRow = pf_row_words(NB);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    uint32_t* xch = pf_smem + kPfStages * kStageWords + warp * 32 * kRow;
+    const int64_t total = ((m + kPfSpan - 1) / kPfSpan) * ncols;
+    int64_t step = total * blockIdx.x / gridDim.x;
+    const int64_t step_end = total * (blockIdx.x + 1) / gridDim.x;
+    if (step >= step_end) return;
+    int ibk = (int)(step / ncols), j = (int)(step - (int64_t)ibk * ncols);
+    const int planes = pc.planes;
+
+    constexpr int kVecs = kPfSpan / 16;                         // 16-byte vectors per plane and step
+    const int sv = threadIdx.x % kVecs, sp = threadIdx.x / kVecs;   // staging: this thread copies vector sv of the planes sp, sp + kPfThreads / kVecs, ...
+    auto issue = [&](int ibk_, int j_, int stage) {
+        const int64_t ib = (int64_t)ibk_ * kPfSpan;
+        if (16 * sv + 16 <= ldp - ib) {                         // ldp is a multiple of 16: whole vectors up to the padded end of the column
+            const int8_t* src = cpm + (int64_t)j_ * ldp + ib + 16 * sv + (int64_t)sp * plane;
+            uint32_t* dst = pf_smem + stage * kStageWords + sp * kPfStrideW + 4 * sv;
+            for (int p = sp; p < planes; p += kPfThreads / kVecs) {
+                cp_async16(dst, src);
+                src += (kPfThreads / kVecs) * plane;
+                dst += (kPfThreads / kVecs) * kPfStrideW;
+            }
+        }
+        cp_async_commit_group();
+    };
+    issue(ibk, j, 0);
+
+    uint32_t bf[KS][NB][2];
+#pragma unroll
+    for (int s = 0; s < KS; ++s)
+#pragma unroll
+        for (int q = 0; q < NB; ++q) {
+            bf[s][q][0] = __ldg(frags + ((s * NB + q) * 2 + 0) * 32 + lane);
+            bf[s][q][1] = __ldg(frags + ((s * NB + q) * 2 + 1) * 32 + lane);
+        }
+    // High word of chunk c of this lane: 1.5 2^52 with the weight 2^(32k) of the chunk, k = (t & 1) NB/2 + c, in its exponent.
+    uint32_t chunk_hi[NB / 2];
+#pragma unroll
+    for (int c = 0; c < NB / 2; ++c) chunk_hi[c] = 0x43380000u + ((uint32_t)(32 * ((t & 1) * (NB / 2) + c)) << 20);
+    int ea[kPfGroups] = {}, ea_block = -1;
+    uint32_t two16;
+    asm("mov.b32 %0, 65536;" : "=r"(two16));
+
+    for (int n = 0; step < step_end; ++step, ++n) {
+        int jn = j + 1, ibkn = ibk;
+        if (jn == ncols) { jn = 0; ++ibkn; }
+        if (step + 1 < step_end) { issue(ibkn, jn, (n + 1) & 1); cp_async_wait_pending<1>(); }
+        else cp_async_wait_pending<0>();
+        __syncthreads();
+        const uint32_t* st = pf_smem + (n & 1) * kStageWords;
+        const int64_t ib = (int64_t)ibk * kPfSpan + 32 * kPfGroups * warp;    // first row of this warp
+        if (ibk != ea_block) {
+#pragma unroll
+            for (int it = 0; it < kPfGroups; ++it) ea[it] = ib + 32 * it + lane < m ? __ldg(eA + ib + 32 * it + lane) : 0;
+            ea_block = ibk;
+        }
+        const int fb = __ldg(eB + j);
+#pragma unroll
+        for (int it = 0; it < kPfGroups; ++it) {
+            int acc[2][NB][4];
+            const uint32_t* col = st + 8 * (kPfGroups * warp + it) + g;
+#pragma unroll
+            for (int s = 0; s < KS; ++s) {
+                uint32_t a0[4], a1[4];                      // A operands of the two 16-row tiles: elements 4g, 4g+1 / 4g+2, 4g+3
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t* p = col + (32 * s + 16 * h + t) * kPfStrideW;
+                    const uint32_t w0 = p[0] ^ 0x80808080u, w1 = p[4 * kPfStrideW] ^ 0x80808080u;      // residue + 128
+                    const uint32_t w2 = p[8 * kPfStrideW] ^ 0x80808080u, w3 = p[12 * kPfStrideW] ^ 0x80808080u;
+                    const uint32_t lo01 = __byte_perm(w0, w1, 0x5140), hi01 = __byte_perm(w0, w1, 0x7362);
+                    const uint32_t lo23 = __byte_perm(w2, w3, 0x5140), hi23 = __byte_perm(w2, w3, 0x7362);
+                    a0[2 * h] = __byte_perm(lo01, lo23, 0x5410);        // element 4g:   row g of tile 0
+                    a0[2 * h + 1] = __byte_perm(lo01, lo23, 0x7632);    // element 4g+1: row g + 8 of tile 0
+                    a1[2 * h] = __byte_perm(hi01, hi23, 0x5410);        // element 4g+2: row g of tile 1
+                    a1[2 * h + 1] = __byte_perm(hi01, hi23, 0x7632);    // element 4g+3: row g + 8 of tile 1
+                }
+#pragma unroll
+                for (int q = 0; q < NB; ++q) {
+                    if (s == 0) {
+                        mma_u8(acc[0][q], a0, bf[s][q][0], bf[s][q][1]);
+                        mma_u8(acc[1][q], a1, bf[s][q][0], bf[s][q][1]);
+                    } else {
+                        mma_u8_acc(acc[0][q], a0, bf[s][q][0], bf[s][q][1]);
+                        mma_u8_acc(acc[1][q], a1, bf[s][q][0], bf[s][q][1]);
+                    }
+                }
+            }
+            // accumulator registers 0, 1 hold row g, columns 2t, 2t+1 (two neighbouring digits); registers 2, 3 the same for row g + 8
+            __syncwarp();                                   // the previous group's reads of the exchange buffer are done
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                unsigned long long chunk[NB / 2];
+#pragma unroll
+                for (int c = 0; c < NB / 2; ++c) {
+                    const uint32_t a = (uint32_t)(acc[e >> 1][2 * c][2 * (e & 1)] + 256 * acc[e >> 1][2 * c][2 * (e & 1) + 1]);
+                    const uint32_t b = (uint32_t)(acc[e >> 1][2 * c + 1][2 * (e & 1)] + 256 * acc[e >> 1][2 * c + 1][2 * (e & 1) + 1]);
+                    chunk[c] = pack_chunk(a, b, chunk_hi[c], two16);           // bits of (1.5 2^52 + a + 2^16 b) 2^(32k)
+                }
+                uint32_t* row = xch + (4 * g + e) * kRow + t * NB;
+                if constexpr (NB % 4 == 0) {
+#pragma unroll
+                    for (int c = 0; c < NB / 2; c += 2) *reinterpret_cast<ulonglong2*>(row + 2 * c) = make_ulonglong2(chunk[c], chunk[c + 1]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < NB / 2; ++c) *reinterpret_cast<unsigned long long*>(row + 2 * c) = chunk[c];
+                }
+            }
+            __syncwarp();
+            double br[NB], bi[NB];                          // lanes 0, 1 of the quad wrote the real part's chunks, lanes 2, 3 the imaginary part's
+            {
+                const double2* row = reinterpret_cast<const double2*>(xch + lane * kRow);
+#pragma unroll
+                for (int c = 0; c < NB / 2; ++c) {
+                    const double2 vr = row[c], vi = row[NB / 2 + c];
+                    br[2 * c] = vr.x; br[2 * c + 1] = vr.y;
+                    bi[2 * c] = vi.x; bi[2 * c + 1] = vi.y;
+                }
+            }
+            const int64_t i = ib + 32 * it + lane;
+            {
+                double re, im;
+                const int eai = ea[it];
+                double hr, lr, hi, li;               // lanes beyond m work on whatever the staging buffer holds; nothing of it is stored
+                crt_finish32<NB>(br, pc.off[0], pc, &hr, &lr);
+                crt_finish32<NB>(bi, pc.off[1], pc, &hi, &li);
+                if (pc.im_hi != 0.0) {               // Eisenstein variant: V sqrt(3)/2 as a double-double product, rounded once below
+                    const double p = hi * pc.im_hi;
+                    li = fma(hi, pc.im_lo, fma(li, pc.im_hi, fma(hi, pc.im_hi, -p)));
+                    hi = p;
+                }
+                const int e = (int)((uint32_t)eai + (uint32_t)fb);
+                if (e > -1000 && e < 1000) {         // 2^e is a normal number: one multiplication
+                    re = (hr + lr) * __longlong_as_double((long long)(e + pc.re_shift + 1023) << 52);
+                    im = (hi + li) * __longlong_as_double((long long)(e + 1023) << 52);
+                } else {
+                    re = scale_pow2(hr + lr, e + pc.re_shift);
+                    im = scale_pow2(hi + li, e);
+                }
+                if (eai == kExpNonFinite || fb == kExpNonFinite) re = im = __longlong_as_double(0x7FF8000000000000ll);
+                T* dst = C + 2 * (i + (int64_t)j * ldc);
+                if (AXPBY) {
+                    double yr = fma(sc.ar, re, -sc.ai * im), yi = fma(sc.ar, im, sc.ai * re);
+                    if (i < m && (sc.br != 0.0 || sc.bi != 0.0)) {
+                        const double cr = (double)dst[0], ci = (double)dst[1];
+                        yr += fma(sc.br, cr, -sc.bi * ci);
+                        yi += fma(sc.br, ci, sc.bi * cr);
+                    }
+                    re = yr;
+                    im = yi;
+                }
+                if (i < m) store_cplx<T>(dst, re, im);
+            }
+        }
+        __syncthreads();                                    // every warp is done with this stage before it is refilled
+        ibk = ibkn;
+        j = jn;
+    }
+}
+
+// The B-operand registers of the contraction, written once per call into the workspace (the kernels read them with
+// coalesced loads; as a kernel argument every lane would read a different word of the constant bank).
+__global__ void __launch_bounds__(256) post_operands_kernel(const __grid_constant__ PostMmaTable tab, uint32_t* __restrict__ dst) {
+    for (int i = threadIdx.x; i < kPostFragWords; i += blockDim.x) dst[i] = tab.bfrag[i];
+}
+
+cudaError_t launch_post_operands(const PostMmaTable& tab, uint32_t* dev_frags, cudaStream_t st, int* launches) {
+    post_operands_kernel<<<1, 256, 0, st>>>(tab, dev_frags);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <typename T, int KS, int NB, bool AXPBY>
+static cudaError_t launch_post_fp_v(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                                    const int32_t* eB, const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc,
+                                    const PostScalars& sc, cudaStream_t st, int* launches) {
+    constexpr size_t smem = (size_t)pf_block_words(KS, NB) * sizeof(uint32_t);
+    static int resident_dev[kMaxDevices] = {};          // thread blocks the device holds at once (0 = not asked yet)
+    int& resident = resident_dev[current_device_slot()];
+    if (!resident) {
+        cudaError_t err = cudaFuncSetAttribute(post_fp_kernel<T, KS, NB, AXPBY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        int per_sm = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, post_fp_kernel<T, KS, NB, AXPBY>, kPfThreads, smem);
+        if (err != cudaSuccess) return err;
+        resident = (per_sm > 0 ? per_sm : 1) * cached_sm_count();
+    }
+    constexpr int64_t kColsPerLaunch = 1 << 20;           // keeps step count times warp count of a launch far inside 63 bits
+    for (int64_t j0 = j_begin; j0 < j_end; j0 += kColsPerLaunch) {
+        const int64_t nj = (j_end - j0 < kColsPerLaunch) ? j_end - j0 : kColsPerLaunch;
+        const int64_t steps = ((m + kPfSpan - 1) / kPfSpan) * nj;
+        const unsigned grid = (unsigned)(steps < resident ? steps : resident);
+        post_fp_kernel<T, KS, NB, AXPBY><<<grid, kPfThreads, smem, st>>>(cpm + j0 * ldp, ldp, m, n * ldp, (int)nj, eA, eB + j0, dev_frags, tab.c,
+                                                                        C + 2 * j0 * ldc, ldc, sc);
+        ++*launches;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T, bool AXPBY>
+static cudaError_t launch_post_fp_t(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                                    const int32_t* eB, const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc,
+                                    const PostScalars& sc, cudaStream_t st, int* launches) {
+#define GEMM2M_POST_CASE(KS, NB)                                                                                                     \
+    if (tab.c.ks == KS && tab.c.nb == NB)                                                                                             \
+        return launch_post_fp_v<T, KS, NB, AXPBY>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, dev_frags, C, ldc, sc, st, launches);
+    GEMM2M_POST_CASE(1, 2) GEMM2M_POST_CASE(1, 4) GEMM2M_POST_CASE(2, 4) GEMM2M_POST_CASE(2, 6)
+#undef GEMM2M_POST_CASE
+    return cudaErrorInvalidValue;
+}
+
+template <typename T>
+cudaError_t launch_post_fp(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
+                           const int32_t* eB, const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc, const double* alpha,
+                           const double* beta, cudaStream_t st, int* launches) {
+    if (m <= 0 || j_end <= j_begin) return cudaSuccess;
+    PostScalars sc{1.0, 0.0, 0.0, 0.0};
+    if (alpha) { sc.ar = alpha[0]; sc.ai = alpha[1]; }
+    if (beta) { sc.br = beta[0]; sc.bi = beta[1]; }
+    const bool plain = sc.ar == 1.0 && sc.ai == 0.0 && sc.br == 0.0 && sc.bi == 0.0;
+    if (plain) return launch_post_fp_t<T, false>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, dev_frags, C, ldc, sc, st, launches);
+    return launch_post_fp_t<T, true>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, dev_frags, C, ldc, sc, st, launches);
+}
+
+template cudaError_t launch_post_fp<double>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const PostMmaTable&, const uint32_t*, double*, int64_t, const double*, const double*, cudaStream_t, int*);
+template cudaError_t launch_post_fp<float>(const int8_t*, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*, const int32_t*, const PostMmaTable&, const uint32_t*, float*, int64_t, const double*, const double*, cudaStream_t, int*);
+
+}  // namespace gemm2m

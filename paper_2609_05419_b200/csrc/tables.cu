@@ -92,6 +92,32 @@ struct Big {
         }
         return out;
     }
+    void shr(int bits) {   // 0 < bits < 32
+        uint32_t c = 0;
+        for (size_t i = w.size(); i-- > 0;) { const uint32_t n = w[i] << (32 - bits); w[i] = (w[i] >> bits) | c; c = n; }
+        trim();
+    }
+    void add_small(uint32_t v) {
+        uint64_t carry = v;
+        for (auto& limb : w) { if (!carry) break; const uint64_t t = (uint64_t)limb + carry; limb = (uint32_t)t; carry = t >> 32; }
+        if (carry) w.push_back((uint32_t)carry);
+    }
+    void add(const Big& o) {
+        if (w.size() < o.w.size()) w.resize(o.w.size(), 0u);
+        uint64_t carry = 0;
+        for (size_t i = 0; i < w.size(); ++i) { const uint64_t t = (uint64_t)w[i] + (i < o.w.size() ? o.w[i] : 0u) + carry; w[i] = (uint32_t)t; carry = t >> 32; }
+        if (carry) w.push_back((uint32_t)carry);
+    }
+    void sub(const Big& o) {   // *this >= o
+        int64_t borrow = 0;
+        for (size_t i = 0; i < w.size(); ++i) {
+            int64_t t = (int64_t)w[i] - (i < o.w.size() ? (int64_t)o.w[i] : 0) - borrow;
+            borrow = t < 0;
+            if (t < 0) t += 4294967296LL;
+            w[i] = (uint32_t)t;
+        }
+        trim();
+    }
     void sub_one() { for (auto& limb : w) { if (limb-- != 0) break; } trim(); }
     void shr1() { uint32_t c = 0; for (size_t i = w.size(); i-- > 0;) { uint32_t n = w[i] & 1u; w[i] = (w[i] >> 1) | (c << 31); c = n; } trim(); }
     double to_double() const { double v = 0; for (size_t i = w.size(); i-- > 0;) v = v * 4294967296.0 + w[i]; return v; }
@@ -297,6 +323,98 @@ void build_crt_table_eis(int nmod, CrtTable* t) {
 }
 void build_crt_table_real(int nmod, CrtTable* t) {
     memoised<CrtTable, kMaxReal>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kRealModuli, nmod, 0, c); });
+}
+
+static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaTable* t) {
+    std::memset(t, 0, sizeof(*t));
+    const int n3 = nmod - n2, planes = 2 * n2 + 3 * n3;
+    const Big M = product_of(nmod, mods);
+    const int ndig = (M.bit_length() + 7) / 8;                        // bytes of a residue modulo M
+    if (ndig > 4 * kPostMaxNB) std::abort();                          // cannot happen: M < 2^185
+    Big ksum[2];                                                      // sum over the planes of the weights, per part
+    auto put = [&](int part, int plane, const Big& W, int coef) {    // weight of `plane` in `part` = coef W (mod M), as bytes
+        if (coef == 0) return;
+        Big G = W;
+        G.mul_small((uint32_t)std::abs(coef));                        // below M/2: |coef| <= m_j / 2
+        if (coef < 0) { Big R = M; R.sub(G); G = R; }
+        ksum[part].add(G);
+        for (int p = 0; p < ndig; ++p) t->digit[part][plane][p] = (uint8_t)G.bits(8 * p, 8);
+    };
+    for (int j = 0; j < nmod; ++j) {
+        Big W;
+        int g, h;
+        folded_weights(nmod, j, M, &W, &g, &h, mods, n2);
+        if (j < n2) {                      // Eq. (2c): X_r takes (C- + C+) g, X_i takes (C- - C+) h
+            put(0, j, W, g);
+            put(0, n2 + j, W, g);
+            put(1, j, W, -h);
+            put(1, n2 + j, W, h);
+        } else {                           // Eq. (1): X_r takes (P1 - P2) g, X_i takes (P3 - P1 - P2) g
+            const int j3 = j - n2, p1 = 2 * n2 + j3, p2 = p1 + n3, p3 = p2 + n3;
+            put(0, p1, W, g);
+            put(0, p2, W, -g);
+            put(1, p1, W, -g);
+            put(1, p2, W, -g);
+            put(1, p3, W, g);
+        }
+    }
+    PostConsts& c = t->c;
+    c.planes = planes;
+    c.ks = (planes + 31) / 32;
+    c.nb = 2 * ((ndig + 7) / 8);           // 32-bit chunks (4 digits each), an even number of them: a lane of the kernel holds whole chunks
+    // M in base 2^32: balanced lower digits, the top digit takes what remains; each stored times its power of 2^32
+    Big rest = M;
+    for (int k = 0; k < c.nb; ++k) {
+        double d;
+        if (k + 1 < c.nb) {
+            const uint32_t low = rest.w.empty() ? 0u : rest.w[0];
+            if (!rest.w.empty()) { rest.w.erase(rest.w.begin()); rest.trim(); }
+            d = (double)low;
+            if (low >= 0x80000000u) { d -= 4294967296.0; rest.add_small(1); }
+        } else {
+            d = rest.to_double();          // below 2^53: exact
+        }
+        c.Mc[k] = std::ldexp(d, 32 * k);
+    }
+    // The kernel contracts (residue + 128) with the weights: 128 times the sum of a part's weights comes off again, chunk
+    // by chunk, together with the offset 1.5 2^52 of the integer-to-double conversion (top chunk: all remaining bits, < 2^46).
+    for (int part = 0; part < 2; ++part) {
+        Big K = ksum[part];
+        K.mul_small(128);
+        for (int k = 0; k < c.nb; ++k) {
+            const double d = k + 1 < c.nb ? (double)K.bits(32 * k, 32) : (double)K.bits(32 * k, 52);
+            c.off[part][k] = std::ldexp(6755399441055744.0 + d, 32 * k);
+        }
+    }
+    c.inv_M = 1.0 / M.to_double();
+    for (int s = 0; s < c.ks; ++s)
+        for (int q = 0; q < c.nb; ++q)
+            for (int hh = 0; hh < 2; ++hh)
+                for (int lane = 0; lane < 32; ++lane) {
+                    const int g = lane >> 2, tt = lane & 3;
+                    // B-operand column g of block q is accumulator column (lane tC = g / 2, register b = g % 2); lanes 0, 1 of
+                    // a quad collect the real part, lanes 2, 3 the imaginary part, each lane nb pairs of neighbouring digits
+                    const int tc = g >> 1, b = g & 1, part = tc >> 1, p = 2 * ((tc & 1) * c.nb + q) + b;
+                    uint32_t word = 0;
+                    for (int r = 0; r < 4; ++r) {
+                        const int plane = 32 * s + 16 * hh + tt + 4 * r;
+                        const uint32_t byte = plane < planes ? (uint32_t)t->digit[part][plane][p] : 0u;
+                        word |= byte << (8 * r);
+                    }
+                    t->bfrag[((s * c.nb + q) * 2 + hh) * 32 + lane] = word;
+                }
+}
+
+void build_post_mma_table(int nmod, PostMmaTable* t) {
+    memoised<PostMmaTable, kMaxMod>(nmod, t, [&](PostMmaTable* c) { build_post_mma_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_post_mma_table_eis(int nmod, PostMmaTable* t) {
+    memoised<PostMmaTable, kMaxEis>(nmod, t, [&](PostMmaTable* c) {
+        build_post_mma_table_for(kEisModuli, nmod, nmod, c);
+        c->c.re_shift = -1;                      // result = (U + V sqrt(-3))/2, the factor sqrt(3)/2 as a double-double
+        c->c.im_hi = 0x1.bb67ae8584caap-1;
+        c->c.im_lo = 0x1.cec95d0b5c1e3p-55;
+    });
 }
 
 static void build_crt_table_int_for(int nmod, CrtTableInt* t) {

@@ -91,7 +91,10 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--panels", type=int, default=0, help="most column panels per call (1 = every phase on the caller's stream, one after the other)")
     a = ap.parse_args()
+    if a.panels:
+        b.debug_set_panels(a.panels)
     if a.op == "int8_yardstick":
         return yardstick(a)
     if a.op == "zgemm_host":

@@ -308,3 +308,90 @@ def test_eisenstein_constants_match_oracle(nmod):
         low = ((y0_bits + x) - (0x4B000000 + (tq - 2 ** 23)) * m) & 0xFF
         res = np.where(low >= 128, low - 256, low)
         assert np.array_equal(res, ((x + m // 2) % m) - m // 2), m
+
+
+def _post_operand_checks(t, mods, M, plane_values, expected, rng_seed):
+    """The tensor-core operand of the post-processing, emulated in exact integers: for residues c_p of every plane the kernel
+    forms sum_p (c_p + 128) digit_p[k] per byte column k, packs four columns into a chunk, takes off[k] off, and removes a
+    multiple of M.  plane_values(rng) -> residues per plane; expected(residues) -> (X_r, X_i) modulo M from the oracle."""
+    planes, nb = t["planes"], t["nb"]
+    assert t["ks"] == (planes + 31) // 32 and nb % 2 == 0 and 4 * nb <= 24
+    nbytes = (M.bit_length() + 7) // 8
+    assert nb == 2 * ((nbytes + 7) // 8) and M >= 2 ** (32 * nb - 64)        # what the quotient estimate relies on
+    weights = [[sum(int(d) << (8 * p) for p, d in enumerate(t["digits"][part, pl])) for pl in range(planes)] for part in range(2)]
+    assert all(0 <= w < M for part in range(2) for w in weights[part])
+    assert (t["digits"][:, :, 4 * nb:] == 0).all()
+    # M in base 2^32, every stored number exact
+    mc = [int(v) for v in t["Mc"]]
+    assert all(float(v) == t["Mc"][k] for k, v in enumerate(mc)) and sum(mc) == M and all(v == 0 for v in mc[nb:])
+    assert all(abs(mc[k]) <= 2 ** 31 * 2 ** (32 * k) and mc[k] % 2 ** (32 * k) == 0 for k in range(nb - 1))
+    # offsets: 1.5 2^52 plus the chunk's share of 128 x (sum of the weights), all exact doubles
+    for part in range(2):
+        off = [int(v) for v in t["off"][part]]
+        assert all(float(v) == t["off"][part][k] for k, v in enumerate(off))
+        share = [off[k] // 2 ** (32 * k) - 3 * 2 ** 51 for k in range(nb)]
+        assert all(off[k] % 2 ** (32 * k) == 0 and 0 <= share[k] < 2 ** 46 for k in range(nb))
+        assert sum(share[k] << (32 * k) for k in range(nb)) == 128 * sum(weights[part])
+    # worst case of the packed sums: every residue at +127 (c + 128 = 255)
+    col_max = max(255 * int(t["digits"][part, :, p].astype(np.int64).sum()) for part in range(2) for p in range(4 * nb))
+    assert col_max < 2 ** 22
+    assert col_max * 257 < 2 ** 31                                            # a = s0 + 256 s1 is a 32-bit unsigned number
+    assert col_max * (1 + 2 ** 8 + 2 ** 16 + 2 ** 24) < 2 ** 47               # the chunk sits far inside the 2^51 of the conversion
+    rng = np.random.default_rng(rng_seed)
+    for trial in range(24):
+        c = plane_values(rng, trial)
+        want = expected(c)
+        for part in range(2):
+            cols = [sum((c[pl] + 128) * int(t["digits"][part, pl, p]) for pl in range(planes)) for p in range(4 * nb)]
+            chunk = [sum(cols[4 * k + b] << (8 * b) for b in range(4)) for k in range(nb)]
+            W = [chunk[k] - (int(t["off"][part][k]) // 2 ** (32 * k) - 3 * 2 ** 51) for k in range(nb)]
+            X1 = sum(W[k] << (32 * k) for k in range(nb))
+            assert X1 == sum(c[pl] * weights[part][pl] for pl in range(planes))
+            assert (X1 - want[part]) % M == 0
+            tq = round(X1 / M) if abs(X1) < 2 ** 1000 else 0
+            lead = sum(W[k] << (32 * k) for k in range(max(nb - 3, 0), nb))
+            assert abs(lead - X1) * 2 ** 17 <= M and abs(tq) < 2 ** 14      # dropped chunks do not move the quotient
+            assert all(abs(W[k] * 2 ** (32 * k) - tq * mc[k]) < 2 ** (47 + 32 * k) for k in range(nb))   # fused multiply-adds exact
+
+
+@pytest.mark.parametrize("nmod", [1, 2, 7, 8, 9, 16, 17, 18, 22, 23, 26])
+def test_post_operands_reproduce_eq_2c_eq_1_and_crt(nmod):
+    mods = staged.hybrid_moduli(nmod)
+    n2 = min(nmod, 22)
+    n3 = nmod - n2
+    roots = [staged.sqrt_minus_one(q) for q in mods[:n2]]
+    M = staged.product(mods)
+    t = b.debug_post_operands(nmod)
+    assert t["planes"] == 2 * n2 + 3 * n3
+
+    def plane_values(rng, trial):
+        lo = lambda m: -(m // 2)
+        hi = lambda m: (m - 1) // 2
+        pick = (lambda m: hi(m)) if trial == 0 else (lambda m: lo(m)) if trial == 1 else (lambda m: int(rng.integers(lo(m), hi(m) + 1)))
+        return [pick(m) for m in mods[:n2]] + [pick(m) for m in mods[:n2]] + [pick(m) for _ in range(3) for m in mods[n2:]]
+
+    def expected(c):
+        post = [staged.post_2m(c[j], c[n2 + j], mods[j], roots[j]) for j in range(n2)]
+        post += [staged.post_3m(c[2 * n2 + j3], c[2 * n2 + n3 + j3], c[2 * n2 + 2 * n3 + j3], mods[n2 + j3]) for j3 in range(n3)]
+        return staged.crt([r for r, _ in post], mods), staged.crt([i for _, i in post], mods)
+
+    _post_operand_checks(t, mods, M, plane_values, expected, nmod)
+
+
+@pytest.mark.parametrize("nmod", [1, 8, 16, 17, 23])
+def test_post_operands_of_the_eisenstein_variant(nmod):
+    from oracle import eisenstein as E
+    mods = E.greedy_eisenstein_moduli()[:nmod]
+    M = staged.product(mods)
+    t = b.debug_post_operands(nmod, eisenstein=True)
+    assert t["planes"] == 2 * nmod
+    state = {}
+
+    def plane_values(rng, trial):
+        ca, cb = (int(v) for v in rng.integers(-10 ** 9, 10 ** 9, 2))
+        state["want"] = ((2 * ca - cb) % M, cb % M)                  # U = 2 c_a - c_b, V = c_b
+        plus = [staged.sym(4 * (ca + E.cube_root_of_unity(m) * cb), m) for m in mods]
+        minus = [staged.sym(4 * (ca + E.cube_root_of_unity(m) ** 2 * cb), m) for m in mods]
+        return plus + minus
+
+    _post_operand_checks(t, mods, M, plane_values, lambda c: state["want"], 100 + nmod)
