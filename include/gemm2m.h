@@ -42,6 +42,8 @@
  *     M reaches about 2^184; useful when a row of A or a column of B spans many binary orders of magnitude.  The
  *     rank-k family and gemm2m_gaussian_int take 2M moduli only.
  *   - One call at a time per workspace: calls that share a workspace must be ordered on the GPU (same stream).
+ *   - Entry points may be called from several host threads, on the same or on different GPUs; they serialise on one
+ *     library-wide mutex for the time it takes to enqueue a call (the GPU work of calls on different GPUs still overlaps).
  *   - Non-finite inputs: a row of A (column of B) that contains an Inf or NaN yields NaN in the whole
  *     corresponding row (column) of C; no error is reported.
  */
@@ -146,8 +148,8 @@ int cgemm2m_ex(char transa, char transb, int64_t m, int64_t n, int64_t k, const 
  * Process-wide; takes effect with the next call.  The rank-k family always uses 0. */
 int gemm2m_set_scaling(int mode);
 
-/* The real Ozaki-II scheme the paper builds on and compares with (Section 3.1; "1 ZGEMM costs about 2.16 DGEMMs",
- * Section 6): C = A B for REAL double matrices (A: m x k, lda >= m; B: k x n, ldb >= k; C: m x n, ldc >= m, real doubles),
+/* The real Ozaki-II scheme the paper builds on and compares with (Section 3.1; Section 6 finds one ZGEMM to cost about
+ * 2.16 real Ozaki-II DGEMMs): C = A B for REAL double matrices (A: m x k, lda >= m; B: k x n, ldb >= k; C: m x n, ldc >= m, real doubles),
  * with ONE real int8 GEMM per modulus of the real modulus set of Section 4 (256, 255, 253, 251, 247, 241, ...; every
  * coprime number qualifies, nmod <= 20, 15 give M ~ 2^117).  Same readings as zgemm2m: power-of-two scale factors from
  * the largest magnitude of a row / column times sqrt(k), truncation, symmetric residues, one rounding.  Workspace:
@@ -208,8 +210,10 @@ int dsyr2k2m(int64_t n, int64_t k, const double* A, int64_t lda, const double* B
  * initialisation, or code on a latency-critical path where an allocation's implicit synchronisation is unacceptable.
  * They cannot provide the workspace the other entry points need.  This call computes, for the rows of A (m x k
  * complex128, column-major, lda >= m, device pointer), exactly the scale exponents e_i (sigma_i = 2^e_i, Algorithm 1
- * step 2) that zgemm2m(m, *, k, ..., nmod) uses, and writes them to e (int32[m], device pointer), using a scratch array
+ * step 2) that zgemm2m(m, *, k, ..., nmod) uses under its default scaling rule (the rule of gemm2m_set_scaling(0), whatever
+ * rule is selected at the time of the call), and writes them to e (int32[m], device pointer), using a scratch array
  * that is built into the library instead of a workspace.  It calls no cudaMalloc/cudaFree and no allocating library.
+ * Returns GEMM2M_ERR_ARCH on a device that is not compute capability 10.0.
  *   - At most GEMM2M_STATIC_MAX_ROWS rows; more returns GEMM2M_ERR_WORKSPACE and launches nothing.
  *   - The built-in scratch (8 bytes per row of the maximum, 512 KB) is held by every GPU that loads the library until the
  *     process exits, is shared by all calls and keeps the last call's contents; the call clears what it uses.  Two calls
@@ -252,14 +256,14 @@ typedef struct {
 } gemm2m_layout;
 int gemm2m_workspace_layout(int op, int64_t m, int64_t n, int64_t k, int nmod, gemm2m_layout* out);
 
+/* Failure handling, exercised without a fault: enqueues a one-thread kernel that waits, with the bounded wait every role of the
+ * GEMM kernel uses, on a barrier nobody ever arrives on.  After budget_ns (checked about every 0.2 ms) the wait gives up, records
+ * its code in the workspace's status word and the kernel returns; gemm2m_device_status() then reports
+ * GEMM2M_ERR_DEVICE_TIMEOUT once and clears the word.  Needs a registered workspace (GEMM2M_ERR_WORKSPACE otherwise). */
+int gemm2m_debug_wait_selftest(uint64_t budget_ns, void* stream);
 /* Which int8 GEMM kernel later calls use: 0 = the tcgen05 kernel on CTA pairs (default), 1 = a plain CUDA-core check
- * kernel kept only so that tests can tell a fault in a tensor-core kernel from one in the pre/post kernels, 2 = the
- * tcgen05 kernel with one CTA per tile. */
+ * kernel kept only so that tests can tell a fault in the tensor-core kernel from one in the pre/post kernels. */
 int gemm2m_debug_set_gemm_kernel(int which);
-/* Which kernel forms the residues of floating-point operands: 0 = the dp4a kernel (default), 1 = the tensor-core kernel
- * (the digit-weight contraction of Eq. (2a) as an int8 MMA with the planes along the TMEM lanes; same planes, bit for
- * bit; measured slower than the default and kept as a selectable variant). */
-int gemm2m_debug_set_residue_kernel(int which);
 /* Largest number of column panels zgemm2m/cgemm2m cut C into (default 8; panels are about 1024 to 2048 columns wide).  With 1 the phases run strictly one after the
  * other on the caller's stream, which is what per-phase bandwidth figures should be measured with. */
 int gemm2m_debug_set_panels(int max_panels);

@@ -14,6 +14,7 @@ OP_GAUSSIAN_INT, OP_ZGEMM, OP_CGEMM, OP_ZHERK, OP_ZHER2K, OP_DSYRK, OP_DSYR2K, O
 OP_ZGEMM_EISENSTEIN = 8
 OP_ZGEMM_HOST = 9
 OK = 0
+ERR_ARG, ERR_NMOD, ERR_WORKSPACE, ERR_CUDA, ERR_ARCH, ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5, 6     # gemm2m_status
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgemm2m.so")
@@ -76,11 +77,11 @@ def lib():
     L.gemm2m_last_launch_count.argtypes = [ctypes.POINTER(i32)]
     L.gemm2m_workspace_layout.argtypes = [i32, i64, i64, i64, i32, ctypes.POINTER(Layout)]
     L.gemm2m_debug_set_gemm_kernel.argtypes = [i32]
+    L.gemm2m_debug_wait_selftest.argtypes = [ctypes.c_uint64, vp]
     L.gemm2m_debug_set_panels.argtypes = [i32]
     L.dgemm_ozaki2.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, i32, vp]
     L.gemm2m_debug_tables_real.argtypes = [i32, i64] + [vp] * 10
     L.gemm2m_set_scaling.argtypes = [i32]
-    L.gemm2m_debug_set_residue_kernel.argtypes = [i32]
     L.gemm2m_debug_tables.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
     L.gemm2m_debug_residue_reduction.argtypes = [i32, vp, vp, vp, vp, vp]
     L.gemm2m_debug_post_operands.argtypes = [i32, i32, vp, vp, vp]
@@ -339,6 +340,11 @@ def last_launch_count():
     return total, [int(x) for x in per]
 
 
+def debug_wait_selftest(budget_ns, stream=None):
+    """Enqueue the bounded-wait self-test (see gemm2m_debug_wait_selftest)."""
+    _check(lib().gemm2m_debug_wait_selftest(int(budget_ns), _stream_ptr(stream)), "gemm2m_debug_wait_selftest")
+
+
 def debug_set_gemm_kernel(which):
     _check(lib().gemm2m_debug_set_gemm_kernel(which), "gemm2m_debug_set_gemm_kernel")
 
@@ -346,11 +352,6 @@ def debug_set_gemm_kernel(which):
 def set_scaling(mode):
     """0 = scale factors from the largest part of each row / column (default), 1 = from a bound of its 2-norm."""
     _check(lib().gemm2m_set_scaling(int(mode)), "gemm2m_set_scaling")
-
-
-def debug_set_residue_kernel(which):
-    """0 = dp4a residue kernel (default), 1 = tensor-core residue kernel."""
-    _check(lib().gemm2m_debug_set_residue_kernel(int(which)), "gemm2m_debug_set_residue_kernel")
 
 
 def debug_set_panels(max_panels):

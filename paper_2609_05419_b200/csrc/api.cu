@@ -42,9 +42,8 @@ struct State {
     Slot* cur_slot = nullptr;     // slot of the call being enqueued
     int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call (1 = no overlap)
     int launches[4] = {0, 0, 0, 0};
-    int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel, 2 = tcgen05 single CTA
+    int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel
     int scaling = 0;              // 0 = largest part times sqrt(2k), 1 = 2-norm rule (zgemm2m / cgemm2m)
-    int residue_kernel = 0;       // 0 = dp4a residue kernel, 1 = tensor-core residue kernel (measured slower; kept selectable)
 };
 State g;
 DevState& D() { return g.dev[g.cur]; }
@@ -193,14 +192,13 @@ int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R
             return GEMM2M_ERR_ARG;
         }
     }
-    if (g.residue_kernel == 0) CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
-    else CK(launch_residues_tc<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, dev_status, D().sm_count, st, &g.launches[1]));
+    (void)dev_status;
+    CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
     return GEMM2M_OK;
 }
 
 int run_gemm(const GemmArgs& a, int64_t klim, cudaStream_t st) {
     if (g.gemm_kernel == 1) CK(launch_gemm_check(a, klim, st, &g.launches[2]));
-    else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(a, klim, D().sm_count, st, &g.launches[2]));
     else CK(launch_gemm_tcgen05_pair(a, klim, D().sm_count, st, &g.launches[2]));
     return GEMM2M_OK;
 }
@@ -799,10 +797,7 @@ int dgemm_ozaki2(int64_t m, int64_t n, int64_t k, const double* A, int64_t lda, 
     if (int s = panel_pipeline(n, st, ph,
             [&](int64_t j0, int64_t j1) {
                 ga.row_begin = j0; ga.row_end = j1;
-                if (g.gemm_kernel == 1) CK(launch_gemm_check(ga, klim, st, &g.launches[2]));
-                else if (g.gemm_kernel == 2) CK(launch_gemm_tcgen05(ga, klim, D().sm_count, st, &g.launches[2]));
-                else CK(launch_gemm_tcgen05_pair(ga, klim, D().sm_count, st, &g.launches[2]));
-                return (int)GEMM2M_OK;
+                return run_gemm(ga, klim, st);
             },
             [&](int64_t j0, int64_t j1, cudaStream_t ps) {
                 return launch_post_real(cpl, c.ldp, m, n, j0, j1, eA, eB, ctab, C, ldc, ps, &g.launches[3]);
@@ -840,6 +835,14 @@ int gemm2m_device_status(void* stream) {
         CK(cudaMemset(D().ws, 0, sizeof(int)));
         return GEMM2M_ERR_DEVICE_TIMEOUT;
     }
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_wait_selftest(uint64_t budget_ns, void* stream) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    if (int s = check_device()) return s;
+    if (!D().ws) return GEMM2M_ERR_WORKSPACE;
+    CK(launch_wait_selftest((int*)D().ws, (unsigned long long)budget_ns, (cudaStream_t)stream));
     return GEMM2M_OK;
 }
 
@@ -887,7 +890,7 @@ int gemm2m_debug_set_panels(int max_panels) {
 
 int gemm2m_debug_set_gemm_kernel(int which) {
     std::lock_guard<std::mutex> lock(g.mu);
-    if (which < 0 || which > 2) return GEMM2M_ERR_ARG;
+    if (which < 0 || which > 1) return GEMM2M_ERR_ARG;
     g.gemm_kernel = which;
     return GEMM2M_OK;
 }
@@ -896,13 +899,6 @@ int gemm2m_set_scaling(int mode) {
     std::lock_guard<std::mutex> lock(g.mu);
     if (mode < 0 || mode > 1) return GEMM2M_ERR_ARG;
     g.scaling = mode;
-    return GEMM2M_OK;
-}
-
-int gemm2m_debug_set_residue_kernel(int which) {
-    std::lock_guard<std::mutex> lock(g.mu);
-    if (which < 0 || which > 1) return GEMM2M_ERR_ARG;
-    g.residue_kernel = which;
     return GEMM2M_OK;
 }
 

@@ -20,7 +20,7 @@ constexpr int kExpNonFinite = INT32_MIN;   // scale-exponent sentinel: row/colum
 
 // Device status word values (written by kernels whose bounded waits give up).
 constexpr int kDevOk = 0;
-constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilogue = 103;
+constexpr int kDevTimeoutProducer = 101, kDevTimeoutMma = 102, kDevTimeoutEpilogue = 103, kDevTimeoutSelfTest = 104;
 
 // Number of 2M moduli among the first nmod, and of residue planes per operand.  Plane order: X+ of the 2M moduli, X- of the
 // 2M moduli, then for the 3M moduli X_r, X_i, X_r + X_i (each group in modulus order).
@@ -169,10 +169,6 @@ cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, 
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
                                                      const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches,
                                                      int64_t plane_rows = 0);
-// The same on the tensor cores (residues_tc.cu): the byte-weight contraction as an int8 MMA, planes along the TMEM lanes.
-template <typename T> cudaError_t launch_residues_tc(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
-                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status,
-                                                     int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).
@@ -199,7 +195,7 @@ cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_
 cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,
                             int64_t ldc, cudaStream_t st, int* launches);
 
-// ---- int8 GEMM (gemm_i8.cu) ----
+// ---- int8 GEMM (gemm_i8_2cta.cu; check kernel: gemm_check.cu) ----
 // For each batch b in [0, nbatch): out[b][r][c] = sym( sum_k rowop[b + row_plane0][r][k] * colop[b + col_plane0][c][k]  mod (modulus of batch entry b) ),
 // r < R, c < Cn, k < Kp (zero padded); planes are [*][rows][Kp] int8; out planes are [R][ldp] int8.
 struct GemmArgs {
@@ -213,8 +209,10 @@ struct GemmArgs {
     ModTable mods;
     int* dev_status;
 };
-cudaError_t launch_gemm_tcgen05(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);        // one CTA per tile
-cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);   // CTA pairs (default)
+cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_count, cudaStream_t st, int* launches);   // CTA pairs
 cudaError_t launch_gemm_check(const GemmArgs& a, int64_t k_limit, cudaStream_t st, int* launches);
+// One thread waits, with the GEMM kernel's bounded wait and a budget of budget_ns, on a barrier nobody arrives on: the wait
+// gives up, records its code in *dev_status and the kernel returns.
+cudaError_t launch_wait_selftest(int* dev_status, unsigned long long budget_ns, cudaStream_t st);
 
 }  // namespace gemm2m

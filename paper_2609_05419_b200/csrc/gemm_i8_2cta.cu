@@ -10,7 +10,11 @@
 // warps 2-5 = epilogue (tcgen05.ld, exact reduction mod m_j, one byte per entry to HBM).
 // Barriers: the leader's full[s] collects the bytes of both CTAs' loads; the MMA's commit is multicast to both CTAs'
 // empty[s] and tmem_full[a]; both CTAs' epilogue warps arrive on the leader's tmem_empty[a].
-// Every wait is bounded in time; on a timeout a code is recorded, both CTAs leave their loops, TMEM is freed.
+// Every wait is bounded in time.  When one gives up, a code is recorded, every role of both CTAs leaves its loop, and before
+// shared memory, barriers and TMEM go away the pair makes sure nothing is still in flight: the MMA issuer commits what it has
+// issued to a barrier of its own and waits for it; the leader's producer squares the byte counts of the stages that only one
+// CTA had got to (both producers publish how many stage fills they issued) and waits for the last fill of every stage, which
+// completes when both CTAs' copies of it have landed.  These waits are bounded too (0.1 s each).
 #include "gemm_ptx.cuh"
 
 namespace gemm2m {
@@ -29,7 +33,7 @@ constexpr int COL_HALF_BYTES = (BN / 2) * BK;    // 16 KB
 constexpr int STAGE_BYTES = ROW_TILE_BYTES + COL_HALF_BYTES;
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 512;                   // two accumulators of 256 columns
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;   // tiles (1024-byte aligned) + barriers and flags
 }  // namespace cfg2
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -52,6 +56,11 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 }
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t cluster_addr) {
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+    return v;
 }
 // TMA load of this CTA's tile whose completion bytes are credited to a barrier that may live in the peer CTA.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y, int z) {
@@ -85,8 +94,10 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
     uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + (size_t)STAGES * STAGE_BYTES);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * STAGES, bar_tempty = bar_tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    const uint32_t bar_drain = bar_tempty + 16;           // give-up path only: the MMA issuer's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile uint32_t* fills_issued = reinterpret_cast<volatile uint32_t*>(tmem_slot + 2);   // stage fills this CTA's producer issued
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();            // 0 = leader
@@ -95,7 +106,9 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 8); }   // 4 warps of each CTA
+        mbar_init(bar_drain, 1);
         *abort_flag = 0;
+        *fills_issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -117,7 +130,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             const uint32_t leader_full = map_to_cta(bar_full, 0);
-            uint32_t stage = 0, phase = 0;
+            uint32_t stage = 0, phase = 0, fills = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < total_tiles; tile += npairs) {
                 int b, tr, tc;
@@ -125,15 +138,17 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
                 const int row0 = tr * (2 * BM) + (int)rank * BM;
                 const int col0 = tc * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < p.kblocks; ++kb) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, kDevTimeoutProducer))) break;
+                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, kDevTimeoutProducer, p.wait_ns))) break;
                     const uint32_t dst = tiles_base + stage * STAGE_BYTES;
                     if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * STAGE_BYTES);   // both CTAs' bytes
                     const int x = (p.kblock0 + kb) * BK;
                     tma_load_3d_pair(dst, &map_row, leader_full + 8 * stage, x, row0, p.row_plane0 + b);
                     tma_load_3d_pair(dst + ROW_TILE_BYTES, &map_col, leader_full + 8 * stage, x, col0, p.col_plane0 + b);
+                    ++fills;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            *fills_issued = fills;
             if (!ok) st_cluster_u32(peer_abort, 1u);
         }
     } else if (warp == 1) {
@@ -146,12 +161,12 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
             int it = 0;
             for (int tile = pair; ok && tile < total_tiles; tile += npairs, ++it) {
                 const int acc = it & 1;
-                if (!(ok = mbar_wait(bar_tempty + 8 * acc, acc_phase[acc] ^ 1u, abort_flag, p.dev_status, kDevTimeoutMma))) break;
+                if (!(ok = mbar_wait(bar_tempty + 8 * acc, acc_phase[acc] ^ 1u, abort_flag, p.dev_status, kDevTimeoutMma, p.wait_ns))) break;
                 acc_phase[acc] ^= 1u;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < p.kblocks; ++kb) {
-                    if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status, kDevTimeoutMma))) break;
+                    if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status, kDevTimeoutMma, p.wait_ns))) break;
                     tcgen05_fence_after();
                     const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
                     const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + ROW_TILE_BYTES);
@@ -164,7 +179,12 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
                 }
                 if (ok) umma_commit_pair(bar_tfull + 8 * acc, 3);    // accumulator complete in both CTAs
             }
-            if (!ok) st_cluster_u32(peer_abort, 1u);
+            if (!ok) {
+                st_cluster_u32(peer_abort, 1u);
+                // MMAs already issued still read both CTAs' shared memory and write both TMEMs: wait until they are through
+                umma_commit_pair(bar_drain, 1);
+                mbar_wait_quiet(bar_drain, 0, kDrainLimitNs);
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
@@ -179,7 +199,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
             decode_tile(p, tile, &b, &tr, &tc);
             const int jm = b;                             // the modulus table has one entry per batch entry
             const ModConsts mc = load_mod_consts(p.mods, jm);
-            if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase[acc], abort_flag, p.dev_status, kDevTimeoutEpilogue))) break;
+            if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase[acc], abort_flag, p.dev_status, kDevTimeoutEpilogue, p.wait_ns))) break;
             acc_phase[acc] ^= 1u;
             tcgen05_fence_after();
             const int64_t row = (int64_t)tr * (2 * BM) + (int64_t)rank * BM + quarter * 32 + lane;
@@ -216,6 +236,29 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync_all();            // neither CTA's shared memory, barriers or TMEM may go away while the peer still uses them
+    // A role that gives up sets its CTA's flag and then the peer's, both before this point, so the two CTAs agree on the flag.
+    if (*abort_flag) {
+        // Bulk copies may still be on their way into either CTA's shared memory, each crediting its bytes to the leader's
+        // full[stage].  The producers run at most STAGES fills apart (a fill of a stage follows the MMAs that consumed the
+        // stage's previous fill, which needed both CTAs' bytes), so every barrier is short of, or ahead by, at most one fill:
+        // the leader takes the missing peer bytes off, or announces the peer bytes it had not got to, and then waits for
+        // the last fill of every stage to complete.
+        if (warp == 0 && lane == 0 && rank == 0) {
+            const uint32_t mine = *fills_issued, peers = ld_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(fills_issued)), 1u));
+            for (uint32_t f = min(mine, peers); f < max(mine, peers); ++f) {
+                const uint32_t bar = bar_full + 8 * (f % STAGES);
+                if (peers < mine) mbar_complete_tx(bar, STAGE_BYTES);
+                else mbar_arrive_expect_tx(bar, STAGE_BYTES);
+            }
+            const uint32_t fills = max(mine, peers);
+            for (uint32_t s = 0; s < (uint32_t)STAGES && s < fills; ++s) {
+                const uint32_t last = s + STAGES * ((fills - 1 - s) / STAGES);       // last fill of stage s
+                mbar_wait_quiet(bar_full + 8 * s, (last / STAGES) & 1u, kDrainLimitNs);
+            }
+        }
+        __syncthreads();
+        cluster_sync_all();
+    }
     if (warp == 1) {
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
@@ -267,6 +310,7 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
     p.out_plane_stride = a.R * a.ldp;
     p.mods = a.mods;
     p.dev_status = a.dev_status;
+    p.wait_ns = kWaitLimitNs;
     p.band = p.tiles_r < 8 ? p.tiles_r : 8;
     const int64_t total_tiles = (int64_t)p.tiles_r * p.tiles_c * p.nbatch;
     if (total_tiles > INT32_MAX) return cudaErrorInvalidValue;
@@ -280,6 +324,24 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
         gemm_i8_tcgen05_pair_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(map_row, map_col, p);   // cluster size is a kernel attribute
         ++*launches;
     }
+    return cudaGetLastError();
+}
+
+// The bounded wait of the GEMM kernel on its own: one thread, one barrier that nobody arrives on.  No pipeline, no bulk copy,
+// no TMEM: the wait runs out after budget_ns, records its code and the kernel returns.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(int* dev_status, unsigned long long budget_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0, &abort_flag, dev_status, kDevTimeoutSelfTest, budget_ns);
+    }
+}
+
+cudaError_t launch_wait_selftest(int* dev_status, unsigned long long budget_ns, cudaStream_t st) {
+    wait_selftest_kernel<<<1, 32, 0, st>>>(dev_status, budget_ns);
     return cudaGetLastError();
 }
 

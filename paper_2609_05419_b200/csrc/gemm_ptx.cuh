@@ -7,7 +7,8 @@
 
 namespace gemm2m {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s budget of every device-side wait
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: default budget of every device-side wait (GemmKernelParams::wait_ns)
+constexpr unsigned long long kDrainLimitNs = 100000000ull;   // 0.1 s: budget of the waits of the give-up path, per barrier
 constexpr int kGemmBK = 128;                                  // bytes of K per pipeline stage (one 128-byte swizzle row)
 
 // ------------------------------------------------------------------------------------------------ PTX helpers
@@ -50,21 +51,34 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait.  Returns false (and records `code`) if the barrier did not complete in time or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int code) {
+// Bounded wait.  Returns false (and records `code`) if the barrier did not complete within limit_ns or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int code,
+                                          unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try_wait_parked(bar, parity, 10000u)) return true;
         if ((spins & 15u) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(dev_status, kDevOk, code);
                 return false;
             }
         }
     }
+}
+
+// Bounded wait of the give-up path: no status, no flag; returns whether the phase completed.
+__device__ __forceinline__ bool mbar_wait_quiet(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+    const unsigned long long t0 = global_timer_ns();
+    while (!mbar_try_wait_parked(bar, parity, 10000u))
+        if (global_timer_ns() - t0 > limit_ns) return false;
+    return true;
+}
+// Takes `bytes` off the pending transaction count of the barrier's current phase (bytes that were announced and will not come).
+__device__ __forceinline__ void mbar_complete_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
@@ -185,6 +199,7 @@ struct GemmKernelParams {
     int tr0;                 // first row tile of this launch (tiles_r counts the row tiles of the launch)
     ModTable mods;
     int* dev_status;
+    unsigned long long wait_ns;   // budget of every device-side wait
 };
 
 // Linear tile index -> (batch, row tile, column tile).  Within a batch the tiles are walked in bands of `band` row tiles,

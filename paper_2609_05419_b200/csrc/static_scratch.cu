@@ -18,15 +18,25 @@ static __device__ __align__(256) unsigned long long g_static_absmax[GEMM2M_STATI
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 unsigned long long* g_scratch_addr[kMaxDevices] = {};   // device address of g_static_absmax, per device
+int g_arch_ok[kMaxDevices] = {};                        // 0 = not asked yet, 1 = compute capability 10.0, -1 = anything else
 
 // In host code the name g_static_absmax is only a handle, not a device address: handing it to a kernel would make
 // the kernel read and write some unrelated location.  The address on the current device comes from the runtime.
-cudaError_t scratch_for_current_device(unsigned long long** out) {
+cudaError_t scratch_for_current_device(unsigned long long** out, bool* arch_ok) {
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_arch_ok[dev]) {
+        int major = 0, minor = 0;
+        err = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (err == cudaSuccess) err = cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev);
+        if (err != cudaSuccess) return err;
+        g_arch_ok[dev] = (major == 10 && minor == 0) ? 1 : -1;
+    }
+    *arch_ok = g_arch_ok[dev] > 0;
+    if (!*arch_ok) return cudaSuccess;                     // the kernels exist for this architecture only
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         err = cudaGetSymbolAddress(&p, g_static_absmax);   // set-up, once per device, with that device current
@@ -46,7 +56,9 @@ extern "C" int gemm2m_zscale_exponents_static(int64_t m, int64_t k, const double
     if (m == 0) return GEMM2M_OK;
     if (!e || (k > 0 && !A)) return GEMM2M_ERR_ARG;
     unsigned long long* scratch = nullptr;
-    if (scratch_for_current_device(&scratch) != cudaSuccess) return GEMM2M_ERR_CUDA;
+    bool arch_ok = false;
+    if (scratch_for_current_device(&scratch, &arch_ok) != cudaSuccess) return GEMM2M_ERR_CUDA;
+    if (!arch_ok) return GEMM2M_ERR_ARCH;
     cudaStream_t st = (cudaStream_t)stream;
     const ScaleTargets sc = scale_targets(nmod, k, false);
     int launches = 0;

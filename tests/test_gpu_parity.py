@@ -18,11 +18,9 @@ TOL_C = 2e-6       # complex64
 @pytest.fixture(autouse=True)
 def _default_kernel():
     b.debug_set_gemm_kernel(0)
-    b.debug_set_residue_kernel(0)
     b.debug_set_panels(8)
     yield
     b.debug_set_gemm_kernel(0)
-    b.debug_set_residue_kernel(0)
     b.debug_set_panels(8)
 
 
@@ -48,7 +46,7 @@ def check_stages_int(st, ref, m, n, k, nmod):
             assert (st["Cpm"][sgn, j, :, :m] == ref["Cpm"][j][sgn].T).all(), ("Cpm", sgn, j)
 
 
-@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])   # check kernel first: isolates pre/post from the tensor-core GEMM
+@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])   # check kernel first: isolates pre/post from the tensor-core GEMM
 @pytest.mark.parametrize("shape,nmod", [((128, 128, 128), 3), ((128, 128, 128), 1), ((128, 128, 128), 2),
                                         ((130, 77, 300), 3), ((1, 1, 1), 1), ((257, 513, 129), 4), ((5, 300, 1000), 8)])
 def test_gaussian_int_bit_exact(shape, nmod, kernel):
@@ -110,7 +108,7 @@ def run_z(A, B, nmod, kernel=0, cplx=torch.complex128, op=None):
         return to_host(C), st
 
 
-@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])
+@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])
 @pytest.mark.parametrize("shape,nmod,dist", [((200, 150, 300), 16, "phi"), ((129, 257, 128), 14, "uniform"),
                                              ((64, 64, 64), 3, "uniform"), ((33, 19, 50), 22, "phi"), ((40, 40, 520), 20, "uniform")])
 def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
@@ -132,7 +130,7 @@ def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
         assert direct.componentwise_error(C, Cref, D) <= TOL_Z
 
 
-@pytest.mark.parametrize("kernel", [1, 2, 0], ids=["checkgemm", "tcgen05-1cta", "tcgen05"])
+@pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])
 @pytest.mark.parametrize("shape,nmod,phi", [((70, 90, 200), 23, 4.0), ((129, 257, 128), 26, 6.0), ((33, 19, 50), 24, 1.0),
                                             ((40, 300, 520), 25, 8.0)])
 def test_zgemm_hybrid_every_stage_against_staged_oracle(shape, nmod, phi, kernel):
@@ -194,31 +192,6 @@ def test_hybrid_beats_the_2m_set_on_a_wide_exponent_span_and_cgemm_accepts_it():
     ref = staged.zgemm2m_staged(A32, B32, 23, out_bits=24)
     for got, want in ((C32.real, ref["C"].real), (C32.imag, ref["C"].imag)):   # 53 then 24 bits: within one float ulp
         assert (np.abs(got.astype(np.float64) - want) <= np.spacing(np.abs(want).astype(np.float32)).astype(np.float64)).all()
-
-
-@pytest.mark.parametrize("shape,nmod,dist,dtype", [((200, 150, 300), 16, "phi", np.complex128), ((129, 257, 128), 14, "uniform", np.complex128),
-                                                   ((33, 19, 50), 22, "phi", np.complex128), ((70, 90, 200), 25, "phi", np.complex128),
-                                                   ((257, 300, 1000), 7, "uniform", np.complex64), ((64, 40, 130), 23, "phi", np.complex64)])
-def test_tensor_core_residue_kernel_gives_the_same_planes(shape, nmod, dist, dtype):
-    """The selectable residue kernel (digit-weight contraction as an int8 MMA): every plane bit-exact against the staged
-    oracle, narrow and wide quantised values, four and two element blocks per instruction, 2M and 3M moduli, ragged tiles."""
-    m, n, k = shape
-    A, B = inputs.complex_inputs(m, n, k, seed=31, dist=dist, phi=2.0, dtype=dtype)
-    b.debug_set_residue_kernel(1)
-    C, st = run_z(A, B, nmod, kernel=1, cplx=torch.complex128 if dtype == np.complex128 else torch.complex64)
-    ref = staged.zgemm2m_staged(A, B, nmod, out_bits=53 if dtype == np.complex128 else 24)
-    n2 = min(nmod, 22)
-    for j in range(n2):
-        for sgn in range(2):
-            assert (st["Apm"][sgn, j, :, :k] == ref["Apm"][j][sgn]).all(), ("Apm", sgn, j)
-            assert (st["Bpm"][sgn, j, :, :k] == ref["Bpm"][j][sgn].T).all(), ("Bpm", sgn, j)
-            assert (st["Apm"][sgn, j, :, k:] == 0).all() and (st["Bpm"][sgn, j, :, k:] == 0).all()     # K padding
-    for j3 in range(nmod - n2):
-        for part in range(3):
-            assert (st["A3"][part, j3, :, :k] == ref["Apm"][22 + j3][part]).all(), ("A3", part, j3)
-            assert (st["B3"][part, j3, :, :k] == ref["Bpm"][22 + j3][part].T).all(), ("B3", part, j3)
-    if dtype == np.complex128:
-        assert ulp_distance(C.real, ref["C"].real).max() <= 1 and ulp_distance(C.imag, ref["C"].imag).max() <= 1
 
 
 @pytest.mark.parametrize("nmod,tol", [(16, TOL_Z), (15, TOL_Z), (14, 1e-13)])

@@ -226,6 +226,23 @@ def test_scaling_rule_and_truncation_invariants():
         assert st["PA"] + st["PB"] == st["Pt"] and 2 ** st["Pt"] <= (st["M"] - 1) // 2 < 2 ** (st["Pt"] + 1)
 
 
+def test_scaling_rule_wastes_less_than_one_bit_beyond_ck():
+    # The largest part of a row quantises into [2^(P - c_k - 1), 2^(P - c_k)): the budget P is used up to the c_k bits the
+    # sqrt(2k) factor of the 2-norm bound takes and less than one more.  An exponent one larger (a bit wasted per operand, which
+    # the overflow bound and the error bound alone would not notice) fails the lower limit.
+    rng = np.random.default_rng(8)
+    for nmod, k in ((7, 64), (16, 300), (16, 8192), (22, 100)):
+        vals = np.concatenate([2.0 ** rng.integers(-300, 300, 6), rng.uniform(1.0, 2.0, 6) * 2.0 ** rng.integers(-40, 40, 6),
+                               [np.nextafter(2.0, 1.0), 5e-324, 1.7e308]])
+        A = np.asfortranarray(np.repeat(vals[:, None], k, axis=1) * (1 + 0j))          # every entry of a row equals its maximum
+        B = np.asfortranarray(np.repeat(vals[None, :], k, axis=0) * (0 + 1j))
+        st = staged.zgemm2m_staged(A, B, nmod, upto="pre")
+        ck = staged.scaling_targets(st["M"], k)[3]
+        for q, P in ((st["Aq"][0][:, 0], st["PA"]), (st["Bq"][1][0, :], st["PB"])):
+            lo, hi = P - ck - 1, P - ck
+            assert all(2 ** lo <= int(v) < 2 ** hi for v in q if lo >= 0), (nmod, k)
+
+
 @pytest.mark.parametrize("nmod", [14, 16, 22])
 def test_staged_float_path_meets_error_bound_and_equals_4m_on_quantised(nmod):
     A, B = inputs.complex_inputs(12, 9, 100, seed=9, dist="phi", phi=0.5)

@@ -18,6 +18,14 @@ from paper_2609_05419_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 from gpu_util import Workspace, empty_dev, to_dev  # noqa: E402
+from oracle import staged  # noqa: E402
+
+
+def exponents_from_oracle(A, k, nmod):
+    """The staged oracle's rule for the rows of A (Algorithm 1 step 2), from the budget of the first nmod moduli."""
+    M = staged.product(staged.hybrid_moduli(nmod))
+    _, PA, _, ck = staged.scaling_targets(M, k)
+    return staged.scaling_exponents(A, 1, PA, ck)
 
 
 def exponents_from_zgemm2m(A, B, nmod):
@@ -48,6 +56,8 @@ def test_static_scratch_entry_point_matches_zgemm2m_on_two_calls_in_a_row():
     assert torch.cuda.memory_allocated() == before
     assert (e1.cpu().numpy() == want1).all()
     assert (e2.cpu().numpy() == want2).all()
+    assert (e1.cpu().numpy() == exponents_from_oracle(A1, k, nmod)).all()      # and against the oracle itself, not only zgemm2m
+    assert (e2.cpu().numpy() == exponents_from_oracle(A2, k, nmod)).all()
     assert want2[5] == 0 and (want2[:5] < want1[:5]).all()
 
 
