@@ -295,35 +295,27 @@ def run_ours(a):
     b.set_profiling(False)
     b.device_status()
     launches_per_step, per_phase = b.last_launch_count()
-    # the same phases strictly one after the other (no panel overlap): what the per-phase bandwidth figures are taken from
-    b.debug_set_panels(1)
-    b.set_profiling(True)
-    for _ in range(5):
-        step()
-    serial, _ = b.phase_ms()
-    b.set_profiling(False)
-    b.debug_set_panels(8)
-    b.device_status()
+    serial = phase                                      # the phases of a call run one after the other on the call's stream
     # whole calls of the two panel modes, alternating in one loop (same clocks, same temperature for both)
     ab = None
     if a.ab_calls > 0:
         pairs = {8: [], 1: []}
         for _ in range(a.ab_calls):
             for panels in (8, 1):
-                b.debug_set_panels(panels)
+                b.debug_set_overlap(panels == 8)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 step()
                 e1.record(stream)
                 pairs[panels].append((e0, e1))
-        b.debug_set_panels(8)
+        b.debug_set_overlap(False)
         torch.cuda.synchronize()
         b.device_status()
         t = {p: [x.elapsed_time(y) for x, y in v] for p, v in pairs.items()}
         ab = {"calls_per_mode": a.ab_calls, "overlap_ms_median": float(np.median(t[8])), "overlap_ms_best": float(min(t[8])),
               "serial_ms_median": float(np.median(t[1])), "serial_ms_best": float(min(t[1])),
-              "note": "whole calls, the two panel modes alternating call by call: post-processing of a panel beside the next panel's "
-                      "GEMMs (default) against every phase on the caller's stream, one after the other"}
+              "note": "whole calls of the two modes alternating call by call: post-processing of a panel on a second stream beside the "
+                      "next panel's GEMMs (gemm2m_debug_set_overlap(1)) against every kernel on the caller's stream, in order (default)"}
 
     # ---- end to end.  zgemm: the library's call on HOST operands (zgemm2m_host): every step uploads A and B from pinned host
     # memory, runs the whole path and downloads C inside the one C-ABI call (A first, B in column panels whose kernels run
@@ -393,10 +385,10 @@ def run_ours(a):
                               "SM clock sampled under load) compares runs taken at different clocks",
                 "launch_ms": phase[2] / gemm_launches, "launches_per_step": gemm_launches, "algorithmic_ops_per_launch": gemm_ops}
     gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else None
-    phases = {"note": "sums of kernel durations per phase in the timed region; post-processing of a panel runs beside the "
-                      "next panel's GEMMs, so the phases add up to more than ms_per_step",
+    phases = {"note": "kernel time per phase and call in the timed region (events recorded by the library around every launch on "
+                      "the call's stream; the phases run one after the other)",
               "scan_ms": phase[0], "residues_ms": phase[1], "gemm_ms": phase[2], "post_ms": phase[3], "calls_averaged": calls}
-    phases_serial = {"note": "5 extra calls with the panel overlap switched off (phases strictly sequential)",
+    phases_serial = {"note": "the same phase times as bytes per second: algorithmic bytes of the phase over its kernel time",
                      "scan_ms": serial[0], "residues_ms": serial[1], "gemm_ms": serial[2], "post_ms": serial[3],
                      "scan_gbs": gbs(scan_bytes, serial[0]), "residues_gbs": gbs(pre_bytes, serial[1]), "post_gbs": gbs(post_bytes, serial[3]),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]}
@@ -408,7 +400,7 @@ def run_ours(a):
         cpu, _ = time_oracle(a, *oracle_operands(a, A, B), a.cpu_seconds)
     line = {"metric": a.metric, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(a.warmup, 3),
             "ms_per_step": ms_step, "ms_per_step_median": float(np.median(per_step)), "ms_per_step_best": float(min(per_step)),
-            "ms_per_step_serial": ab["serial_ms_median"] if ab else None,
+            "ms_per_step_serial": ab["serial_ms_median"] if ab else None, "ms_per_step_overlap": ab["overlap_ms_median"] if ab else None,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
             "data": "synthetic",
             "config": {"workload": workload_name(a),

@@ -24,12 +24,16 @@
  *   - All matrix pointers are DEVICE pointers owned by the caller (zgemm2m_host alone takes host pointers).  The library never allocates or frees device
  *     memory inside a call; it uses the caller-provided workspace registered with gemm2m_set_workspace().
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and
- *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  zgemm2m and cgemm2m
- *     additionally use one library-owned stream, forked from and joined back into `stream` with events: work enqueued
- *     on `stream` after the call still sees the finished result.  (zgemm2m_host uses two more, for its copies.)
+ *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  Every kernel of a call
+ *     runs on `stream`, in order.  (zgemm2m_host alone uses library-owned streams, for its copies and the work that runs
+ *     beside them, forked from and joined back into `stream` with events: work enqueued on `stream` after the call still
+ *     sees the finished result.  So does every entry point while gemm2m_debug_set_overlap(1) is in force.)
  *   - Because a call only enqueues (kernels, memsets, event records and waits), it can be captured into a CUDA graph
- *     and replayed; the library-owned stream joins the capture through its fork/join events.  Make one call outside any
- *     capture first: it creates that stream and its events.  (gemm2m_set_profiling must be off during a capture.)
+ *     and replayed; a library-owned stream joins the capture through its fork/join events.  Make one call outside any
+ *     capture first: it creates such streams and events, and leaves in the workspace the constant operand of the
+ *     post-processing, which later calls with the same modulus count reuse.  (gemm2m_set_profiling must be off during a capture.)
+ *   - The workspace belongs to the library while it is registered: besides the status word it keeps that operand between
+ *     calls.  Register it again (gemm2m_set_workspace) after writing to it.
  *   - Argument errors are detected on the host before anything is launched.  m, n or k equal to 0 is valid:
  *     nothing is computed for m = 0 or n = 0, and C is set to zero for k = 0.
  *   - `nmod` selects the first nmod moduli of the set of Section 4 (241, 233, 229, 221, 205, ... , 37, 29; 22 in
@@ -264,9 +268,13 @@ int gemm2m_debug_wait_selftest(uint64_t budget_ns, void* stream);
 /* Which int8 GEMM kernel later calls use: 0 = the tcgen05 kernel on CTA pairs (default), 1 = a plain CUDA-core check
  * kernel kept only so that tests can tell a fault in the tensor-core kernel from one in the pre/post kernels. */
 int gemm2m_debug_set_gemm_kernel(int which);
-/* Largest number of column panels zgemm2m/cgemm2m cut C into (default 8; panels are about 1024 to 2048 columns wide).  With 1 the phases run strictly one after the
- * other on the caller's stream, which is what per-phase bandwidth figures should be measured with. */
+/* Largest number of panels the output is cut into (default 8; panels are about 1024 to 2048 columns wide; the GEMMs of a panel
+ * are one launch, its post-processing the next). */
 int gemm2m_debug_set_panels(int max_panels);
+/* 0 (default): every kernel of a call runs on the caller's stream, in order.  1: the post-processing of a panel (and, for
+ * large operands, the exponent scan of B) runs on a library-owned stream beside the next panel's GEMMs, forked from and joined
+ * back into the caller's stream with events.  Kept for measurement: it does not pay on a GPU whose GEMM phase is power-limited. */
+int gemm2m_debug_set_overlap(int enabled);
 
 /* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host
  * pointers, any may be NULL), so that CPU tests can check them against an independent computation:

@@ -354,6 +354,10 @@ def set_scaling(mode):
     _check(lib().gemm2m_set_scaling(int(mode)), "gemm2m_set_scaling")
 
 
+def debug_set_overlap(enabled):
+    _check(lib().gemm2m_debug_set_overlap(1 if enabled else 0), "gemm2m_debug_set_overlap")
+
+
 def debug_set_panels(max_panels):
     _check(lib().gemm2m_debug_set_panels(max_panels), "gemm2m_debug_set_panels")
 

@@ -27,6 +27,7 @@ struct DevState {
     cudaEvent_t call_begin = nullptr, a_ready = nullptr, b_ready[kHostPanels] = {}, g_ready[kHostPanels] = {}, c_ready[kHostPanels] = {}, c_done = nullptr;
     int sm_count = 0;
     int arch_ok = -1;
+    int frags_key = 0;            // which post-processing operand the workspace holds: 0 = none, else 1 + nmod (+ 64 for the Eisenstein set)
 };
 
 struct State {
@@ -40,7 +41,8 @@ struct State {
     Slot slots[kProfSlots];       // timed intervals (phase, start, end) of the profiled calls
     int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
     Slot* cur_slot = nullptr;     // slot of the call being enqueued
-    int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call (1 = no overlap)
+    int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call
+    int overlap = 0;              // 1 = post-processing of a panel (and the scan of B) on the library's stream beside the next kernels
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel
     int scaling = 0;              // 0 = largest part times sqrt(2k), 1 = 2-norm rule (zgemm2m / cgemm2m)
@@ -182,18 +184,19 @@ constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kern
 
 // hex: the Eisenstein variant's lattice rounding in front of the same residue arithmetic (complex double only).
 template <typename T>
-int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st, bool hex = false) {
+int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
+                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st, bool hex = false,
+                 ScaleFrom from = ScaleFrom()) {
     if (hex) {
         if constexpr (sizeof(T) == 8) {
-            CK(launch_residues_hex(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
+            CK(launch_residues_hex(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1], from));
             return GEMM2M_OK;
         } else {
             return GEMM2M_ERR_ARG;
         }
     }
     (void)dev_status;
-    CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1]));
+    CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1], 0, from));
     return GEMM2M_OK;
 }
 
@@ -203,26 +206,30 @@ int run_gemm(const GemmArgs& a, int64_t klim, cudaStream_t st) {
     return GEMM2M_OK;
 }
 
-// Panel pipeline shared by every entry point: the rows [0, n) of the GEMM's row operand (columns of C for the GEMMs, rows of the
+// Panel loop shared by every entry point: the rows [0, n) of the GEMM's row operand (columns of C for the GEMMs, rows of the
 // lower triangle for the rank-k family) are cut into panels of about 1024 rows up to four of them, then of about 2048 rows
 // (more, narrower panels also keep the operand slices of a launch inside the L2: 16384 columns in 8 panels measured 6-8 %
 // faster than in 4).  gemm(r0, r1) enqueues the GEMMs of a panel on the caller's stream; post(r0, r1, stream) its
-// post-processing, which runs on the library's stream beside the GEMMs of the next panel, except for the last panel.  The
-// call is complete on the caller's stream only when the library's stream has been joined back.
+// post-processing, by default on the same stream right behind them.  With the overlap switched on (gemm2m_debug_set_overlap)
+// the post-processing of every panel but the last runs on the library's stream beside the GEMMs of the next panel, and the
+// call is complete on the caller's stream only when the library's stream has been joined back.  Measured with whole calls of
+// the two modes alternating in one loop, the overlap gains 0.4 % at 8192^3 and loses 0.8 % for cgemm2m at 16384 x 16384 x
+// 4096: the GEMM phase runs at the board's power limit, and what runs beside it slows it down by what it hides.
 template <typename GemmFn, typename PostFn>
 int panel_pipeline(int64_t n, cudaStream_t st, Phases& ph, GemmFn gemm, PostFn post) {
     int panels = (int)(n / 1024);
     if (panels > 4) panels = (int)(n / 2048) > 4 ? (int)(n / 2048) : 4;
     panels = panels < 1 ? 1 : (panels > g.max_panels ? g.max_panels : panels);
     const int64_t panel_rows = round_up((n + panels - 1) / panels, 256);
-    if (panels > 1) { if (int s = ensure_side_stream()) return s; }
+    const bool overlap = g.overlap && panels > 1;
+    if (overlap) { if (int s = ensure_side_stream()) return s; }
     for (int pnl = 0; pnl < panels; ++pnl) {
         const int64_t r0 = pnl * panel_rows, r1 = (r0 + panel_rows < n) ? r0 + panel_rows : n;
         if (r0 >= r1) break;
         CK(ph.begin(2, st));
         if (int s = gemm(r0, r1)) return s;
         CK(ph.end(st));
-        const bool last = r1 >= n;
+        const bool last = r1 >= n || !overlap;
         cudaStream_t ps = last ? st : D().side;
         if (!last) {
             CK(cudaEventRecord(D().panel_done[pnl], st));
@@ -232,7 +239,7 @@ int panel_pipeline(int64_t n, cudaStream_t st, Phases& ph, GemmFn gemm, PostFn p
         CK(post(r0, r1, ps));
         CK(ph.end(ps));
     }
-    if (panels > 1) {
+    if (overlap) {
         CK(cudaEventRecord(D().side_done, D().side));
         CK(cudaStreamWaitEvent(st, D().side_done, 0));
     }
@@ -295,13 +302,18 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
 
     Phases ph;
     if (int s = begin_call(&ph)) return s;
-    // step 2: scale factors.  The scan of B (bandwidth-bound) runs on the library's side stream beside the scan and the
-    // residues of A (which are bound by arithmetic); the residues of B wait for it.  (With the panel overlap switched off
-    // everything stays on the caller's stream, one phase after the other.)
-    if (int s = ensure_side_stream()) return s;
-    cudaStream_t sb = g.max_panels > 1 ? D().side : st;
+    // step 2: scale factors.  Everything runs on the caller's stream, one phase after the other.  (With the overlap switched
+    // on, the scan of B, bandwidth-bound, runs on the library's stream beside the scan and the residues of A, which are bound
+    // by arithmetic, and the residues of B wait for it; not for small operands, whose scan is shorter than a fork and join.)
+    const bool side_scan = g.overlap && k * n >= (1ll << 24);
+    if (side_scan) { if (int s = ensure_side_stream()) return s; }
+    cudaStream_t sb = side_scan ? D().side : st;
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
-    CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
+    const int frags_key = 1 + nmod + (eis ? 64 : 0);           // the operand of the post-processing stays in the workspace between calls
+    if (D().frags_key != frags_key) {
+        CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
+        D().frags_key = frags_key;
+    }
     if (sb != st) {
         CK(cudaEventRecord(D().panel_done[0], st));
         CK(cudaStreamWaitEvent(sb, D().panel_done[0], 0));
@@ -312,7 +324,8 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // columns of op(B) are columns of B as stored ('N') or its rows ('T', 'C')
     if (tb == 'N') CK(launch_scan_cols<T>(B, k, n, ldb, absB, sb, &g.launches[0]));
     else CK(launch_scan_rows<T>(B, n, k, ldb, absB, sb, &g.launches[0]));
-    if (!two_norm_mode) CK(launch_exponents<T>(absB, n, sc.PB, sc.ck, eB, sb, &g.launches[0]));
+    // (largest-part rule: the residue kernels form the exponents from the maxima themselves)
+    if (!two_norm_mode) {}
     else if (tb == 'N') CK(launch_exponents_2norm<T>(B, k, n, ldb, false, absB, qB, sc.PB, eB, sb, &g.launches[0]));
     else CK(launch_exponents_2norm<T>(B, n, k, ldb, true, absB, qB, sc.PB, eB, sb, &g.launches[0]));
     CK(ph.end(sb));
@@ -321,15 +334,20 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C')
     if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
     else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0]));
-    if (!two_norm_mode) CK(launch_exponents<T>(absA, m, sc.PA, sc.ck, eA, st, &g.launches[0]));     // (2-norm rule: not for k > 2^22,
+    if (!two_norm_mode) {}                                                                          // (2-norm rule: not for k > 2^22,
     else if (ta == 'N') CK(launch_exponents_2norm<T>(A, m, k, lda, true, absA, qA, sc.PA, eA, st, &g.launches[0]));   // where the sums
     else CK(launch_exponents_2norm<T>(A, k, m, lda, false, absA, qA, sc.PA, eA, st, &g.launches[0]));   // of squares would not fit 64 bits)
     CK(ph.end(st));
     // step 3 + Eq. (2a)
     CK(ph.begin(1, st));
-    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st, eis)) return s;
+    ScaleFrom fromA, fromB;
+    if (!two_norm_mode) {
+        fromA.absmax = (const unsigned long long*)absA; fromA.P = sc.PA; fromA.ck = sc.ck;
+        fromB.absmax = (const unsigned long long*)absB; fromB.P = sc.PB; fromB.ck = sc.ck;
+    }
+    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st, eis, fromA)) return s;
     if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st, eis)) return s;
+    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st, eis, fromB)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: while the tensor cores work on panel p + 1 (this stream), Eq. (2c) + steps 5-7 of
@@ -429,7 +447,10 @@ int zgemm_host(int64_t m, int64_t n, int64_t k, const double* hA, int64_t lda, c
     }
     // A: steps 2-4 as in zgemm2m
     CK(cudaMemsetAsync(ws + c.off_abs_a, 0, (size_t)(c.off_exp_a - c.off_abs_a), st));
-    CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
+    if (D().frags_key != 1 + nmod) {
+        CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
+        D().frags_key = 1 + nmod;
+    }
     CK(cudaStreamWaitEvent(st, D().a_ready, 0));
     CK(ph.begin(0, st));
     CK(launch_scan_rows<double>(dA, m, k, m, absA, st, &g.launches[0]));
@@ -537,6 +558,7 @@ int gemm2m_set_workspace(void* dev_ptr, size_t bytes) {
     select_device();
     D().ws = dev_ptr;
     D().ws_bytes = bytes;
+    D().frags_key = 0;
     if (dev_ptr) CK(cudaMemset(dev_ptr, 0, 256));   // device status word
     return GEMM2M_OK;
 }
@@ -885,6 +907,12 @@ int gemm2m_debug_set_panels(int max_panels) {
     std::lock_guard<std::mutex> lock(g.mu);
     if (max_panels < 1 || max_panels > State::kMaxPanels) return GEMM2M_ERR_ARG;
     g.max_panels = max_panels;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_set_overlap(int enabled) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    g.overlap = enabled ? 1 : 0;
     return GEMM2M_OK;
 }
 

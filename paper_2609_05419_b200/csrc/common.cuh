@@ -111,6 +111,13 @@ struct CrtTableInt {
 
 struct ScaleTargets { int Pt, PA, PB, ck; };
 
+// Where a residue kernel takes its scale exponents from: the array e (absmax == null), or the scan's per-row maxima, from
+// which it forms e = floor(log2 mu) + 1 + c_k - P itself and leaves it in e (one kernel launch less per operand).
+struct ScaleFrom {
+    const unsigned long long* absmax = nullptr;
+    int P = 0, ck = 0;
+};
+
 // Function attributes (dynamic shared memory size, cluster occupancy) belong to a device: launchers cache "done" per device.
 constexpr int kMaxDevices = 64;
 inline int current_device_slot() {
@@ -162,13 +169,13 @@ template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t row
 // Quantise + residues.  k_contiguous = false: operand row r is row r of the column-major matrix X (A: m x k);
 // true: operand row r is column r of X (B: k x n).
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
-cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches);
+cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
+                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, ScaleFrom from = ScaleFrom());
 // plane_rows: rows of a whole plane when the launch covers a row range of the operand only (X, e and planes then point at the
 // first row of the range); 0 = R.
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
-                                                     const int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches,
-                                                     int64_t plane_rows = 0);
+                                                     int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches,
+                                                     int64_t plane_rows = 0, ScaleFrom from = ScaleFrom());
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);
 // Columns [j_begin, j_end) of C only (n stays the full column count: it fixes the plane stride).

@@ -27,13 +27,19 @@ static_assert(kPfSpan % 128 == 0, "plane stride = 8 mod 32 words");
 // Words per element in the exchange buffer: 2 parts x NB chunks of 8 bytes, plus a pad that keeps the 16-byte accesses of a
 // warp on distinct banks.
 __host__ __device__ constexpr int pf_row_words(int nb) { return 4 * nb + 4; }
-__host__ __device__ constexpr int pf_block_words(int ks, int nb) { return kPfStages * 32 * ks * kPfStrideW + kPfWarps * 32 * pf_row_words(nb); }
+__host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfStages * 16 * kh * kPfStrideW + kPfWarps * 32 * pf_row_words(nb); }
 
 // D = A B, A: 16 x 32 bytes (row-major fragments), B: 32 x 8 bytes (column-major fragments), D: 16 x 8 int32; unsigned bytes.
 __device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
+}
+// The same with K = 16 (A: 16 x 16, B: 16 x 8): for operands of at most 16 planes.
+__device__ __forceinline__ void mma_u8_k16(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(b0), "r"(0));
 }
 __device__ __forceinline__ void mma_u8_acc(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -105,14 +111,16 @@ template <> __device__ __forceinline__ void store_cplx<float>(float* dst, double
 // and passes the chunks through shared memory so that lane L ends up with all chunks of element L, which it finishes and
 // stores (consecutive lanes, consecutive i).  Many warps per SM matter more here than long steps: the per-element finish is a
 // chain of dependent FP64 operations.
-template <typename T, int KS, int NB, bool AXPBY>
+// KH: 16-plane halves of K that are staged and contracted (1, 2 or 4).
+template <typename T, int KH, int NB, bool AXPBY>
 __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __restrict__ cpm, int64_t ldp, int64_t m, int64_t plane, int ncols,
                                                              const int32_t* __restrict__ eA, const int32_t* __restrict__ eB,
                                                              const uint32_t* __restrict__ frags, const __grid_constant__ PostConsts pc,
                                                              T* __restrict__ C, int64_t ldc, const PostScalars sc) {
     static_assert(NB % 2 == 0, "whole chunks per lane");
     extern __shared__ __align__(16) uint32_t pf_smem[];
-    constexpr int kStageWords = 32 * KS * kPfStrideW;
+    constexpr int KS = (KH + 1) / 2, kHalves = KH == 1 ? 1 : 2;     // K-steps of 32 planes; halves of a step in use
+    constexpr int kStageWords = 16 * KH * kPfStrideW;
     constexpr int kRow = pf_row_words(NB);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     uint32_t* xch = pf_smem + kPfStages * kStageWords + warp * 32 * kRow;
@@ -146,7 +154,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
 #pragma unroll
         for (int q = 0; q < NB; ++q) {
             bf[s][q][0] = __ldg(frags + ((s * NB + q) * 2 + 0) * 32 + lane);
-            bf[s][q][1] = __ldg(frags + ((s * NB + q) * 2 + 1) * 32 + lane);
+            bf[s][q][1] = kHalves > 1 ? __ldg(frags + ((s * NB + q) * 2 + 1) * 32 + lane) : 0u;
         }
     // High word of chunk c of this lane: 1.5 2^52 with the weight 2^(32k) of the chunk, k = (t & 1) NB/2 + c, in its exponent.
     uint32_t chunk_hi[NB / 2];
@@ -178,7 +186,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
             for (int s = 0; s < KS; ++s) {
                 uint32_t a0[4], a1[4];                      // A operands of the two 16-row tiles: elements 4g, 4g+1 / 4g+2, 4g+3
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < kHalves; ++h) {
                     const uint32_t* p = col + (32 * s + 16 * h + t) * kPfStrideW;
                     const uint32_t w0 = p[0] ^ 0x80808080u, w1 = p[4 * kPfStrideW] ^ 0x80808080u;      // residue + 128
                     const uint32_t w2 = p[8 * kPfStrideW] ^ 0x80808080u, w3 = p[12 * kPfStrideW] ^ 0x80808080u;
@@ -191,7 +199,10 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                 }
 #pragma unroll
                 for (int q = 0; q < NB; ++q) {
-                    if (s == 0) {
+                    if (KH == 1) {
+                        mma_u8_k16(acc[0][q], a0[0], a0[1], bf[s][q][0]);
+                        mma_u8_k16(acc[1][q], a1[0], a1[1], bf[s][q][0]);
+                    } else if (s == 0) {
                         mma_u8(acc[0][q], a0, bf[s][q][0], bf[s][q][1]);
                         mma_u8(acc[1][q], a1, bf[s][q][0], bf[s][q][1]);
                     } else {
@@ -284,18 +295,18 @@ cudaError_t launch_post_operands(const PostMmaTable& tab, uint32_t* dev_frags, c
     return cudaGetLastError();
 }
 
-template <typename T, int KS, int NB, bool AXPBY>
+template <typename T, int KH, int NB, bool AXPBY>
 static cudaError_t launch_post_fp_v(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
                                     const int32_t* eB, const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc,
                                     const PostScalars& sc, cudaStream_t st, int* launches) {
-    constexpr size_t smem = (size_t)pf_block_words(KS, NB) * sizeof(uint32_t);
+    constexpr size_t smem = (size_t)pf_block_words(KH, NB) * sizeof(uint32_t);
     static int resident_dev[kMaxDevices] = {};          // thread blocks the device holds at once (0 = not asked yet)
     int& resident = resident_dev[current_device_slot()];
     if (!resident) {
-        cudaError_t err = cudaFuncSetAttribute(post_fp_kernel<T, KS, NB, AXPBY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t err = cudaFuncSetAttribute(post_fp_kernel<T, KH, NB, AXPBY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         int per_sm = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, post_fp_kernel<T, KS, NB, AXPBY>, kPfThreads, smem);
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, post_fp_kernel<T, KH, NB, AXPBY>, kPfThreads, smem);
         if (err != cudaSuccess) return err;
         resident = (per_sm > 0 ? per_sm : 1) * cached_sm_count();
     }
@@ -304,7 +315,7 @@ static cudaError_t launch_post_fp_v(const int8_t* cpm, int64_t ldp, int64_t m, i
         const int64_t nj = (j_end - j0 < kColsPerLaunch) ? j_end - j0 : kColsPerLaunch;
         const int64_t steps = ((m + kPfSpan - 1) / kPfSpan) * nj;
         const unsigned grid = (unsigned)(steps < resident ? steps : resident);
-        post_fp_kernel<T, KS, NB, AXPBY><<<grid, kPfThreads, smem, st>>>(cpm + j0 * ldp, ldp, m, n * ldp, (int)nj, eA, eB + j0, dev_frags, tab.c,
+        post_fp_kernel<T, KH, NB, AXPBY><<<grid, kPfThreads, smem, st>>>(cpm + j0 * ldp, ldp, m, n * ldp, (int)nj, eA, eB + j0, dev_frags, tab.c,
                                                                         C + 2 * j0 * ldc, ldc, sc);
         ++*launches;
     }
@@ -315,10 +326,11 @@ template <typename T, bool AXPBY>
 static cudaError_t launch_post_fp_t(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, int64_t j_begin, int64_t j_end, const int32_t* eA,
                                     const int32_t* eB, const PostMmaTable& tab, const uint32_t* dev_frags, T* C, int64_t ldc,
                                     const PostScalars& sc, cudaStream_t st, int* launches) {
-#define GEMM2M_POST_CASE(KS, NB)                                                                                                     \
-    if (tab.c.ks == KS && tab.c.nb == NB)                                                                                             \
-        return launch_post_fp_v<T, KS, NB, AXPBY>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, dev_frags, C, ldc, sc, st, launches);
-    GEMM2M_POST_CASE(1, 2) GEMM2M_POST_CASE(1, 4) GEMM2M_POST_CASE(2, 4) GEMM2M_POST_CASE(2, 6)
+    const int kh = tab.c.planes <= 16 ? 1 : 2 * tab.c.ks;           // 16-plane halves of K in use
+#define GEMM2M_POST_CASE(KH, NB)                                                                                                     \
+    if (kh == KH && tab.c.nb == NB)                                                                                                   \
+        return launch_post_fp_v<T, KH, NB, AXPBY>(cpm, ldp, m, n, j_begin, j_end, eA, eB, tab, dev_frags, C, ldc, sc, st, launches);
+    GEMM2M_POST_CASE(1, 2) GEMM2M_POST_CASE(2, 4) GEMM2M_POST_CASE(4, 4) GEMM2M_POST_CASE(4, 6)
 #undef GEMM2M_POST_CASE
     return cudaErrorInvalidValue;
 }

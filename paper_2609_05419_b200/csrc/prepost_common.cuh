@@ -16,6 +16,17 @@ template <> struct FpBits<float> {
     __device__ static U mag(float v) { return (U)(__float_as_uint(v) & 0x7FFFFFFFu); }
 };
 
+// Scale exponent of a row / column from the bit pattern of its largest |Re| or |Im| (Algorithm 1 step 2):
+// e = floor(log2 mu) + 1 + c_k - P; 0 for an all-zero row; the sentinel for a row that holds an Inf or NaN.
+template <typename T>
+__device__ __forceinline__ int scale_exponent(unsigned long long absmax_bits, int P, int ck) {
+    if (absmax_bits == 0) return 0;
+    const int E = (int)(absmax_bits >> FpBits<T>::kMantBits);
+    if (E == FpBits<T>::kExpMax) return kExpNonFinite;
+    const int x = E ? E - FpBits<T>::kBias : (63 - __clzll((long long)absmax_bits)) - (FpBits<T>::kBias - 1 + FpBits<T>::kMantBits);
+    return x + 1 + ck - P;
+}
+
 template <typename T> struct Cplx { T re, im; };
 template <typename T> __device__ __forceinline__ Cplx<T> load_cplx(const T* p);
 template <> __device__ __forceinline__ Cplx<double> load_cplx<double>(const double* p) {

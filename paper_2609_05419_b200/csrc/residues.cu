@@ -1,6 +1,6 @@
 // Algorithm 1 steps 3 + 4 (Eq. 2a; Eq. 1 for the 3M moduli of the hybrid; Section 3.1 for real inputs): quantisation and
 // residue planes.  Bound by integer / FP32 arithmetic throughput rather than by HBM bandwidth.
-#include "prepost_common.cuh"
+#include "residues_common.cuh"
 
 namespace gemm2m {
 
@@ -11,23 +11,6 @@ namespace gemm2m {
 // vectors into every plane.
 // =====================================================================================================
 struct QPair { long long re, im; };   // quantised parts, two's complement
-
-// trunc(v 2^-e) for a finite v given by its bit pattern; the scaling rule guarantees |result| < 2^62 in the narrow mode.
-template <typename T>
-__device__ __forceinline__ long long quantise_part(T v, int e) {
-    using F = FpBits<T>;
-    const unsigned long long mag = F::mag(v);
-    const int E = (int)(mag >> F::kMantBits);
-    unsigned long long mant = mag & ((1ull << F::kMantBits) - 1);
-    if (E) mant |= (1ull << F::kMantBits);
-    // v = mant 2^(max(E,1) - bias - mantbits)
-    const int sh = max(E, 1) - (F::kBias + F::kMantBits) - e;
-    const bool neg = (sizeof(T) == 8) ? (__double_as_longlong((double)v) < 0) : (__float_as_int((float)v) < 0);
-    unsigned long long q;
-    if (sh >= 0) q = mant << min(sh, 63);
-    else q = (-sh > 63) ? 0ull : (mant >> (-sh));
-    return neg ? -(long long)q : (long long)q;
-}
 
 // Wide mode: |result| < 2^92 (19 or more moduli; 2^76 without the hybrid's 3M moduli); returned as the low 32 bits and the
 // signed upper 64 bits of the 96-bit two's complement value.
@@ -232,32 +215,10 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
     }
 }
 
-// ---- floating-point inputs: persistent blocks, raw elements copied asynchronously into a two-stage ring -------------
-#ifndef GEMM2M_RES_ROWS
-#define GEMM2M_RES_ROWS 8
-#endif
-constexpr int kResRows = GEMM2M_RES_ROWS, kResK = 128, kResRun = 8, kResThreads = kResRows * kResK / kResRun;
-constexpr int kResBlocksPerSm = 640 / kResThreads;   // 5 blocks of 128: up to 96 registers per thread measured faster than 6 blocks at 80
-constexpr int kResIThreads = 256;
-constexpr int kResRowStride = kResK + kResK / kResRun + 1;   // in elements: one pad per run of 8 + odd row stride -> no bank conflicts
-constexpr int kResStages = 2;
-
-template <typename T> struct RawCplx;
-template <> struct RawCplx<double> { using type = double2; };
-template <> struct RawCplx<float> { using type = float2; };
-
-template <int BYTES>
-__device__ __forceinline__ void cp_async_zfill(void* smem_dst, const void* gmem_src, bool valid) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    const int src_bytes = valid ? BYTES : 0;   // 0 source bytes: the destination is filled with zeros
-    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"(d), "l"(gmem_src), "n"(BYTES), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
+// ---- floating-point inputs: persistent blocks, raw elements copied asynchronously into a two-stage ring (residues_common.cuh)
 template <typename T, bool WIDE, int NMOD, bool HEX = false>
 __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K,
-                                                                     int64_t Kp, const int32_t* __restrict__ e,
+                                                                     int64_t Kp, int32_t* __restrict__ e, const ScaleFrom from,
                                                                      const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes,
                                                                      int64_t plane_rows) {
     using Raw = typename RawCplx<T>::type;
@@ -307,7 +268,14 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
         const int g = t & (kResK / kResRun - 1), r = t / (kResK / kResRun);
         const int64_t row = row0 + r;
         if (row < R) {
-            const int ex = __ldg(e + row);
+            // the scale exponent: given, or formed here from the scan's maximum (and left in e for the post-processing)
+            int ex;
+            if (from.absmax) {
+                ex = scale_exponent<T>(from.absmax[row], from.P, from.ck);
+                if (k0 == 0 && g == 0) e[row] = ex;
+            } else {
+                ex = e[row];
+            }
             // Narrow mode, ordinary exponents: x 2^-e is an exact FP64 product (or underflows towards zero, where the
             // truncation is zero anyway) and its truncation to int64 is one conversion; |x 2^-e| < 2^62 by the scaling rule.
             const bool fast = !WIDE && ex > -1000 && ex < 1000;
@@ -364,8 +332,9 @@ constexpr size_t kResSmemBytes(size_t elem) { return (size_t)kResStages * kResRo
 
 
 template <typename T>
-cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, int64_t plane_rows) {
+cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
+                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, int64_t plane_rows,
+                               ScaleFrom from) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
     static bool attr_set_dev[kMaxDevices] = {};
@@ -387,20 +356,20 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
     // saves two instructions per (element, modulus) -- 13 % of the kernel's time at 16 moduli.
     const int spec = (!wide && tab.n2 == tab.nmod) ? tab.nmod : 0;
     switch (spec) {
-#define GEMM2M_RES_CASE(N) case N: residues_fp_kernel<T, false, N><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R); break;
+#define GEMM2M_RES_CASE(N) case N: residues_fp_kernel<T, false, N><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R); break;
         GEMM2M_RES_CASE(7) GEMM2M_RES_CASE(8) GEMM2M_RES_CASE(14) GEMM2M_RES_CASE(15) GEMM2M_RES_CASE(16)
 #undef GEMM2M_RES_CASE
         default:
-            if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
-            else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
+            if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+            else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
     }
     ++*launches;
     return cudaGetLastError();
 }
 
 // Eisenstein variant: the same kernel with the lattice rounding in front (complex double operands, 96-bit coordinates).
-cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, const int32_t* e,
-                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches) {
+cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
+                                const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, ScaleFrom from) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
     constexpr int64_t plane_rows = 0;
     constexpr size_t smem = kResSmemBytes(2 * sizeof(double));
@@ -416,9 +385,9 @@ cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, 
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
     const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
-    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
-    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
-    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, planes, plane_rows ? plane_rows : R);
+    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
     ++*launches;
     return cudaGetLastError();
 }
@@ -599,7 +568,7 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
     return cudaGetLastError();
 }
 
-template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t);
-template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, const int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t);
+template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
+template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
 
 }  // namespace gemm2m

@@ -56,20 +56,7 @@ template <typename T>
 __global__ void exponents_kernel(const unsigned long long* __restrict__ absmax, int64_t count, int P, int ck, int32_t* __restrict__ e) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= count) return;
-    const unsigned long long b = absmax[i];
-    int out;
-    if (b == 0) {
-        out = 0;
-    } else {
-        const int E = (int)(b >> FpBits<T>::kMantBits);
-        if (E == FpBits<T>::kExpMax) {
-            out = kExpNonFinite;
-        } else {
-            const int x = E ? E - FpBits<T>::kBias : (63 - __clzll((long long)b)) - (FpBits<T>::kBias - 1 + FpBits<T>::kMantBits);
-            out = x + 1 + ck - P;
-        }
-    }
-    e[i] = out;
+    e[i] = scale_exponent<T>(absmax[i], P, ck);
 }
 
 // ---- real matrices (real Ozaki-II scheme, Section 3.1): the same scans over scalar elements ----------------

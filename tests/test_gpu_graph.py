@@ -12,10 +12,19 @@ pytestmark = pytest.mark.gpu
 from gpu_util import Workspace, empty_dev, to_dev, to_host  # noqa: E402
 
 
-def test_zgemm2m_replays_from_a_cuda_graph_bit_for_bit():
-    m, n, k, nmod = 300, 2304, 256, 16                     # 2304 columns: two panels, so the side stream is part of the capture
+@pytest.mark.parametrize("overlap", [False, True], ids=["in-order", "overlap"])
+def test_zgemm2m_replays_from_a_cuda_graph_bit_for_bit(overlap):
+    m, n, k, nmod = 300, 2304, 256, 16                     # 2304 columns: two panels; with the overlap on, the library's stream is part of the capture
     A, B = inputs.complex_inputs(m, n, k, seed=71)
     A2, B2 = inputs.complex_inputs(m, n, k, seed=72)
+    b.debug_set_overlap(overlap)
+    try:
+        _replay_case(m, n, k, nmod, A, B, A2, B2)
+    finally:
+        b.debug_set_overlap(False)
+
+
+def _replay_case(m, n, k, nmod, A, B, A2, B2):
     with Workspace(b.workspace_bytes(b.OP_ZGEMM, m, n, k, nmod)):
         dA, dB = to_dev(A), to_dev(B)
         C_direct = empty_dev(m, n, torch.complex128)
