@@ -215,6 +215,9 @@ int run_gemm(const GemmArgs& a, int64_t klim, cudaStream_t st) {
 // call is complete on the caller's stream only when the library's stream has been joined back.  Measured with whole calls of
 // the two modes alternating in one loop, the overlap gains 0.4 % at 8192^3 and loses 0.8 % for cgemm2m at 16384 x 16384 x
 // 4096: the GEMM phase runs at the board's power limit, and what runs beside it slows it down by what it hides.
+// (Panel count at 8192 columns, 30 back-to-back calls each: 1 panel 17.4-17.7 ms, 2 panels 17.2-17.4, 4 panels 15.7-16.3,
+// 8 panels 16.5-16.7: fewer launches would read the planes of A less often, but the short post-processing launches between the
+// GEMM launches let the power-limited clock recover, which is worth more.)
 template <typename GemmFn, typename PostFn>
 int panel_pipeline(int64_t n, cudaStream_t st, Phases& ph, GemmFn gemm, PostFn post) {
     int panels = (int)(n / 1024);
