@@ -296,14 +296,15 @@ int gemm2m_debug_tables(int nmod, int64_t k, int herk, int* scale, double* crt_g
 int gemm2m_debug_tables_real(int nmod, int64_t k, int* moduli, int* scale, double* crt_g, double* crt_m, int* nchunks, int32_t* y0_bits, float* cq,
                              float* inv_m, int32_t* xmax, double* margin);
 int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float* inv_m, int32_t* xmax, double* margin);
-/* Operand of the tensor-core contraction in the post-processing of the complex GEMMs (tests only; host pointers, any may be
- * NULL; eisenstein != 0 selects the Eisenstein set).  Eq. (2c) (Eq. (1) for a 3M modulus) and the CRT of Section 3.1 are folded
+/* Operand of the tensor-core contraction in the post-processing (tests only; host pointers, any may be NULL; variant 0 = the
+ * complex GEMMs, 1 = the Eisenstein set, 2 = the rank-k family, whose planes are the C+ planes read directly, in K slots
+ * 0 .. nmod-1, and mirrored, in slots H .. H+nmod-1 with H = nmod rounded up to 16).  Eq. (2c) (Eq. (1) for a 3M modulus) and the CRT of Section 3.1 are folded
  * into one weight per residue plane and part (real, imaginary), reduced to [0, M) and written in bytes:
  *   dims[3]   = residue planes, K-steps of 32 planes, chunks of four bytes (nb)
  *   digits    = [2][planes][24] bytes, least significant first: weight of the plane in the real / imaginary part
  *   consts[19]= M in base 2^32 (6 numbers, each times its power of 2^32; lower digits balanced), then per part the 6 numbers
  *               (1.5 2^52 + digit k of 128 x the sum of the part's weights) 2^(32k), then 1/M. */
-int gemm2m_debug_post_operands(int eisenstein, int nmod, uint8_t* digits, int* dims, double* consts);
+int gemm2m_debug_post_operands(int variant, int nmod, uint8_t* digits, int* dims, double* consts);
 /* The same for the Eisenstein set (tests only): scale[4], crt_gr / crt_gi[nmod*5] = digits of sym(4^-1 q_j)(M/m_j) and of
  * sym(-(4 d_j)^-1 q_j)(M/m_j), crt_m[5], nchunks, and the reduction constants. */
 int gemm2m_debug_tables_eisenstein(int nmod, int64_t k, int* scale, double* crt_gr, double* crt_gi, double* crt_m, int* nchunks,

@@ -378,15 +378,16 @@ def debug_tables(nmod, k, herk=False):
                 nchunks=int(nch[0]), res_w=w)
 
 
-def debug_post_operands(nmod, eisenstein=False):
-    """Operand of the post-processing contraction of the complex GEMMs (see gemm2m_debug_post_operands)."""
+def debug_post_operands(nmod, eisenstein=False, herk=False):
+    """Operand of the post-processing contraction (see gemm2m_debug_post_operands)."""
     import numpy as np
     dims = np.zeros(3, dtype=np.int32)
     consts = np.zeros(19, dtype=np.float64)
     ptr = lambda a: ctypes.c_void_p(a.ctypes.data)
-    _check(lib().gemm2m_debug_post_operands(1 if eisenstein else 0, nmod, None, ptr(dims), None), "gemm2m_debug_post_operands")
+    variant = 2 if herk else 1 if eisenstein else 0
+    _check(lib().gemm2m_debug_post_operands(variant, nmod, None, ptr(dims), None), "gemm2m_debug_post_operands")
     digits = np.zeros((2, int(dims[0]), 24), dtype=np.uint8)
-    _check(lib().gemm2m_debug_post_operands(1 if eisenstein else 0, nmod, ptr(digits), ptr(dims), ptr(consts)), "gemm2m_debug_post_operands")
+    _check(lib().gemm2m_debug_post_operands(variant, nmod, ptr(digits), ptr(dims), ptr(consts)), "gemm2m_debug_post_operands")
     return dict(planes=int(dims[0]), ks=int(dims[1]), nb=int(dims[2]), digits=digits, Mc=consts[0:6], off=consts[6:18].reshape(2, 6),
                 inv_M=float(consts[18]))
 

@@ -7,8 +7,8 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["api.cu", "tables.cu", "scan.cu", "residues.cu", "post.cu", "post_fp.cu", "gemm_check.cu", "gemm_i8_2cta.cu", "static_scratch.cu"]
-HEADERS = ["common.cuh", "gemm_ptx.cuh", "prepost_common.cuh", "residues_common.cuh", "post_common.cuh", os.path.join("..", "..", "include", "gemm2m.h")]
+SOURCES = ["api.cu", "tables.cu", "scan.cu", "residues.cu", "post.cu", "post_fp.cu", "post_herk.cu", "gemm_check.cu", "gemm_i8_2cta.cu", "static_scratch.cu"]
+HEADERS = ["common.cuh", "gemm_ptx.cuh", "prepost_common.cuh", "residues_common.cuh", "post_common.cuh", "post_mma.cuh", os.path.join("..", "..", "include", "gemm2m.h")]
 LIB = os.path.join(HERE, "libgemm2m.so")
 
 

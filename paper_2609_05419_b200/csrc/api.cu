@@ -684,10 +684,15 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
     const bool wide = sc.PA - sc.ck > 62;
     ResidueTable rtab;
     build_residue_table(nmod, &rtab);
-    CrtTable ctab;
-    build_crt_table(nmod, &ctab);
+    PostMmaTable ptab;
+    build_post_mma_table_herk(nmod, &ptab);
+    uint32_t* frags = (uint32_t*)(ws + c.off_frags);
     Phases ph;
     if (int s = begin_call(&ph)) return s;
+    if (D().frags_key != 128 + nmod) {                       // the operand of the post-processing stays in the workspace between calls
+        CK(launch_post_operands(ptab, frags, st, &g.launches[3]));
+        D().frags_key = 128 + nmod;
+    }
     CK(ph.begin(0, st));
     const double* ZA = A;
     const double* ZB = B;
@@ -744,7 +749,7 @@ static int rank_update(int op, int64_t n, int64_t k, const double* A, int64_t ld
                 return (int)GEMM2M_OK;
             },
             [&](int64_t r0, int64_t r1, cudaStream_t ps) {
-                return launch_post_herk(cp, c.ldp, n, r0, r1, eA, ctab, C, ldc, real_in, ps, &g.launches[3]);
+                return launch_post_herk(cp, c.ldp, n, r0, r1, eA, ptab, frags, C, ldc, real_in, ps, &g.launches[3]);
             })) return s;
     ph.done();
     return GEMM2M_OK;
@@ -996,10 +1001,11 @@ int gemm2m_debug_residue_reduction(int nmod, int32_t* y0_bits, float* cq, float*
     return GEMM2M_OK;
 }
 
-int gemm2m_debug_post_operands(int eisenstein, int nmod, uint8_t* digits, int* dims, double* consts) {
-    if (nmod < 1 || nmod > (eisenstein ? kMaxEis : kMaxMod)) return GEMM2M_ERR_ARG;
+int gemm2m_debug_post_operands(int variant, int nmod, uint8_t* digits, int* dims, double* consts) {
+    if (variant < 0 || variant > 2 || nmod < 1 || nmod > (variant == 1 ? kMaxEis : variant == 2 ? kMax2M : kMaxMod)) return GEMM2M_ERR_ARG;
     PostMmaTable t;
-    if (eisenstein) build_post_mma_table_eis(nmod, &t);
+    if (variant == 1) build_post_mma_table_eis(nmod, &t);
+    else if (variant == 2) build_post_mma_table_herk(nmod, &t);
     else build_post_mma_table(nmod, &t);
     if (dims) { dims[0] = t.c.planes; dims[1] = t.c.ks; dims[2] = t.c.nb; }
     if (digits)

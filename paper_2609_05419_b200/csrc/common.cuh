@@ -96,8 +96,9 @@ struct PostConsts {
 };
 struct PostMmaTable {
     PostConsts c;
+    int nmod;                                  // moduli the table was built for
     uint32_t bfrag[kPostFragWords];            // host copy; launch_post_operands writes it to device memory
-    uint8_t digit[2][kMaxPlanes][4 * kPostMaxNB];  // [part][plane][p]: the digits themselves (host side; for tests)
+    uint8_t digit[2][32 * kPostMaxKS][4 * kPostMaxNB];   // [part][plane (K slot)][p]: the digits themselves (host side; for tests)
 };
 
 // CRT constants for the exact int64 result (nmod <= 8, M < 2^62).
@@ -137,6 +138,9 @@ void build_crt_table(int nmod, CrtTable* t);
 void build_crt_table_int(int nmod, CrtTableInt* t);
 void build_post_mma_table(int nmod, PostMmaTable* t);
 void build_post_mma_table_eis(int nmod, PostMmaTable* t);
+// Rank-k family (Section 5): the planes are the C+ planes read directly (K slots 0 .. nmod-1) and read mirrored, as C- = C+^T
+// (K slots H .. H + nmod - 1 with H = nmod rounded up to 16, so that every 16-slot half of K holds planes of one kind).
+void build_post_mma_table_herk(int nmod, PostMmaTable* t);
 ScaleTargets scale_targets(int nmod, int64_t k, bool herk);
 // The same for the real Ozaki-II scheme (dgemm_ozaki2): moduli 256, 255, 253, ..., one residue plane per modulus.
 int real_modulus_value(int j);
@@ -195,8 +199,8 @@ cudaError_t launch_post_real(const int8_t* cp, int64_t ldp, int64_t m, int64_t n
 template <typename T> cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double* beta, cudaStream_t st, int* launches);
 // real_out: C is a real matrix (SYRK / SYR2K through Z = A1 + i A2): only the real part is formed and stored.
 // Rows [i_begin, i_end) of the lower triangle only (i_begin a multiple of 64): they need the GEMM output rows below i_end.
-cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const CrtTable& tab,
-                             double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches);
+cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const PostMmaTable& tab,
+                             const uint32_t* dev_frags, double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches);
 // Z[i, p] = X[i, p] + i X[i, p + k2] for p < k2 = ceil(k / 2) (zero beyond column k): the complex matrix whose HERK is the SYRK of X.
 cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_t k, double* Z, cudaStream_t st, int* launches);
 cudaError_t launch_post_int(const int8_t* cpm, int64_t ldp, int64_t m, int64_t n, const CrtTableInt& tab, int64_t* Cr, int64_t* Ci,

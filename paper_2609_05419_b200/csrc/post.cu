@@ -160,90 +160,6 @@ cudaError_t launch_scale_c(T* C, int64_t m, int64_t n, int64_t ldc, const double
 template cudaError_t launch_scale_c<double>(double*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
 template cudaError_t launch_scale_c<float>(float*, int64_t, int64_t, int64_t, const double*, cudaStream_t, int*);
 
-// HERK (Section 5): only C+ = A+ A-^T was computed; C- = C+^T.  cp: [nmod][n][ldp] with cp[j][col][row] = C+_j[row, col].
-// A block handles 64 rows i x 16 columns j of the lower triangle.  It needs C+[i, j] (rows of cp along i: 16 runs of 64
-// bytes per modulus) and C-[i, j] = C+[j, i] (rows of cp along j: 64 runs of 16 bytes per modulus); both are pulled into
-// shared memory with asynchronous 16-byte copies, then each thread combines 4 consecutive i of one column.
-// Lower triangle only; on the diagonal C- - C+ = 0, so the imaginary part is exactly zero.
-constexpr int kHerkI = 64, kHerkJ = 16, kHerkThreads = 256;
-constexpr int kHerkMirrorSlots = kHerkI + kHerkI / 8;                      // 16-byte slots, one pad slot per 8 rows (bank spread)
-constexpr int kHerkPlaneBytes = kHerkJ * kHerkI + kHerkMirrorSlots * 16;   // direct + mirrored bytes per modulus
-
-template <int NCH, bool REAL_OUT>
-__global__ void __launch_bounds__(kHerkThreads) post_herk_kernel(const int8_t* __restrict__ cp, int64_t ldp, int64_t n, int64_t i_begin,
-                                                                 const int32_t* __restrict__ eA, const __grid_constant__ CrtTable tab,
-                                                                 double* __restrict__ C, int64_t ldc) {
-    extern __shared__ __align__(16) unsigned char herk_smem[];
-    const int64_t ibase = i_begin + (int64_t)blockIdx.x * kHerkI, jbase = (int64_t)blockIdx.y * kHerkJ;
-    if (ibase + kHerkI - 1 < jbase) return;                                // tile entirely above the diagonal
-    const int nmod = tab.nmod;
-    const int64_t plane = n * ldp;
-    const int t = threadIdx.x;
-    // direct part: for each modulus and each column j of the tile, 64 bytes along i (4 copies of 16 bytes)
-    for (int idx = t; idx < nmod * kHerkJ * (kHerkI / 16); idx += kHerkThreads) {
-        const int v = idx & 3, jj = (idx >> 2) & (kHerkJ - 1), jm = idx / (kHerkJ * 4);
-        const int64_t i = ibase + 16 * v, j = jbase + jj;
-        if (j < n && i < ldp) cp_async16(herk_smem + jm * kHerkPlaneBytes + jj * kHerkI + 16 * v, cp + (int64_t)jm * plane + j * ldp + i);
-    }
-    // mirrored part: for each modulus and each row i of the tile, the 16 bytes C+[jbase .. jbase+15, i]
-    for (int idx = t; idx < nmod * kHerkI; idx += kHerkThreads) {
-        const int ii = idx & (kHerkI - 1), jm = idx / kHerkI;
-        const int64_t i = ibase + ii;
-        if (i < n && jbase < ldp)
-            cp_async16(herk_smem + jm * kHerkPlaneBytes + kHerkJ * kHerkI + (ii + (ii >> 3)) * 16, cp + (int64_t)jm * plane + i * ldp + jbase);
-    }
-    cp_async_wait_all();
-    __syncthreads();
-    const int g = t & 15, jj = t >> 4;                                     // 4 consecutive rows i0 .. i0+3 of column j
-    const int64_t i0 = ibase + 4 * g, j = jbase + jj;
-    if (j >= n || i0 >= n || i0 + 3 < j) return;
-    double Sr[4][NCH], Si[4][NCH];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) Sr[e][c] = Si[e][c] = 0.0;
-    }
-#pragma unroll 2
-    for (int jm = 0; jm < nmod; ++jm) {
-        const unsigned char* base = herk_smem + jm * kHerkPlaneBytes;
-        const uint32_t wp = *reinterpret_cast<const uint32_t*>(base + jj * kHerkI + 4 * g);      // C+[i0..i0+3, j]
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int ii = 4 * g + e;
-            const int cpv = sbyte(wp, e);
-            const int cmv = (int)(int8_t)base[kHerkJ * kHerkI + (ii + (ii >> 3)) * 16 + jj];    // C-[i, j] = C+[j, i]
-            const double vr = int_to_double(cmv + cpv), vi = int_to_double(cmv - cpv);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                Sr[e][c] = fma(vr, tab.gr[jm][c], Sr[e][c]);
-                if (!REAL_OUT) Si[e][c] = fma(vi, tab.gi[jm][c], Si[e][c]);
-            }
-        }
-    }
-    const int ej = __ldg(eA + j);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int64_t i = i0 + e;
-        if (i < n && i >= j) {
-            const int ei = __ldg(eA + i);
-            double re, im = 0.0;
-            if (ei == kExpNonFinite || ej == kExpNonFinite) {
-                re = im = __longlong_as_double(0x7FF8000000000000ll);
-            } else {
-                double h, l;
-                crt_finish<NCH>(Sr[e], tab, &h, &l);
-                re = scale_pow2(h + l, ei + ej);
-                if (!REAL_OUT) {
-                    crt_finish<NCH>(Si[e], tab, &h, &l);
-                    im = scale_pow2(h + l, ei + ej);
-                }
-            }
-            if (REAL_OUT) C[i + j * ldc] = re;
-            else *reinterpret_cast<double2*>(C + 2 * (i + j * ldc)) = make_double2(re, im);
-        }
-    }
-}
-
 __global__ void __launch_bounds__(256) pack_real_pair_kernel(const double* __restrict__ X, int64_t ld, int64_t n, int64_t k, int64_t k2,
                                                              double* __restrict__ Z) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -264,41 +180,6 @@ cudaError_t launch_pack_real_pair(const double* X, int64_t ld, int64_t n, int64_
         ++*launches;
     }
     return cudaGetLastError();
-}
-
-template <bool REAL_OUT>
-static cudaError_t launch_post_herk_t(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA,
-                                      const CrtTable& tab, double* C, int64_t ldc, cudaStream_t st, int* launches) {
-    const size_t smem = (size_t)kMaxMod * kHerkPlaneBytes;
-    static bool attr_set_dev[kMaxDevices] = {};
-    bool& attr_set = attr_set_dev[current_device_slot()];
-    if (!attr_set) {
-        cudaError_t err = cudaFuncSetAttribute(post_herk_kernel<1, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<2, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<3, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err == cudaSuccess) err = cudaFuncSetAttribute(post_herk_kernel<4, REAL_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return err;
-        attr_set = true;
-    }
-    const size_t use = (size_t)tab.nmod * kHerkPlaneBytes;
-    const int64_t tiles_j = (i_end + kHerkJ - 1) / kHerkJ;  // lower triangle: columns up to the last row of the range
-    if (tiles_j > 65535) return cudaErrorInvalidValue;     // n beyond 65535 * 16 columns: far beyond any workspace
-    dim3 grid((unsigned)((i_end - i_begin + kHerkI - 1) / kHerkI), (unsigned)tiles_j);
-    switch (tab.nchunks) {
-        case 1: post_herk_kernel<1, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
-        case 2: post_herk_kernel<2, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
-        case 3: post_herk_kernel<3, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
-        default: post_herk_kernel<4, REAL_OUT><<<grid, kHerkThreads, use, st>>>(cp, ldp, n, i_begin, eA, tab, C, ldc); break;
-    }
-    ++*launches;
-    return cudaGetLastError();
-}
-
-cudaError_t launch_post_herk(const int8_t* cp, int64_t ldp, int64_t n, int64_t i_begin, int64_t i_end, const int32_t* eA, const CrtTable& tab,
-                             double* C, int64_t ldc, bool real_out, cudaStream_t st, int* launches) {
-    if (n <= 0 || i_end <= i_begin) return cudaSuccess;
-    return real_out ? launch_post_herk_t<true>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches)
-                    : launch_post_herk_t<false>(cp, ldp, n, i_begin, i_end, eA, tab, C, ldc, st, launches);
 }
 
 // Exact integer variant for gemm2m_gaussian_int: X = sum_j sym(v_j g_j mod m_j) (M/m_j) mod M in int64 (M < 2^62).

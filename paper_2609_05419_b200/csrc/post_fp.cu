@@ -6,7 +6,7 @@
 // sum is non-negative, at most 56 . 255 . 255 < 2^22).  What is left per element is to add the digit columns up (integer, then
 // FP64 on 32-bit-spaced chunks), remove the multiple of M, round once and scale by 2^(e_i + f_j).
 // Bound by HBM traffic: 1 byte per plane read, 16 (8) bytes written per element.
-#include "post_common.cuh"
+#include "post_mma.cuh"
 
 namespace gemm2m {
 
@@ -24,82 +24,7 @@ constexpr int kPfStrideW = kPfSpan / 4 + 8;     // words per staged plane: + 8, 
 constexpr int kPfStages = 2;                    // staging ring: the next step is on its way while this one is processed
 static_assert(kPfSpan % 128 == 0, "plane stride = 8 mod 32 words");
 
-// Words per element in the exchange buffer: 2 parts x NB chunks of 8 bytes, plus a pad that keeps the 16-byte accesses of a
-// warp on distinct banks.
-__host__ __device__ constexpr int pf_row_words(int nb) { return 4 * nb + 4; }
 __host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfStages * 16 * kh * kPfStrideW + kPfWarps * 32 * pf_row_words(nb); }
-
-// D = A B, A: 16 x 32 bytes (row-major fragments), B: 32 x 8 bytes (column-major fragments), D: 16 x 8 int32; unsigned bytes.
-__device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
-}
-// The same with K = 16 (A: 16 x 16, B: 16 x 8): for operands of at most 16 planes.
-__device__ __forceinline__ void mma_u8_k16(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-    asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
-        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-        : "r"(a0), "r"(a1), "r"(b0), "r"(0));
-}
-__device__ __forceinline__ void mma_u8_acc(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// hi:lo = b 2^16 + (hi_word 2^32 + a): four digit-column sums s0..s3 packed as a = s0 + 2^8 s1, b = s2 + 2^8 s3 (both below
-// 2^31) under the high word of a double, one wide multiply-add.
-// (two16 holds 65536 in a register: with the constant in the instruction the compiler splits the product into a shift pair.)
-__device__ __forceinline__ unsigned long long pack_chunk(uint32_t a, uint32_t b, uint32_t hi_word, uint32_t two16) {
-    unsigned long long r;
-    asm("{\n\t.reg .b64 c;\n\tmov.b64 c, {%1, %2};\n\tmad.wide.u32 %0, %3, %4, c;\n\t}" : "=l"(r) : "r"(a), "r"(hi_word), "r"(b), "r"(two16));
-    return r;
-}
-
-// Lifted X (exact integer, |X| <= M/2) of one part from its NB chunks, returned as an unevaluated sum hi + lo with
-// |lo| <= ulp(hi)/2.  Chunk k arrives as the bit pattern of the double (1.5 2^52 + V_k) 2^(32k), with
-// V_k = s_4k + 2^8 s_(4k+1) + 2^16 s_(4k+2) + 2^24 s_(4k+3) < 2^46.1 the four digit-column sums it covers; off[k] takes the
-// conversion offset and the chunk's share of 128 sum_planes W_p off again, exactly, which leaves W_k with
-// X' = sum_k W_k 2^(32k) = sum_planes residue_p W_p = X + t M.
-// t = rint(X'/M) from the three leading chunks: M >= 2^(32 NB - 64) (its bytes fill more than NB - 2 chunks), so the
-// rest is below 2^-17 M; |t| < 2^14, and |X/M| stays away from 1/2 by the scaling rule.  W_k - t Mc_k is exact
-// (|t Mc_k| < 2^46 before the weight).  The chunks are then added with error-free transformations, neighbours first, so
-// hi + lo equals X to 2^-105 relative.
-template <int NB>
-__device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const double (&off)[kPostMaxNB], const PostConsts& pc, double* hi, double* lo) {
-    double W[NB];
-#pragma unroll
-    for (int k = 0; k < NB; ++k) W[k] = bits[k] - off[k];
-    double lead = W[NB - 1];
-#pragma unroll
-    for (int k = NB - 2; k >= 0 && k >= NB - 3; --k) lead += W[k];
-    const double t = rint(lead * pc.inv_M);
-#pragma unroll
-    for (int k = 0; k < NB; ++k) W[k] = fma(-t, pc.Mc[k], W[k]);
-    double ph[NB / 2], l = 0.0;
-#pragma unroll
-    for (int k = 0; k < NB / 2; ++k) {
-        const double a = W[2 * k + 1], b = W[2 * k];
-        const double s = a + b;                                              // TwoSum
-        const double bb = s - a;
-        l += (a - (s - bb)) + (b - bb);
-        ph[k] = s;
-    }
-    double h = ph[NB / 2 - 1];
-#pragma unroll
-    for (int k = NB / 2 - 2; k >= 0; --k) {
-        const double s = h + ph[k];
-        const double bb = s - h;
-        l += (h - (s - bb)) + (ph[k] - bb);
-        h = s;
-    }
-    *hi = h;
-    *lo = l;
-}
-
-template <typename T> __device__ __forceinline__ void store_cplx(T* dst, double re, double im);
-template <> __device__ __forceinline__ void store_cplx<double>(double* dst, double re, double im) { *reinterpret_cast<double2*>(dst) = make_double2(re, im); }
-template <> __device__ __forceinline__ void store_cplx<float>(float* dst, double re, double im) { *reinterpret_cast<float2*>(dst) = make_float2((float)re, (float)im); }
 
 // cpm: [planes][n][ldp] int8 (row index i contiguous); plane = n ldp is the plane stride; ncols columns starting at the
 // pointers given.  The work is cut into steps of kPfSpan consecutive i of one column j, numbered column by column within a

@@ -325,9 +325,12 @@ void build_crt_table_real(int nmod, CrtTable* t) {
     memoised<CrtTable, kMaxReal>(nmod, t, [&](CrtTable* c) { build_crt_table_for(kRealModuli, nmod, 0, c); });
 }
 
-static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaTable* t) {
+// herk: the plane order of the rank-k family (see build_post_mma_table_herk).
+static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaTable* t, bool herk = false) {
     std::memset(t, 0, sizeof(*t));
-    const int n3 = nmod - n2, planes = 2 * n2 + 3 * n3;
+    const int n3 = nmod - n2, herk_half = 16 * ((n2 + 15) / 16);
+    const int planes = herk ? 2 * herk_half : 2 * n2 + 3 * n3;
+    auto slot = [&](int plane) { return herk && plane >= n2 ? herk_half + (plane - n2) : plane; };
     const Big M = product_of(nmod, mods);
     const int ndig = (M.bit_length() + 7) / 8;                        // bytes of a residue modulo M
     if (ndig > 4 * kPostMaxNB) std::abort();                          // cannot happen: M < 2^185
@@ -338,7 +341,7 @@ static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaT
         G.mul_small((uint32_t)std::abs(coef));                        // below M/2: |coef| <= m_j / 2
         if (coef < 0) { Big R = M; R.sub(G); G = R; }
         ksum[part].add(G);
-        for (int p = 0; p < ndig; ++p) t->digit[part][plane][p] = (uint8_t)G.bits(8 * p, 8);
+        for (int p = 0; p < ndig; ++p) t->digit[part][slot(plane)][p] = (uint8_t)G.bits(8 * p, 8);
     };
     for (int j = 0; j < nmod; ++j) {
         Big W;
@@ -359,6 +362,7 @@ static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaT
         }
     }
     PostConsts& c = t->c;
+    t->nmod = nmod;
     c.planes = planes;
     c.ks = (planes + 31) / 32;
     c.nb = 2 * ((ndig + 7) / 8);           // 32-bit chunks (4 digits each), an even number of them: a lane of the kernel holds whole chunks
@@ -407,6 +411,12 @@ static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaT
 
 void build_post_mma_table(int nmod, PostMmaTable* t) {
     memoised<PostMmaTable, kMaxMod>(nmod, t, [&](PostMmaTable* c) { build_post_mma_table_for(kModuli, nmod, count_2m(nmod), c); });
+}
+void build_post_mma_table_herk(int nmod, PostMmaTable* t) {
+    static PostMmaTable cache[kMax2M + 1];
+    static std::once_flag once[kMax2M + 1];
+    std::call_once(once[nmod], [&] { build_post_mma_table_for(kModuli, nmod, nmod, &cache[nmod], true); });
+    *t = cache[nmod];
 }
 void build_post_mma_table_eis(int nmod, PostMmaTable* t) {
     memoised<PostMmaTable, kMaxEis>(nmod, t, [&](PostMmaTable* c) {

@@ -395,3 +395,27 @@ def test_post_operands_of_the_eisenstein_variant(nmod):
         return plus + minus
 
     _post_operand_checks(t, mods, M, plane_values, lambda c: state["want"], 100 + nmod)
+
+
+@pytest.mark.parametrize("nmod", [1, 7, 16, 17, 22])
+def test_post_operands_of_the_rank_k_family(nmod):
+    # Section 5: C- = C+^T, so the kernel reads the C+ planes twice; K slots 0 .. nmod-1 hold c+ = C+[i, j], slots H .. H+nmod-1
+    # (H = nmod rounded up to 16) hold c- = C+[j, i]; the padding slots carry zero weights.
+    mods = staged.greedy_2m_moduli()[:nmod]
+    roots = [staged.sqrt_minus_one(q) for q in mods]
+    M = staged.product(mods)
+    H = 16 * ((nmod + 15) // 16)
+    t = b.debug_post_operands(nmod, herk=True)
+    assert t["planes"] == 2 * H and t["ks"] == H // 16
+    assert (t["digits"][:, nmod:H] == 0).all() and (t["digits"][:, H + nmod:] == 0).all()
+
+    def plane_values(rng, trial):
+        pick = (lambda m: (m - 1) // 2) if trial == 0 else (lambda m: -(m // 2)) if trial == 1 else (lambda m: int(rng.integers(-(m // 2), (m - 1) // 2 + 1)))
+        pad = [int(rng.integers(-128, 128)) for _ in range(H - nmod)]              # whatever the padding slots hold must not matter
+        return [pick(m) for m in mods] + pad + [pick(m) for m in mods] + pad
+
+    def expected(c):
+        post = [staged.post_2m(c[j], c[H + j], mods[j], roots[j]) for j in range(nmod)]
+        return staged.crt([r for r, _ in post], mods), staged.crt([i for _, i in post], mods)
+
+    _post_operand_checks(t, mods, M, plane_values, expected, 200 + nmod)
