@@ -22,9 +22,13 @@ constexpr int kPfThreads = 32 * kPfWarps;
 constexpr int kPfSpan = 32 * kPfGroups * kPfWarps;      // consecutive row indices i per step of a block
 constexpr int kPfStrideW = kPfSpan / 4 + 8;     // words per staged plane: + 8, so that the 32 fragment loads of a warp hit 32 banks
 constexpr int kPfStages = 2;                    // staging ring: the next step is on its way while this one is processed
+constexpr int kPfIlp = 1;                       // groups of a warp whose elements are finished together (one exchange buffer each);
+                                                // 2 and 4 measured 5 and 15 % slower at 8192^3: fewer blocks fit, and the compiler
+                                                // does not interleave the finishes anyway
+static_assert(kPfGroups % kPfIlp == 0, "whole batches of groups");
 static_assert(kPfSpan % 128 == 0, "plane stride = 8 mod 32 words");
 
-__host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfStages * 16 * kh * kPfStrideW + kPfWarps * 32 * pf_row_words(nb); }
+__host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfStages * 16 * kh * kPfStrideW + kPfWarps * kPfIlp * 32 * pf_row_words(nb); }
 
 // cpm: [planes][n][ldp] int8 (row index i contiguous); plane = n ldp is the plane stride; ncols columns starting at the
 // pointers given.  The work is cut into steps of kPfSpan consecutive i of one column j, numbered column by column within a
@@ -48,7 +52,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
     constexpr int kStageWords = 16 * KH * kPfStrideW;
     constexpr int kRow = pf_row_words(NB);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    uint32_t* xch = pf_smem + kPfStages * kStageWords + warp * 32 * kRow;
+    uint32_t* xch = pf_smem + kPfStages * kStageWords + warp * kPfIlp * 32 * kRow;
     const int64_t total = ((m + kPfSpan - 1) / kPfSpan) * ncols;
     int64_t step = total * blockIdx.x / gridDim.x;
     const int64_t step_end = total * (blockIdx.x + 1) / gridDim.x;
@@ -103,8 +107,10 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
             ea_block = ibk;
         }
         const int fb = __ldg(eB + j);
-#pragma unroll
-        for (int it = 0; it < kPfGroups; ++it) {
+        T* dst0 = C + 2 * (ib + lane + (int64_t)j * ldc);     // this lane's element of the warp's first group
+        const int64_t rows_left = m - ib - lane;               // group `it` is inside the matrix for this lane if 32 it < rows_left
+        // MMA phase of group `it`: operand gather, contraction, chunks into the exchange buffer xb
+        auto contract = [&](int it, uint32_t* xb) {
             int acc[2][NB][4];
             const uint32_t* col = st + 8 * (kPfGroups * warp + it) + g;
 #pragma unroll
@@ -137,7 +143,6 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                 }
             }
             // accumulator registers 0, 1 hold row g, columns 2t, 2t+1 (two neighbouring digits); registers 2, 3 the same for row g + 8
-            __syncwarp();                                   // the previous group's reads of the exchange buffer are done
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 unsigned long long chunk[NB / 2];
@@ -147,7 +152,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     const uint32_t b = (uint32_t)(acc[e >> 1][2 * c + 1][2 * (e & 1)] + 256 * acc[e >> 1][2 * c + 1][2 * (e & 1) + 1]);
                     chunk[c] = pack_chunk(a, b, chunk_hi[c], two16);           // bits of (1.5 2^52 + a + 2^16 b) 2^(32k)
                 }
-                uint32_t* row = xch + (4 * g + e) * kRow + t * NB;
+                uint32_t* row = xb + (4 * g + e) * kRow + t * NB;
                 if constexpr (NB % 4 == 0) {
 #pragma unroll
                     for (int c = 0; c < NB / 2; c += 2) *reinterpret_cast<ulonglong2*>(row + 2 * c) = make_ulonglong2(chunk[c], chunk[c + 1]);
@@ -156,42 +161,58 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     for (int c = 0; c < NB / 2; ++c) *reinterpret_cast<unsigned long long*>(row + 2 * c) = chunk[c];
                 }
             }
+        };
+        // kPfIlp groups at a time: their contractions first, then the FP64 finishes of all of them
+#pragma unroll
+        for (int ip = 0; ip < kPfGroups; ip += kPfIlp) {
+            __syncwarp();                                   // the previous groups' reads of the exchange buffers are done
+#pragma unroll
+            for (int u = 0; u < kPfIlp; ++u) contract(ip + u, xch + u * 32 * kRow);
             __syncwarp();
-            double br[NB], bi[NB];                          // lanes 0, 1 of the quad wrote the real part's chunks, lanes 2, 3 the imaginary part's
-            {
-                const double2* row = reinterpret_cast<const double2*>(xch + lane * kRow);
+            double br[kPfIlp][NB], bi[kPfIlp][NB];          // lanes 0, 1 of a quad wrote the real part's chunks, lanes 2, 3 the imaginary part's
+#pragma unroll
+            for (int u = 0; u < kPfIlp; ++u) {
+                const double2* row = reinterpret_cast<const double2*>(xch + u * 32 * kRow + lane * kRow);
 #pragma unroll
                 for (int c = 0; c < NB / 2; ++c) {
                     const double2 vr = row[c], vi = row[NB / 2 + c];
-                    br[2 * c] = vr.x; br[2 * c + 1] = vr.y;
-                    bi[2 * c] = vi.x; bi[2 * c + 1] = vi.y;
+                    br[u][2 * c] = vr.x; br[u][2 * c + 1] = vr.y;
+                    bi[u][2 * c] = vi.x; bi[u][2 * c + 1] = vi.y;
                 }
             }
-            const int64_t i = ib + 32 * it + lane;
-            {
-                double re, im;
-                const int eai = ea[it];
-                double hr, lr, hi, li;               // lanes beyond m work on whatever the staging buffer holds; nothing of it is stored
-                crt_finish32<NB>(br, pc.off[0], pc, &hr, &lr);
-                crt_finish32<NB>(bi, pc.off[1], pc, &hi, &li);
-                if (pc.im_hi != 0.0) {               // Eisenstein variant: V sqrt(3)/2 as a double-double product, rounded once below
+            double xr[kPfIlp], xi[kPfIlp];                  // lanes beyond m work on whatever the staging buffer holds; nothing of it is stored
+#pragma unroll
+            for (int u = 0; u < kPfIlp; ++u) {
+                double hr, lr, hi, li;
+                crt_finish32<NB>(br[u], pc.off[0], pc, &hr, &lr);
+                crt_finish32<NB>(bi[u], pc.off[1], pc, &hi, &li);
+                if (pc.im_hi != 0.0) {                       // Eisenstein variant: V sqrt(3)/2 as a double-double product, rounded once below
                     const double p = hi * pc.im_hi;
                     li = fma(hi, pc.im_lo, fma(li, pc.im_hi, fma(hi, pc.im_hi, -p)));
                     hi = p;
                 }
+                xr[u] = NB == 2 ? hr : hr + lr;              // the one rounding of the lifted integers
+                xi[u] = hi + li;
+            }
+#pragma unroll
+            for (int u = 0; u < kPfIlp; ++u) {
+                const int it = ip + u;
+                double re, im;
+                const int eai = ea[it];
                 const int e = (int)((uint32_t)eai + (uint32_t)fb);
-                if (e > -1000 && e < 1000) {         // 2^e is a normal number: one multiplication
-                    re = (hr + lr) * __longlong_as_double((long long)(e + pc.re_shift + 1023) << 52);
-                    im = (hi + li) * __longlong_as_double((long long)(e + 1023) << 52);
+                const bool bad = eai == kExpNonFinite || fb == kExpNonFinite;     // an Inf or NaN in the row of A or the column of B
+                if (bad || (unsigned)(e + 999) < 1999u) {
+                    // 2^e is a normal number: one multiplication by a factor built from its exponent (a NaN for a bad row / column)
+                    re = xr[u] * __hiloint2double(bad ? 0x7FF80000 : (e + pc.re_shift + 1023) << 20, 0);
+                    im = xi[u] * __hiloint2double(bad ? 0x7FF80000 : (e + 1023) << 20, 0);
                 } else {
-                    re = scale_pow2(hr + lr, e + pc.re_shift);
-                    im = scale_pow2(hi + li, e);
+                    re = scale_pow2(xr[u], e + pc.re_shift);
+                    im = scale_pow2(xi[u], e);
                 }
-                if (eai == kExpNonFinite || fb == kExpNonFinite) re = im = __longlong_as_double(0x7FF8000000000000ll);
-                T* dst = C + 2 * (i + (int64_t)j * ldc);
+                T* dst = dst0 + 64 * it;
                 if (AXPBY) {
                     double yr = fma(sc.ar, re, -sc.ai * im), yi = fma(sc.ar, im, sc.ai * re);
-                    if (i < m && (sc.br != 0.0 || sc.bi != 0.0)) {
+                    if (32 * it < rows_left && (sc.br != 0.0 || sc.bi != 0.0)) {
                         const double cr = (double)dst[0], ci = (double)dst[1];
                         yr += fma(sc.br, cr, -sc.bi * ci);
                         yi += fma(sc.br, ci, sc.bi * cr);
@@ -199,7 +220,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     re = yr;
                     im = yi;
                 }
-                if (i < m) store_cplx<T>(dst, re, im);
+                if (32 * it < rows_left) store_cplx<T>(dst, re, im);
             }
         }
         __syncthreads();                                    // every warp is done with this stage before it is refilled

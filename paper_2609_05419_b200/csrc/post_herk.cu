@@ -170,11 +170,11 @@ __global__ void __launch_bounds__(kHkThreads) post_herk_kernel(const int8_t* __r
             crt_finish32<NB>(br, pc.off[0], pc, &hr, &lr);
             const int e = (int)((uint32_t)ei_lane + (uint32_t)ej);
             const bool fast = e > -1000 && e < 1000;        // 2^e is a normal number: one multiplication
-            re = fast ? (hr + lr) * __longlong_as_double((long long)(e + 1023) << 52) : scale_pow2(hr + lr, e);
+            re = fast ? (NB == 2 ? hr : hr + lr) * __longlong_as_double((long long)(e + 1023) << 52) : scale_pow2(NB == 2 ? hr : hr + lr, e);
             if (!REAL_OUT) {
                 double hi, li;
                 crt_finish32<NB>(bi, pc.off[1], pc, &hi, &li);
-                im = fast ? (hi + li) * __longlong_as_double((long long)(e + 1023) << 52) : scale_pow2(hi + li, e);
+                im = fast ? (NB == 2 ? hi : hi + li) * __longlong_as_double((long long)(e + 1023) << 52) : scale_pow2(NB == 2 ? hi : hi + li, e);
             }
             if (ei_lane == kExpNonFinite || ej == kExpNonFinite) re = im = __longlong_as_double(0x7FF8000000000000ll);
             if (i < n && j < n && i >= j) {

@@ -44,7 +44,7 @@ __device__ __forceinline__ unsigned long long pack_chunk(uint32_t a, uint32_t b,
 // t = rint(X'/M) from the three leading chunks: M >= 2^(32 NB - 64) (its bytes fill more than NB - 2 chunks), so the
 // rest is below 2^-17 M; |t| < 2^14, and |X/M| stays away from 1/2 by the scaling rule.  W_k - t Mc_k is exact
 // (|t Mc_k| < 2^46 before the weight).  The chunks are then added with error-free transformations, neighbours first, so
-// hi + lo equals X to 2^-105 relative.
+// hi + lo equals X to 2^-105 relative (two chunks: hi alone is X rounded once, lo = 0).
 template <int NB>
 __device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const double (&off)[kPostMaxNB], const PostConsts& pc, double* hi, double* lo) {
     double W[NB];
@@ -56,6 +56,11 @@ __device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const dou
     const double t = rint(lead * pc.inv_M);
 #pragma unroll
     for (int k = 0; k < NB; ++k) W[k] = fma(-t, pc.Mc[k], W[k]);
+    if (NB == 2) {               // two exact terms: their floating-point sum is the correctly rounded X already
+        *hi = W[1] + W[0];
+        *lo = 0.0;
+        return;
+    }
     double ph[NB / 2], l = 0.0;
 #pragma unroll
     for (int k = 0; k < NB / 2; ++k) {
