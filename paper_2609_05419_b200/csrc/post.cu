@@ -30,7 +30,7 @@ template <int NCH>
 __device__ __forceinline__ void crt_finish(double (&S)[NCH], const CrtTable& tab, double* hi, double* lo) {
     const double t = rint(NCH > 1 ? fma(S[NCH - 1], tab.q_hi, S[NCH > 1 ? NCH - 2 : 0] * tab.q_lo) : S[0] * tab.q_hi);
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) S[c] = fma(-t, tab.Mc[c], S[c]);          // exact: |t| < 2^12, digits < 2^40
+    for (int c = 0; c < NCH; ++c) S[c] = fma(-t, tab.Mc[c], S[c]);          // exact: |S[c]| + |t| Mc[c] < 2^53 for every modulus count (host test)
     const double two40 = 1099511627776.0, inv40 = 1.0 / 1099511627776.0;
 #pragma unroll
     for (int c = 0; c + 1 < NCH; ++c) {                                     // carry into canonical digits [0, 2^40)

@@ -281,7 +281,7 @@ def test_cgemm_parity(shape, nmod):
     assert (np.abs(C.real.astype(np.float64) - ref["C"].real) <= spacing).all()
 
 
-@pytest.mark.parametrize("n,k,nmod", [(96, 200, 16), (257, 129, 16), (130, 300, 17), (64, 64, 21)])
+@pytest.mark.parametrize("n,k,nmod", [(96, 200, 16), (257, 129, 16), (130, 300, 17), (64, 64, 21), (70, 50, 7), (33, 40, 8), (20, 10, 1)])
 def test_zherk_parity(n, k, nmod):
     A = inputs.herk_input(n, k, seed=9)
     with Workspace(max(b.workspace_bytes(b.OP_ZHERK, n, n, k, nmod), b.workspace_bytes(b.OP_ZGEMM, n, n, k, nmod))) as ws:
@@ -302,7 +302,8 @@ def test_zherk_parity(n, k, nmod):
     assert (Ch[~low] == -5.0).all()                                           # strict upper triangle untouched
     assert (np.diag(Ch).imag == 0).all()
     Cref, D = direct.zgemm4m_dd(A, np.asfortranarray(A.conj().T))
-    assert direct.componentwise_error(Ch[low], Cref[low], D[low]) <= TOL_Z
+    if nmod >= 16:                                                            # fewer moduli: the error bound is that of their M; the stages are still exact
+        assert direct.componentwise_error(Ch[low], Cref[low], D[low]) <= TOL_Z
     assert ulp_distance(Ch[low].real, ref["C"][low].real).max() <= 1 and ulp_distance(Ch[low].imag, ref["C"][low].imag).max() <= 1
     if ref["Pt"] % 2 == 0:                                                    # same scale split: identical integers, identical bits
         assert (Ch[low] == Cg[low]).all()

@@ -180,6 +180,13 @@ def test_real_scheme_constants_match_oracle(nmod):
         W = M // m
         assert val(t["g"][j]) == staged.sym(pow(W % m, -1, m) if m > 1 else 0, m) * W
     assert 2 ** t["Pt"] / M < 0.494 or nmod == 1                      # margin of the quotient estimate in the post kernel
+    # exactness of the post kernel's digit arithmetic: every digit-column sum, and what is left of it after t M has come off,
+    # stays an exact integer in a double for the worst residues (all at -128)
+    G = [abs(val(t["g"][j])) for j in range(nmod)]
+    t_max = -(-sum(128 * g for g in G) // M) + 1
+    for c in range(t["nchunks"]):
+        col = sum(128 * abs(int(t["g"][j][c])) for j in range(nmod))
+        assert col + t_max * int(t["Mc"][c]) < 2 ** 53, (nmod, c)
     # the residue kernels' reduction, exhaustively, as for the 2M moduli
     assert (t["margin"] > 1.0).all()
     for j, m in enumerate(mods):
@@ -316,6 +323,8 @@ def _post_operand_checks(t, mods, M, plane_values, expected, rng_seed):
     multiple of M.  plane_values(rng) -> residues per plane; expected(residues) -> (X_r, X_i) modulo M from the oracle."""
     planes, nb = t["planes"], t["nb"]
     assert t["ks"] == (planes + 31) // 32 and nb % 2 == 0 and 4 * nb <= 24
+    Pt = ((M - 1) // 2).bit_length() - 1                              # |X| <= 2^Pt by the scaling rule: the quotient estimate (off by
+    assert 2 ** Pt / M + 2 ** -16 < 0.5                               # less than 2^-17) rounds to the right multiple of M
     nbytes = (M.bit_length() + 7) // 8
     assert nb == 2 * ((nbytes + 7) // 8) and M >= 2 ** (32 * nb - 64)        # what the quotient estimate relies on
     weights = [[sum(int(d) << (8 * p) for p, d in enumerate(t["digits"][part, pl])) for pl in range(planes)] for part in range(2)]
