@@ -179,12 +179,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
                 }
                 if (ok) umma_commit_pair(bar_tfull + 8 * acc, 3);    // accumulator complete in both CTAs
             }
-            if (!ok) {
-                st_cluster_u32(peer_abort, 1u);
-                // MMAs already issued still read both CTAs' shared memory and write both TMEMs: wait until they are through
-                umma_commit_pair(bar_drain, 1);
-                mbar_wait_quiet(bar_drain, 0, kDrainLimitNs);
-            }
+            if (!ok) st_cluster_u32(peer_abort, 1u);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
@@ -243,6 +238,12 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
         // stage's previous fill, which needed both CTAs' bytes), so every barrier is short of, or ahead by, at most one fill:
         // the leader takes the missing peer bytes off, or announces the peer bytes it had not got to, and then waits for
         // the last fill of every stage to complete.
+        if (warp == 1 && lane == 0 && rank == 0) {
+            // MMAs already issued (by this thread, whichever role gave up) still read both CTAs' shared memory and write both
+            // TMEMs: commit them to a barrier of their own and wait until they are through
+            umma_commit_pair(bar_drain, 1);
+            mbar_wait_quiet(bar_drain, 0, kDrainLimitNs);
+        }
         if (warp == 0 && lane == 0 && rank == 0) {
             const uint32_t mine = *fills_issued, peers = ld_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(fills_issued)), 1u));
             for (uint32_t f = min(mine, peers); f < max(mine, peers); ++f) {
