@@ -25,7 +25,8 @@
  *     memory inside a call; it uses the caller-provided workspace registered with gemm2m_set_workspace().
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and
  *     return immediately.  The return value is a gemm2m_status; it is the only error channel.  Every kernel of a call
- *     runs on `stream`, in order.  (zgemm2m_host alone uses library-owned streams, for its copies and the work that runs
+ *     runs on `stream`, in order (some are launched as programmatic dependents of the kernel before them: such a kernel may
+ *     become resident early, and waits on the device for every earlier kernel before it touches global memory).  (zgemm2m_host alone uses library-owned streams, for its copies and the work that runs
  *     beside them, forked from and joined back into `stream` with events: work enqueued on `stream` after the call still
  *     sees the finished result.  So does every entry point while gemm2m_debug_set_overlap(1) is in force.)
  *   - Because a call only enqueues (kernels, memsets, event records and waits), it can be captured into a CUDA graph
@@ -275,6 +276,11 @@ int gemm2m_debug_set_panels(int max_panels);
  * large operands, the exponent scan of B) runs on a library-owned stream beside the next panel's GEMMs, forked from and joined
  * back into the caller's stream with events.  Kept for measurement: it does not pay on a GPU whose GEMM phase is power-limited. */
 int gemm2m_debug_set_overlap(int enabled);
+/* 1 (default): the residue, GEMM and post-processing kernels of a call are launched as programmatic dependents of the kernel
+ * before them on the stream: a kernel may become resident while its predecessor drains, and waits on the device for the
+ * predecessor's completion before it touches global memory, so results and ordering are those of plain launches.  0: plain
+ * launches.  Kept for measurement (it matters for small problems, where launch latency is a visible share of a call). */
+int gemm2m_debug_set_chained_launch(int enabled);
 
 /* Host-only: copies the constants the library uses for `nmod` moduli and inner dimension k into caller arrays (host
  * pointers, any may be NULL), so that CPU tests can check them against an independent computation:

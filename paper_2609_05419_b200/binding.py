@@ -358,6 +358,10 @@ def debug_set_overlap(enabled):
     _check(lib().gemm2m_debug_set_overlap(1 if enabled else 0), "gemm2m_debug_set_overlap")
 
 
+def debug_set_chained_launch(enabled):
+    _check(lib().gemm2m_debug_set_chained_launch(1 if enabled else 0), "gemm2m_debug_set_chained_launch")
+
+
 def debug_set_panels(max_panels):
     _check(lib().gemm2m_debug_set_panels(max_panels), "gemm2m_debug_set_panels")
 

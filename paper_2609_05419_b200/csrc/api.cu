@@ -42,12 +42,16 @@ struct State {
     int prof_calls = 0;           // profiled calls since profiling was switched on (each uses slot prof_calls % kProfSlots)
     Slot* cur_slot = nullptr;     // slot of the call being enqueued
     int max_panels = 8;           // most column panels per zgemm2m/cgemm2m call
+    int chained = 1;              // 1 = the residue, GEMM and post-processing kernels are launched as programmatic dependents
     int overlap = 0;              // 1 = post-processing of a panel (and the scan of B) on the library's stream beside the next kernels
     int launches[4] = {0, 0, 0, 0};
     int gemm_kernel = 0;          // 0 = tcgen05 CTA pairs, 1 = check kernel
     int scaling = 0;              // 0 = largest part times sqrt(2k), 1 = 2-norm rule (zgemm2m / cgemm2m)
 };
 State g;
+}  // namespace
+bool gemm2m::chained_launch_enabled() { return g.chained != 0; }   // read while a call holds the library mutex
+namespace {
 DevState& D() { return g.dev[g.cur]; }
 thread_local char g_cuda_err[256] = "no error";
 
@@ -335,8 +339,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     if (sb != st) CK(cudaEventRecord(D().side_done, sb));
     CK(ph.begin(0, st));
     // rows of op(A) are rows of A as stored ('N') or its columns ('T', 'C')
-    if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0]));
-    else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0]));
+    const bool after_kernel = sb == st && !ph.on;          // directly behind the scan of B (no event in between)
+    if (ta == 'N') CK(launch_scan_rows<T>(A, m, k, lda, absA, st, &g.launches[0], after_kernel));
+    else CK(launch_scan_cols<T>(A, k, m, lda, absA, st, &g.launches[0], after_kernel));
     if (!two_norm_mode) {}                                                                          // (2-norm rule: not for k > 2^22,
     else if (ta == 'N') CK(launch_exponents_2norm<T>(A, m, k, lda, true, absA, qA, sc.PA, eA, st, &g.launches[0]));   // where the sums
     else CK(launch_exponents_2norm<T>(A, k, m, lda, false, absA, qA, sc.PA, eA, st, &g.launches[0]));   // of squares would not fit 64 bits)
@@ -921,6 +926,12 @@ int gemm2m_debug_set_panels(int max_panels) {
 int gemm2m_debug_set_overlap(int enabled) {
     std::lock_guard<std::mutex> lock(g.mu);
     g.overlap = enabled ? 1 : 0;
+    return GEMM2M_OK;
+}
+
+int gemm2m_debug_set_chained_launch(int enabled) {
+    std::lock_guard<std::mutex> lock(g.mu);
+    g.chained = enabled ? 1 : 0;
     return GEMM2M_OK;
 }
 

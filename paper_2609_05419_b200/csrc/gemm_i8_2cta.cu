@@ -121,6 +121,7 @@ gemm_i8_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_row, const _
     cluster_sync_all();                                  // the peer's barriers exist before anything signals them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    wait_for_prior_kernels();                            // barriers and TMEM are set up; the planes are read from here on
 
     const int tiles_per_batch = p.tiles_r * p.tiles_c;
     const int total_tiles = tiles_per_batch * p.nbatch;
@@ -322,7 +323,8 @@ cudaError_t launch_gemm_tcgen05_pair(const GemmArgs& a, int64_t k_limit, int sm_
         p.kblock0 = kb0;
         p.kblocks = (kblocks_total - kb0 < chunk) ? kblocks_total - kb0 : chunk;
         p.accumulate = (kb0 > 0 || a.accumulate) ? 1 : 0;
-        gemm_i8_tcgen05_pair_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(map_row, map_col, p);   // cluster size is a kernel attribute
+        cudaError_t err = launch_chained(gemm_i8_tcgen05_pair_kernel, dim3(2 * pairs), dim3(THREADS), SMEM_BYTES, st, map_row, map_col, p);   // cluster size is a kernel attribute
+        if (err != cudaSuccess) return err;
         ++*launches;
     }
     return cudaGetLastError();

@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                                                              T* __restrict__ C, int64_t ldc, const PostScalars sc) {
     static_assert(NB % 2 == 0, "whole chunks per lane");
     extern __shared__ __align__(16) uint32_t pf_smem[];
+    wait_for_prior_kernels();
     constexpr int KS = (KH + 1) / 2, kHalves = KH == 1 ? 1 : 2;     // K-steps of 32 planes; halves of a step in use
     constexpr int kStageWords = 16 * KH * kPfStrideW;
     constexpr int kRow = pf_row_words(NB);
@@ -261,7 +262,7 @@ static cudaError_t launch_post_fp_v(const int8_t* cpm, int64_t ldp, int64_t m, i
         const int64_t nj = (j_end - j0 < kColsPerLaunch) ? j_end - j0 : kColsPerLaunch;
         const int64_t steps = ((m + kPfSpan - 1) / kPfSpan) * nj;
         const unsigned grid = (unsigned)(steps < resident ? steps : resident);
-        post_fp_kernel<T, KH, NB, AXPBY><<<grid, kPfThreads, smem, st>>>(cpm + j0 * ldp, ldp, m, n * ldp, (int)nj, eA, eB + j0, dev_frags, tab.c,
+        launch_chained(post_fp_kernel<T, KH, NB, AXPBY>, dim3(grid), dim3(kPfThreads), smem, st, cpm + j0 * ldp, ldp, m, n * ldp, (int)nj, eA, eB + j0, dev_frags, tab.c,
                                                                         C + 2 * j0 * ldc, ldc, sc);
         ++*launches;
     }

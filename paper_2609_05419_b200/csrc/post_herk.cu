@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(kHkThreads) post_herk_kernel(const int8_t* __r
                                                                const int32_t* __restrict__ eA, const uint32_t* __restrict__ frags,
                                                                const __grid_constant__ PostConsts pc, double* __restrict__ C, int64_t ldc) {
     extern __shared__ __align__(16) uint32_t hk_smem[];
+    wait_for_prior_kernels();
     constexpr int KS = HV;                                   // K-steps of 32 slots: HV halves direct + HV halves mirrored
     constexpr int kRow = pf_row_words(NB);
     uint32_t* sdir = hk_smem;
@@ -199,7 +200,7 @@ static cudaError_t launch_post_herk_v(const int8_t* cp, int64_t ldp, int64_t n, 
     const int64_t tiles_j = (i_end + kHkJ - 1) / kHkJ;     // lower triangle: columns up to the last row of the range
     if (tiles_j > 65535) return cudaErrorInvalidValue;     // n beyond 65535 * 16 columns: far beyond any workspace
     dim3 grid((unsigned)((i_end - i_begin + kHkI - 1) / kHkI), (unsigned)tiles_j);
-    post_herk_kernel<HV, NB, REAL_OUT><<<grid, kHkThreads, smem, st>>>(cp, ldp, n, i_begin, nmod, eA, dev_frags, tab.c, C, ldc);
+    launch_chained(post_herk_kernel<HV, NB, REAL_OUT>, grid, dim3(kHkThreads), smem, st, cp, ldp, n, i_begin, nmod, eA, dev_frags, tab.c, C, ldc);
     return cudaGetLastError();
 }
 

@@ -223,6 +223,7 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
                                                                      int64_t plane_rows) {
     using Raw = typename RawCplx<T>::type;
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    wait_for_prior_kernels();
     Raw* ring = reinterpret_cast<Raw*>(smem_raw);
     constexpr int kStageElems = kResRows * kResRowStride;
     const int t = threadIdx.x;
@@ -356,12 +357,12 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
     // saves two instructions per (element, modulus) -- 13 % of the kernel's time at 16 moduli.
     const int spec = (!wide && tab.n2 == tab.nmod) ? tab.nmod : 0;
     switch (spec) {
-#define GEMM2M_RES_CASE(N) case N: residues_fp_kernel<T, false, N><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R); break;
+#define GEMM2M_RES_CASE(N) case N: launch_chained(residues_fp_kernel<T, false, N>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R); break;
         GEMM2M_RES_CASE(7) GEMM2M_RES_CASE(8) GEMM2M_RES_CASE(14) GEMM2M_RES_CASE(15) GEMM2M_RES_CASE(16)
 #undef GEMM2M_RES_CASE
         default:
-            if (wide) residues_fp_kernel<T, true, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
-            else residues_fp_kernel<T, false, 0><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+            if (wide) launch_chained(residues_fp_kernel<T, true, 0>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+            else launch_chained(residues_fp_kernel<T, false, 0>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
     }
     ++*launches;
     return cudaGetLastError();
@@ -385,9 +386,9 @@ cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, 
     const int64_t total = ((R + kResRows - 1) / kResRows) * (Kp / kResK);
     const int64_t resident = (int64_t)cached_sm_count() * kResBlocksPerSm;
     const unsigned grid = (unsigned)(total < resident ? total : resident);
-    if (wide) residues_fp_kernel<double, true, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
-    else if (tab.nmod == 16) residues_fp_kernel<double, false, 16, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
-    else residues_fp_kernel<double, false, 0, true><<<grid, kResThreads, smem, st>>>(X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+    if (wide) launch_chained(residues_fp_kernel<double, true, 0, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+    else if (tab.nmod == 16) launch_chained(residues_fp_kernel<double, false, 16, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+    else launch_chained(residues_fp_kernel<double, false, 0, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
     ++*launches;
     return cudaGetLastError();
 }

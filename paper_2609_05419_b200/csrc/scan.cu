@@ -16,6 +16,7 @@ constexpr int kScanColsSpan = 2048;   // rows handled by one warp of scan_cols
 template <typename T>
 __global__ void __launch_bounds__(kScanThreads) scan_rows_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
                                                                  unsigned long long* __restrict__ absmax) {
+    wait_for_prior_kernels();
     const int64_t r = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
     if (r >= rows) return;
     const int64_t c0 = (int64_t)blockIdx.y * span;
@@ -34,6 +35,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_rows_kernel(const T* __rest
 template <typename T>
 __global__ void __launch_bounds__(kScanThreads) scan_cols_kernel(const T* __restrict__ X, int64_t rows, int64_t cols, int64_t ld, int64_t span,
                                                                  unsigned long long* __restrict__ absmax) {
+    wait_for_prior_kernels();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t c = (int64_t)blockIdx.x * (kScanThreads / 32) + warp;
     if (c >= cols) return;
@@ -224,26 +226,28 @@ template cudaError_t launch_exponents_2norm<double>(const double*, int64_t, int6
 template cudaError_t launch_exponents_2norm<float>(const float*, int64_t, int64_t, int64_t, bool, const uint64_t*, uint64_t*, int, int32_t*, cudaStream_t, int*);
 
 template <typename T>
-cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
+cudaError_t launch_scan_rows(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches, bool chained) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
     int64_t span = kScanRowsSpan;
     const int64_t row_blocks = (rows + kScanThreads - 1) / kScanThreads;
     while (span > 8 && row_blocks * ((cols + span - 1) / span) < 4 * cached_sm_count()) span /= 2;   // small matrices: enough blocks to fill the GPU
     while ((cols + span - 1) / span > 65535) span *= 2;        // grid.y limit
     dim3 grid((unsigned)row_blocks, (unsigned)((cols + span - 1) / span));
-    scan_rows_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    if (chained) launch_chained(scan_rows_kernel<T>, grid, dim3(kScanThreads), 0, st, X, rows, cols, ld, span, (unsigned long long*)absmax);
+    else scan_rows_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
     ++*launches;
     return cudaGetLastError();
 }
 template <typename T>
-cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches) {
+cudaError_t launch_scan_cols(const T* X, int64_t rows, int64_t cols, int64_t ld, uint64_t* absmax, cudaStream_t st, int* launches, bool chained) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
     int64_t span = kScanColsSpan;
     const int64_t col_blocks = (cols + kScanThreads / 32 - 1) / (kScanThreads / 32);
     while (span > 256 && col_blocks * ((rows + span - 1) / span) < 4 * cached_sm_count()) span /= 2;
     while ((rows + span - 1) / span > 65535) span *= 2;        // grid.y limit
     dim3 grid((unsigned)col_blocks, (unsigned)((rows + span - 1) / span));
-    scan_cols_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
+    if (chained) launch_chained(scan_cols_kernel<T>, grid, dim3(kScanThreads), 0, st, X, rows, cols, ld, span, (unsigned long long*)absmax);
+    else scan_cols_kernel<T><<<grid, kScanThreads, 0, st>>>(X, rows, cols, ld, span, (unsigned long long*)absmax);
     ++*launches;
     return cudaGetLastError();
 }
@@ -255,10 +259,10 @@ cudaError_t launch_exponents(const uint64_t* absmax, int64_t count, int P, int c
     return cudaGetLastError();
 }
 
-template cudaError_t launch_scan_rows<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
-template cudaError_t launch_scan_rows<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
-template cudaError_t launch_scan_cols<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
-template cudaError_t launch_scan_cols<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*);
+template cudaError_t launch_scan_rows<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*, bool);
+template cudaError_t launch_scan_rows<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*, bool);
+template cudaError_t launch_scan_cols<double>(const double*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*, bool);
+template cudaError_t launch_scan_cols<float>(const float*, int64_t, int64_t, int64_t, uint64_t*, cudaStream_t, int*, bool);
 template cudaError_t launch_exponents<double>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
 template cudaError_t launch_exponents<float>(const uint64_t*, int64_t, int, int, int32_t*, cudaStream_t, int*);
 
