@@ -20,10 +20,12 @@ def _default_kernel():
     b.debug_set_gemm_kernel(0)
     b.debug_set_panels(8)
     b.debug_set_overlap(False)
+    b.debug_set_chained_launch(True)
     yield
     b.debug_set_gemm_kernel(0)
     b.debug_set_panels(8)
     b.debug_set_overlap(False)
+    b.debug_set_chained_launch(True)
 
 
 def run_int(Ar, Ai, Br, Bi, nmod, kernel=0, ldc=None):
@@ -322,6 +324,38 @@ def test_device_status_and_launch_counts():
             b.set_profiling(False)
     assert calls == 1 and all(x >= 0 for x in ms) and sum(ms) > 0
     assert per == [2, 2, 1, 2] and total == 7             # two scans, two residue launches, one GEMM launch, the post-processing's operand and its launch
+
+
+def test_chained_launches_are_bitwise_identical_to_plain_ones_in_a_stream_of_calls():
+    # The residue, GEMM and post-processing kernels are launched as programmatic dependents: a kernel may be resident before
+    # the one in front of it has finished, and must not touch memory until it has.  Calls on different operands, sharing one
+    # workspace, are enqueued back to back without a synchronisation in between; a kernel that read planes, exponents or C
+    # early would pick up the previous call's.
+    shapes = [(300, 200, 260), (129, 1100, 96), (520, 130, 1030)]
+    ops = [inputs.complex_inputs(m, n, k, seed=40 + i, dist="phi", phi=1.0) for i, (m, n, k) in enumerate(shapes)]
+    H = inputs.complex_inputs(260, 1, 300, seed=44)[0]
+    dev = [(to_dev(A), to_dev(B)) for A, B in ops]
+    dH = to_dev(H)
+    need = max([b.workspace_bytes(b.OP_ZGEMM, m, n, k, 16) for m, n, k in shapes] + [b.workspace_bytes(b.OP_ZHERK, 260, 260, 300, 16)])
+    results = {}
+    with Workspace(need):
+        for chained in (False, True):
+            b.debug_set_chained_launch(chained)
+            outs = []
+            for rep in range(6):
+                for (m, n, k), (dA, dB) in zip(shapes, dev):
+                    C = empty_dev(m, n, torch.complex128, fill=float(rep))
+                    b.zgemm2m(dA, dB, C, 16 if rep % 2 == 0 else 12)
+                    outs.append(C)
+                Ch = empty_dev(260, 260, torch.complex128, fill=1.0)
+                b.zherk2m(dH, Ch, 16)
+                outs.append(Ch)
+            b.device_status()
+            results[chained] = [to_host(C) for C in outs]
+    for x, y in zip(results[False], results[True]):
+        assert (x == y).all()
+    ref = staged.zgemm2m_staged(ops[0][0], ops[0][1], 16)["C"]
+    assert (results[True][0] == ref).mean() > 0.999
 
 
 def test_panel_pipeline_is_bitwise_identical_and_joins_the_callers_stream():
