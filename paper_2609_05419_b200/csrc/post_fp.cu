@@ -20,13 +20,13 @@ constexpr int kPfWarps = GEMM2M_POST_WARPS;     // warps per block
 constexpr int kPfGroups = GEMM2M_POST_GROUPS;   // MMA groups of 32 elements per warp and step
 constexpr int kPfThreads = 32 * kPfWarps;
 constexpr int kPfSpan = 32 * kPfGroups * kPfWarps;      // consecutive row indices i per step of a block
-constexpr int kPfStrideW = kPfSpan / 4 + 8;     // words per staged plane: + 8, so that the 32 fragment loads of a warp hit 32 banks
+constexpr int kPfStrideW = kPfSpan / 4 + 4;     // words per staged plane: + 4, so that the 16-byte rows of 8 consecutive planes cover the 32 banks
 constexpr int kPfStages = 2;                    // staging ring: the next step is on its way while this one is processed
 constexpr int kPfIlp = 1;                       // groups of a warp whose elements are finished together (one exchange buffer each);
-                                                // 2 and 4 measured 5 and 15 % slower at 8192^3: fewer blocks fit, and the compiler
-                                                // does not interleave the finishes anyway
+                                                // 2 and 4 measured 5 and 15 % slower at 8192^3 (fewer blocks fit), also with the
+                                                // finishes written out step by step across the groups
 static_assert(kPfGroups % kPfIlp == 0, "whole batches of groups");
-static_assert(kPfSpan % 128 == 0, "plane stride = 8 mod 32 words");
+static_assert(kPfSpan % 128 == 0, "plane stride = 4 mod 32 words");
 
 __host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfStages * 16 * kh * kPfStrideW + kPfWarps * kPfIlp * 32 * pf_row_words(nb); }
 
@@ -34,9 +34,10 @@ __host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfSta
 // pointers given.  The work is cut into steps of kPfSpan consecutive i of one column j, numbered column by column within a
 // block of rows; every thread block takes an equal, contiguous share of the steps.  The planes x kPfSpan residue bytes of a step
 // are pulled into shared memory with asynchronous 16-byte copies while the previous step is processed.  A warp owns 32 kPfGroups
-// of the i; for each group of 32 it gathers the MMA operand (rows = elements, K = planes; lane (g, t) takes the word of
-// elements 4g..4g+3 of the planes t, t+4, t+8, t+12 of each half K-step, moves the bytes to [0, 255] and transposes the 4 x 4
-// bytes), multiplies by the digit matrix held in registers, packs each run of four digit-column sums into one 64-bit chunk,
+// of the i; for each group of 32 it loads the MMA operand (rows = elements, K = planes) with the transposing 8-bit matrix load
+// (a staged plane's 16 consecutive element bytes are one row of the matrix in shared memory; the load hands lane (g, t) the
+// bytes of planes 4t..4t+3 for elements g and g + 8, which is the operand fragment), moves the bytes to [0, 255],
+// multiplies by the digit matrix held in registers, packs each run of four digit-column sums into one 64-bit chunk,
 // and passes the chunks through shared memory so that lane L ends up with all chunks of element L, which it finishes and
 // stores (consecutive lanes, consecutive i).  Many warps per SM matter more here than long steps: the per-element finish is a
 // chain of dependent FP64 operations.
@@ -113,22 +114,23 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
         // MMA phase of group `it`: operand gather, contraction, chunks into the exchange buffer xb
         auto contract = [&](int it, uint32_t* xb) {
             int acc[2][NB][4];
-            const uint32_t* col = st + 8 * (kPfGroups * warp + it) + g;
+            // rows of the staged planes holding this group's 32 elements: lane L addresses plane L of the K-step (16 bytes = elements 0..15)
+            const uint32_t rows = (uint32_t)__cvta_generic_to_shared(st) + (kHalves > 1 ? lane : (lane & 15)) * (4 * kPfStrideW) + 32 * (kPfGroups * warp + it);
 #pragma unroll
             for (int s = 0; s < KS; ++s) {
-                uint32_t a0[4], a1[4];                      // A operands of the two 16-row tiles: elements 4g, 4g+1 / 4g+2, 4g+3
-#pragma unroll
-                for (int h = 0; h < kHalves; ++h) {
-                    const uint32_t* p = col + (32 * s + 16 * h + t) * kPfStrideW;
-                    const uint32_t w0 = p[0] ^ 0x80808080u, w1 = p[4 * kPfStrideW] ^ 0x80808080u;      // residue + 128
-                    const uint32_t w2 = p[8 * kPfStrideW] ^ 0x80808080u, w3 = p[12 * kPfStrideW] ^ 0x80808080u;
-                    const uint32_t lo01 = __byte_perm(w0, w1, 0x5140), hi01 = __byte_perm(w0, w1, 0x7362);
-                    const uint32_t lo23 = __byte_perm(w2, w3, 0x5140), hi23 = __byte_perm(w2, w3, 0x7362);
-                    a0[2 * h] = __byte_perm(lo01, lo23, 0x5410);        // element 4g:   row g of tile 0
-                    a0[2 * h + 1] = __byte_perm(lo01, lo23, 0x7632);    // element 4g+1: row g + 8 of tile 0
-                    a1[2 * h] = __byte_perm(hi01, hi23, 0x5410);        // element 4g+2: row g of tile 1
-                    a1[2 * h + 1] = __byte_perm(hi01, hi23, 0x7632);    // element 4g+3: row g + 8 of tile 1
+                uint32_t a0[4], a1[4];                      // A operands of the two 16-row tiles: elements 0..15 and 16..31 of the group
+                if (kHalves > 1) {
+                    load_a_k32(a0, rows + s * (32 * 4 * kPfStrideW));
+                    load_a_k32(a1, rows + s * (32 * 4 * kPfStrideW) + 16);
+                } else {
+                    uint32_t x0[2], x1[2];
+                    load_a_k16(x0, rows);
+                    load_a_k16(x1, rows + 16);
+                    a0[0] = x0[0]; a0[1] = x0[1]; a1[0] = x1[0]; a1[1] = x1[1];
+                    a0[2] = a0[3] = a1[2] = a1[3] = 0u;
                 }
+#pragma unroll
+                for (int r = 0; r < 2 * kHalves; ++r) { a0[r] ^= 0x80808080u; a1[r] ^= 0x80808080u; }      // residue + 128
 #pragma unroll
                 for (int q = 0; q < NB; ++q) {
                     if (KH == 1) {
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     }
                 }
             }
-            // accumulator registers 0, 1 hold row g, columns 2t, 2t+1 (two neighbouring digits); registers 2, 3 the same for row g + 8
+            // accumulator registers 0, 1 hold row g (element g of the tile), columns 2t, 2t+1 (two neighbouring digits); registers 2, 3 the same for row g + 8
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 unsigned long long chunk[NB / 2];
@@ -153,7 +155,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     const uint32_t b = (uint32_t)(acc[e >> 1][2 * c + 1][2 * (e & 1)] + 256 * acc[e >> 1][2 * c + 1][2 * (e & 1) + 1]);
                     chunk[c] = pack_chunk(a, b, chunk_hi[c], two16);           // bits of (1.5 2^52 + a + 2^16 b) 2^(32k)
                 }
-                uint32_t* row = xb + (4 * g + e) * kRow + t * NB;
+                uint32_t* row = xb + (16 * (e >> 1) + 8 * (e & 1) + g) * kRow + t * NB;     // tile e / 2, row g or g + 8 of it
                 if constexpr (NB % 4 == 0) {
 #pragma unroll
                     for (int c = 0; c < NB / 2; c += 2) *reinterpret_cast<ulonglong2*>(row + 2 * c) = make_ulonglong2(chunk[c], chunk[c + 1]);

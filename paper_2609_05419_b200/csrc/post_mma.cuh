@@ -15,6 +15,16 @@ __device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint
         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(0));
 }
+// A operand straight from shared memory: 16 (x1) or 32 (x2) rows of 16 bytes, row r = the bytes of K index r for 16
+// consecutive elements, loaded transposed.  Lane (g, t) receives, per 16 rows, the bytes of K = 4t .. 4t+3 for element g and
+// for element g + 8: the A fragment of the 8-bit MMAs.  Lanes 0..15 (x2: 0..31) supply the row addresses (16-byte aligned).
+__device__ __forceinline__ void load_a_k16(uint32_t (&a)[2], uint32_t row_addr) {
+    asm volatile("ldmatrix.sync.aligned.m16n16.x1.trans.shared.b8 {%0, %1}, [%2];" : "=r"(a[0]), "=r"(a[1]) : "r"(row_addr) : "memory");
+}
+__device__ __forceinline__ void load_a_k32(uint32_t (&a)[4], uint32_t row_addr) {
+    asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(row_addr) : "memory");
+}
 // The same with K = 16 (A: 16 x 16, B: 16 x 8): for operands of at most 16 planes.
 __device__ __forceinline__ void mma_u8_k16(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
     asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"

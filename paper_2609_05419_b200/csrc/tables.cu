@@ -401,7 +401,9 @@ static void build_post_mma_table_for(const int* mods, int nmod, int n2, PostMmaT
                     const int tc = g >> 1, b = g & 1, part = tc >> 1, p = 2 * ((tc & 1) * c.nb + q) + b;
                     uint32_t word = 0;
                     for (int r = 0; r < 4; ++r) {
-                        const int plane = 32 * s + 16 * hh + tt + 4 * r;
+                        // K index 4 tt + r of the half: the complex GEMMs' kernel loads its operand with the planes in their order,
+                        // the rank-k kernel gathers the planes tt, tt + 4, tt + 8, tt + 12 into one register
+                        const int plane = 32 * s + 16 * hh + (herk ? tt + 4 * r : 4 * tt + r);
                         const uint32_t byte = plane < planes ? (uint32_t)t->digit[part][plane][p] : 0u;
                         word |= byte << (8 * r);
                     }
