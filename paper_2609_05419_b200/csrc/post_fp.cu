@@ -21,7 +21,11 @@ constexpr int kPfGroups = GEMM2M_POST_GROUPS;   // MMA groups of 32 elements per
 constexpr int kPfThreads = 32 * kPfWarps;
 constexpr int kPfSpan = 32 * kPfGroups * kPfWarps;      // consecutive row indices i per step of a block
 constexpr int kPfStrideW = kPfSpan / 4 + 4;     // words per staged plane: + 4, so that the 16-byte rows of 8 consecutive planes cover the 32 banks
-constexpr int kPfStages = 2;                    // staging ring: the next step is on its way while this one is processed
+#ifndef GEMM2M_POST_STAGES
+#define GEMM2M_POST_STAGES 2
+#endif
+constexpr int kPfStages = GEMM2M_POST_STAGES;   // staging ring: the next step is on its way while this one is processed (3 stages of 512 rows,
+                                                // 3 or 4 stages of 256 rows: 5-14 % slower at 8192^3)
 constexpr int kPfIlp = 1;                       // groups of a warp whose elements are finished together (one exchange buffer each);
                                                 // 2 and 4 measured 5 and 15 % slower at 8192^3 (fewer blocks fit), also with the
                                                 // finishes written out step by step across the groups
@@ -38,8 +42,8 @@ __host__ __device__ constexpr int pf_block_words(int kh, int nb) { return kPfSta
 // (a staged plane's 16 consecutive element bytes are one row of the matrix in shared memory; the load hands lane (g, t) the
 // bytes of planes 4t..4t+3 for elements g and g + 8, which is the operand fragment), moves the bytes to [0, 255],
 // multiplies by the digit matrix held in registers, packs each run of four digit-column sums into one 64-bit chunk,
-// and passes the chunks through shared memory so that lane L ends up with all chunks of element L, which it finishes and
-// stores (consecutive lanes, consecutive i).  Many warps per SM matter more here than long steps: the per-element finish is a
+// and passes the chunks through shared memory so that every lane ends up with all chunks of one element, which it finishes and
+// stores (the 32 lanes of a warp cover 32 consecutive i).  Many warps per SM matter more here than long steps: the per-element finish is a
 // chain of dependent FP64 operations.
 // KH: 16-plane halves of K that are staged and contracted (1, 2 or 4).
 template <typename T, int KH, int NB, bool AXPBY>
@@ -54,6 +58,9 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
     constexpr int kStageWords = 16 * KH * kPfStrideW;
     constexpr int kRow = pf_row_words(NB);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    // The element of a group that this lane finishes: exchange row `lane` = 4 g' + e' holds row g' (e' odd: g' + 8) of the 16-element
+    // tile e' / 2 (a row order in which the 16-byte stores of the chunks and the 16-byte loads of the rows are both free of bank conflicts)
+    const int el = 16 * ((lane >> 1) & 1) + 8 * (lane & 1) + (lane >> 2);
     uint32_t* xch = pf_smem + kPfStages * kStageWords + warp * kPfIlp * 32 * kRow;
     const int64_t total = ((m + kPfSpan - 1) / kPfSpan) * ncols;
     int64_t step = total * blockIdx.x / gridDim.x;
@@ -77,7 +84,16 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
         }
         cp_async_commit_group();
     };
-    issue(ibk, j, 0);
+    // the ring is filled kPfStages - 1 steps ahead: (pibk, pj) is the step the next copy is for
+    int pibk = ibk, pj = j;
+    int64_t pstep = step;
+#pragma unroll
+    for (int a = 0; a < kPfStages - 1; ++a) {
+        if (pstep < step_end) issue(pibk, pj, a);
+        else cp_async_commit_group();
+        ++pstep;
+        if (++pj == ncols) { pj = 0; ++pibk; }
+    }
 
     uint32_t bf[KS][NB][2];
 #pragma unroll
@@ -98,19 +114,22 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
     for (int n = 0; step < step_end; ++step, ++n) {
         int jn = j + 1, ibkn = ibk;
         if (jn == ncols) { jn = 0; ++ibkn; }
-        if (step + 1 < step_end) { issue(ibkn, jn, (n + 1) & 1); cp_async_wait_pending<1>(); }
-        else cp_async_wait_pending<0>();
+        if (pstep < step_end) issue(pibk, pj, (n + kPfStages - 1) % kPfStages);
+        else cp_async_commit_group();                       // an empty group keeps the count of pending groups uniform
+        ++pstep;
+        if (++pj == ncols) { pj = 0; ++pibk; }
+        cp_async_wait_pending<kPfStages - 1>();
         __syncthreads();
-        const uint32_t* st = pf_smem + (n & 1) * kStageWords;
+        const uint32_t* st = pf_smem + (n % kPfStages) * kStageWords;
         const int64_t ib = (int64_t)ibk * kPfSpan + 32 * kPfGroups * warp;    // first row of this warp
         if (ibk != ea_block) {
 #pragma unroll
-            for (int it = 0; it < kPfGroups; ++it) ea[it] = ib + 32 * it + lane < m ? __ldg(eA + ib + 32 * it + lane) : 0;
+            for (int it = 0; it < kPfGroups; ++it) ea[it] = ib + 32 * it + el < m ? __ldg(eA + ib + 32 * it + el) : 0;
             ea_block = ibk;
         }
         const int fb = __ldg(eB + j);
-        T* dst0 = C + 2 * (ib + lane + (int64_t)j * ldc);     // this lane's element of the warp's first group
-        const int64_t rows_left = m - ib - lane;               // group `it` is inside the matrix for this lane if 32 it < rows_left
+        T* dst0 = C + 2 * (ib + el + (int64_t)j * ldc);       // this lane's element of the warp's first group
+        const int64_t rows_left = m - ib - el;               // group `it` is inside the matrix for this lane if 32 it < rows_left
         // MMA phase of group `it`: operand gather, contraction, chunks into the exchange buffer xb
         auto contract = [&](int it, uint32_t* xb) {
             int acc[2][NB][4];
@@ -155,7 +174,7 @@ __global__ void __launch_bounds__(kPfThreads) post_fp_kernel(const int8_t* __res
                     const uint32_t b = (uint32_t)(acc[e >> 1][2 * c + 1][2 * (e & 1)] + 256 * acc[e >> 1][2 * c + 1][2 * (e & 1) + 1]);
                     chunk[c] = pack_chunk(a, b, chunk_hi[c], two16);           // bits of (1.5 2^52 + a + 2^16 b) 2^(32k)
                 }
-                uint32_t* row = xb + (16 * (e >> 1) + 8 * (e & 1) + g) * kRow + t * NB;     // tile e / 2, row g or g + 8 of it
+                uint32_t* row = xb + (4 * g + e) * kRow + t * NB;     // tile e / 2, row g or g + 8 of it: finished by lane 4 g + e
                 if constexpr (NB % 4 == 0) {
 #pragma unroll
                     for (int c = 0; c < NB / 2; c += 2) *reinterpret_cast<ulonglong2*>(row + 2 * c) = make_ulonglong2(chunk[c], chunk[c + 1]);
