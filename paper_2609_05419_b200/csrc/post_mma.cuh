@@ -46,15 +46,15 @@ __device__ __forceinline__ unsigned long long pack_chunk(uint32_t a, uint32_t b,
     return r;
 }
 
-// Lifted X (exact integer, |X| <= M/2) of one part from its NB chunks, returned as an unevaluated sum hi + lo with
-// |lo| <= ulp(hi)/2.  Chunk k arrives as the bit pattern of the double (1.5 2^52 + V_k) 2^(32k), with
+// Lifted X (exact integer, |X| <= M/2) of one part from its NB chunks, returned as an unevaluated sum hi + lo (not
+// normalised: lo collects the error terms of the additions, whose own sum is rounded: X = hi + lo up to a few 2^-106 of the
+// largest intermediate sum, which exceeds |X| only where chunks cancel, i.e. for entries far below the scale of their row and column).  Chunk k arrives as the bit pattern of the double (1.5 2^52 + V_k) 2^(32k), with
 // V_k = s_4k + 2^8 s_(4k+1) + 2^16 s_(4k+2) + 2^24 s_(4k+3) < 2^46.1 the four digit-column sums it covers; off[k] takes the
 // conversion offset and the chunk's share of 128 sum_planes W_p off again, exactly, which leaves W_k with
 // X' = sum_k W_k 2^(32k) = sum_planes residue_p W_p = X + t M.
 // t = rint(X'/M) from the three leading chunks: M >= 2^(32 NB - 64) (its bytes fill more than NB - 2 chunks), so the
 // rest is below 2^-17 M; |t| < 2^14, and |X/M| stays away from 1/2 by the scaling rule.  W_k - t Mc_k is exact
-// (|t Mc_k| < 2^46 before the weight).  The chunks are then added with error-free transformations, neighbours first, so
-// hi + lo equals X to 2^-105 relative (two chunks: hi alone is X rounded once, lo = 0).
+// (|t Mc_k| < 2^46 before the weight).  The chunks are then added with error-free transformations, neighbours first (below; two chunks: hi alone is X rounded once, lo = 0).
 template <int NB>
 __device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const double (&off)[kPostMaxNB], const PostConsts& pc, double* hi, double* lo) {
     double W[NB];
@@ -71,21 +71,25 @@ __device__ __forceinline__ void crt_finish32(const double (&bits)[NB], const dou
         *lo = 0.0;
         return;
     }
+    // Error-free additions in three operations each (s = a + b, z = s - a, e = b - z): exact whenever a is a whole multiple of
+    // ulp(b), whatever the magnitudes.  First loop: a = W[2k+1] is a multiple of 2^(64k+32), |b| = |W[2k]| < 2^(64k+48) has an ulp
+    // of at most 2^(64k-4).  Second loop: h, a rounded sum of pairs above k, is a multiple of 2^(64k+64), and |ph[k]| < 2^(64k+81)
+    // has an ulp of at most 2^(64k+29).
     double ph[NB / 2], l = 0.0;
 #pragma unroll
     for (int k = 0; k < NB / 2; ++k) {
         const double a = W[2 * k + 1], b = W[2 * k];
-        const double s = a + b;                                              // TwoSum
-        const double bb = s - a;
-        l += (a - (s - bb)) + (b - bb);
+        const double s = a + b;
+        const double z = s - a;
+        l += b - z;
         ph[k] = s;
     }
     double h = ph[NB / 2 - 1];
 #pragma unroll
     for (int k = NB / 2 - 2; k >= 0; --k) {
         const double s = h + ph[k];
-        const double bb = s - h;
-        l += (h - (s - bb)) + (ph[k] - bb);
+        const double z = s - h;
+        l += ph[k] - z;
         h = s;
     }
     *hi = h;

@@ -361,6 +361,53 @@ def _post_operand_checks(t, mods, M, plane_values, expected, rng_seed):
             lead = sum(W[k] << (32 * k) for k in range(max(nb - 3, 0), nb))
             assert abs(lead - X1) * 2 ** 17 <= M and abs(tq) < 2 ** 14      # dropped chunks do not move the quotient
             assert all(abs(W[k] * 2 ** (32 * k) - tq * mc[k]) < 2 ** (47 + 32 * k) for k in range(nb))   # fused multiply-adds exact
+            if abs(X1 - tq * M) * 2 <= M and nb > 2:
+                _check_three_op_sums([W[k] * 2 ** (32 * k) - tq * mc[k] for k in range(nb)], X1 - tq * M)
+
+
+def _check_three_op_sums(terms, X, rounded=True):
+    """The finish adds its chunks with three-operation error-free additions (s = a + b, z = s - a, e = b - z), which are exact
+    when a is a whole multiple of ulp(b).  Emulated here in IEEE doubles (Python floats) in the kernel's order: neighbours
+    first, then from the top down; every step must be error-free, so hi plus the error terms is X exactly; the error terms'
+    own floating-point sum is off by at most a few 2^-106 of the largest intermediate sum."""
+    Wf = [float(v) for v in terms]
+    assert all(int(w) == v for w, v in zip(Wf, terms))
+    errs, sums = [], [1.0]
+
+    def add(a, b):
+        s = a + b
+        z = s - a
+        e = b - z
+        assert int(s) + int(e) == int(a) + int(b), (a, b)
+        errs.append(e)
+        sums.append(abs(s))
+        return s
+
+    ph = [add(Wf[2 * k + 1], Wf[2 * k]) for k in range(len(Wf) // 2)]
+    h = ph[-1]
+    for k in range(len(ph) - 2, -1, -1):
+        h = add(h, ph[k])
+    assert int(h) + sum(int(e) for e in errs) == X
+    lo = 0.0
+    for e in errs:
+        lo += e
+    slack = abs(int(h) + int(lo) - X)
+    assert slack * 2 ** 104 <= int(max(sums))
+    if rounded and slack * 2 ** 70 <= abs(X):                      # chunks that cancel to a tiny X aside, the result is X rounded once
+        assert h + lo == float(X)
+
+
+def test_three_operation_sums_hold_for_adversarial_magnitudes():
+    # small or zero upper terms beside full-size lower ones: the case the usual |a| >= |b| condition does not cover
+    rng = np.random.default_rng(5)
+    for nb in (4, 6):
+        for trial in range(2000):
+            terms = []
+            for k in range(nb):
+                mag = int(rng.integers(0, 48))
+                v = int(rng.integers(-2 ** mag, 2 ** mag + 1)) if rng.random() > 0.2 else 0
+                terms.append(v * 2 ** (32 * k))
+            _check_three_op_sums(terms, sum(terms), rounded=False)   # (ties between the error terms decide the last bit here)
 
 
 @pytest.mark.parametrize("nmod", [1, 2, 7, 8, 9, 16, 17, 18, 22, 23, 26])
