@@ -189,18 +189,18 @@ constexpr int64_t kMaxRows = 65535LL * 32;   // grid.y limit of the residue kern
 // hex: the Eisenstein variant's lattice rounding in front of the same residue arithmetic (complex double only).
 template <typename T>
 int run_residues(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
-                 const ResidueTable& tab, bool wide, int8_t* planes, int* dev_status, cudaStream_t st, bool hex = false,
+                 const ResidueTable& tab, int width, int8_t* planes, int* dev_status, cudaStream_t st, bool hex = false,
                  ScaleFrom from = ScaleFrom()) {
     if (hex) {
         if constexpr (sizeof(T) == 8) {
-            CK(launch_residues_hex(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1], from));
+            CK(launch_residues_hex(X, ld, k_contiguous, conj, R, K, Kp, e, tab, width == 1, planes, st, &g.launches[1], from));
             return GEMM2M_OK;
         } else {
             return GEMM2M_ERR_ARG;
         }
     }
     (void)dev_status;
-    CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, wide, planes, st, &g.launches[1], 0, from));
+    CK(launch_residues_fp<T>(X, ld, k_contiguous, conj, R, K, Kp, e, tab, width, planes, st, &g.launches[1], 0, from));
     return GEMM2M_OK;
 }
 
@@ -306,6 +306,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
     // (Eisenstein variant: the coordinate u reaches 2^(P - c_k + 1) + 1)
     const int head = eis ? 2 : 0;
     const bool wideA = two_norm_mode ? sc.PA > 61 : sc.PA - sc.ck + head > 62, wideB = two_norm_mode ? sc.PB > 61 : sc.PB - sc.ck + head > 62;
+    // narrow: every quantised part stays below 2^30 in magnitude (the same bounds, 32 bits down), which halves the residue kernel's byte-weight chains
+    const bool narrowA = !eis && (two_norm_mode ? sc.PA <= 29 : sc.PA - sc.ck + head <= 30), narrowB = !eis && (two_norm_mode ? sc.PB <= 29 : sc.PB - sc.ck + head <= 30);
+    const int widthA = wideA ? 1 : narrowA ? 2 : 0, widthB = wideB ? 1 : narrowB ? 2 : 0;
 
     Phases ph;
     if (int s = begin_call(&ph)) return s;
@@ -353,9 +356,9 @@ int xgemm2m(int op, char transa, char transb, int64_t m, int64_t n, int64_t k, c
         fromA.absmax = (const unsigned long long*)absA; fromA.P = sc.PA; fromA.ck = sc.ck;
         fromB.absmax = (const unsigned long long*)absB; fromB.P = sc.PB; fromB.ck = sc.ck;
     }
-    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, wideA, apm, dev_status, st, eis, fromA)) return s;
+    if (int s = run_residues<T>(A, lda, ta != 'N', ta == 'C', m, k, c.kp, eA, rtab, widthA, apm, dev_status, st, eis, fromA)) return s;
     if (sb != st) CK(cudaStreamWaitEvent(st, D().side_done, 0));
-    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, wideB, bpm, dev_status, st, eis, fromB)) return s;
+    if (int s = run_residues<T>(B, ldb, tb == 'N', tb == 'C', n, k, c.kp, eB, rtab, widthB, bpm, dev_status, st, eis, fromB)) return s;
     CK(ph.end(st));
     // Eq. (2b): 2 real int8 GEMMs per 2M modulus (3 per 3M modulus of the hybrid, Eq. (1)); TMEM lanes = columns of C (rows of Bpm), TMEM columns = rows of C (rows of Apm).
     // The columns of C are cut into panels: one GEMM launch and one launch of Eq. (2c) + steps 5-7 per panel, in order.

@@ -202,10 +202,11 @@ template <typename T> cudaError_t launch_exponents_2norm(const T* X, int64_t row
 // conj: the operand is the complex conjugate of X.  wide = quantised values may need more than 62 bits (P - c_k > 62).
 cudaError_t launch_residues_hex(const double* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
                                 const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, ScaleFrom from = ScaleFrom());
+// width: 0 = quantised values of up to 62 bits, 1 = wide (up to 94 bits), 2 = narrow (|value| < 2^31: half the byte-weight chain).
 // plane_rows: rows of a whole plane when the launch covers a row range of the operand only (X, e and planes then point at the
 // first row of the range); 0 = R.
 template <typename T> cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp,
-                                                     int32_t* e, const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches,
+                                                     int32_t* e, const ResidueTable& tab, int width, int8_t* planes, cudaStream_t st, int* launches,
                                                      int64_t plane_rows = 0, ScaleFrom from = ScaleFrom());
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
                                  const ResidueTable& tab, int8_t* planes, cudaStream_t st, int* launches);

@@ -134,13 +134,18 @@ __device__ __forceinline__ void store_run(int8_t* dst, const uint32_t (&w)[NE / 
 }
 
 // One 2M modulus (index j) of emit_run: X+ into plane j, X- into plane n2 + j.
-template <int NE, bool WIDE>
+template <int NE, bool WIDE, bool NARROW>
 __device__ __forceinline__ void emit_2m(int j, int n2, const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tr, const uint32_t* ti,
                                         const ResidueTable& tab, int8_t* dst, int64_t plane_stride) {
     const int neg_m = -tab.m[j], y0 = tab.magic[j];
     const float inv_m = tab.inv_m[j], cq = tab.cq[j];
     const uint32_t wl = tab.w_lo[j], wh = tab.w_hi[j], sl = tab.ws_lo[j], sh = tab.ws_hi[j];
     const uint32_t wt = WIDE ? tab.w_top[j] : 0u, st = WIDE ? tab.ws_top[j] : 0u;
+    // Narrow mode: every part fits 32 bits and arrives as u = x + 2^31 (four unsigned bytes): one dp4a per part, and the 2^31 comes
+    // off again as 128 times the weight of byte 3 (of the real part's weights at the start of the chain, of the imaginary part's
+    // weights, which carry the factor s, where the chain continues).
+    const int y0n = NARROW ? y0 - 128 * (int)(int8_t)(wl >> 24) : y0;
+    const int kin = NARROW ? 128 * (int)(int8_t)(sl >> 24) : 0;
     uint32_t pw[NE / 4], mw[NE / 4];
 #pragma unroll
     for (int w = 0; w < NE / 4; ++w) {
@@ -148,11 +153,11 @@ __device__ __forceinline__ void emit_2m(int j, int n2, const Digits (&dr)[NE], c
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const int i = 4 * w + b;
-            int Ry = dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
+            int Ry = NARROW ? dp4a_us(dr[i].lo, wl, y0n) : dp4a_ss(dr[i].hi, wh, dp4a_us(dr[i].lo, wl, y0));  // A_r mod m (unreduced) on top of the bits of Y0
             if (WIDE) Ry = dp4a_ss(tr[i], wt, Ry);                      // digits 8..11 of the 96-bit value
             // The imaginary part's weights continue the same chain: no separate addition for the "+" sum of Eq. (2a),
             // and the "-" sum is 2 Ry - yp, a three-input integer add that does not compete with the dp4a's for their pipe.
-            int yp = dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, Ry));
+            int yp = NARROW ? dp4a_us(di[i].lo, sl, Ry - kin) : dp4a_ss(di[i].hi, sh, dp4a_us(di[i].lo, sl, Ry));
             if (WIDE) yp = dp4a_ss(ti[i], st, yp);
             const int ym = (int)(2u * (uint32_t)Ry - (uint32_t)yp);     // the doubled bit pattern wraps, the difference does not
             sym_reduce_pm(yp, ym, neg_m, inv_m, cq, &bp[b], &bm[b]);
@@ -169,18 +174,18 @@ __device__ __forceinline__ void emit_2m(int j, int n2, const Digits (&dr)[NE], c
 // moduli of the hybrid.  dst points at plane 0, this row, first k of the run; tr / ti (wide mode) hold the four top digits
 // of each part.  NMOD > 0: exactly NMOD moduli, all of them 2M moduli, known at compile time: the loop is unrolled and the
 // per-modulus constants become constant-bank operands instead of loads.
-template <int NE, bool WIDE, int NMOD>
+template <int NE, bool WIDE, int NMOD, bool NARROW>
 __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&di)[NE], const uint32_t* tr, const uint32_t* ti,
                                          const ResidueTable& tab, int8_t* dst, int64_t plane_stride) {
     static_assert(NE == 8 || NE == 16, "runs of 8 or 16 elements");
     if constexpr (NMOD > 0) {
 #pragma unroll
-        for (int j = 0; j < NMOD; ++j) emit_2m<NE, WIDE>(j, NMOD, dr, di, tr, ti, tab, dst, plane_stride);
+        for (int j = 0; j < NMOD; ++j) emit_2m<NE, WIDE, NARROW>(j, NMOD, dr, di, tr, ti, tab, dst, plane_stride);
         return;
     }
     const int nmod = tab.nmod, n2 = tab.n2;
 #pragma unroll 1
-    for (int j = 0; j < n2; ++j) emit_2m<NE, WIDE>(j, n2, dr, di, tr, ti, tab, dst, plane_stride);
+    for (int j = 0; j < n2; ++j) emit_2m<NE, WIDE, NARROW>(j, n2, dr, di, tr, ti, tab, dst, plane_stride);
     const int n3 = nmod - n2;
     int8_t* dst3 = dst + (int64_t)(2 * n2) * plane_stride;
 #pragma unroll 1
@@ -216,7 +221,7 @@ __device__ __forceinline__ void emit_run(const Digits (&dr)[NE], const Digits (&
 }
 
 // ---- floating-point inputs: persistent blocks, raw elements copied asynchronously into a two-stage ring (residues_common.cuh)
-template <typename T, bool WIDE, int NMOD, bool HEX = false>
+template <typename T, bool WIDE, int NMOD, bool HEX = false, bool NARROW = false>
 __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kernel(const T* __restrict__ X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K,
                                                                      int64_t Kp, int32_t* __restrict__ e, const ScaleFrom from,
                                                                      const __grid_constant__ ResidueTable tab, int8_t* __restrict__ planes,
@@ -319,11 +324,16 @@ __global__ void __launch_bounds__(kResThreads, kResBlocksPerSm) residues_fp_kern
                         qr = quantise_part<T>(v.x, ex);
                         qi = quantise_part<T>(v.y, ex);
                     }
-                    dr[i] = split_digits(qr);
-                    di[i] = split_digits(qi);
+                    if (NARROW) {              // |q| < 2^31: the low word plus 2^31 as four unsigned bytes
+                        dr[i].lo = (uint32_t)(unsigned long long)qr ^ 0x80000000u; dr[i].hi = 0u;
+                        di[i].lo = (uint32_t)(unsigned long long)qi ^ 0x80000000u; di[i].hi = 0u;
+                    } else {
+                        dr[i] = split_digits(qr);
+                        di[i] = split_digits(qi);
+                    }
                 }
             }
-            emit_run<kResRun, WIDE, NMOD>(dr, di, tr, ti, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
+            emit_run<kResRun, WIDE, NMOD, NARROW>(dr, di, tr, ti, tab, planes + row * Kp + k0 + kResRun * g, plane_stride);
         }
         __syncthreads();   // everyone is done with this stage before it is refilled
     }
@@ -334,9 +344,11 @@ constexpr size_t kResSmemBytes(size_t elem) { return (size_t)kResStages * kResRo
 
 template <typename T>
 cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool conj, int64_t R, int64_t K, int64_t Kp, int32_t* e,
-                               const ResidueTable& tab, bool wide, int8_t* planes, cudaStream_t st, int* launches, int64_t plane_rows,
+                               const ResidueTable& tab, int width, int8_t* planes, cudaStream_t st, int* launches, int64_t plane_rows,
                                ScaleFrom from) {
     if (R <= 0 || Kp <= 0) return cudaSuccess;
+    const bool wide = width == 1;
+    const bool narrow = width == 2 && tab.n2 == tab.nmod;      // (the 3M moduli of the hybrid only come with wide values)
     constexpr size_t smem = kResSmemBytes(2 * sizeof(T));
     static bool attr_set_dev[kMaxDevices] = {};
     bool& attr_set = attr_set_dev[current_device_slot()];
@@ -346,6 +358,9 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
 #define GEMM2M_RES_ATTR(N) if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, false, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         GEMM2M_RES_ATTR(7) GEMM2M_RES_ATTR(8) GEMM2M_RES_ATTR(14) GEMM2M_RES_ATTR(15) GEMM2M_RES_ATTR(16)
 #undef GEMM2M_RES_ATTR
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, false, 7, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err == cudaSuccess) err = cudaFuncSetAttribute(residues_fp_kernel<T, false, 8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         attr_set = true;
     }
@@ -356,6 +371,14 @@ cudaError_t launch_residues_fp(const T* X, int64_t ld, bool k_contiguous, bool c
     // get a specialisation with the modulus loop unrolled: the per-modulus constants become constant-bank operands, which
     // saves two instructions per (element, modulus) -- 13 % of the kernel's time at 16 moduli.
     const int spec = (!wide && tab.n2 == tab.nmod) ? tab.nmod : 0;
+    if (narrow) {
+        // Values below 2^31 (few moduli: single precision, or the fastest double-precision settings): one dp4a per part
+        if (spec == 7) launch_chained(residues_fp_kernel<T, false, 7, false, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+        else if (spec == 8) launch_chained(residues_fp_kernel<T, false, 8, false, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+        else launch_chained(residues_fp_kernel<T, false, 0, false, true>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R);
+        ++*launches;
+        return cudaGetLastError();
+    }
     switch (spec) {
 #define GEMM2M_RES_CASE(N) case N: launch_chained(residues_fp_kernel<T, false, N>, grid, dim3(kResThreads), smem, st, X, ld, k_contiguous, conj, R, K, Kp, e, from, tab, planes, plane_rows ? plane_rows : R); break;
         GEMM2M_RES_CASE(7) GEMM2M_RES_CASE(8) GEMM2M_RES_CASE(14) GEMM2M_RES_CASE(15) GEMM2M_RES_CASE(16)
@@ -549,7 +572,7 @@ __global__ void __launch_bounds__(kResIThreads) residues_int8_kernel(const int8_
     }
     const int64_t row = row0 + r;
     if (row >= R) return;
-    emit_run<kResIRun, false, 0>(dr, di, nullptr, nullptr, tab, planes + row * Kp + k0 + kResIRun * g, R * Kp);
+    emit_run<kResIRun, false, 0, false>(dr, di, nullptr, nullptr, tab, planes + row * Kp + k0 + kResIRun * g, R * Kp);
 }
 
 cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld, bool k_contiguous, int64_t R, int64_t K, int64_t Kp,
@@ -569,7 +592,7 @@ cudaError_t launch_residues_int8(const int8_t* Xr, const int8_t* Xi, int64_t ld,
     return cudaGetLastError();
 }
 
-template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
-template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, bool, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
+template cudaError_t launch_residues_fp<double>(const double*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, int, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
+template cudaError_t launch_residues_fp<float>(const float*, int64_t, bool, bool, int64_t, int64_t, int64_t, int32_t*, const ResidueTable&, int, int8_t*, cudaStream_t, int*, int64_t, ScaleFrom);
 
 }  // namespace gemm2m

@@ -114,7 +114,10 @@ def run_z(A, B, nmod, kernel=0, cplx=torch.complex128, op=None):
 
 @pytest.mark.parametrize("kernel", [1, 0], ids=["checkgemm", "tcgen05"])
 @pytest.mark.parametrize("shape,nmod,dist", [((200, 150, 300), 16, "phi"), ((129, 257, 128), 14, "uniform"),
-                                             ((64, 64, 64), 3, "uniform"), ((33, 19, 50), 22, "phi"), ((40, 40, 520), 20, "uniform")])
+                                             ((64, 64, 64), 3, "uniform"), ((33, 19, 50), 22, "phi"), ((40, 40, 520), 20, "uniform"),
+                                             # few moduli: quantised parts below 2^31 take the residue kernel's 32-bit path
+                                             ((96, 80, 260), 8, "phi"), ((50, 70, 90), 7, "uniform"), ((70, 33, 130), 10, "phi"),
+                                             ((33, 70, 40), 11, "uniform")])
 def test_zgemm_every_stage_against_staged_oracle(shape, nmod, dist, kernel):
     m, n, k = shape
     A, B = inputs.complex_inputs(m, n, k, seed=7, dist=dist, phi=1.0)
