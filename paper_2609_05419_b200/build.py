@@ -40,6 +40,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_issue_rates(out_dir: str | None = None) -> str:
+    """Compiles csrc/issue_rates.cu (a stand-alone microbenchmark of instruction issue rates, not part of the library) into
+    an executable under out_dir (default: next to this file, as issue_rates.bin) and returns its path."""
+    exe = os.path.join(out_dir or HERE, "issue_rates.bin")
+    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
+           os.path.join(CSRC, "issue_rates.cu"), "-o", exe + ".tmp"]
+    subprocess.run(cmd, check=True)
+    os.replace(exe + ".tmp", exe)
+    return exe
+
+
 if __name__ == "__main__":
     import sys
     print(build(force=True, verbose="-v" in sys.argv))
