@@ -37,7 +37,9 @@ def run(A, B, nmod, cplx=torch.complex128, kernel=0, ta="N", tb="N"):
 
 @pytest.mark.parametrize("shape,nmod,dist,ta,tb", [((200, 150, 300), 16, "phi", "N", "N"), ((129, 257, 1000), 14, "uniform", "T", "N"),
                                                    ((33, 19, 50), 22, "phi", "N", "C"), ((70, 90, 200), 25, "phi", "C", "T"),
-                                                   ((64, 64, 2100), 17, "phi", "N", "N")])
+                                                   ((64, 64, 2100), 17, "phi", "N", "N"),
+                                                   # few moduli: the residue kernel's 32-bit form under this rule (P_A <= 29)
+                                                   ((90, 70, 260), 7, "phi", "N", "N"), ((50, 60, 130), 8, "uniform", "C", "N")])
 def test_2norm_rule_every_stage(shape, nmod, dist, ta, tb):
     m, n, k = shape
     A, B = inputs.complex_inputs(m, n, k, seed=81, dist=dist, phi=2.0)
